@@ -1,0 +1,168 @@
+/*
+ * libfgmp -- the FGMP linear layer (fine-grained mixed-precision NVFP4/FP8 weights and
+ * activations) for NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes only.
+ *
+ * Orientation (Section 3: Y = W x X, blocks run along the dot-product dimension):
+ *   activations X [M, K], weights W [N, K], output Y [M, N]; K is contiguous in X and W.
+ * A block is 16 consecutive elements along K (Section 4: block size = NVFP4 microscale
+ * block = vector length 16).  Each block is stored either as NVFP4 (16 E2M1 codes + one
+ * E4M3 microscale, times an FP32 tensor scale) or as FP8 E4M3 (times an FP32 tensor
+ * scale, no microscale), with one metadata bit per block (Section 4, Section 5.1).
+ *
+ * Conventions for every entry point
+ *   - every data pointer is a DEVICE pointer owned by the caller, unless it says "host";
+ *   - the library allocates no device memory: scratch comes in through `workspace`
+ *     (size from fgmp_workspace_bytes); a workspace may be reused once the call that used
+ *     it has completed on its stream;
+ *   - calls are asynchronous on `cuda_stream` (a cudaStream_t, may be NULL for the default
+ *     stream); the return value reports argument validation and launch errors only;
+ *   - requirements: K % 64 == 0, K >= 64, rows >= 1, bf16 inputs finite, input pointers
+ *     16-byte aligned, leading dimensions multiples of 8 elements;
+ *   - a packed tensor is an opaque device blob (layout below) produced by the two
+ *     quantizers and consumed by fgmp_linear / fgmp_unpack; it must be 1024-byte aligned.
+ *
+ * Packed blob layout (all sections 1024-byte aligned, in this order)
+ *   header  256 B : fgmp_packed_header (device-written)
+ *   codes4        : rows * K/2 bytes, row-major; two E2M1 codes per byte, even element in
+ *                   the low nibble; all-zero for FP8 blocks
+ *   sf            : E4M3 microscales in 512-byte tiles of 128 rows x 4 blocks:
+ *                   byte of (row r, block kb) = ((r/128) * (K/64) + kb/4) * 512
+ *                                               + (r%32)*16 + ((r%128)/32)*4 + kb%4;
+ *                   0x00 for FP8 blocks and for padding rows
+ *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
+ *                   1 = FP8
+ *   wordptr       : (weights only) one uint32 per mask word = number of FP8 blocks that
+ *                   precede the word's first block in row-major block order
+ *   codes8        : weights: the FP8 blocks only, 16 bytes each, in row-major block order
+ *                   (capacity max_fp8_blocks); activations: a dense rows*K byte plane of
+ *                   which only the FP8 blocks are written.
+ */
+#ifndef FGMP_H
+#define FGMP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FGMP_OK = 0,
+    FGMP_ERR_INVALID_ARG = -1, /* NULL pointer, bad enum, non-finite or non-positive scale   */
+    FGMP_ERR_SHAPE = -2,       /* K % 64, leading dimension, alignment                       */
+    FGMP_ERR_WORKSPACE = -3,   /* workspace or output blob too small                         */
+    FGMP_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed                          */
+    FGMP_ERR_ARCH = -5,        /* current device is not compute capability 10.x              */
+    FGMP_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (see fgmp_check)        */
+    FGMP_ERR_CAPACITY = -7     /* more FP8 blocks than the packed blob has room for          */
+} fgmp_status;
+
+/* Which block score decides the precision.
+ *   FGMP_SCORE_LP_ERROR : sum_i f_i (v_i - Q_NVFP4(v_i))^2          (Eq. 6)
+ *   FGMP_SCORE_HP_TO_LP : sum_i f_i (Q_NVFP4(v_i) - Q_FP8(v_i))^2   (Eq. 7-8)          */
+typedef enum { FGMP_SCORE_LP_ERROR = 0, FGMP_SCORE_HP_TO_LP = 1 } fgmp_score_mode;
+
+/* NVFP4 microscale of weight blocks: dynamic max, or the sensitivity-weighted brute-force
+ * search over all 126 positive finite E4M3 scales (Eq. 11).  Activations always use
+ * dynamic max (Section 3.3). */
+typedef enum { FGMP_CLIP_NONE = 0, FGMP_CLIP_SW_BRUTE = 1 } fgmp_clip_mode;
+
+typedef struct {
+    float scale_fp4;    /* FP32 tensor scale of the NVFP4 part; 0 = derive amax/(6*448)
+                           on the device (weights only)                                     */
+    int fp8_log2_ratio; /* FP8 tensor scale = scale_fp4 * 2^ratio, -8 <= ratio <= 8        */
+} fgmp_scales;
+
+/* First 256 bytes of a packed blob (device memory). */
+typedef struct {
+    uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
+    uint32_t version;        /* layout version, 1                                           */
+    int64_t rows, K;
+    float scale_fp4;         /* tensor scale actually used                                  */
+    int32_t fp8_log2_ratio;
+    int64_t n_fp8;           /* number of FP8 blocks                                        */
+    float tau_eff;           /* weights, fraction mode: smallest selected score             */
+    uint32_t kind;           /* 0 = activations, 1 = weights                                */
+    int64_t capacity;        /* weights: room for this many FP8 blocks                      */
+    int32_t error;           /* 0, or FGMP_ERR_CAPACITY                                     */
+    int32_t reserved[49];
+} fgmp_packed_header;
+
+enum { FGMP_OP_QUANTIZE_WEIGHTS = 0, FGMP_OP_QUANTIZE_ACTIVATIONS = 1, FGMP_OP_LINEAR = 2,
+       FGMP_OP_CALIBRATE_TAU = 3 };
+
+/* ---- sizes (pure host functions; return 0 for invalid shapes) ---- */
+size_t fgmp_weights_bytes(int64_t N, int64_t K, int64_t max_fp8_blocks);
+size_t fgmp_acts_bytes(int64_t M, int64_t K);
+/* scratch needed by one call of `op` (FGMP_OP_*); M or N is ignored where it has no meaning */
+size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K);
+
+/* ---- offline: weight packing (Section 3.1-3.3; Eq. 8, 9, 11) ----
+ * W_bf16 [N, ldw] bf16, fisher_elem [N, ldf] fp32 (per-element diagonal Fisher information,
+ * the g^2 of Eq. 6).  Per block: microscale (dynamic max or Eq. 11 search), score under that
+ * scale (Eq. 6 or Eq. 8).  fp8_fraction >= 0: exactly floor(fraction * N*K/16 + 0.5) blocks
+ * with the largest scores are kept in FP8 (Eq. 9: the top-R percentile of one tensor; equal
+ * scores are taken in row-major block order) and tau is ignored; fp8_fraction < 0: a block
+ * is FP8 iff score > tau.  The blob must have room for the result
+ * (packed_bytes >= fgmp_weights_bytes(N, K, max_fp8_blocks)); if threshold mode finds
+ * more FP8 blocks than that, header.error = FGMP_ERR_CAPACITY and the blob is invalid.
+ * tau_eff_out (device float, may be NULL) receives the smallest selected score. */
+fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, const float* fisher_elem, int64_t ldf,
+                                  int64_t N, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
+                                  fgmp_clip_mode cm, double fp8_fraction, float tau,
+                                  void* packed_out, size_t packed_bytes, float* tau_eff_out,
+                                  void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- online: activation quantizer (Section 4.2) ----
+ * X_bf16 [M, ldx] bf16, fisher_chan [K] fp32 (average squared gradient per input channel).
+ * Per block: dynamic-max NVFP4 scale, NVFP4 rounding, the score, FP8 iff score > tau
+ * (tau is calibrated offline and fixed; +inf = all NVFP4, negative = all FP8), then the
+ * block is written in its format.  sc.scale_fp4 must be > 0.  No workspace needed
+ * (workspace may be NULL). */
+fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                                      int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm, float tau,
+                                      void* packed_out, size_t packed_bytes,
+                                      void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- offline: activation threshold for a target FP8 fraction (Eq. 9, local threshold) ----
+ * Scores every block of a calibration batch X and writes to tau_out (device float) the
+ * value midway (in fp32) between the k-th and (k+1)-th largest score, k = floor(fraction *
+ * blocks + 0.5), so that exactly k blocks of this batch exceed it unless scores tie. */
+fgmp_status fgmp_calibrate_tau(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                               int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
+                               double fp8_fraction, float* tau_out,
+                               void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- the mixed-precision GEMM (Section 4.1) ----
+ * Y[m, n] = sum over blocks of dot16(A[m, kb], W[n, kb]) with each block pair multiplied in
+ * its own formats (FP4xFP4, FP4xFP8, FP8xFP4, FP8xFP8), microscales and tensor scales
+ * applied, accumulated in FP32.  Y is fp32 (y_is_bf16 = 0) or bf16 [M, ldy].  The first
+ * 256 bytes of the workspace hold a status word that fgmp_check reads. */
+fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
+                        void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                        void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* Synchronizes the stream and returns the device-side status recorded in a workspace used
+ * by fgmp_linear (FGMP_OK or FGMP_ERR_TIMEOUT). */
+fgmp_status fgmp_check(const void* workspace, void* cuda_stream);
+
+/* ---- parity support: packed -> canonical arrays (device) ----
+ * codes4 [rows*K/2] (0 for FP8 blocks), codes8 [rows*K] (0 for FP4 blocks), scales
+ * [rows*K/16] E4M3 (0 for FP8 blocks), mask [rows*ceil(K/16/32)], scores is not stored.
+ * Any output pointer may be NULL. */
+fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, uint8_t* codes4, uint8_t* codes8,
+                        uint8_t* scales, uint32_t* mask, void* cuda_stream);
+
+/* Block scores only (parity support and calibration): scores [M*K/16] fp32, activations. */
+fgmp_status fgmp_activation_scores(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                                   int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
+                                   float* scores, void* cuda_stream);
+
+const char* fgmp_status_string(fgmp_status s);
+int fgmp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FGMP_H */

@@ -1,0 +1,10 @@
+"""B200-native FGMP linear layer: thin Python binding over the C-ABI library libfgmp.so.
+
+Every step of the path runs in the CUDA kernels of the library; this package only
+marshals arguments (torch tensors give device memory and streams).
+"""
+from .binding import (  # noqa: F401
+    FgmpError, PackedTensor, SCORE_LP_ERROR, SCORE_HP_TO_LP, CLIP_NONE, CLIP_SW_BRUTE,
+    acts_bytes, weights_bytes, workspace_bytes, quantize_weights, quantize_activations,
+    calibrate_tau, activation_scores, linear, check, unpack, version, status_string, library_path,
+)

@@ -1,0 +1,160 @@
+// Shared device/host helpers of libfgmp: packed-blob layout arithmetic, number-format
+// conversions and the pinned single-precision quantization sequence.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "fgmp.h"
+
+#define FGMP_MAGIC 0x504d4746u
+#define FGMP_BS 16
+
+// ---------------------------------------------------------------- blob layout
+struct PackedLayout {
+    int64_t rows, K, KB, MW;          // KB = K/16 blocks per row, MW = mask words per row
+    size_t off_codes4, off_sf, off_mask, off_wordptr, off_codes8, total;
+};
+
+__host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
+
+// kind 0 = activations (dense FP8 plane), 1 = weights (compact FP8 list, capacity blocks)
+__host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int kind, int64_t capacity)
+{
+    PackedLayout L;
+    L.rows = rows; L.K = K; L.KB = K / 16; L.MW = (L.KB + 31) / 32;
+    size_t o = 1024;                                   // header section
+    L.off_codes4 = o;  o = fgmp_align1k(o + (size_t)rows * (size_t)(K / 2));
+    L.off_sf = o;      o = fgmp_align1k(o + (size_t)((rows + 127) / 128) * (size_t)(K / 64) * 512);
+    L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
+    L.off_wordptr = o; if (kind == 1) o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
+    L.off_codes8 = o;
+    o = fgmp_align1k(o + (kind == 1 ? (size_t)capacity * 16 : (size_t)rows * (size_t)K));
+    L.total = o;
+    return L;
+}
+
+// byte offset of the microscale of (row r, block kb) inside the sf section
+__host__ __device__ inline size_t fgmp_sf_offset(int64_t r, int64_t kb, int64_t K)
+{
+    return ((size_t)(r >> 7) * (size_t)(K >> 6) + (size_t)(kb >> 2)) * 512
+         + (size_t)(r & 31) * 16 + (size_t)((r & 127) >> 5) * 4 + (size_t)(kb & 3);
+}
+
+// ---------------------------------------------------------------- conversions
+#ifdef __CUDACC__
+
+// two floats -> two E2M1 codes in one byte: `lo` in bits 0..3, `hi` in bits 4..7.
+// Round to nearest even, saturating to +-6 (cvt.rn.satfinite.e2m1x2.f32).
+__device__ __forceinline__ uint32_t f32x2_to_e2m1x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("{\n\t.reg .b8 t;\n\tcvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n\tcvt.u32.u8 %0, t;\n\t}"
+        : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// two floats -> two E4M3 codes: `lo` in bits 0..7, `hi` in bits 8..15 (satfinite, RNE).
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// byte of two E2M1 codes -> two floats (exact)
+__device__ __forceinline__ float2 e2m1x2_to_f32x2(uint32_t byte)
+{
+    uint32_t h2;
+    asm("{\n\t.reg .b8 t;\n\tcvt.u8.u32 t, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, t;\n\t}" : "=r"(h2) : "r"(byte));
+    __half2 h = *reinterpret_cast<__half2*>(&h2);
+    return __half22float2(h);
+}
+
+// two E4M3 codes (low 16 bits) -> two floats (exact)
+__device__ __forceinline__ float2 e4m3x2_to_f32x2(uint32_t two)
+{
+    uint32_t h2;
+    uint16_t s = (uint16_t)two;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(s));
+    __half2 h = *reinterpret_cast<__half2*>(&h2);
+    return __half22float2(h);
+}
+
+__device__ __forceinline__ float e4m3_to_f32(uint32_t code) { return e4m3x2_to_f32x2(code & 0xff).x; }
+
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t pair) { return __uint_as_float(pair << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t pair) { return __uint_as_float(pair & 0xffff0000u); }
+
+// ---------------------------------------------------------------- block math
+// One block of 16 values in registers.  Every step below is a single IEEE fp32 operation
+// (no contraction): this sequence is what makes codes and scores reproducible bit for bit.
+
+struct BlockQ {
+    uint32_t c4[2];     // 16 E2M1 codes, element i in nibble i
+    float score;
+};
+
+// dynamic-max microscale code: E4M3(amax * k6), k6 = 1 / (6 * s4)
+__device__ __forceinline__ uint32_t block_dynamic_scale(const float (&v)[16], float k6)
+{
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+    return f32x2_to_e4m3x2(__fmul_rn(amax, k6), 0.f) & 0x7f;
+}
+
+// NVFP4 rounding under microscale code `sc`; dq receives the dequantized values
+__device__ __forceinline__ void block_nvfp4(const float (&v)[16], uint32_t sc, float s4,
+                                            uint32_t (&c4)[2], float (&dq)[16])
+{
+    float d = __fmul_rn(e4m3_to_f32(sc), s4);
+    float inv = (d == 0.f) ? 0.f : __fdiv_rn(1.0f, d);
+    c4[0] = 0; c4[1] = 0;
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        float y0 = __fmul_rn(v[i], inv), y1 = __fmul_rn(v[i + 1], inv);
+        // inv == 0 (zero scale): keep only the signs, as -0.0 * 0 = -0.0 does
+        uint32_t b = f32x2_to_e2m1x2(y0, y1);
+        float2 q = e2m1x2_to_f32x2(b);
+        dq[i] = __fmul_rn(q.x, d);
+        dq[i + 1] = __fmul_rn(q.y, d);
+        c4[i >> 3] |= b << ((i & 7) * 4);
+    }
+}
+
+// FP8 rounding of the block: 16 E4M3 codes in 4 words, dq8 = dequantized values
+__device__ __forceinline__ void block_fp8(const float (&v)[16], float inv8, float s8,
+                                          uint32_t (&c8)[4], float (&dq)[16])
+{
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        uint32_t two = f32x2_to_e4m3x2(__fmul_rn(v[i], inv8), __fmul_rn(v[i + 1], inv8));
+        float2 q = e4m3x2_to_f32x2(two);
+        dq[i] = __fmul_rn(q.x, s8);
+        dq[i + 1] = __fmul_rn(q.y, s8);
+        if ((i & 3) == 0) c8[i >> 2] = two; else c8[i >> 2] |= two << 16;
+    }
+}
+
+// sum_i (f_i * e_i) * e_i, in element order
+__device__ __forceinline__ float weighted_sq_sum(const float (&a)[16], const float (&b)[16],
+                                                 const float (&f)[16])
+{
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        float e = __fsub_rn(a[i], b[i]);
+        s = __fadd_rn(s, __fmul_rn(__fmul_rn(f[i], e), e));
+    }
+    return s;
+}
+
+// 16 bf16 (two 128-bit words) -> 16 floats
+__device__ __forceinline__ void unpack_bf16x16(const uint4& a, const uint4& b, float (&v)[16])
+{
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { v[2 * i] = bf16lo_to_f32(w[i]); v[2 * i + 1] = bf16hi_to_f32(w[i]); }
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,441 @@
+// fgmp_linear: the mixed-precision GEMM (Section 4.1 of the paper).
+//
+// General path ("common container"): every block of both operands, whatever its format, is
+// an exact bf16 number once its microscale is folded in (E2M1 x E4M3 scale has at most 6
+// significant bits, E4M3 has 4).  A streaming pass expands the packed operands into bf16
+// planes, and a persistent tcgen05 kernel multiplies them with FP32 accumulation in TMEM;
+// the two FP32 tensor scales are applied in the epilogue.  All four block-pair products of
+// the paper's datapath (FP4xFP4, FP4xFP8, FP8xFP4, FP8xFP8) are therefore exact products.
+//
+// Kernel structure (one CTA per SM, 192 threads):
+//   warp 0    : TMA producer   (global -> 128B-swizzled shared tiles, mbarrier complete_tx)
+//   warp 1    : MMA issuer     (tcgen05.mma kind::f16, accumulators in TMEM, double buffered)
+//   warps 2-5 : epilogue       (tcgen05.ld -> scale -> global), overlapped with the next tile
+// Every wait on an mbarrier is bounded; on expiry the CTA records FGMP_ERR_TIMEOUT and leaves.
+#include <cuda.h>
+#include "fgmp_common.cuh"
+#include "fgmp_host.h"
+
+namespace {
+
+// ------------------------------------------------------------------ expand to bf16 planes
+// plane[r, k] = e2m1 * e4m3scale (NVFP4 block) or e4m3 * 2^ratio (FP8 block); exact in bf16.
+__global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, int kind,
+                                                     uint4* plane)
+{
+    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
+    const PackedLayout L = fgmp_layout(rows, K, kind, 0);
+    const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t* wordptr = reinterpret_cast<const uint32_t*>(blob + L.off_wordptr);
+    const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
+    const int64_t nblk = rows * L.KB;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
+        int64_t r = b / L.KB, kb = b % L.KB;
+        uint32_t word = pmask[r * L.MW + (kb >> 5)];
+        bool is8 = (word >> (kb & 31)) & 1;
+        float v[16];
+        if (is8) {
+            size_t src = (kind == 1)
+                ? L.off_codes8 + (size_t)(wordptr[r * L.MW + (kb >> 5)] + __popc(word & ((1u << (kb & 31)) - 1u))) * 16
+                : L.off_codes8 + (size_t)(r * K + kb * 16);
+            uint4 c = *reinterpret_cast<const uint4*>(blob + src);
+            const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float2 a = e4m3x2_to_f32x2(w[i] & 0xffff), bb = e4m3x2_to_f32x2(w[i] >> 16);
+                v[4 * i] = a.x * r8; v[4 * i + 1] = a.y * r8; v[4 * i + 2] = bb.x * r8; v[4 * i + 3] = bb.y * r8;
+            }
+        } else {
+            uint2 c = *reinterpret_cast<const uint2*>(blob + L.off_codes4 + (r * K) / 2 + kb * 8);
+            float d = e4m3_to_f32(blob[L.off_sf + fgmp_sf_offset(r, kb, K)]);
+            const uint32_t w[2] = {c.x, c.y};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float2 q = e2m1x2_to_f32x2((w[i >> 2] >> ((i & 3) * 8)) & 0xff);
+                v[2 * i] = q.x * d; v[2 * i + 1] = q.y * d;
+            }
+        }
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)   // exact: the low 16 bits of every value are zero
+            o[i] = (__float_as_uint(v[2 * i]) >> 16) | (__float_as_uint(v[2 * i + 1]) & 0xffff0000u);
+        uint4* dst = plane + (r * K) / 8 + kb * 2;
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: gives up after ~2 s (or when another thread of the CTA already gave up),
+// records the failure and returns false.  `abort_flag` lives in shared memory.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+{
+    const unsigned long long t0 = globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > 2000000000ull) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, (int)FGMP_ERR_TIMEOUT);
+            atomicExch(status + 1, where);
+            return false;
+        }
+        __nanosleep(64);
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, where);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart (tile base 1024-byte aligned)
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
+{
+    uint64_t d = (uint64_t)((saddr & 0x3ffff) >> 4);
+    d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset: 8 rows x 128 B
+    d |= (uint64_t)1 << 46;                 // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+    return d;
+}
+
+// ------------------------------------------------------------------ bf16 tcgen05 GEMM
+constexpr int BM = 128, BN = 128, BK = 64;          // BK bf16 = one 128-byte swizzle row
+constexpr int STAGES = 6;
+constexpr int UMMA_K = 16;
+constexpr int GEMM_THREADS = 192;
+constexpr uint32_t A_TILE_BYTES = BM * BK * 2, B_TILE_BYTES = BN * BK * 2;
+constexpr uint32_t STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
+constexpr uint32_t TMEM_COLS = 2 * BN;              // two accumulator buffers
+constexpr size_t GEMM_SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=BN, M=BM
+constexpr uint32_t IDESC_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct GemmParams {
+    void* Y; int64_t ldy; int y_is_bf16;
+    int64_t M, N, K;
+    const fgmp_packed_header* ha; const fgmp_packed_header* hw;
+    int* status;
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) acc_full, [2S+2..2S+4) acc_empty
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
+    const uint32_t accf0 = smem_u32(bars + 2 * STAGES), acce0 = smem_u32(bars + 2 * STAGES + 2);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int64_t tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const int64_t num_tiles = tiles_m * tiles_n;
+    const int num_kb = (int)(p.K / BK);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                const int32_t m0 = (int32_t)((t % tiles_m) * BM), n0 = (int32_t)((t / tiles_m) * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!(ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1))) break;
+                    const uint32_t fb = full0 + 8 * stage;
+                    mbar_expect_tx(fb, STAGE_BYTES);
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+                    tma_load_2d(sa, &tmA, kb * BK, m0, fb);
+                    tma_load_2d(sa + A_TILE_BYTES, &tmB, kb * BK, n0, fb);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            int64_t it = 0;
+            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+                const int acc = (int)(it & 1); const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
+                if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+                    const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sa + A_TILE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_f16(d_tmem, adesc + (uint64_t)(k * UMMA_K * 2 / 16), bdesc + (uint64_t)(k * UMMA_K * 2 / 16),
+                                 IDESC_BF16, (kb | k) ? 1u : 0u);
+                    umma_commit(empty0 + 8 * stage);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(accf0 + 8 * acc);
+            }
+        }
+    } else {
+        const int q = warp & 3;                        // TMEM lane quadrant this warp may read
+        const float alpha = __fmul_rn(p.ha->scale_fp4, p.hw->scale_fp4);
+        bool ok = true;
+        int64_t it = 0;
+        for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+            const int acc = (int)(it & 1); const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
+            const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+            if (!(ok = mbar_wait(accf0 + 8 * acc, acc_phase, abort_flag, p.status, 4))) break;
+            tc_fence_after();
+            const int64_t row = m0 + q * 32 + lane;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+                const int64_t col0 = n0 + c * 32;
+                if (row < p.M) {
+                    if (p.y_is_bf16) {
+                        __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
+                        if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t o[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * u]) * alpha,
+                                                                             __uint_as_float(r[j + 2 * u + 1]) * alpha);
+                                    o[u] = *reinterpret_cast<uint32_t*>(&h);
+                                }
+                                *reinterpret_cast<uint4*>(y + j) = make_uint4(o[0], o[1], o[2], o[3]);
+                            }
+                        } else {
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) y[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
+                        }
+                    } else {
+                        float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
+                        if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
+                                                                                __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
+                        } else {
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) y[j] = __uint_as_float(r[j]) * alpha;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acce0 + 8 * acc);
+        }
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies and MMAs that may still be in flight time to land before the CTA's
+        // shared memory and TMEM are released
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major [rows, K] tensor, box = [box_rows, 64 elements], 128-byte swizzle
+bool make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K)
+{
+    return 1024 + fgmp_align1k((size_t)M * K * 2) + fgmp_align1k((size_t)N * K * 2);
+}
+
+extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
+                                   void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                   void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!packed_acts || !packed_weights || !Y || !workspace) return FGMP_ERR_INVALID_ARG;
+    if (M < 1 || N < 1 || K < 64 || (K % 64) != 0 || ldy < N) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
+        ((uintptr_t)Y & 15)) return FGMP_ERR_SHAPE;
+    if (ws_bytes < fgmp_ws_linear(M, N, K)) return FGMP_ERR_WORKSPACE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    int* status = reinterpret_cast<int*>(ws);
+    uint8_t* planeA = ws + 1024;
+    uint8_t* planeW = planeA + fgmp_align1k((size_t)M * K * 2);
+
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM) != cudaSuccess)
+            return FGMP_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    CUtensorMap tmA, tmB;
+    if (!make_tmap_bf16(&tmA, planeA, M, K, BM) || !make_tmap_bf16(&tmB, planeW, N, K, BN)) return FGMP_ERR_CUDA;
+
+    if (cudaMemsetAsync(status, 0, 256, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    const int sms = fgmp_sm_count();
+    {
+        int64_t nb = M * (K / 16);
+        int g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
+        expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, 0, reinterpret_cast<uint4*>(planeA));
+        nb = N * (K / 16);
+        g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
+        expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_weights, N, K, 1, reinterpret_cast<uint4*>(planeW));
+    }
+    GemmParams p;
+    p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K;
+    p.ha = reinterpret_cast<const fgmp_packed_header*>(packed_acts);
+    p.hw = reinterpret_cast<const fgmp_packed_header*>(packed_weights);
+    p.status = status;
+    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(tmA, tmB, p);
+    return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_check(const void* workspace, void* cuda_stream)
+{
+    if (!workspace) return FGMP_ERR_INVALID_ARG;
+    int host[2] = {0, 0};
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FGMP_ERR_CUDA;
+    return host[0] == 0 ? FGMP_OK : (fgmp_status)host[0];
+}
+
+extern "C" size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K)
+{
+    if (K < 64 || (K % 64) != 0) return 0;
+    switch (op) {
+        case FGMP_OP_QUANTIZE_WEIGHTS: return N >= 1 ? fgmp_ws_quantize_weights(N, K) : 0;
+        case FGMP_OP_QUANTIZE_ACTIVATIONS: return 0;
+        case FGMP_OP_LINEAR: return (M >= 1 && N >= 1) ? fgmp_ws_linear(M, N, K) : 0;
+        case FGMP_OP_CALIBRATE_TAU: return M >= 1 ? fgmp_ws_calibrate(M, K) : 0;
+    }
+    return 0;
+}

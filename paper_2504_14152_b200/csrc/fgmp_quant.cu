@@ -1,0 +1,230 @@
+// Online activation quantizer (Section 4.2 of the paper), block scores, and the
+// packed -> canonical unpacker.
+//
+// Thread mapping: one thread owns one 16-element block column (kb) and walks down the rows
+// of its CTA, so the 16 per-channel Fisher weights stay in registers.  A warp covers 32
+// consecutive blocks of one row = one mask word, produced with a ballot.
+#include "fgmp_common.cuh"
+#include "fgmp_host.h"
+
+namespace {
+
+constexpr int QA_THREADS = 256;
+
+struct ActParams {
+    const uint4* X; int64_t ldx8;        // row stride in 16-byte units
+    const float* fisher;
+    int64_t M, K, KB, MW;
+    float s4, k6, s8, inv8, tau;
+    uint8_t* codes4; uint8_t* sf; uint32_t* mask; uint8_t* codes8;   // codes8: dense plane
+    float* scores;                       // optional (score-only kernel)
+    int rows_per_cta;
+};
+
+template <int MODE, bool SCORE_ONLY>
+__global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
+{
+    const int64_t kb = (int64_t)blockIdx.x * QA_THREADS + threadIdx.x;
+    const bool active = kb < p.KB;
+    const int64_t m0 = (int64_t)blockIdx.y * p.rows_per_cta;
+    const int64_t m1 = min(m0 + (int64_t)p.rows_per_cta, p.M);
+
+    float f[16];
+    if (active) {
+        const float4* fp = reinterpret_cast<const float4*>(p.fisher + kb * 16);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 t = __ldg(fp + i);
+            f[4 * i] = t.x; f[4 * i + 1] = t.y; f[4 * i + 2] = t.z; f[4 * i + 3] = t.w;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) f[i] = 0.f;
+    }
+
+    for (int64_t m = m0; m < m1; ++m) {
+        bool is8 = false;
+        if (active) {
+            const uint4* xp = p.X + m * p.ldx8 + kb * 2;
+            uint4 xa = __ldcs(xp), xb = __ldcs(xp + 1);
+            float v[16], dq4[16];
+            unpack_bf16x16(xa, xb, v);
+            uint32_t sc = block_dynamic_scale(v, p.k6);
+            uint32_t c4[2];
+            block_nvfp4(v, sc, p.s4, c4, dq4);
+            float score;
+            uint32_t c8[4];
+            if (MODE == 0) {
+                score = weighted_sq_sum(v, dq4, f);
+            } else {
+                float dq8[16];
+                block_fp8(v, p.inv8, p.s8, c8, dq8);
+                score = weighted_sq_sum(dq4, dq8, f);
+            }
+            if (SCORE_ONLY) {
+                p.scores[m * p.KB + kb] = score;
+            } else {
+                is8 = score > p.tau;
+                if (is8) {
+                    if (MODE == 0) {
+                        float dq8[16];
+                        block_fp8(v, p.inv8, p.s8, c8, dq8);
+                    }
+                    *reinterpret_cast<uint4*>(p.codes8 + m * p.K + kb * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
+                    c4[0] = 0; c4[1] = 0; sc = 0;
+                }
+                *reinterpret_cast<uint2*>(p.codes4 + (m * p.K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
+                p.sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)sc;
+            }
+        }
+        if (!SCORE_ONLY) {
+            uint32_t word = __ballot_sync(0xffffffffu, is8);
+            int64_t w = kb >> 5;
+            if ((threadIdx.x & 31) == 0 && w < p.MW) p.mask[m * p.MW + w] = word;
+        }
+    }
+}
+
+// zero the microscales of the padding rows (rows M .. 128*ceil(M/128)) so that a GEMM that
+// loads whole 128-row scale tiles reads zeros there
+__global__ void sf_pad_zero_kernel(uint8_t* sf, int64_t M, int64_t K)
+{
+    const int64_t Mpad = (M + 127) & ~(int64_t)127;
+    const int64_t KB = K / 16;
+    const int64_t n = (Mpad - M) * KB;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t r = M + i / KB, kb = i % KB;
+        sf[fgmp_sf_offset(r, kb, K)] = 0;
+    }
+}
+
+__global__ void act_header_kernel(fgmp_packed_header* h, int64_t M, int64_t K, float s4, int ratio)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        h->magic = FGMP_MAGIC; h->version = 1; h->rows = M; h->K = K; h->scale_fp4 = s4;
+        h->fp8_log2_ratio = ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+        h->error = 0;
+    }
+}
+
+// packed -> canonical arrays; one thread per block
+__global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
+                              uint8_t* codes4, uint8_t* codes8, uint8_t* scales, uint32_t* mask)
+{
+    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
+    const int kind = (int)h->kind;
+    const PackedLayout L = fgmp_layout(rows, K, kind, kind ? h->capacity : 0);
+    const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t* wordptr = reinterpret_cast<const uint32_t*>(blob + L.off_wordptr);
+    const int64_t nblk = rows * L.KB;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
+        int64_t r = b / L.KB, kb = b % L.KB;
+        uint32_t word = pmask[r * L.MW + (kb >> 5)];
+        bool is8 = (word >> (kb & 31)) & 1;
+        if (mask && (kb & 31) == 0) mask[r * L.MW + (kb >> 5)] = word;
+        if (scales) scales[b] = blob[L.off_sf + fgmp_sf_offset(r, kb, K)];
+        if (codes4) {
+            uint2 c = *reinterpret_cast<const uint2*>(blob + L.off_codes4 + (r * K) / 2 + kb * 8);
+            *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) = c;
+        }
+        if (codes8) {
+            uint4 c = make_uint4(0, 0, 0, 0);
+            if (is8) {
+                size_t src;
+                if (kind == 1) {
+                    uint32_t pos = wordptr[r * L.MW + (kb >> 5)] + __popc(word & ((1u << (kb & 31)) - 1u));
+                    src = L.off_codes8 + (size_t)pos * 16;
+                } else {
+                    src = L.off_codes8 + (size_t)(r * K + kb * 16);
+                }
+                c = *reinterpret_cast<const uint4*>(blob + src);
+            }
+            *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) = c;
+        }
+    }
+}
+
+fgmp_status check_act_args(const void* X, int64_t ldx, const float* fisher, int64_t M, int64_t K, fgmp_scales sc, int sm)
+{
+    if (!X || !fisher) return FGMP_ERR_INVALID_ARG;
+    if (sm != 0 && sm != 1) return FGMP_ERR_INVALID_ARG;
+    if (!(sc.scale_fp4 > 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
+    if (sc.fp8_log2_ratio < -8 || sc.fp8_log2_ratio > 8) return FGMP_ERR_INVALID_ARG;
+    if (M < 1 || K < 64 || (K % 64) != 0 || ldx < K || (ldx % 8) != 0) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)X & 15) || ((uintptr_t)fisher & 15)) return FGMP_ERR_SHAPE;
+    return FGMP_OK;
+}
+
+ActParams make_act_params(const void* X, int64_t ldx, const float* fisher, int64_t M, int64_t K, fgmp_scales sc, float tau)
+{
+    ActParams p{};
+    p.X = reinterpret_cast<const uint4*>(X); p.ldx8 = ldx / 8; p.fisher = fisher;
+    p.M = M; p.K = K; p.KB = K / 16; p.MW = (p.KB + 31) / 32;
+    p.s4 = sc.scale_fp4;
+    p.k6 = 1.0f / (6.0f * sc.scale_fp4);
+    p.s8 = ldexpf(sc.scale_fp4, sc.fp8_log2_ratio);
+    p.inv8 = 1.0f / p.s8;
+    p.tau = tau;
+    // enough CTAs to fill the machine when M is small, few row-loop iterations otherwise
+    p.rows_per_cta = (M >= 2048) ? 8 : (M >= 256 ? 4 : 1);
+    return p;
+}
+
+}  // namespace
+
+extern "C" fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                                                 int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm, float tau,
+                                                 void* packed_out, size_t packed_bytes,
+                                                 void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    (void)workspace; (void)ws_bytes;
+    fgmp_status st = check_act_args(X_bf16, ldx, fisher_chan, M, K, sc, (int)sm);
+    if (st != FGMP_OK) return st;
+    if (!packed_out || ((uintptr_t)packed_out & 1023)) return packed_out ? FGMP_ERR_SHAPE : FGMP_ERR_INVALID_ARG;
+    if (tau != tau) return FGMP_ERR_INVALID_ARG;
+    const PackedLayout L = fgmp_layout(M, K, 0, 0);
+    if (packed_bytes < L.total) return FGMP_ERR_WORKSPACE;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint8_t* blob = (uint8_t*)packed_out;
+
+    ActParams p = make_act_params(X_bf16, ldx, fisher_chan, M, K, sc, tau);
+    p.codes4 = blob + L.off_codes4; p.sf = blob + L.off_sf;
+    p.mask = reinterpret_cast<uint32_t*>(blob + L.off_mask); p.codes8 = blob + L.off_codes8;
+    dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((M + p.rows_per_cta - 1) / p.rows_per_cta));
+    act_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), M, K, sc.scale_fp4, sc.fp8_log2_ratio);
+    if (M % 128) sf_pad_zero_kernel<<<64, 256, 0, s>>>(p.sf, M, K);
+    if (sm == FGMP_SCORE_LP_ERROR) quant_act_kernel<0, false><<<grid, QA_THREADS, 0, s>>>(p);
+    else                           quant_act_kernel<1, false><<<grid, QA_THREADS, 0, s>>>(p);
+    return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_activation_scores(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                                              int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
+                                              float* scores, void* cuda_stream)
+{
+    fgmp_status st = check_act_args(X_bf16, ldx, fisher_chan, M, K, sc, (int)sm);
+    if (st != FGMP_OK) return st;
+    if (!scores) return FGMP_ERR_INVALID_ARG;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    ActParams p = make_act_params(X_bf16, ldx, fisher_chan, M, K, sc, 0.f);
+    p.scores = scores;
+    dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((M + p.rows_per_cta - 1) / p.rows_per_cta));
+    if (sm == FGMP_SCORE_LP_ERROR) quant_act_kernel<0, true><<<grid, QA_THREADS, 0, s>>>(p);
+    else                           quant_act_kernel<1, true><<<grid, QA_THREADS, 0, s>>>(p);
+    return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, uint8_t* codes4, uint8_t* codes8,
+                                   uint8_t* scales, uint32_t* mask, void* cuda_stream)
+{
+    if (!packed) return FGMP_ERR_INVALID_ARG;
+    if (rows < 1 || K < 64 || (K % 64) != 0 || ((uintptr_t)packed & 1023)) return FGMP_ERR_SHAPE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    int64_t nblk = rows * (K / 16);
+    int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);
+    unpack_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask);
+    return fgmp_launch_status();
+}

@@ -1,0 +1,475 @@
+// Offline weight packer: tensor scale, sensitivity-weighted clip search (Eq. 11), block
+// scores (Eq. 6 / Eq. 8), exact top-R selection (Eq. 9) and emission of the packed blob.
+// Also the activation-threshold calibration (Eq. 9 applied to a calibration batch), which
+// reuses the selection kernels.
+#include "fgmp_common.cuh"
+#include "fgmp_host.h"
+
+namespace {
+
+// Device-resident state of one packing call (lives at the start of the workspace).
+struct SelectState {
+    uint32_t hist[256];
+    uint32_t amax_bits;      // max |w| as fp32 bits
+    float s4;                // NVFP4 tensor scale in use
+    uint32_t prefix;         // radix-select prefix (high bits of the k-th largest score)
+    uint32_t pad0;
+    unsigned long long krem; // how many blocks are still to be taken inside the prefix group
+    float tau;               // threshold: FP8 iff score > tau, or == tau within the first need_eq
+    uint32_t use_eq;
+    unsigned long long need_eq;
+    unsigned long long n_fp8;
+    float next_below;        // calibration: largest score strictly below tau
+    uint32_t pad1;
+};
+
+constexpr size_t STATE_BYTES = 2048;
+
+__global__ void state_init_kernel(SelectState* st, float s4_given, unsigned long long k)
+{
+    int t = threadIdx.x;
+    if (t < 256) st->hist[t] = 0;
+    if (t == 0) {
+        st->amax_bits = 0; st->s4 = s4_given; st->prefix = 0; st->krem = k; st->tau = 0.f;
+        st->use_eq = 0; st->need_eq = 0; st->n_fp8 = 0; st->next_below = 0.f;
+    }
+}
+
+__global__ void w_amax_kernel(const uint4* W, int64_t ldw8, int64_t N, int64_t K8, SelectState* st)
+{
+    uint32_t m = 0;
+    const int64_t total = N * K8;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t n = i / K8, c = i % K8;
+        uint4 x = __ldg(W + n * ldw8 + c);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            m = max(m, (w[j] << 16) & 0x7fffffffu);
+            m = max(m, w[j] & 0x7fff0000u);
+        }
+    }
+    for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(&st->amax_bits, m);
+}
+
+__global__ void w_scale_kernel(SelectState* st)
+{
+    if (threadIdx.x == 0) st->s4 = __fdiv_rn(__uint_as_float(st->amax_bits), 2688.0f);
+}
+
+__device__ __forceinline__ void load_block(const uint4* W, int64_t ldw8, const float* F, int64_t ldf,
+                                           int64_t n, int64_t kb, float (&v)[16], float (&f)[16])
+{
+    const uint4* wp = W + n * ldw8 + kb * 2;
+    unpack_bf16x16(__ldg(wp), __ldg(wp + 1), v);
+    if (F) {
+        const float4* fp = reinterpret_cast<const float4*>(F + n * ldf + kb * 16);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 t = __ldg(fp + i);
+            f[4 * i] = t.x; f[4 * i + 1] = t.y; f[4 * i + 2] = t.z; f[4 * i + 3] = t.w;
+        }
+    }
+}
+
+// per block: microscale (dynamic max or Eq. 11 brute force) and the score under it
+template <int MODE, bool CLIP>
+__global__ void __launch_bounds__(256) w_score_kernel(const uint4* W, int64_t ldw8, const float* F, int64_t ldf,
+                                                      int64_t N, int64_t KB, int ratio, const SelectState* st,
+                                                      uint8_t* sc_out, float* scores)
+{
+    __shared__ float s_d[128], s_inv[128];
+    const float s4 = st->s4;
+    if (CLIP) {
+        if (threadIdx.x < 127) {
+            float d = __fmul_rn(e4m3_to_f32(threadIdx.x), s4);
+            s_d[threadIdx.x] = d;
+            s_inv[threadIdx.x] = (d == 0.f) ? 0.f : __fdiv_rn(1.0f, d);
+        }
+        __syncthreads();
+    }
+    const float k6 = __fdiv_rn(1.0f, __fmul_rn(6.0f, s4));
+    const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
+    const float inv8 = __fdiv_rn(1.0f, s8);
+    const int64_t B = N * KB;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
+        float v[16], f[16];
+        load_block(W, ldw8, F, ldf, b / KB, b % KB, v, f);
+        uint32_t sc = block_dynamic_scale(v, k6);
+        if (CLIP) {
+            // incumbent = dynamic max; ascending scan, strict improvement only
+            float best;
+            {
+                float d = s_d[sc], inv = s_inv[sc];
+                best = 0.f;
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float2 q = e2m1x2_to_f32x2(f32x2_to_e2m1x2(__fmul_rn(v[i], inv), __fmul_rn(v[i + 1], inv)));
+                    float e0 = __fsub_rn(__fmul_rn(q.x, d), v[i]);
+                    best = __fadd_rn(best, __fmul_rn(__fmul_rn(f[i], e0), e0));
+                    float e1 = __fsub_rn(__fmul_rn(q.y, d), v[i + 1]);
+                    best = __fadd_rn(best, __fmul_rn(__fmul_rn(f[i + 1], e1), e1));
+                }
+            }
+            for (uint32_t c = 1; c <= 0x7e; ++c) {
+                float d = s_d[c], inv = s_inv[c];
+                float j = 0.f;
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float2 q = e2m1x2_to_f32x2(f32x2_to_e2m1x2(__fmul_rn(v[i], inv), __fmul_rn(v[i + 1], inv)));
+                    float e0 = __fsub_rn(__fmul_rn(q.x, d), v[i]);
+                    j = __fadd_rn(j, __fmul_rn(__fmul_rn(f[i], e0), e0));
+                    float e1 = __fsub_rn(__fmul_rn(q.y, d), v[i + 1]);
+                    j = __fadd_rn(j, __fmul_rn(__fmul_rn(f[i + 1], e1), e1));
+                }
+                if (j < best) { best = j; sc = c; }
+            }
+        }
+        uint32_t c4[2];
+        float dq4[16];
+        block_nvfp4(v, sc, s4, c4, dq4);
+        float score;
+        if (MODE == 0) {
+            score = weighted_sq_sum(v, dq4, f);
+        } else {
+            uint32_t c8[4];
+            float dq8[16];
+            block_fp8(v, inv8, s8, c8, dq8);
+            score = weighted_sq_sum(dq4, dq8, f);
+        }
+        sc_out[b] = (uint8_t)sc;
+        scores[b] = score;
+    }
+}
+
+// ------------------------------------------------------------ radix select (k-th largest)
+// Scores are >= 0, so their fp32 bit patterns order like unsigned integers.
+__global__ void select_hist_kernel(const float* scores, int64_t B, int pass, SelectState* st)
+{
+    __shared__ uint32_t h[256];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const int shift = 24 - 8 * pass;
+    const uint32_t prefix = st->prefix;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
+        uint32_t u = __float_as_uint(scores[b]);
+        if (pass == 0 || (u >> (shift + 8)) == prefix) atomicAdd(&h[(u >> shift) & 255], 1u);
+    }
+    __syncthreads();
+    if (h[threadIdx.x]) atomicAdd(&st->hist[threadIdx.x], h[threadIdx.x]);
+}
+
+__global__ void select_pick_kernel(SelectState* st, int pass)
+{
+    if (threadIdx.x == 0) {
+        unsigned long long krem = st->krem, cum = 0;
+        int bin = 255;
+        for (; bin > 0; --bin) {
+            if (cum + st->hist[bin] >= krem) break;
+            cum += st->hist[bin];
+        }
+        st->prefix = (st->prefix << 8) | (uint32_t)bin;
+        st->krem = krem - cum;
+        if (pass == 3) {
+            st->tau = __uint_as_float(st->prefix);
+            st->need_eq = st->krem;          // of the blocks equal to tau, take this many
+            st->use_eq = 1;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < 256) st->hist[threadIdx.x] = 0;
+}
+
+// largest score strictly below tau (calibration: the (k+1)-th largest when there are no ties)
+__global__ void next_below_kernel(const float* scores, int64_t B, SelectState* st)
+{
+    const float tau = st->tau;
+    uint32_t m = 0;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
+        float s = scores[b];
+        if (s < tau) m = max(m, __float_as_uint(s));
+    }
+    for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<uint32_t*>(&st->next_below), m);
+}
+
+__global__ void calib_finish_kernel(const SelectState* st, float* tau_out, int all_or_none)
+{
+    if (threadIdx.x == 0) {
+        if (all_or_none == 1) *tau_out = __int_as_float(0x7f800000);   // k = 0: nothing exceeds +inf
+        else if (all_or_none == 2) *tau_out = -1.0f;                   // k = all
+        else {
+            // midway between the k-th largest score and the next one below it; if fp32 cannot
+            // separate them, the lower neighbour itself (score > tau still selects the top k)
+            float t = __fmul_rn(0.5f, __fadd_rn(st->tau, st->next_below));
+            *tau_out = (t < st->tau && t >= st->next_below) ? t : st->next_below;
+        }
+    }
+}
+
+// ------------------------------------------------------------ mask, prefix sums, emission
+// per mask word: how many of its blocks have score == tau
+__global__ void w_eqcount_kernel(const float* scores, int64_t N, int64_t KB, int64_t MW, const SelectState* st, uint32_t* cnt)
+{
+    const float tau = st->tau;
+    const int lane = threadIdx.x & 31;
+    const int64_t nw = N * MW;
+    for (int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < nw; w += ((int64_t)gridDim.x * blockDim.x) >> 5) {
+        int64_t n = w / MW, kb = (w % MW) * 32 + lane;
+        bool eq = kb < KB && scores[n * KB + kb] == tau;
+        uint32_t bal = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) cnt[w] = __popc(bal);
+    }
+}
+
+__global__ void w_mask_kernel(const float* scores, int64_t N, int64_t KB, int64_t MW, const SelectState* st,
+                              const uint32_t* eqprefix, uint32_t* mask, uint32_t* wcnt)
+{
+    const float tau = st->tau;
+    const bool use_eq = st->use_eq != 0;
+    const unsigned long long need_eq = st->need_eq;
+    const int lane = threadIdx.x & 31;
+    const int64_t nw = N * MW;
+    for (int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < nw; w += ((int64_t)gridDim.x * blockDim.x) >> 5) {
+        int64_t n = w / MW, kb = (w % MW) * 32 + lane;
+        float s = kb < KB ? scores[n * KB + kb] : -1.f;
+        bool gt = kb < KB && s > tau;
+        bool eq = use_eq && kb < KB && s == tau;
+        uint32_t eqbal = __ballot_sync(0xffffffffu, eq);
+        bool take = gt;
+        if (eq) {
+            unsigned long long rank = (unsigned long long)eqprefix[w] + __popc(eqbal & ((1u << lane) - 1u));
+            take = rank < need_eq;
+        }
+        uint32_t word = __ballot_sync(0xffffffffu, take);
+        if (lane == 0) { mask[w] = word; wcnt[w] = __popc(word); }
+    }
+}
+
+// exclusive prefix sum of n uint32 by one CTA of 1024 threads; total -> *total_out (may be NULL)
+__global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t* out, int64_t n, unsigned long long* total_out)
+{
+    __shared__ uint32_t warp_sums[32];
+    __shared__ unsigned long long carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int64_t base = 0; base < n; base += 1024) {
+        int64_t i = base + threadIdx.x;
+        uint32_t x = i < n ? in[i] : 0;
+        uint32_t incl = x;
+        for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+        if (lane == 31) warp_sums[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            uint32_t s = warp_sums[lane], si = s;
+            for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xffffffffu, si, o); if (lane >= o) si += y; }
+            warp_sums[lane] = si - s;       // exclusive warp offsets
+        }
+        __syncthreads();
+        unsigned long long carry = carry_s;
+        if (i < n) out[i] = (uint32_t)(carry + warp_sums[wid] + incl - x);
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = carry + warp_sums[31] + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && total_out) *total_out = carry_s;
+}
+
+__global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw8, int64_t N, int64_t K, int ratio,
+                                                     const SelectState* st, const uint8_t* sc_in,
+                                                     uint8_t* blob, PackedLayout L, int64_t capacity)
+{
+    const float s4 = st->s4;
+    const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
+    const float inv8 = __fdiv_rn(1.0f, s8);
+    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t* wordptr = reinterpret_cast<const uint32_t*>(blob + L.off_wordptr);
+    const int64_t B = N * L.KB;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
+        int64_t n = b / L.KB, kb = b % L.KB;
+        float v[16], f[16];
+        load_block(W, ldw8, nullptr, 0, n, kb, v, f);
+        uint32_t word = mask[n * L.MW + (kb >> 5)];
+        bool is8 = (word >> (kb & 31)) & 1;
+        uint32_t c4[2] = {0, 0};
+        uint32_t sc = 0;
+        if (is8) {
+            uint32_t c8[4];
+            float dq8[16];
+            block_fp8(v, inv8, s8, c8, dq8);
+            int64_t pos = (int64_t)wordptr[n * L.MW + (kb >> 5)] + __popc(word & ((1u << (kb & 31)) - 1u));
+            if (pos < capacity)
+                *reinterpret_cast<uint4*>(blob + L.off_codes8 + (size_t)pos * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
+        } else {
+            float dq4[16];
+            sc = sc_in[b];
+            block_nvfp4(v, sc, s4, c4, dq4);
+        }
+        *reinterpret_cast<uint2*>(blob + L.off_codes4 + (n * K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
+        blob[L.off_sf + fgmp_sf_offset(n, kb, K)] = (uint8_t)sc;
+    }
+    // microscales of the padding rows
+    const int64_t Npad = (N + 127) & ~(int64_t)127;
+    const int64_t npad = (Npad - N) * L.KB;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < npad; i += (int64_t)gridDim.x * blockDim.x)
+        blob[L.off_sf + fgmp_sf_offset(N + i / L.KB, i % L.KB, K)] = 0;
+}
+
+__global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, int64_t N, int64_t K, int ratio,
+                                int64_t capacity, int fraction_mode, float tau_given, float* tau_eff_out)
+{
+    if (threadIdx.x == 0) {
+        h->magic = FGMP_MAGIC; h->version = 1; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
+        h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = capacity;
+        float teff = fraction_mode ? st->tau : tau_given;
+        h->tau_eff = teff;
+        h->error = ((int64_t)st->n_fp8 > capacity) ? (int32_t)FGMP_ERR_CAPACITY : 0;
+        if (tau_eff_out) *tau_eff_out = teff;
+    }
+}
+
+__global__ void set_tau_kernel(SelectState* st, float tau)
+{
+    if (threadIdx.x == 0) { st->tau = tau; st->use_eq = 0; st->need_eq = 0; }
+}
+
+int grid_for(int64_t work_items, int threads, int max_ctas_per_sm)
+{
+    int64_t g = (work_items + threads - 1) / threads;
+    int64_t cap = (int64_t)fgmp_sm_count() * max_ctas_per_sm;
+    if (g > cap) g = cap;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+// runs the 4-pass radix select for the k-th largest of scores[0..B)
+void run_select(const float* scores, int64_t B, SelectState* st, cudaStream_t s)
+{
+    int g = grid_for(B, 256, 8);
+    for (int pass = 0; pass < 4; ++pass) {
+        select_hist_kernel<<<g, 256, 0, s>>>(scores, B, pass, st);
+        select_pick_kernel<<<1, 256, 0, s>>>(st, pass);
+    }
+}
+
+size_t ws_weights_bytes(int64_t N, int64_t K)
+{
+    int64_t KB = K / 16, MW = (KB + 31) / 32, B = N * KB, NW = N * MW;
+    return STATE_BYTES + fgmp_align1k((size_t)B * 4) + fgmp_align1k((size_t)B) + 2 * fgmp_align1k((size_t)NW * 4);
+}
+
+}  // namespace
+
+size_t fgmp_ws_quantize_weights(int64_t N, int64_t K) { return ws_weights_bytes(N, K); }
+size_t fgmp_ws_calibrate(int64_t M, int64_t K) { return STATE_BYTES + fgmp_align1k((size_t)M * (K / 16) * 4); }
+
+extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, const float* fisher_elem, int64_t ldf,
+                                             int64_t N, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
+                                             fgmp_clip_mode cm, double fp8_fraction, float tau,
+                                             void* packed_out, size_t packed_bytes, float* tau_eff_out,
+                                             void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!W_bf16 || !fisher_elem || !packed_out || !workspace) return FGMP_ERR_INVALID_ARG;
+    if ((int)sm < 0 || (int)sm > 1 || (int)cm < 0 || (int)cm > 1) return FGMP_ERR_INVALID_ARG;
+    if (!(sc.scale_fp4 >= 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
+    if (sc.fp8_log2_ratio < -8 || sc.fp8_log2_ratio > 8) return FGMP_ERR_INVALID_ARG;
+    if (fp8_fraction != fp8_fraction || fp8_fraction > 1.0) return FGMP_ERR_INVALID_ARG;
+    if (fp8_fraction < 0 && tau != tau) return FGMP_ERR_INVALID_ARG;
+    if (N < 1 || K < 64 || (K % 64) != 0 || ldw < K || (ldw % 8) != 0 || ldf < K || (ldf % 4) != 0) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)W_bf16 & 15) || ((uintptr_t)fisher_elem & 15) || ((uintptr_t)packed_out & 1023) ||
+        ((uintptr_t)workspace & 255)) return FGMP_ERR_SHAPE;
+    const int64_t KB = K / 16, MW = (KB + 31) / 32, B = N * KB, NW = N * MW;
+    if (B >= ((int64_t)1 << 32)) return FGMP_ERR_SHAPE;
+    const bool fraction_mode = fp8_fraction >= 0.0;
+    int64_t k = 0;
+    if (fraction_mode) {
+        k = (int64_t)floor(fp8_fraction * (double)B + 0.5);
+        if (k > B) k = B;
+    }
+    // capacity: what the blob can hold
+    const PackedLayout L0 = fgmp_layout(N, K, 1, 0);
+    if (packed_bytes < L0.total) return FGMP_ERR_WORKSPACE;
+    int64_t capacity = (int64_t)((packed_bytes - L0.off_codes8) / 16);
+    if (capacity > B) capacity = B;
+    if (fraction_mode && capacity < k) return FGMP_ERR_WORKSPACE;
+    const PackedLayout L = fgmp_layout(N, K, 1, capacity);
+    if (ws_bytes < ws_weights_bytes(N, K)) return FGMP_ERR_WORKSPACE;
+    fgmp_status stt;
+    if ((stt = fgmp_require_sm100()) != FGMP_OK) return stt;
+
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    SelectState* st = reinterpret_cast<SelectState*>(ws);
+    float* scores = reinterpret_cast<float*>(ws + STATE_BYTES);
+    uint8_t* sc_tmp = ws + STATE_BYTES + fgmp_align1k((size_t)B * 4);
+    uint32_t* tmp_a = reinterpret_cast<uint32_t*>(sc_tmp + fgmp_align1k((size_t)B));
+    uint32_t* tmp_b = reinterpret_cast<uint32_t*>((uint8_t*)tmp_a + fgmp_align1k((size_t)NW * 4));
+    uint8_t* blob = (uint8_t*)packed_out;
+    const uint4* W = reinterpret_cast<const uint4*>(W_bf16);
+    const int ratio = sc.fp8_log2_ratio;
+
+    state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k);
+    if (sc.scale_fp4 == 0.f) {
+        w_amax_kernel<<<grid_for(N * (K / 8), 256, 8), 256, 0, s>>>(W, ldw / 8, N, K / 8, st);
+        w_scale_kernel<<<1, 32, 0, s>>>(st);
+    }
+    {
+        int g = grid_for(B, 256, 4);
+        if (sm == FGMP_SCORE_LP_ERROR) {
+            if (cm == FGMP_CLIP_SW_BRUTE) w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
+            else                          w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
+        } else {
+            if (cm == FGMP_CLIP_SW_BRUTE) w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
+            else                          w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
+        }
+    }
+    uint32_t* mask = reinterpret_cast<uint32_t*>(blob + L.off_mask);
+    uint32_t* wordptr = reinterpret_cast<uint32_t*>(blob + L.off_wordptr);
+    const int gw = grid_for(NW * 32, 256, 8);
+    if (fraction_mode && k > 0) {
+        run_select(scores, B, st, s);
+        w_eqcount_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_a);
+        scan_kernel<<<1, 1024, 0, s>>>(tmp_a, tmp_b, NW, nullptr);
+    } else {
+        // k == 0: nothing is FP8 (tau_eff = +inf); threshold mode: the given tau
+        set_tau_kernel<<<1, 32, 0, s>>>(st, fraction_mode ? INFINITY : tau);
+    }
+    w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a);
+    scan_kernel<<<1, 1024, 0, s>>>(tmp_a, wordptr, NW, &st->n_fp8);
+    w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, ratio, st, sc_tmp, blob, L, capacity);
+    w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, N, K, ratio, capacity,
+                                     fraction_mode ? 1 : 0, tau, tau_eff_out);
+    return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_calibrate_tau(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                                          int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
+                                          double fp8_fraction, float* tau_out,
+                                          void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!tau_out || !workspace) return FGMP_ERR_INVALID_ARG;
+    if (!(fp8_fraction >= 0.0) || fp8_fraction > 1.0) return FGMP_ERR_INVALID_ARG;
+    if (M < 1 || K < 64 || (K % 64) != 0) return FGMP_ERR_SHAPE;
+    if ((uintptr_t)workspace & 255) return FGMP_ERR_SHAPE;
+    const int64_t B = M * (K / 16);
+    if (ws_bytes < fgmp_ws_calibrate(M, K)) return FGMP_ERR_WORKSPACE;
+    uint8_t* ws = (uint8_t*)workspace;
+    SelectState* st = reinterpret_cast<SelectState*>(ws);
+    float* scores = reinterpret_cast<float*>(ws + STATE_BYTES);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    fgmp_status stt = fgmp_activation_scores(X_bf16, ldx, fisher_chan, M, K, sc, sm, scores, cuda_stream);
+    if (stt != FGMP_OK) return stt;
+    int64_t k = (int64_t)floor(fp8_fraction * (double)B + 0.5);
+    if (k > B) k = B;
+    state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k);
+    if (k == 0 || k == B) {
+        calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, k == 0 ? 1 : 2);
+    } else {
+        run_select(scores, B, st, s);
+        next_below_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(scores, B, st);
+        calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, 0);
+    }
+    return fgmp_launch_status();
+}

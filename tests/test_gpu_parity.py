@@ -1,0 +1,264 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Bars: codes, microscales and masks bit-exact (a block whose fp32 score lies within
+1e-6*tau of tau is excused); GEMM outputs within 2e-3 * sum|a||w| of the oracle's fp64 result.
+"""
+import numpy as np
+import pytest
+import torch
+
+import fgmp_inputs as gi
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+GEMM_TOL = 2e-3
+
+
+@pytest.fixture(scope="module")
+def fg():
+    import paper_2504_14152_b200 as fg_
+    assert torch.cuda.is_available()
+    assert torch.cuda.get_device_capability()[0] == 10, "these kernels are sm_100a only"
+    return fg_
+
+
+def tau_for_fraction(scores: np.ndarray, frac: float) -> float:
+    k = int(np.floor(frac * scores.size + 0.5))
+    if k == 0:
+        return float("inf")
+    if k == scores.size:
+        return -1.0
+    s = np.sort(scores.ravel())[::-1]
+    return float(np.float32(0.5) * (s[k - 1] + s[k]))
+
+
+def compare_packed(fg, packed, q: oracle.Quantized, tau=None, what=""):
+    c4, c8, sc, mk = [t.cpu().numpy() for t in fg.unpack(packed)]
+    mk = mk.view(np.uint32)
+    KB = q.K // 16
+    excused = np.zeros((q.rows, KB), bool)
+    if tau is not None and np.isfinite(tau) and tau > 0:
+        excused = np.abs(q.scores.reshape(q.rows, KB) - np.float32(tau)) <= 1e-6 * tau
+    g = oracle.Quantized(q.rows, q.K, c4, c8, sc, mk, q.scores, q.scale_fp4, q.ratio)
+    ok_mask = (g.mask_bits() == q.mask_bits()) | excused
+    assert ok_mask.all(), f"{what}: {np.count_nonzero(~ok_mask)} mask bits differ"
+    keep = ~excused
+    assert np.array_equal(sc.reshape(q.rows, KB)[keep], q.scales.reshape(q.rows, KB)[keep]), f"{what}: microscales differ"
+    d4 = (c4.reshape(q.rows, KB, 8) != q.codes4.reshape(q.rows, KB, 8)).any(-1) & keep
+    assert not d4.any(), f"{what}: {d4.sum()} NVFP4 blocks differ, first at {np.argwhere(d4)[:3].tolist()}"
+    d8 = (c8.reshape(q.rows, KB, 16) != q.codes8.reshape(q.rows, KB, 16)).any(-1) & keep
+    assert not d8.any(), f"{what}: {d8.sum()} FP8 blocks differ, first at {np.argwhere(d8)[:3].tolist()}"
+    return int(excused.sum())
+
+
+def gpu_quant_acts(fg, x, fx, s4, tau, mode=0, ratio=3):
+    return fg.quantize_activations(x.cuda(), fx.cuda(), scale_fp4=s4, ratio=ratio, score_mode=mode, tau=tau)
+
+
+# ------------------------------------------------------------------ conversions
+
+@pytest.mark.parametrize("order", ["sorted", "shuffled"])
+def test_every_bf16_value_converts_like_the_oracle(fg, order):
+    """All 65 536 bf16 bit patterns (non-finite ones replaced by zero) through the quantizer,
+    as NVFP4 (codes + microscales) and as FP8, for several tensor scales."""
+    bits = np.arange(65536, dtype=np.uint32)
+    f = (bits << 16).view(np.float32)
+    bits = np.where(np.isfinite(f), bits, 0).astype(np.uint16)
+    if order == "shuffled":
+        bits = np.random.default_rng(3).permutation(bits)
+    xb = bits.reshape(64, 1024)
+    x = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16)
+    fx = torch.ones(1024)
+    for s4 in (1.0, 2.0 ** -7 * 1.37, 3.1e-5, 41.0):
+        for tau in (float("inf"), -1.0):
+            for mode in (0, 1):
+                q = oracle.quantize_activations(xb, fx.numpy(), s4, tau=tau, mode=mode)
+                p = gpu_quant_acts(fg, x, fx, s4, tau, mode)
+                compare_packed(fg, p, q, what=f"s4={s4} tau={tau} mode={mode}")
+                if tau == float("inf"):
+                    sg = fg.activation_scores(x.cuda(), fx.cuda(), scale_fp4=s4, score_mode=mode).cpu().numpy()
+                    assert np.array_equal(sg.ravel().view(np.uint32), q.scores.view(np.uint32))
+
+
+# ------------------------------------------------------------------ activations
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_activations_tiny_config(fg, mode):
+    wl = gi.tiny(0)
+    x, fx = wl.x(), wl.fx()
+    s4 = gi.tensor_scale(x)
+    xb = gi.bf16_bits(x)
+    scores = oracle.quantize_activations(xb, fx.numpy(), s4, tau=np.inf, mode=mode).scores
+    sg = fg.activation_scores(x.cuda(), fx.cuda(), scale_fp4=s4, score_mode=mode).cpu().numpy()
+    assert np.array_equal(sg.ravel().view(np.uint32), scores.view(np.uint32))
+    tau = tau_for_fraction(scores, wl.fp8_fraction)
+    q = oracle.quantize_activations(xb, fx.numpy(), s4, tau=tau, mode=mode)
+    p = gpu_quant_acts(fg, x, fx, s4, tau, mode)
+    compare_packed(fg, p, q, tau, "tiny")
+    assert q.mask_bits().sum() == int(np.floor(0.1 * scores.size + 0.5))
+    # calibration entry point reproduces the threshold (Eq. 9)
+    tg = fg.calibrate_tau(x.cuda(), fx.cuda(), scale_fp4=s4, score_mode=mode, fp8_fraction=wl.fp8_fraction)
+    assert np.float32(tg.item()) == np.float32(tau)
+    h = p.header()
+    assert h["magic"] == 0x504D4746 and h["rows"] == wl.M and h["K"] == wl.K and h["kind"] == 0
+
+
+@pytest.mark.parametrize("M,K", [(1, 4096), (16, 4096), (77, 11008), (300, 5120), (129, 64), (2048, 1024)])
+def test_activations_ragged_shapes(fg, M, K):
+    wl = gi.llama("a", M, 1, K, seed=M + K)
+    x, fx = wl.x(), wl.fx()
+    s4 = gi.tensor_scale(x)
+    xb = gi.bf16_bits(x)
+    scores = oracle.quantize_activations(xb, fx.numpy(), s4, tau=np.inf).scores
+    for frac in (0.1, 0.0, 1.0):
+        tau = tau_for_fraction(scores, frac)
+        q = oracle.quantize_activations(xb, fx.numpy(), s4, tau=tau)
+        p = gpu_quant_acts(fg, x, fx, s4, tau)
+        compare_packed(fg, p, q, tau, f"M={M} K={K} frac={frac}")
+
+
+def test_activations_strided_input_and_zero_blocks(fg):
+    wl = gi.llama("a", 40, 1, 1024, seed=9)
+    big = torch.zeros(40, 2048, dtype=torch.bfloat16)
+    x = wl.x()
+    x[:, 64:96] = 0                      # all-zero blocks
+    x[3, 70] = -0.0
+    big[:, :1024] = x
+    fx = wl.fx()
+    s4 = gi.tensor_scale(x)
+    q = oracle.quantize_activations(gi.bf16_bits(x), fx.numpy(), s4, tau=1e-3)
+    xg = big.cuda()[:, :1024]            # row stride 2048
+    assert xg.stride(0) == 2048
+    p = fg.quantize_activations(xg, fx.cuda(), scale_fp4=s4, tau=1e-3)
+    compare_packed(fg, p, q, 1e-3, "strided")
+
+
+def test_argument_validation(fg):
+    x = torch.zeros(4, 100, dtype=torch.bfloat16, device="cuda")       # K % 64 != 0
+    with pytest.raises(fg.FgmpError) as e:
+        fg.quantize_activations(x, torch.ones(100, device="cuda"), scale_fp4=1.0, tau=0.0)
+    assert e.value.code == -2
+    x = torch.zeros(4, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(fg.FgmpError) as e:
+        fg.quantize_activations(x, torch.ones(128, device="cuda"), scale_fp4=0.0, tau=0.0)
+    assert e.value.code == -1
+    with pytest.raises(fg.FgmpError) as e:
+        fg.quantize_activations(x, torch.ones(128, device="cuda"), scale_fp4=1.0, tau=0.0,
+                                out=torch.empty(2048, dtype=torch.uint8, device="cuda"))
+    assert e.value.code in (-2, -3)
+
+
+# ---------------------------------------------------------------------- weights
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("clip", [False, True])
+def test_weights_tiny_config(fg, mode, clip):
+    wl = gi.tiny(0)
+    w, fw = wl.w(), wl.fw()
+    wb = gi.bf16_bits(w)
+    for frac in (0.1, 0.0, 0.3, 1.0):
+        q = oracle.quantize_weights(wb, fw.numpy(), clip=clip, mode=mode, fp8_fraction=frac)
+        p = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=int(clip), score_mode=mode, fp8_fraction=frac)
+        compare_packed(fg, p, q, None, f"tiny clip={clip} mode={mode} frac={frac}")
+        h = p.header()
+        assert h["n_fp8"] == q.mask_bits().sum() == int(np.floor(frac * 4096 + 0.5))
+        assert np.float32(h["scale_fp4"]) == np.float32(q.scale_fp4) and h["error"] == 0
+        if 0 < frac:
+            assert np.float32(h["tau_eff"]) == np.float32(q.tau_eff)
+    # threshold mode with the oracle's effective threshold selects the strictly larger ones
+    q = oracle.quantize_weights(wb, fw.numpy(), clip=clip, mode=mode, fp8_fraction=0.1)
+    qt = oracle.quantize_weights(wb, fw.numpy(), clip=clip, mode=mode, fp8_fraction=-1.0, tau=q.tau_eff)
+    pt = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=int(clip), score_mode=mode, fp8_fraction=-1.0,
+                             tau=q.tau_eff)
+    compare_packed(fg, pt, qt, None, "threshold mode")
+    # given tensor scale
+    q = oracle.quantize_weights(wb, fw.numpy(), scale_fp4=3e-5, clip=clip, mode=mode, fp8_fraction=0.2)
+    p = fg.quantize_weights(w.cuda(), fw.cuda(), scale_fp4=3e-5, clip_mode=int(clip), score_mode=mode, fp8_fraction=0.2)
+    compare_packed(fg, p, q, None, "given scale")
+
+
+def test_weights_ties_take_the_lower_block_index(fg):
+    row = gi.weights(1, 64, 5)
+    w = row.repeat(96, 1)                                   # every row identical -> massive ties
+    w = torch.cat([w[:, :16]] * 4, dim=1).contiguous()      # and every block identical
+    fw = torch.ones(96, 64)
+    for frac in (0.37, 0.5, 0.011):
+        q = oracle.quantize_weights(gi.bf16_bits(w), fw.numpy(), clip=False, fp8_fraction=frac)
+        p = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=0, fp8_fraction=frac)
+        compare_packed(fg, p, q, None, f"ties frac={frac}")
+        k = int(np.floor(frac * 96 * 4 + 0.5))
+        assert q.mask_bits().ravel()[:k].all() and not q.mask_bits().ravel()[k:].any()
+
+
+@pytest.mark.parametrize("N,K,clip", [(11008, 4096, False), (384, 4096, True), (200, 11008, True), (5120, 1024, False)])
+def test_weights_llama_shapes(fg, N, K, clip):
+    wl = gi.llama("w", 1, N, K, seed=1)
+    w, fw = wl.w(), wl.fw()
+    q = oracle.quantize_weights(gi.bf16_bits(w), fw.numpy(), clip=clip, fp8_fraction=0.1)
+    p = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=int(clip), fp8_fraction=0.1)
+    compare_packed(fg, p, q, None, f"N={N} K={K}")
+    assert p.header()["n_fp8"] == int(np.floor(0.1 * N * K / 16 + 0.5))
+
+
+# ------------------------------------------------------------------------- GEMM
+
+def quantize_both(fg, wl, frac_a, frac_w, mode=0, clip=True):
+    x, w, fx, fw = wl.x(), wl.w(), wl.fx(), wl.fw()
+    s4 = gi.tensor_scale(x)
+    xb, wb = gi.bf16_bits(x), gi.bf16_bits(w)
+    scores = oracle.quantize_activations(xb, fx.numpy(), s4, tau=np.inf, mode=mode).scores
+    tau = tau_for_fraction(scores, frac_a)
+    qa = oracle.quantize_activations(xb, fx.numpy(), s4, tau=tau, mode=mode)
+    qw = oracle.quantize_weights(wb, fw.numpy(), clip=clip, mode=mode, fp8_fraction=frac_w)
+    pa = fg.quantize_activations(x.cuda(), fx.cuda(), scale_fp4=s4, score_mode=mode, tau=tau)
+    pw = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=int(clip), score_mode=mode, fp8_fraction=frac_w)
+    return qa, qw, pa, pw
+
+
+@pytest.mark.parametrize("frac_a,frac_w", [(0.1, 0.1), (0.0, 0.0), (1.0, 1.0), (0.0, 1.0), (1.0, 0.0), (0.3, 0.2)])
+def test_linear_tiny_config(fg, frac_a, frac_w):
+    wl = gi.tiny(0)
+    qa, qw, pa, pw = quantize_both(fg, wl, frac_a, frac_w)
+    Y, S = oracle.linear(qa, qw)
+    y = fg.linear(pa, pw)
+    fg.check(fg.linear.last_workspace)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - Y)
+    assert (err <= GEMM_TOL * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    # the common-container path is exact up to fp32 accumulation: far inside the bar
+    assert (err <= 1e-5 * S + 1e-30).all()
+    # bf16 output: the oracle's value rounded to bf16, within one bf16 step plus the bar
+    yb = fg.linear(pa, pw, out_dtype=torch.bfloat16).float().cpu().numpy().astype(np.float64)
+    assert (np.abs(yb - Y) <= GEMM_TOL * S + np.abs(Y) * 2.0 ** -8 + 1e-30).all()
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 256, 256), (16, 11008, 4096), (77, 300, 1024), (129, 136, 64), (384, 1000, 2048)])
+def test_linear_ragged_shapes(fg, M, N, K):
+    wl = gi.llama("l", M, N, K, seed=2)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    y = fg.linear(pa, pw).cpu().numpy().astype(np.float64)
+    fg.check(fg.linear.last_workspace)
+    rng = np.random.default_rng(0)
+    ns = 4000
+    ms = np.r_[rng.integers(0, M, ns), [0, M - 1, 0, M - 1]]
+    nn = np.r_[rng.integers(0, N, ns), [0, N - 1, N - 1, 0]]
+    Y, S = oracle.linear_sampled(qa, qw, ms, nn)
+    err = np.abs(y[ms, nn] - Y)
+    assert (err <= GEMM_TOL * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    assert np.isfinite(y).all()
+
+
+def test_linear_prefill_shape_sampled(fg):
+    """Llama-2-7B o_proj at M=4096 (one of the prefill benchmark shapes), sampled outputs."""
+    wl = gi.llama("o_proj", 4096, 4096, 4096, seed=0)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    y = fg.linear(pa, pw).cpu().numpy().astype(np.float64)
+    fg.check(fg.linear.last_workspace)
+    rng = np.random.default_rng(1)
+    ms, nn = rng.integers(0, 4096, 3000), rng.integers(0, 4096, 3000)
+    Y, S = oracle.linear_sampled(qa, qw, ms, nn)
+    err = np.abs(y[ms, nn] - Y)
+    assert (err <= GEMM_TOL * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    # two runs give the same bits
+    y2 = fg.linear(pa, pw).cpu().numpy().astype(np.float64)
+    assert np.array_equal(y, y2)
