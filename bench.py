@@ -1,0 +1,392 @@
+#!/usr/bin/env python
+"""Benchmark of the FGMP linear layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Default workload: Llama-2-7B FC1 at decode (M=16 tokens, K=4096, N=11008, 10% FP8 blocks in
+weights and activations); metric = packed-weight GB/s.  One step = the online path: quantize
+the step's activations (bf16 -> mixed NVFP4/FP8) and run the mixed-precision GEMM against
+offline-packed weights.  Weight packing is offline in the method and is timed separately
+(reported under "offline").  The step rotates over several weight copies so that the working
+set exceeds L2.  Prints ONE JSON line (rank 0).
+
+With N > 1 (torchrun) every rank runs an independent replica of the same workload on its own
+GPU ("weak" scaling, no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import fgmp_inputs as gi  # noqa: E402
+
+L2_BYTES = 126e6
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def algorithmic_weight_bytes(N, K, p):
+    B = N * K // 16
+    n8 = int(np.floor(p * B + 0.5))
+    return (B - n8) * 9 + n8 * 16 + B / 8.0
+
+
+def algorithmic_act_bytes(M, K, p):
+    B = M * K // 16
+    n8 = int(np.floor(p * B + 0.5))
+    return (B - n8) * 9 + n8 * 16 + B / 8.0
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl" if torch.cuda.is_available() else "gloo")
+    return world, rank, local
+
+
+def barrier_and_sync(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+WORKLOADS = {
+    # name: (M, N, K, fp8 fraction, kind)
+    "llama2-7b-fc1-decode": (16, 11008, 4096, 0.10, "decode"),
+    "llama2-7b-qkvo-prefill": (4096, 4096, 4096, 0.10, "prefill"),
+    "llama2-7b-fc1-prefill": (4096, 11008, 4096, 0.10, "prefill"),
+    "llama2-7b-fc2-prefill": (4096, 4096, 11008, 0.10, "prefill"),
+    "tiny": (64, 256, 256, 0.10, "decode"),
+}
+
+
+def run_ours(args, world, rank, local):
+    import paper_2504_14152_b200 as fg
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    M, N, K, p, kind = WORKLOADS[args.workload]
+    if args.m:
+        M = args.m
+    wl = gi.llama(args.workload, M, N, K, p, seed=0) if args.workload != "tiny" else gi.tiny(0)
+    x_cpu, w_cpu, fx, fw = wl.x(), wl.w(), wl.fx().to(dev), wl.fw().to(dev)
+    s4 = gi.tensor_scale(x_cpu)
+    wbytes = algorithmic_weight_bytes(N, K, p)
+    # enough distinct weight copies that weights alone exceed L2
+    n_copies = max(2, int(np.ceil(1.5 * L2_BYTES / wbytes))) if kind == "decode" else 2
+    n_copies = min(n_copies, 16)
+
+    # ---- offline: pack the weights (timed, reported separately)
+    w_dev = w_cpu.to(dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    packed_w = []
+    pw_ms = []
+    for i in range(n_copies):
+        ev[0].record()
+        packed_w.append(fg.quantize_weights(w_dev, fw, clip_mode=fg.CLIP_SW_BRUTE, fp8_fraction=p))
+        ev[1].record()
+        torch.cuda.synchronize()
+        pw_ms.append(ev[0].elapsed_time(ev[1]))
+    # ---- offline: activation threshold for the target fraction (Eq. 9 on this batch)
+    x_dev = x_cpu.to(dev)
+    tau = float(fg.calibrate_tau(x_dev, fx, scale_fp4=s4, fp8_fraction=p).item())
+
+    acts_buf = fg.binding._alloc_aligned(fg.acts_bytes(M, K), dev)
+    ws = fg.binding._alloc_aligned(fg.workspace_bytes(fg.binding.OP_LINEAR, M, N, K), dev)
+    y = torch.empty(M, N, dtype=torch.float32, device=dev)
+    # distinct activation copies as well (small at decode, > L2 in total at prefill with the planes)
+    n_x = 4
+    xs = [x_dev] + [x_dev.clone() for _ in range(n_x - 1)]
+
+    def step(i):
+        pa = fg.quantize_activations(xs[i % n_x], fx, scale_fp4=s4, tau=tau, out=acts_buf)
+        fg.linear(pa, packed_w[i % n_copies], out=y, workspace=ws)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    fg.check(ws)
+
+    timed = ("expand_weights", "gemm_bf16_tcgen05", "decode_gemm", "quant_act")
+    barrier_and_sync(world)
+    with ClockSampler(local) as clk:
+        fg.profile_begin(timed)
+        ev[0].record()
+        for i in range(args.steps):
+            step(i)
+        ev[1].record()
+        barrier_and_sync(world)
+        prof = fg.profile_end()
+    ms = ev[0].elapsed_time(ev[1])
+    fg.check(ws)
+    ms = max_over_ranks(ms, world)
+    clocks = clk.summary()
+
+    # ---- end to end: host buffers, H2D of the step's activations and D2H of its result inside
+    x_host = x_cpu.pin_memory()
+    y_host = torch.empty(M, N, dtype=torch.float32).pin_memory()
+    x_in = torch.empty_like(x_dev)
+
+    def step_e2e(i):
+        x_in.copy_(x_host, non_blocking=True)
+        pa = fg.quantize_activations(x_in, fx, scale_fp4=s4, tau=tau, out=acts_buf)
+        fg.linear(pa, packed_w[i % n_copies], out=y, workspace=ws)
+        y_host.copy_(y, non_blocking=True)
+
+    for i in range(3):
+        step_e2e(i)
+    barrier_and_sync(world)
+    t0 = time.perf_counter()
+    ev[0].record()
+    for i in range(args.steps):
+        step_e2e(i)
+    ev[1].record()
+    barrier_and_sync(world)
+    e2e_wall_ms = (time.perf_counter() - t0) * 1e3
+    e2e_ms = max(ev[0].elapsed_time(ev[1]), 0.0)
+    e2e_ms = max_over_ranks(max(e2e_ms, e2e_wall_ms if args.steps else 0.0), world)
+
+    flops = 2.0 * M * N * K
+    if kind == "decode":
+        metric, unit = "FGMP linear weight GB/s (decode)", "GB/s"
+        per_step_units = wbytes / 1e9
+    else:
+        metric, unit = "FGMP linear TFLOP/s (prefill)", "TFLOP/s"
+        per_step_units = flops / 1e12
+    value = world * per_step_units * args.steps / (ms / 1e3)
+    e2e_value = world * per_step_units * args.steps / (e2e_ms / 1e3)
+
+    peaks = measured_peaks()
+    launches = sum(v[0] for v in prof.values())
+    # dominant kernel = the timed kernel with the largest share
+    dom = max(((k, v) for k, v in prof.items() if v[1] > 0), key=lambda kv: kv[1][1], default=None)
+    roofline = None
+    if dom:
+        name, (n_l, tot_ms) = dom
+        avg_s = tot_ms / n_l / 1e3
+        if kind == "decode":
+            alg = wbytes + algorithmic_act_bytes(M, K, p) + M * N * 4
+            ach = alg / avg_s / 1e9
+            roofline = {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"], "traffic": load_traffic(name, args.workload),
+                        "peak_source": peaks["source"], "avg_kernel_us": avg_s * 1e6,
+                        "algorithmic_bytes_per_launch": alg}
+        else:
+            ach = flops / avg_s / 1e12
+            pk = peaks["bf16_tflops_sustained"]
+            roofline = {"kernel": name, "bound": "tensor", "achieved": ach, "peak": pk, "unit": "TFLOP/s",
+                        "frac": ach / pk, "traffic": load_traffic(name, args.workload),
+                        "peak_source": peaks["source"] + " bf16 sustained (common-container path runs at the f16 rate)",
+                        "avg_kernel_us": avg_s * 1e6}
+    out = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "nvfp4+e4m3 operands, f32 accumulate", "data": "synthetic",
+        "config": {"workload": args.workload, "M": M, "N": N, "K": K, "fp8_fraction_weights": p,
+                   "fp8_fraction_activations": p, "score_mode": "lp_error(Eq.6)", "clip": "sw_brute(Eq.11)",
+                   "l2": f"rotating {n_copies} packed weight copies ({n_copies * wbytes / 1e6:.0f} MB > 126 MB L2)"
+                   if kind == "decode" else "operands + bf16 planes exceed L2",
+                   "step": "quantize_activations + linear (online path); weight packing is offline"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": x_cpu.numel() * 2,
+                "d2h_bytes_per_step": M * N * 4, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": launches,
+        "kernels": {k: {"launches": v[0], "avg_us": (v[1] / v[0] * 1e3 if v[1] else None)} for k, v in prof.items()},
+        "roofline": roofline,
+        "offline": {"quantize_weights_ms": statistics.median(pw_ms), "weights_shape": [N, K],
+                    "packed_MB": fg.weights_bytes(N, K, int(p * N * K / 16 + 0.5) + 1) / 1e6,
+                    "algorithmic_MB": wbytes / 1e6},
+    }
+    if rank == 0 and not args.no_cpu_baseline and world >= 1:
+        out["cpu_baseline"] = cpu_baseline(args, wl, p, kind, per_step_units, unit)
+    return out
+
+
+def load_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of the kernel, from the committed ncu summary (None if absent)."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        try:
+            return json.load(open(path)).get(workload, {}).get(kernel)
+        except Exception:
+            return None
+    return None
+
+
+def cpu_baseline(args, wl, p, kind, per_step_units, unit, budget_s=20.0, max_steps=None):
+    """The oracle, as it stands, on the host cores: the same online step (activation quantizer +
+    fp64 GEMM over decoded operands), on a bounded sample of the workload."""
+    import oracle
+    x, w, fx, fw = wl.x(), wl.w(), wl.fx().numpy(), wl.fw().numpy()
+    M, N, K = wl.M, wl.N, wl.K
+    # bound the sample: a slice of the weight rows (and of the tokens at prefill)
+    n_rows = min(N, 1024 if kind == "decode" else 256)
+    m_rows = min(M, 16 if kind == "decode" else 64)
+    s4 = gi.tensor_scale(x)
+    xb = gi.bf16_bits(x)[:m_rows].copy()
+    qw = oracle.quantize_weights(gi.bf16_bits(w)[:n_rows].copy(), fw[:n_rows].copy(), clip=False, fp8_fraction=p)
+    scores = oracle.quantize_activations(xb, fx, s4, tau=np.inf).scores
+    k = int(np.floor(p * scores.size + 0.5))
+    srt = np.sort(scores)[::-1]
+    tau = float(np.float32(0.5) * (srt[k - 1] + srt[k])) if 0 < k < scores.size else float("inf")
+    frac = (n_rows / N) * (m_rows / M)
+    t0 = time.perf_counter()
+    steps = 0
+    while True:
+        qa = oracle.quantize_activations(xb, fx, s4, tau=tau)
+        oracle.linear(qa, qw)
+        steps += 1
+        el = time.perf_counter() - t0
+        if el > budget_s or (max_steps and steps >= max_steps):
+            break
+    sec_per_full_step = el / steps / frac
+    return {"value": per_step_units / sec_per_full_step, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{steps} steps of tokens[:{m_rows}] x weight rows[:{n_rows}] (fraction {frac:.4g} of one step, "
+                      f"scaled linearly); weights pre-packed by the oracle without clip search (untimed)",
+            "seconds_per_full_step": sec_per_full_step}
+
+
+def run_reference(args, world, rank):
+    """The CPU oracle as the reference arm (there is no reference implementation to install)."""
+    if rank != 0:
+        return None
+    M, N, K, p, kind = WORKLOADS[args.workload]
+    if args.m:
+        M = args.m
+    wl = gi.llama(args.workload, M, N, K, p, seed=0) if args.workload != "tiny" else gi.tiny(0)
+    flops = 2.0 * M * N * K
+    if kind == "decode":
+        metric, unit, units = "FGMP linear weight GB/s (decode)", "GB/s", algorithmic_weight_bytes(N, K, p) / 1e9
+    else:
+        metric, unit, units = "FGMP linear TFLOP/s (prefill)", "TFLOP/s", flops / 1e12
+    # warm-up (also builds the oracle) then K bounded-sample steps
+    cpu_baseline(args, wl, p, kind, units, unit, budget_s=0.0, max_steps=max(1, min(args.warmup, 1)))
+    cb = cpu_baseline(args, wl, p, kind, units, unit, budget_s=1e9, max_steps=max(1, args.steps))
+    return {
+        "impl": "reference", "metric": metric, "value": cb["value"], "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": cb["seconds_per_full_step"] * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64 accumulate over decoded nvfp4/e4m3 operands",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "M": M, "N": N, "K": K, "fp8_fraction_weights": p,
+                   "fp8_fraction_activations": p},
+        "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": cb["value"], "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2-7b-fc1-decode", choices=sorted(WORKLOADS))
+    ap.add_argument("--m", type=int, default=0, help="override the token count M")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        if rank != 0:
+            return 0
+        if args.steps == 200:
+            args.steps = 3
+        out = run_reference(args, int(os.environ.get("WORLD_SIZE", "1")), rank)
+        print(json.dumps(out))
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the FGMP kernels have no CPU fallback")
+    world, rank, local = dist_setup(args.gpus)
+    out = run_ours(args, world, rank, local)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

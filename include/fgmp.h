@@ -159,6 +159,17 @@ fgmp_status fgmp_activation_scores(const void* X_bf16, int64_t ldx, const float*
                                    int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
                                    float* scores, void* cuda_stream);
 
+/* ---- measurement support (the paper has no counterpart) ----
+ * Between fgmp_profile_begin and fgmp_profile_end (host calls, same thread as the launches)
+ * the library counts every kernel it launches, per kernel id, and brackets the launches of
+ * the ids selected in `timed_kernel_mask` (bit i = id i) with CUDA events on their launch
+ * stream.  fgmp_profile_end synchronizes those events and fills launches[i] and ms_total[i]
+ * (host arrays of length n; ms_total is 0 for ids that were not selected).  Both return the
+ * number of kernel ids; fgmp_kernel_name(i) names id i. */
+int fgmp_profile_begin(unsigned timed_kernel_mask);
+int fgmp_profile_end(int n, long long* launches, float* ms_total);
+const char* fgmp_kernel_name(int id);
+
 const char* fgmp_status_string(fgmp_status s);
 int fgmp_version(void);
 

@@ -62,6 +62,12 @@ def _load():
     L.fgmp_unpack.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp]
     L.fgmp_activation_scores.restype = ci
     L.fgmp_activation_scores.argtypes = [vp, i64, vp, i64, i64, _Scales, ci, vp, vp]
+    L.fgmp_profile_begin.restype = ci
+    L.fgmp_profile_begin.argtypes = [ctypes.c_uint]
+    L.fgmp_profile_end.restype = ci
+    L.fgmp_profile_end.argtypes = [ci, vp, vp]
+    L.fgmp_kernel_name.restype = ctypes.c_char_p
+    L.fgmp_kernel_name.argtypes = [ci]
     L.fgmp_status_string.restype = ctypes.c_char_p
     L.fgmp_status_string.argtypes = [ci]
     L.fgmp_version.restype = ci
@@ -230,3 +236,34 @@ def unpack(p: PackedTensor):
     _ok(L.fgmp_unpack(p.blob.data_ptr(), p.rows, p.K, codes4.data_ptr(), codes8.data_ptr(), scales.data_ptr(),
                       mask.data_ptr(), _stream()), "fgmp_unpack")
     return codes4, codes8, scales, mask
+
+
+def kernel_names() -> list[str]:
+    L = _load()
+    names = []
+    while True:
+        name = L.fgmp_kernel_name(len(names)).decode()
+        if not name:
+            return names
+        names.append(name)
+
+
+def profile_begin(timed_kernels: list[str] | tuple[str, ...] = ()) -> None:
+    """Start counting kernel launches; launches of the named kernels are also timed with
+    CUDA events on their stream."""
+    names = kernel_names()
+    mask = 0
+    for k in timed_kernels:
+        mask |= 1 << names.index(k)
+    _load().fgmp_profile_begin(mask)
+
+
+def profile_end() -> dict:
+    """{kernel name: (launches, total ms or 0.0)} since profile_begin."""
+    L = _load()
+    names = kernel_names()
+    n = len(names)
+    launches = (ctypes.c_longlong * n)()
+    ms = (ctypes.c_float * n)()
+    L.fgmp_profile_end(n, launches, ms)
+    return {names[i]: (int(launches[i]), float(ms[i])) for i in range(n) if launches[i]}

@@ -402,10 +402,10 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     {
         int64_t nb = M * (K / 16);
         int g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
-        expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, 0, reinterpret_cast<uint4*>(planeA));
+        FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, 0, reinterpret_cast<uint4*>(planeA)));
         nb = N * (K / 16);
         g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
-        expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_weights, N, K, 1, reinterpret_cast<uint4*>(planeW));
+        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_weights, N, K, 1, reinterpret_cast<uint4*>(planeW)));
     }
     GemmParams p;
     p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K;
@@ -414,7 +414,7 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     p.status = status;
     const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(tmA, tmB, p);
+    FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(tmA, tmB, p));
     return fgmp_launch_status();
 }
 

@@ -1,6 +1,8 @@
 // Host utilities: device capability check, status strings, size queries.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
+#include <vector>
+#include <mutex>
 
 namespace {
 struct DevInfo { int checked; int major; int sms; };
@@ -65,4 +67,76 @@ extern "C" size_t fgmp_acts_bytes(int64_t M, int64_t K)
 {
     if (M < 1 || K < 64 || (K % 64) != 0) return 0;
     return fgmp_layout(M, K, 0, 0).total;
+}
+
+// ------------------------------------------------------------------ launch accounting
+namespace {
+struct ProfRec { int id; cudaEvent_t a, b; };
+std::mutex g_prof_mu;
+bool g_prof_on = false;
+unsigned g_prof_mask = 0;
+long long g_prof_count[FGMP_K_COUNT];
+std::vector<ProfRec> g_prof_recs;
+std::vector<cudaEvent_t> g_event_pool;
+const char* const g_kernel_names[FGMP_K_COUNT] = {
+    "quant_act", "act_aux", "unpack", "expand_acts", "expand_weights", "gemm_bf16_tcgen05",
+    "w_amax", "w_score_clip", "select", "w_mask", "scan", "w_emit", "w_aux", "act_scores", "decode_gemm"};
+cudaEvent_t get_event()
+{
+    if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+}  // namespace
+
+FgmpLaunchScope::FgmpLaunchScope(int id_, cudaStream_t s_) : id(id_), s(s_), stop(nullptr)
+{
+    if (!g_prof_on) return;
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_count[id]++;
+    if (g_prof_mask & (1u << id)) {
+        ProfRec r{id, get_event(), get_event()};
+        if (r.a && r.b) {
+            cudaEventRecord(r.a, s);
+            stop = r.b;
+            g_prof_recs.push_back(r);
+        }
+    }
+}
+
+FgmpLaunchScope::~FgmpLaunchScope()
+{
+    if (stop) cudaEventRecord(stop, s);
+}
+
+extern "C" int fgmp_profile_begin(unsigned timed_kernel_mask)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    for (int i = 0; i < FGMP_K_COUNT; ++i) g_prof_count[i] = 0;
+    for (auto& r : g_prof_recs) { g_event_pool.push_back(r.a); g_event_pool.push_back(r.b); }
+    g_prof_recs.clear();
+    g_prof_mask = timed_kernel_mask;
+    g_prof_on = true;
+    return FGMP_K_COUNT;
+}
+
+extern "C" int fgmp_profile_end(int n, long long* launches, float* ms_total)
+{
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = false;
+    for (int i = 0; i < n && i < FGMP_K_COUNT; ++i) { launches[i] = g_prof_count[i]; ms_total[i] = 0.f; }
+    for (auto& r : g_prof_recs) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.b) == cudaSuccess && cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess && r.id < n)
+            ms_total[r.id] += ms;
+        g_event_pool.push_back(r.a); g_event_pool.push_back(r.b);
+    }
+    g_prof_recs.clear();
+    return FGMP_K_COUNT;
+}
+
+extern "C" const char* fgmp_kernel_name(int id)
+{
+    return (id >= 0 && id < FGMP_K_COUNT) ? g_kernel_names[id] : "";
 }

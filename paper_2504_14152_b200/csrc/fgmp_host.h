@@ -13,3 +13,18 @@ int fgmp_sm_count();
 size_t fgmp_ws_quantize_weights(int64_t N, int64_t K);
 size_t fgmp_ws_calibrate(int64_t M, int64_t K);
 size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K);
+
+// ---- launch accounting (see fgmp_profile_begin in fgmp.h) ----
+enum FgmpKernelId {
+    FGMP_K_ACT_QUANT = 0, FGMP_K_ACT_AUX, FGMP_K_UNPACK, FGMP_K_EXPAND_A, FGMP_K_EXPAND_W, FGMP_K_GEMM_BF16,
+    FGMP_K_W_AMAX, FGMP_K_W_SCORE, FGMP_K_SELECT, FGMP_K_W_MASK, FGMP_K_SCAN, FGMP_K_W_EMIT, FGMP_K_W_AUX,
+    FGMP_K_ACT_SCORES, FGMP_K_DECODE, FGMP_K_COUNT
+};
+// Brackets one kernel launch: counts it and, when event timing of this kernel id is on,
+// records a CUDA event before and after it on the launch stream.
+struct FgmpLaunchScope {
+    int id; cudaStream_t s; cudaEvent_t stop;
+    FgmpLaunchScope(int id, cudaStream_t s);
+    ~FgmpLaunchScope();
+};
+#define FGMP_LAUNCH(id, stream, ...) do { FgmpLaunchScope fgmp_scope_(id, stream); __VA_ARGS__; } while (0)

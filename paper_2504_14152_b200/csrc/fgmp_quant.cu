@@ -192,10 +192,10 @@ extern "C" fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx
     p.codes4 = blob + L.off_codes4; p.sf = blob + L.off_sf;
     p.mask = reinterpret_cast<uint32_t*>(blob + L.off_mask); p.codes8 = blob + L.off_codes8;
     dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((M + p.rows_per_cta - 1) / p.rows_per_cta));
-    act_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), M, K, sc.scale_fp4, sc.fp8_log2_ratio);
-    if (M % 128) sf_pad_zero_kernel<<<64, 256, 0, s>>>(p.sf, M, K);
-    if (sm == FGMP_SCORE_LP_ERROR) quant_act_kernel<0, false><<<grid, QA_THREADS, 0, s>>>(p);
-    else                           quant_act_kernel<1, false><<<grid, QA_THREADS, 0, s>>>(p);
+    FGMP_LAUNCH(FGMP_K_ACT_AUX, s, act_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), M, K, sc.scale_fp4, sc.fp8_log2_ratio));
+    if (M % 128) FGMP_LAUNCH(FGMP_K_ACT_AUX, s, sf_pad_zero_kernel<<<64, 256, 0, s>>>(p.sf, M, K));
+    if (sm == FGMP_SCORE_LP_ERROR) FGMP_LAUNCH(FGMP_K_ACT_QUANT, s, quant_act_kernel<0, false><<<grid, QA_THREADS, 0, s>>>(p));
+    else                           FGMP_LAUNCH(FGMP_K_ACT_QUANT, s, quant_act_kernel<1, false><<<grid, QA_THREADS, 0, s>>>(p));
     return fgmp_launch_status();
 }
 
@@ -211,8 +211,8 @@ extern "C" fgmp_status fgmp_activation_scores(const void* X_bf16, int64_t ldx, c
     ActParams p = make_act_params(X_bf16, ldx, fisher_chan, M, K, sc, 0.f);
     p.scores = scores;
     dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((M + p.rows_per_cta - 1) / p.rows_per_cta));
-    if (sm == FGMP_SCORE_LP_ERROR) quant_act_kernel<0, true><<<grid, QA_THREADS, 0, s>>>(p);
-    else                           quant_act_kernel<1, true><<<grid, QA_THREADS, 0, s>>>(p);
+    if (sm == FGMP_SCORE_LP_ERROR) FGMP_LAUNCH(FGMP_K_ACT_SCORES, s, quant_act_kernel<0, true><<<grid, QA_THREADS, 0, s>>>(p));
+    else                           FGMP_LAUNCH(FGMP_K_ACT_SCORES, s, quant_act_kernel<1, true><<<grid, QA_THREADS, 0, s>>>(p));
     return fgmp_launch_status();
 }
 
@@ -225,6 +225,6 @@ extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, 
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
     int64_t nblk = rows * (K / 16);
     int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);
-    unpack_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask);
+    FGMP_LAUNCH(FGMP_K_UNPACK, (cudaStream_t)cuda_stream, unpack_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
     return fgmp_launch_status();
 }

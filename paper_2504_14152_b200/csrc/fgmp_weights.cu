@@ -349,8 +349,8 @@ void run_select(const float* scores, int64_t B, SelectState* st, cudaStream_t s)
 {
     int g = grid_for(B, 256, 8);
     for (int pass = 0; pass < 4; ++pass) {
-        select_hist_kernel<<<g, 256, 0, s>>>(scores, B, pass, st);
-        select_pick_kernel<<<1, 256, 0, s>>>(st, pass);
+        FGMP_LAUNCH(FGMP_K_SELECT, s, select_hist_kernel<<<g, 256, 0, s>>>(scores, B, pass, st));
+        FGMP_LAUNCH(FGMP_K_SELECT, s, select_pick_kernel<<<1, 256, 0, s>>>(st, pass));
     }
 }
 
@@ -410,19 +410,19 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     const uint4* W = reinterpret_cast<const uint4*>(W_bf16);
     const int ratio = sc.fp8_log2_ratio;
 
-    state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k);
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k));
     if (sc.scale_fp4 == 0.f) {
-        w_amax_kernel<<<grid_for(N * (K / 8), 256, 8), 256, 0, s>>>(W, ldw / 8, N, K / 8, st);
-        w_scale_kernel<<<1, 32, 0, s>>>(st);
+        FGMP_LAUNCH(FGMP_K_W_AMAX, s, w_amax_kernel<<<grid_for(N * (K / 8), 256, 8), 256, 0, s>>>(W, ldw / 8, N, K / 8, st));
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, w_scale_kernel<<<1, 32, 0, s>>>(st));
     }
     {
         int g = grid_for(B, 256, 4);
         if (sm == FGMP_SCORE_LP_ERROR) {
-            if (cm == FGMP_CLIP_SW_BRUTE) w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
-            else                          w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
+            if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+            else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
         } else {
-            if (cm == FGMP_CLIP_SW_BRUTE) w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
-            else                          w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores);
+            if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+            else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
         }
     }
     uint32_t* mask = reinterpret_cast<uint32_t*>(blob + L.off_mask);
@@ -430,17 +430,17 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     const int gw = grid_for(NW * 32, 256, 8);
     if (fraction_mode && k > 0) {
         run_select(scores, B, st, s);
-        w_eqcount_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_a);
-        scan_kernel<<<1, 1024, 0, s>>>(tmp_a, tmp_b, NW, nullptr);
+        FGMP_LAUNCH(FGMP_K_W_MASK, s, w_eqcount_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_a));
+        FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, tmp_b, NW, nullptr));
     } else {
         // k == 0: nothing is FP8 (tau_eff = +inf); threshold mode: the given tau
-        set_tau_kernel<<<1, 32, 0, s>>>(st, fraction_mode ? INFINITY : tau);
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, set_tau_kernel<<<1, 32, 0, s>>>(st, fraction_mode ? INFINITY : tau));
     }
-    w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a);
-    scan_kernel<<<1, 1024, 0, s>>>(tmp_a, wordptr, NW, &st->n_fp8);
-    w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, ratio, st, sc_tmp, blob, L, capacity);
-    w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, N, K, ratio, capacity,
-                                     fraction_mode ? 1 : 0, tau, tau_eff_out);
+    FGMP_LAUNCH(FGMP_K_W_MASK, s, w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a));
+    FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, wordptr, NW, &st->n_fp8));
+    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, ratio, st, sc_tmp, blob, L, capacity));
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, N, K, ratio, capacity,
+                                     fraction_mode ? 1 : 0, tau, tau_eff_out));
     return fgmp_launch_status();
 }
 
@@ -463,13 +463,13 @@ extern "C" fgmp_status fgmp_calibrate_tau(const void* X_bf16, int64_t ldx, const
     if (stt != FGMP_OK) return stt;
     int64_t k = (int64_t)floor(fp8_fraction * (double)B + 0.5);
     if (k > B) k = B;
-    state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k);
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k));
     if (k == 0 || k == B) {
-        calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, k == 0 ? 1 : 2);
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, k == 0 ? 1 : 2));
     } else {
         run_select(scores, B, st, s);
-        next_below_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(scores, B, st);
-        calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, 0);
+        FGMP_LAUNCH(FGMP_K_SELECT, s, next_below_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(scores, B, st));
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, 0));
     }
     return fgmp_launch_status();
 }
