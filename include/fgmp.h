@@ -31,11 +31,15 @@
  *                   0x00 for FP8 blocks and for padding rows
  *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
  *                   1 = FP8
- *   wordptr       : (weights only) one uint32 per mask word = number of FP8 blocks that
- *                   precede the word's first block in row-major block order
- *   codes8        : weights: the FP8 blocks only, 16 bytes each, in row-major block order
- *                   (capacity max_fp8_blocks); activations: a dense rows*K byte plane of
- *                   which only the FP8 blocks are written.
+ *   ctptr, rowoff : (weights only) index of the FP8 list: ctptr[t*C + c] (uint32, C = ceil(K/256))
+ *                   = list position of the first FP8 block of 128-row tile t and 256-element
+ *                   K chunk c; rowoff[(t*C + c)*128 + r%128] (uint16) = offset of row r's
+ *                   first FP8 block inside that (tile, chunk)
+ *   atrue         : (activations with rows <= 16 only) fp16 copy of the quantized values
+ *                   divided by the tensor scale, [K/16][16 tokens][16]; rows >= M are zero
+ *   codes8        : weights: the FP8 blocks only, 16 bytes each, ordered by (tile, chunk, row,
+ *                   block) (capacity max_fp8_blocks); activations: a dense rows*K byte plane
+ *                   of which only the FP8 blocks are written.
  */
 #ifndef FGMP_H
 #define FGMP_H
@@ -71,7 +75,7 @@ typedef enum { FGMP_CLIP_NONE = 0, FGMP_CLIP_SW_BRUTE = 1 } fgmp_clip_mode;
 typedef struct {
     float scale_fp4;    /* FP32 tensor scale of the NVFP4 part; 0 = derive amax/(6*448)
                            on the device (weights only)                                     */
-    int fp8_log2_ratio; /* FP8 tensor scale = scale_fp4 * 2^ratio, -8 <= ratio <= 8        */
+    int fp8_log2_ratio; /* FP8 tensor scale = scale_fp4 * 2^ratio, -7 <= ratio <= 7        */
 } fgmp_scales;
 
 /* First 256 bytes of a packed blob (device memory). */

@@ -10,23 +10,34 @@
 #define FGMP_BS 16
 
 // ---------------------------------------------------------------- blob layout
+// Weights keep their FP8 blocks in a compact list ordered by (128-row tile, 256-element K
+// chunk, row, block): the blocks one GEMM CTA needs for one pipeline stage are contiguous.
+//   ctptr [tiles*chunks + 1] uint32 : list index of the first FP8 block of each (tile, chunk)
+//   rowoff[tiles*chunks*128] uint16 : offset of a row's first FP8 block inside its (tile, chunk)
+// Activations keep a dense FP8 plane (only FP8 blocks are written) and, when rows <= 16, a
+// dequantized fp16 copy `atrue` laid out [K/16 blocks][16 tokens][16 elements] whose values
+// are value / tensor scale (E2M1 x microscale, or E4M3 x 2^ratio); rows >= M are zero.
 struct PackedLayout {
     int64_t rows, K, KB, MW;          // KB = K/16 blocks per row, MW = mask words per row
-    size_t off_codes4, off_sf, off_mask, off_wordptr, off_codes8, total;
+    int64_t tiles, chunks;            // 128-row tiles, 16-block K chunks
+    size_t off_codes4, off_sf, off_mask, off_ctptr, off_rowoff, off_atrue, off_codes8, total;
 };
 
 __host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 
-// kind 0 = activations (dense FP8 plane), 1 = weights (compact FP8 list, capacity blocks)
+// kind 0 = activations, 1 = weights (capacity = room for that many FP8 blocks)
 __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int kind, int64_t capacity)
 {
     PackedLayout L;
     L.rows = rows; L.K = K; L.KB = K / 16; L.MW = (L.KB + 31) / 32;
+    L.tiles = (rows + 127) / 128; L.chunks = (L.KB + 15) / 16;
     size_t o = 1024;                                   // header section
     L.off_codes4 = o;  o = fgmp_align1k(o + (size_t)rows * (size_t)(K / 2));
-    L.off_sf = o;      o = fgmp_align1k(o + (size_t)((rows + 127) / 128) * (size_t)(K / 64) * 512);
+    L.off_sf = o;      o = fgmp_align1k(o + (size_t)L.tiles * (size_t)(K / 64) * 512);
     L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
-    L.off_wordptr = o; if (kind == 1) o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
+    L.off_ctptr = o;   if (kind == 1) o = fgmp_align1k(o + ((size_t)L.tiles * L.chunks + 1) * 4);
+    L.off_rowoff = o;  if (kind == 1) o = fgmp_align1k(o + (size_t)L.tiles * L.chunks * 128 * 2);
+    L.off_atrue = o;   if (kind == 0 && rows <= 16) o = fgmp_align1k(o + (size_t)L.KB * 512);
     L.off_codes8 = o;
     o = fgmp_align1k(o + (kind == 1 ? (size_t)capacity * 16 : (size_t)rows * (size_t)K));
     L.total = o;
@@ -39,6 +50,19 @@ __host__ __device__ inline size_t fgmp_sf_offset(int64_t r, int64_t kb, int64_t 
     return ((size_t)(r >> 7) * (size_t)(K >> 6) + (size_t)(kb >> 2)) * 512
          + (size_t)(r & 31) * 16 + (size_t)((r & 127) >> 5) * 4 + (size_t)(kb & 3);
 }
+
+#ifdef __CUDACC__
+// list index of FP8 block (r, kb) of a packed weight tensor; `word` is the row's mask word
+// that holds kb
+__device__ __forceinline__ uint32_t fgmp_fp8_pos(const uint8_t* blob, const PackedLayout& L, int64_t r, int64_t kb, uint32_t word)
+{
+    const int64_t ct = (r >> 7) * L.chunks + (kb >> 4);
+    const uint32_t half = (word >> (((kb >> 4) & 1) * 16)) & 0xffffu;
+    const uint32_t* ctptr = reinterpret_cast<const uint32_t*>(blob + L.off_ctptr);
+    const uint16_t* rowoff = reinterpret_cast<const uint16_t*>(blob + L.off_rowoff);
+    return ctptr[ct] + rowoff[ct * 128 + (r & 127)] + __popc(half & ((1u << (kb & 15)) - 1u));
+}
+#endif
 
 // ---------------------------------------------------------------- conversions
 #ifdef __CUDACC__

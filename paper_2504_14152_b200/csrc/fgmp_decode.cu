@@ -1,0 +1,434 @@
+// fgmp_linear for decode-sized batches (M <= 16 tokens): a weight-streaming kernel that
+// reads the packed weights exactly once (Section 4.1 of the paper: the four block-pair
+// products, FP32 accumulation).
+//
+// Decomposition (exact).  With A4z / W4z the NVFP4 planes (zero in FP8 blocks), W8 the FP8
+// blocks of the weights and At the true activation values (fp16 copy, either format):
+//     Y = A4z.W4z^T            tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
+//                              weights are the 128-row MMA operand, the 16 tokens are N
+//       + At.W8^T              only where a weight block is FP8   } mma.sync m16n8k16 on
+//       + At[FP8 blocks].W4z^T only where an activation block is FP8 } gathered 8-row groups
+// Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all
+// SMs stream the same number of bytes; tiles shared by several CTAs are reduced in a fixed
+// order by the CTA that arrives last (deterministic).
+//
+// Warp roles (320 threads): warp 0 = producer (TMA tensor + bulk copies), warp 1 = MMA issuer
+// and TMEM owner, warps 2-9 = FP8 corrections on CUDA-core-fed mma.sync, then epilogue.
+#include "fgmp_common.cuh"
+#include "fgmp_host.h"
+#include "fgmp_ptx.cuh"
+#include <cuda_fp16.h>
+
+namespace {
+
+constexpr int DEC_THREADS = 320;
+constexpr int DEC_CORR_WARPS = 8;
+constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
+constexpr uint32_t W4_BYTES = 128 * 128;        // 128 rows x 256 E2M1
+constexpr uint32_t A4_BYTES = TOK * 128;
+constexpr uint32_t SF_BYTES = 2048;             // 4 scale tiles of 512 B
+constexpr uint32_t ATRUE_BYTES = 16 * 512;      // 16 blocks x 16 tokens x 16 fp16
+constexpr uint32_t OFF_A4 = W4_BYTES, OFF_SFW = OFF_A4 + A4_BYTES, OFF_SFA = OFF_SFW + SF_BYTES,
+                   OFF_ATRUE = OFF_SFA + SF_BYTES, OFF_FP8 = OFF_ATRUE + ATRUE_BYTES;      // 30720
+constexpr uint32_t FP8_CAP_BLOCKS = 512;        // staged FP8 blocks per (tile, chunk); more are read from global
+constexpr uint32_t DEC_STAGE_BYTES = OFF_FP8 + FP8_CAP_BLOCKS * 16;                       // 38912
+constexpr int DEC_STAGES = 5;
+constexpr int CORR_LD = 17;                     // padded row of the correction tile (floats)
+constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 16 accumulator columns + 5 stages x 32 scale columns
+constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + 128 * CORR_LD * 4 + 1024 + 512;
+
+// kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
+constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
+
+struct DecParams {
+    const uint8_t* wblob; const uint8_t* ablob;
+    PackedLayout LW, LA;
+    float* Y; void* Ybf; int64_t ldy; int y_is_bf16;
+    int64_t M, N, K;
+    int64_t total;            // tiles * chunks
+    int64_t chunks;
+    int* status; uint32_t* counters; float* partials; int maxseg;
+};
+
+struct StageMeta { uint32_t p0, cnt; };
+
+__device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
+
+__global__ void __launch_bounds__(DEC_THREADS, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, DecParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    float* corr = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(corr) + 128 * CORR_LD * 4);
+    // bars: [0,S) full, [S,2S) empty, [2S,2S+2) acc_full, [2S+2,2S+4) acc_empty
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + DEC_STAGES);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + DEC_STAGES);
+    const uint32_t accf0 = smem_u32(bars + 2 * DEC_STAGES), acce0 = smem_u32(bars + 2 * DEC_STAGES + 2);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + DEC_CORR_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 32 * DEC_CORR_WARPS); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // this CTA's span of (tile, chunk) units
+    const int64_t G = gridDim.x, C = p.chunks;
+    const int64_t u_begin = ((int64_t)blockIdx.x * p.total) / G, u_end = ((int64_t)(blockIdx.x + 1) * p.total) / G;
+    const uint32_t* ctptr = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_ctptr);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            const uint8_t* sfw = p.wblob + p.LW.off_sf;
+            const uint8_t* sfa = p.ablob + p.LA.off_sf;
+            const uint8_t* atrue = p.ablob + p.LA.off_atrue;
+            const uint8_t* fp8 = p.wblob + p.LW.off_codes8;
+            uint32_t nxt0 = 0, nxt1 = 0;
+            if (u_begin < u_end) { nxt0 = __ldg(ctptr + u_begin); nxt1 = __ldg(ctptr + u_begin + 1); }
+            for (int64_t u = u_begin; u < u_end; ++u) {
+                const int64_t tile = u / C, c = u % C;
+                const uint32_t p0 = nxt0, p1 = nxt1;
+                if (u + 1 < u_end) { nxt0 = p1; nxt1 = __ldg(ctptr + u + 2); }
+                if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) break;
+                const uint32_t cnt = p1 - p0, staged = cnt < FP8_CAP_BLOCKS ? cnt : FP8_CAP_BLOCKS;
+                smeta[stage].p0 = p0; smeta[stage].cnt = cnt;
+                const uint32_t fb = full0 + 8 * stage;
+                const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
+                mbar_expect_tx(fb, OFF_FP8 + staged * 16);
+                tma_load_2d(sb, &tmW, (int32_t)(c * 128), (int32_t)(tile * 128), fb);
+                tma_load_2d(sb + OFF_A4, &tmA, (int32_t)(c * 128), 0, fb);
+                bulk_load(sb + OFF_SFW, sfw + ((size_t)tile * (p.K >> 6) + (size_t)c * 4) * 512, SF_BYTES, fb);
+                bulk_load(sb + OFF_SFA, sfa + (size_t)c * 4 * 512, SF_BYTES, fb);
+                bulk_load(sb + OFF_ATRUE, atrue + (size_t)c * ATRUE_BYTES, ATRUE_BYTES, fb);
+                if (staged) bulk_load(sb + OFF_FP8, fp8 + (size_t)p0 * 16, staged * 16, fb);
+                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            int seg = 0;
+            for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+                const int64_t tile = u / C;
+                const int64_t seg_end = min(u_end, (tile + 1) * C);
+                const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
+                if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
+                bool first = true;
+                for (; u < seg_end; ++u) {
+                    if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
+                    tc_fence_after();
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
+                    const uint32_t sf_t = tmem_base + 32 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        tmem_cp_sf(sf_t + 4 * j, smem_desc_sf(sb + OFF_SFW + 512 * j));
+                        tmem_cp_sf(sf_t + 16 + 4 * j, smem_desc_sf(sb + OFF_SFA + 512 * j));
+                    }
+                    const uint64_t adesc = smem_desc_sw128(sb), bdesc = smem_desc_sw128(sb + OFF_A4);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        umma_nvf4(d_tmem, adesc + 2 * j, bdesc + 2 * j, IDESC_NVF4, sf_t + 4 * j, sf_t + 16 + 4 * j,
+                                  (first && j == 0) ? 0u : 1u);
+                    }
+                    first = false;
+                    umma_commit(empty0 + 8 * stage);
+                    if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(accf0 + 8 * acc);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ corrections + epilogue
+        // A warp may read TMEM lanes [32q, 32q+32), q = warp % 4; two warps share a quadrant and
+        // each owns 16 of its rows, for the corrections and for the epilogue alike, so that the
+        // correction sums never cross warps.
+        const int q = warp & 3, h = (warp - 2) >> 2;
+        const int rowbase = 32 * q + 16 * h;           // first owned row inside the tile
+        const int slice = 2 * q + h;                   // 0..7
+        const int g = lane >> 2, t = lane & 3;
+        const uint32_t* wmask = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_mask);
+        const uint16_t* rowoff = reinterpret_cast<const uint16_t*>(p.wblob + p.LW.off_rowoff);
+        const uint32_t* amask = reinterpret_cast<const uint32_t*>(p.ablob + p.LA.off_mask);
+        const uint8_t* fp8 = p.wblob + p.LW.off_codes8;
+        const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
+        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+        const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
+        const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
+        const int64_t MWw = p.LW.MW, MWa = p.LA.MW;
+        const bool tok0 = g < p.M, tok1 = g + 8 < p.M;
+        float* mycorr = corr + rowbase * CORR_LD;
+
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
+            const int64_t n0 = tile * 128 + rowbase + g, n1 = n0 + 8;       // own rows (B fragments)
+            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+
+            // per-chunk metadata of the own rows / tokens, fetched one chunk ahead
+            uint32_t wm[2], ro[2], am[2];
+            auto fetch_meta = [&](int64_t uu, uint32_t (&wm_)[2], uint32_t (&ro_)[2], uint32_t (&am_)[2]) {
+                const int64_t c = uu % C;
+                const int sh = (int)(c & 1) * 16;
+                wm_[0] = n0 < p.N ? (__ldg(wmask + n0 * MWw + (c >> 1)) >> sh) & 0xffffu : 0u;
+                wm_[1] = n1 < p.N ? (__ldg(wmask + n1 * MWw + (c >> 1)) >> sh) & 0xffffu : 0u;
+                ro_[0] = __ldg(rowoff + uu * 128 + rowbase + g);
+                ro_[1] = __ldg(rowoff + uu * 128 + rowbase + 8 + g);
+                am_[0] = tok0 ? (__ldg(amask + (int64_t)g * MWa + (c >> 1)) >> sh) & 0xffffu : 0u;
+                am_[1] = tok1 ? (__ldg(amask + (int64_t)(g + 8) * MWa + (c >> 1)) >> sh) & 0xffffu : 0u;
+            };
+            fetch_meta(u, wm, ro, am);
+
+            for (; u < seg_end; ++u) {
+                uint32_t wm_n[2] = {0, 0}, ro_n[2] = {0, 0}, am_n[2] = {0, 0};
+                if (u + 1 < seg_end) fetch_meta(u + 1, wm_n, ro_n, am_n);
+                // which blocks of this chunk need work at all (any of the 8 rows / 16 tokens)
+                uint32_t ow0 = wm[0], ow1 = wm[1], oa = am[0] | am[1];
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) {
+                    ow0 |= __shfl_xor_sync(0xffffffffu, ow0, o);
+                    ow1 |= __shfl_xor_sync(0xffffffffu, ow1, o);
+                    oa |= __shfl_xor_sync(0xffffffffu, oa, o);
+                }
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+                const uint32_t list0 = smeta[stage].p0;
+                uint32_t todo = ow0 | ow1 | oa;
+                while (todo) {
+                    const int kb = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const uint32_t bit = 1u << kb;
+                    // A fragment: true activation values of tokens g and g+8, elements 4t..4t+3 of block kb
+                    const uint2 at0 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + g * 32 + t * 8);
+                    const uint2 at1 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + (g + 8) * 32 + t * 8);
+                    // (1) FP8 weight blocks
+#pragma unroll
+                    for (int rg = 0; rg < 2; ++rg) {
+                        if (!((rg ? ow1 : ow0) & bit)) continue;
+                        uint32_t b0 = 0, b1 = 0;
+                        if (wm[rg] & bit) {
+                            const uint32_t idx = ro[rg] + __popc(wm[rg] & (bit - 1u));
+                            uint32_t raw;
+                            if (idx < FP8_CAP_BLOCKS) raw = *reinterpret_cast<const uint32_t*>(sb + OFF_FP8 + idx * 16 + t * 4);
+                            else raw = __ldg(reinterpret_cast<const uint32_t*>(fp8 + ((size_t)list0 + idx) * 16 + t * 4));
+                            uint32_t h0, h1;
+                            uint16_t lo = (uint16_t)raw, hi = (uint16_t)(raw >> 16);
+                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(lo));
+                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(hi));
+                            __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), rw2), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), rw2);
+                            b0 = *reinterpret_cast<uint32_t*>(&x0); b1 = *reinterpret_cast<uint32_t*>(&x1);
+                        }
+                        mma_f16_16816(acc[rg], at0.x, at1.x, at0.y, at1.y, b0, b1);
+                    }
+                    // (2) FP8 activation blocks against the NVFP4 weights of this stage
+                    if (oa & bit) {
+                        const uint32_t a0 = (am[0] & bit) ? at0.x : 0u, a2 = (am[0] & bit) ? at0.y : 0u;
+                        const uint32_t a1 = (am[1] & bit) ? at1.x : 0u, a3 = (am[1] & bit) ? at1.y : 0u;
+#pragma unroll
+                        for (int rg = 0; rg < 2; ++rg) {
+                            const int r = rowbase + 8 * rg + g;            // row inside the tile
+                            const uint32_t codes = *reinterpret_cast<const uint16_t*>(
+                                sb + r * 128 + ((((uint32_t)kb >> 1) ^ ((uint32_t)r & 7u)) << 4) + (kb & 1) * 8 + t * 2);
+                            const uint32_t sfb = sb[OFF_SFW + (kb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)];
+                            uint32_t q0, q1, sc2;
+                            asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
+                                : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
+                            uint16_t s16 = (uint16_t)(sfb | (sfb << 8));
+                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
+                            __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&q0), *reinterpret_cast<__half2*>(&sc2));
+                            __half2 x1 = __hmul2(*reinterpret_cast<__half2*>(&q1), *reinterpret_cast<__half2*>(&sc2));
+                            mma_f16_16816(acc[rg], a0, a1, a2, a3, *reinterpret_cast<uint32_t*>(&x0), *reinterpret_cast<uint32_t*>(&x1));
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+                wm[0] = wm_n[0]; wm[1] = wm_n[1]; ro[0] = ro_n[0]; ro[1] = ro_n[1]; am[0] = am_n[0]; am[1] = am_n[1];
+            }
+            if (!ok) break;
+
+            // transpose the correction sums through this warp's private rows of the tile:
+            // mycorr[row][token]
+#pragma unroll
+            for (int rg = 0; rg < 2; ++rg) {
+                const int r = 8 * rg + 2 * t;
+                mycorr[r * CORR_LD + g] = acc[rg][0];
+                mycorr[(r + 1) * CORR_LD + g] = acc[rg][1];
+                mycorr[r * CORR_LD + g + 8] = acc[rg][2];
+                mycorr[(r + 1) * CORR_LD + g + 8] = acc[rg][3];
+            }
+            __syncwarp();
+
+            const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
+            if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
+            tc_fence_after();
+            uint32_t rr[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
+            tc_fence_before();
+            mbar_arrive(acce0 + 8 * accb);
+            // lanes 16h .. 16h+15 hold this warp's rows
+            const bool mine = (lane >> 4) == h;
+            const int lr = lane & 15;
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]) + mycorr[lr * CORR_LD + j];
+            __syncwarp();
+            const int64_t n = tile * 128 + rowbase + lr;
+            const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
+            bool write_out = whole;
+            if (!whole) {
+                // partial tile: publish, and let the warp that arrives last add everything up
+                const int64_t c_first = cta_of_unit(tile * C, G, p.total);
+                const int64_t c_last = cta_of_unit((tile + 1) * C - 1, G, p.total);
+                const int nseg = (int)(c_last - c_first + 1);
+                const int slot = (int)(blockIdx.x - c_first);
+                if (mine) {
+                    float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + rowbase + lr) * 16;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+                }
+                __threadfence();
+                __syncwarp();
+                uint32_t old = 0;
+                if (lane == 0) old = atomicAdd(p.counters + tile * 8 + slice, 1u);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old == (uint32_t)(nseg - 1)) {
+                    __threadfence();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                    if (mine) {
+                        for (int sgi = 0; sgi < nseg; ++sgi) {
+                            const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + rowbase + lr) * 16;
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4) {
+                                float4 x = __ldcg(reinterpret_cast<const float4*>(src + j));
+                                v[j] += x.x; v[j + 1] += x.y; v[j + 2] += x.z; v[j + 3] += x.w;
+                            }
+                        }
+                    }
+                    write_out = true;
+                }
+            }
+            if (write_out && mine && n < p.N) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    if (j < p.M) {
+                        if (p.y_is_bf16) reinterpret_cast<__nv_bfloat16*>(p.Ybf)[(int64_t)j * p.ldy + n] = __float2bfloat16_rn(v[j] * alpha);
+                        else p.Y[(int64_t)j * p.ldy + n] = v[j] * alpha;
+                    }
+                }
+            }
+        }
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, DEC_TMEM_COLS);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D byte tensor [rows, row_bytes], box = [box_rows, 128 bytes], 128-byte swizzle
+bool make_tmap_u8(CUtensorMap* map, const void* base, int64_t rows, int64_t row_bytes, int box_rows)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) return false;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    cuuint32_t box[2] = {128, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct DecPlan { int64_t tiles, chunks, total; int grid; int maxseg; };
+
+DecPlan decode_plan(int64_t N, int64_t K)
+{
+    DecPlan d;
+    d.tiles = (N + 127) / 128; d.chunks = K / 256; d.total = d.tiles * d.chunks;
+    const int sms = fgmp_sm_count();
+    d.grid = (int)(d.total < sms ? d.total : sms);
+    // a tile of `chunks` units meets at most this many CTA spans of >= floor(total/grid) units
+    const int64_t span = d.total / d.grid;
+    d.maxseg = (int)((d.chunks + span - 1) / span + 1);
+    return d;
+}
+
+}  // namespace
+
+bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K)
+{
+    return M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0;
+}
+
+size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K)
+{
+    if (!fgmp_decode_supported(M, N, K)) return 0;
+    const DecPlan d = decode_plan(N, K);
+    return 1024 + fgmp_align1k((size_t)d.tiles * 32) + (size_t)d.tiles * d.maxseg * 128 * 16 * 4;
+}
+
+fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
+                               int64_t M, int64_t N, int64_t K, void* workspace, cudaStream_t s)
+{
+    const DecPlan d = decode_plan(N, K);
+    uint8_t* ws = (uint8_t*)workspace;
+    DecParams p;
+    p.wblob = (const uint8_t*)packed_weights; p.ablob = (const uint8_t*)packed_acts;
+    p.LW = fgmp_layout(N, K, 1, 0); p.LA = fgmp_layout(M, K, 0, 0);
+    p.Y = (float*)Y; p.Ybf = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16;
+    p.M = M; p.N = N; p.K = K; p.total = d.total; p.chunks = d.chunks;
+    p.status = reinterpret_cast<int*>(ws);
+    p.counters = reinterpret_cast<uint32_t*>(ws + 1024);
+    p.partials = reinterpret_cast<float*>(ws + 1024 + fgmp_align1k((size_t)d.tiles * 32));
+    p.maxseg = d.maxseg;
+
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess)
+            return FGMP_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    CUtensorMap tmW, tmA;
+    if (!make_tmap_u8(&tmW, p.wblob + p.LW.off_codes4, N, K / 2, 128) ||
+        !make_tmap_u8(&tmA, p.ablob + p.LA.off_codes4, M, K / 2, TOK)) return FGMP_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, 1024 + (size_t)d.tiles * 32, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    FGMP_LAUNCH(FGMP_K_DECODE, s, decode_kernel<<<d.grid, DEC_THREADS, DEC_SMEM, s>>>(tmW, tmA, p));
+    return fgmp_launch_status();
+}

@@ -15,6 +15,7 @@
 #include <cuda.h>
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
+#include "fgmp_ptx.cuh"
 
 namespace {
 
@@ -26,7 +27,6 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
     const PackedLayout L = fgmp_layout(rows, K, kind, 0);
     const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const uint32_t* wordptr = reinterpret_cast<const uint32_t*>(blob + L.off_wordptr);
     const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
     const int64_t nblk = rows * L.KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
         float v[16];
         if (is8) {
             size_t src = (kind == 1)
-                ? L.off_codes8 + (size_t)(wordptr[r * L.MW + (kb >> 5)] + __popc(word & ((1u << (kb & 31)) - 1u))) * 16
+                ? L.off_codes8 + (size_t)fgmp_fp8_pos(blob, L, r, kb, word) * 16
                 : L.off_codes8 + (size_t)(r * K + kb * 16);
             uint4 c = *reinterpret_cast<const uint4*>(blob + src);
             const uint32_t w[4] = {c.x, c.y, c.z, c.w};
@@ -63,113 +63,6 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
         dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
         dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
     }
-}
-
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait: gives up after ~2 s (or when another thread of the CTA already gave up),
-// records the failure and returns false.  `abort_flag` lives in shared memory.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
-{
-    const unsigned long long t0 = globaltimer_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > 2000000000ull) {
-            *abort_flag = 1;
-            atomicCAS(status, 0, (int)FGMP_ERR_TIMEOUT);
-            atomicExch(status + 1, where);
-            return false;
-        }
-        __nanosleep(64);
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, where);
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes,
-// 8-row groups 1024 bytes apart (tile base 1024-byte aligned)
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
-{
-    uint64_t d = (uint64_t)((saddr & 0x3ffff) >> 4);
-    d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset: 8 rows x 128 B
-    d |= (uint64_t)1 << 46;                 // descriptor version for sm_100
-    d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
-    return d;
 }
 
 // ------------------------------------------------------------------ bf16 tcgen05 GEMM
@@ -366,6 +259,7 @@ bool make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t K,
 
 size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K)
 {
+    if (fgmp_decode_supported(M, N, K)) return fgmp_ws_decode(M, N, K);
     return 1024 + fgmp_align1k((size_t)M * K * 2) + fgmp_align1k((size_t)N * K * 2);
 }
 
@@ -381,6 +275,8 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     fgmp_status st;
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
     cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (fgmp_decode_supported(M, N, K))
+        return fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, s);
     uint8_t* ws = (uint8_t*)workspace;
     int* status = reinterpret_cast<int*>(ws);
     uint8_t* planeA = ws + 1024;

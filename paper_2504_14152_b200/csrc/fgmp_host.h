@@ -13,6 +13,11 @@ int fgmp_sm_count();
 size_t fgmp_ws_quantize_weights(int64_t N, int64_t K);
 size_t fgmp_ws_calibrate(int64_t M, int64_t K);
 size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K);
+// weight-streaming kernel for M <= 16 tokens and K % 256 == 0
+bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K);
+size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K);
+fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
+                               int64_t M, int64_t N, int64_t K, void* workspace, cudaStream_t s);
 
 // ---- launch accounting (see fgmp_profile_begin in fgmp.h) ----
 enum FgmpKernelId {

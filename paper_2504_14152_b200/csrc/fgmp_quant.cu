@@ -18,6 +18,10 @@ struct ActParams {
     float s4, k6, s8, inv8, tau;
     uint8_t* codes4; uint8_t* sf; uint32_t* mask; uint8_t* codes8;   // codes8: dense plane
     float* scores;                       // optional (score-only kernel)
+    uint4* atrue;                        // optional fp16 copy [KB][16][16] (M <= 16)
+    fgmp_packed_header* header;
+    float r8;                            // 2^ratio
+    int ratio;
     int rows_per_cta;
 };
 
@@ -28,6 +32,22 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     const bool active = kb < p.KB;
     const int64_t m0 = (int64_t)blockIdx.y * p.rows_per_cta;
     const int64_t m1 = min(m0 + (int64_t)p.rows_per_cta, p.M);
+    if (!SCORE_ONLY) {
+        if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+            fgmp_packed_header* h = p.header;
+            h->magic = FGMP_MAGIC; h->version = 1; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+            h->error = 0;
+        }
+        // token rows M..15 of the fp16 copy are zero (the grid covers 16 rows in that mode)
+        if (p.atrue && m0 >= p.M) {
+            if (active) {
+                uint4* dst = p.atrue + (kb * 16 + m0) * 2;
+                dst[0] = make_uint4(0, 0, 0, 0); dst[1] = make_uint4(0, 0, 0, 0);
+            }
+            return;
+        }
+    }
 
     float f[16];
     if (active) {
@@ -73,6 +93,28 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                     *reinterpret_cast<uint4*>(p.codes8 + m * p.K + kb * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
                     c4[0] = 0; c4[1] = 0; sc = 0;
                 }
+                if (p.atrue) {
+                    // value / tensor scale, exact in fp16: E2M1 x microscale or E4M3 x 2^ratio
+                    uint32_t o[8];
+                    if (is8) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float2 a = e4m3x2_to_f32x2(c8[i] & 0xffff), b = e4m3x2_to_f32x2(c8[i] >> 16);
+                            __half2 h0 = __floats2half2_rn(a.x * p.r8, a.y * p.r8), h1 = __floats2half2_rn(b.x * p.r8, b.y * p.r8);
+                            o[2 * i] = *reinterpret_cast<uint32_t*>(&h0); o[2 * i + 1] = *reinterpret_cast<uint32_t*>(&h1);
+                        }
+                    } else {
+                        const float d = e4m3_to_f32(sc);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            float2 q = e2m1x2_to_f32x2((c4[i >> 2] >> ((i & 3) * 8)) & 0xff);
+                            __half2 h = __floats2half2_rn(q.x * d, q.y * d);
+                            o[i] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                    }
+                    uint4* dst = p.atrue + (kb * 16 + m) * 2;
+                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]); dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
                 *reinterpret_cast<uint2*>(p.codes4 + (m * p.K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
                 p.sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)sc;
             }
@@ -85,28 +127,6 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     }
 }
 
-// zero the microscales of the padding rows (rows M .. 128*ceil(M/128)) so that a GEMM that
-// loads whole 128-row scale tiles reads zeros there
-__global__ void sf_pad_zero_kernel(uint8_t* sf, int64_t M, int64_t K)
-{
-    const int64_t Mpad = (M + 127) & ~(int64_t)127;
-    const int64_t KB = K / 16;
-    const int64_t n = (Mpad - M) * KB;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t r = M + i / KB, kb = i % KB;
-        sf[fgmp_sf_offset(r, kb, K)] = 0;
-    }
-}
-
-__global__ void act_header_kernel(fgmp_packed_header* h, int64_t M, int64_t K, float s4, int ratio)
-{
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        h->magic = FGMP_MAGIC; h->version = 1; h->rows = M; h->K = K; h->scale_fp4 = s4;
-        h->fp8_log2_ratio = ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
-        h->error = 0;
-    }
-}
-
 // packed -> canonical arrays; one thread per block
 __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
                               uint8_t* codes4, uint8_t* codes8, uint8_t* scales, uint32_t* mask)
@@ -115,7 +135,6 @@ __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
     const int kind = (int)h->kind;
     const PackedLayout L = fgmp_layout(rows, K, kind, kind ? h->capacity : 0);
     const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const uint32_t* wordptr = reinterpret_cast<const uint32_t*>(blob + L.off_wordptr);
     const int64_t nblk = rows * L.KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
         int64_t r = b / L.KB, kb = b % L.KB;
@@ -132,8 +151,7 @@ __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
             if (is8) {
                 size_t src;
                 if (kind == 1) {
-                    uint32_t pos = wordptr[r * L.MW + (kb >> 5)] + __popc(word & ((1u << (kb & 31)) - 1u));
-                    src = L.off_codes8 + (size_t)pos * 16;
+                    src = L.off_codes8 + (size_t)fgmp_fp8_pos(blob, L, r, kb, word) * 16;
                 } else {
                     src = L.off_codes8 + (size_t)(r * K + kb * 16);
                 }
@@ -149,7 +167,7 @@ fgmp_status check_act_args(const void* X, int64_t ldx, const float* fisher, int6
     if (!X || !fisher) return FGMP_ERR_INVALID_ARG;
     if (sm != 0 && sm != 1) return FGMP_ERR_INVALID_ARG;
     if (!(sc.scale_fp4 > 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc.fp8_log2_ratio < -8 || sc.fp8_log2_ratio > 8) return FGMP_ERR_INVALID_ARG;
+    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
     if (M < 1 || K < 64 || (K % 64) != 0 || ldx < K || (ldx % 8) != 0) return FGMP_ERR_SHAPE;
     if (((uintptr_t)X & 15) || ((uintptr_t)fisher & 15)) return FGMP_ERR_SHAPE;
     return FGMP_OK;
@@ -165,6 +183,8 @@ ActParams make_act_params(const void* X, int64_t ldx, const float* fisher, int64
     p.s8 = ldexpf(sc.scale_fp4, sc.fp8_log2_ratio);
     p.inv8 = 1.0f / p.s8;
     p.tau = tau;
+    p.ratio = sc.fp8_log2_ratio;
+    p.r8 = ldexpf(1.0f, sc.fp8_log2_ratio);
     // enough CTAs to fill the machine when M is small, few row-loop iterations otherwise
     p.rows_per_cta = (M >= 2048) ? 8 : (M >= 256 ? 4 : 1);
     return p;
@@ -191,9 +211,14 @@ extern "C" fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx
     ActParams p = make_act_params(X_bf16, ldx, fisher_chan, M, K, sc, tau);
     p.codes4 = blob + L.off_codes4; p.sf = blob + L.off_sf;
     p.mask = reinterpret_cast<uint32_t*>(blob + L.off_mask); p.codes8 = blob + L.off_codes8;
-    dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((M + p.rows_per_cta - 1) / p.rows_per_cta));
-    FGMP_LAUNCH(FGMP_K_ACT_AUX, s, act_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), M, K, sc.scale_fp4, sc.fp8_log2_ratio));
-    if (M % 128) FGMP_LAUNCH(FGMP_K_ACT_AUX, s, sf_pad_zero_kernel<<<64, 256, 0, s>>>(p.sf, M, K));
+    p.header = reinterpret_cast<fgmp_packed_header*>(blob);
+    int64_t grid_rows = M;
+    if (M <= 16) {                     // decode-sized batch: also emit the fp16 copy, 16 token rows
+        p.atrue = reinterpret_cast<uint4*>(blob + L.off_atrue);
+        p.rows_per_cta = 1;
+        grid_rows = 16;
+    }
+    dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((grid_rows + p.rows_per_cta - 1) / p.rows_per_cta));
     if (sm == FGMP_SCORE_LP_ERROR) FGMP_LAUNCH(FGMP_K_ACT_QUANT, s, quant_act_kernel<0, false><<<grid, QA_THREADS, 0, s>>>(p));
     else                           FGMP_LAUNCH(FGMP_K_ACT_QUANT, s, quant_act_kernel<1, false><<<grid, QA_THREADS, 0, s>>>(p));
     return fgmp_launch_status();

@@ -248,7 +248,8 @@ __global__ void w_mask_kernel(const float* scores, int64_t N, int64_t KB, int64_
 }
 
 // exclusive prefix sum of n uint32 by one CTA of 1024 threads; total -> *total_out (may be NULL)
-__global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t* out, int64_t n, unsigned long long* total_out)
+__global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t* out, int64_t n, unsigned long long* total_out,
+                                                    int append_total)
 {
     __shared__ uint32_t warp_sums[32];
     __shared__ unsigned long long carry_s;
@@ -275,6 +276,30 @@ __global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t
         __syncthreads();
     }
     if (threadIdx.x == 0 && total_out) *total_out = carry_s;
+    if (threadIdx.x == 0 && append_total) out[n] = (uint32_t)carry_s;
+}
+
+// per (128-row tile, 16-block K chunk): rowoff = exclusive prefix over the tile's rows of the
+// number of FP8 blocks each row has in the chunk; ctcnt = their total.  One CTA of 128 threads
+// per (tile, chunk).
+__global__ void __launch_bounds__(128) w_ctcount_kernel(const uint32_t* mask, int64_t N, int64_t MW, int64_t chunks,
+                                                        uint16_t* rowoff, uint32_t* ctcnt)
+{
+    __shared__ uint32_t wsum[4];
+    const int64_t ct = blockIdx.x;
+    const int64_t tile = ct / chunks, chunk = ct % chunks;
+    const int64_t r = tile * 128 + threadIdx.x;
+    uint32_t cnt = 0;
+    if (r < N) cnt = __popc((mask[r * MW + (chunk >> 1)] >> ((chunk & 1) * 16)) & 0xffffu);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    uint32_t incl = cnt;
+    for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+    if (lane == 31) wsum[wid] = incl;
+    __syncthreads();
+    uint32_t base = 0;
+    for (int w = 0; w < wid; ++w) base += wsum[w];
+    rowoff[ct * 128 + threadIdx.x] = (uint16_t)(base + incl - cnt);
+    if (threadIdx.x == 127) ctcnt[ct] = base + incl;
 }
 
 __global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw8, int64_t N, int64_t K, int ratio,
@@ -285,7 +310,6 @@ __global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw
     const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
     const float inv8 = __fdiv_rn(1.0f, s8);
     const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const uint32_t* wordptr = reinterpret_cast<const uint32_t*>(blob + L.off_wordptr);
     const int64_t B = N * L.KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
         int64_t n = b / L.KB, kb = b % L.KB;
@@ -299,7 +323,7 @@ __global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw
             uint32_t c8[4];
             float dq8[16];
             block_fp8(v, inv8, s8, c8, dq8);
-            int64_t pos = (int64_t)wordptr[n * L.MW + (kb >> 5)] + __popc(word & ((1u << (kb & 31)) - 1u));
+            int64_t pos = (int64_t)fgmp_fp8_pos(blob, L, n, kb, word);
             if (pos < capacity)
                 *reinterpret_cast<uint4*>(blob + L.off_codes8 + (size_t)pos * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
         } else {
@@ -354,10 +378,18 @@ void run_select(const float* scores, int64_t B, SelectState* st, cudaStream_t s)
     }
 }
 
+// words in each of the two scratch arrays: one per mask word, or one per (tile, chunk) + 1
+int64_t tmp_words(int64_t N, int64_t K)
+{
+    int64_t KB = K / 16, MW = (KB + 31) / 32;
+    int64_t nct = ((N + 127) / 128) * ((KB + 15) / 16) + 1;
+    return N * MW > nct ? N * MW : nct;
+}
+
 size_t ws_weights_bytes(int64_t N, int64_t K)
 {
-    int64_t KB = K / 16, MW = (KB + 31) / 32, B = N * KB, NW = N * MW;
-    return STATE_BYTES + fgmp_align1k((size_t)B * 4) + fgmp_align1k((size_t)B) + 2 * fgmp_align1k((size_t)NW * 4);
+    int64_t KB = K / 16, MW = (KB + 31) / 32, B = N * KB;
+    return STATE_BYTES + fgmp_align1k((size_t)B * 4) + fgmp_align1k((size_t)B) + 2 * fgmp_align1k((size_t)tmp_words(N, K) * 4);
 }
 
 }  // namespace
@@ -374,7 +406,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     if (!W_bf16 || !fisher_elem || !packed_out || !workspace) return FGMP_ERR_INVALID_ARG;
     if ((int)sm < 0 || (int)sm > 1 || (int)cm < 0 || (int)cm > 1) return FGMP_ERR_INVALID_ARG;
     if (!(sc.scale_fp4 >= 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc.fp8_log2_ratio < -8 || sc.fp8_log2_ratio > 8) return FGMP_ERR_INVALID_ARG;
+    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
     if (fp8_fraction != fp8_fraction || fp8_fraction > 1.0) return FGMP_ERR_INVALID_ARG;
     if (fp8_fraction < 0 && tau != tau) return FGMP_ERR_INVALID_ARG;
     if (N < 1 || K < 64 || (K % 64) != 0 || ldw < K || (ldw % 8) != 0 || ldf < K || (ldf % 4) != 0) return FGMP_ERR_SHAPE;
@@ -405,7 +437,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     float* scores = reinterpret_cast<float*>(ws + STATE_BYTES);
     uint8_t* sc_tmp = ws + STATE_BYTES + fgmp_align1k((size_t)B * 4);
     uint32_t* tmp_a = reinterpret_cast<uint32_t*>(sc_tmp + fgmp_align1k((size_t)B));
-    uint32_t* tmp_b = reinterpret_cast<uint32_t*>((uint8_t*)tmp_a + fgmp_align1k((size_t)NW * 4));
+    uint32_t* tmp_b = reinterpret_cast<uint32_t*>((uint8_t*)tmp_a + fgmp_align1k((size_t)tmp_words(N, K) * 4));
     uint8_t* blob = (uint8_t*)packed_out;
     const uint4* W = reinterpret_cast<const uint4*>(W_bf16);
     const int ratio = sc.fp8_log2_ratio;
@@ -426,18 +458,21 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
         }
     }
     uint32_t* mask = reinterpret_cast<uint32_t*>(blob + L.off_mask);
-    uint32_t* wordptr = reinterpret_cast<uint32_t*>(blob + L.off_wordptr);
+    uint32_t* ctptr = reinterpret_cast<uint32_t*>(blob + L.off_ctptr);
+    uint16_t* rowoff = reinterpret_cast<uint16_t*>(blob + L.off_rowoff);
+    const int64_t NCT = L.tiles * L.chunks;
     const int gw = grid_for(NW * 32, 256, 8);
     if (fraction_mode && k > 0) {
         run_select(scores, B, st, s);
         FGMP_LAUNCH(FGMP_K_W_MASK, s, w_eqcount_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_a));
-        FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, tmp_b, NW, nullptr));
+        FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, tmp_b, NW, nullptr, 0));
     } else {
         // k == 0: nothing is FP8 (tau_eff = +inf); threshold mode: the given tau
         FGMP_LAUNCH(FGMP_K_W_AUX, s, set_tau_kernel<<<1, 32, 0, s>>>(st, fraction_mode ? INFINITY : tau));
     }
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a));
-    FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, wordptr, NW, &st->n_fp8));
+    FGMP_LAUNCH(FGMP_K_W_MASK, s, w_ctcount_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, N, MW, L.chunks, rowoff, tmp_a));
+    FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, ctptr, NCT, &st->n_fp8, 1));
     FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, ratio, st, sc_tmp, blob, L, capacity));
     FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, N, K, ratio, capacity,
                                      fraction_mode ? 1 : 0, tau, tau_eff_out));

@@ -262,3 +262,40 @@ def test_linear_prefill_shape_sampled(fg):
     # two runs give the same bits
     y2 = fg.linear(pa, pw).cpu().numpy().astype(np.float64)
     assert np.array_equal(y, y2)
+
+
+# ------------------------------------------------------------ decode kernel (M <= 16)
+
+@pytest.mark.parametrize("frac_a,frac_w", [(0.0, 0.0), (0.1, 0.1), (0.0, 0.1), (0.1, 0.0), (1.0, 1.0), (0.0, 1.0),
+                                            (1.0, 0.0), (0.3, 0.3)])
+@pytest.mark.parametrize("M", [16, 5])
+def test_decode_kernel_block_pair_cases(fg, M, frac_a, frac_w):
+    """Weight-streaming path: every combination of block formats, full output against the oracle.
+    30% FP8 exceeds the staged FP8 capacity of a pipeline stage and takes the global-memory route."""
+    wl = gi.llama("d", M, 640, 1024, seed=11)
+    qa, qw, pa, pw = quantize_both(fg, wl, frac_a, frac_w, clip=False)
+    Y, S = oracle.linear(qa, qw)
+    y = fg.linear(pa, pw)
+    fg.check(fg.linear.last_workspace)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - Y)
+    assert (err <= GEMM_TOL * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    assert (err <= 1e-5 * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    y2 = fg.linear(pa, pw)
+    assert torch.equal(y, y2), "stream-K reduction must be deterministic"
+    yb = fg.linear(pa, pw, out_dtype=torch.bfloat16).float().cpu().numpy().astype(np.float64)
+    assert (np.abs(yb - Y) <= GEMM_TOL * S + np.abs(Y) * 2.0 ** -8 + 1e-30).all()
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 11008, 4096), (16, 4096, 11008), (8, 300, 256), (2, 129, 5120), (16, 13824, 5120)])
+def test_decode_kernel_shapes(fg, M, N, K):
+    wl = gi.llama("d", M, N, K, seed=4)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    y = fg.linear(pa, pw).cpu().numpy().astype(np.float64)
+    fg.check(fg.linear.last_workspace)
+    rng = np.random.default_rng(0)
+    ms = np.r_[rng.integers(0, M, 6000), [0, M - 1, 0, M - 1]]
+    nn = np.r_[rng.integers(0, N, 6000), [0, N - 1, N - 1, 0]]
+    Y, S = oracle.linear_sampled(qa, qw, ms, nn)
+    err = np.abs(y[ms, nn] - Y)
+    assert (err <= GEMM_TOL * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    assert np.isfinite(y).all()
