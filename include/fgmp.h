@@ -147,6 +147,31 @@ fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
                         void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                         void* workspace, size_t ws_bytes, void* cuda_stream);
 
+/* ---- fgmp_linear for callers that cannot allocate (the paper has no counterpart) ----
+ * Some callers have no way to hand the library a workspace: code that runs where cudaMalloc is
+ * forbidden (inside a region that must not touch the allocator, a host that pre-sized its
+ * memory pool and gave all of it away, a plugin interface with no scratch argument).  This
+ * variant of fgmp_linear for decode-sized batches (1 <= M <= 16 tokens, K % 256 == 0) keeps its
+ * scratch -- status word, stream-K tile counters and partial sums -- in a fixed array inside the
+ * library image instead: FGMP_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the
+ * library, held until the process exits.  It calls no allocation routine of any kind.
+ *   - Inputs and outputs are passed as for fgmp_linear; results are bit-identical to it.
+ *   - Shapes whose scratch need (fgmp_workspace_bytes(FGMP_OP_LINEAR, M, N, K)) exceeds
+ *     FGMP_STATIC_SCRATCH_BYTES return FGMP_ERR_WORKSPACE; M > 16 or K % 256 != 0 returns
+ *     FGMP_ERR_SHAPE.  Llama-2-70B FC1/FC2 (28672 x 8192) needs 3.5 MiB and fits.
+ *   - The first call on each device looks up the array's device address (a host-side query,
+ *     made with that device current); make that first call outside any stream capture.
+ *   - All calls on one GPU share the array and each call starts by clearing the part that
+ *     must be zero, so calls must not overlap on the GPU: two calls in flight at once (two
+ *     streams, two host threads) race on the scratch and give wrong results.  Calls ordered
+ *     on one stream are fine.
+ *   - status_out (device, 2 x int32, may be NULL) receives what fgmp_check would report for
+ *     this call: word 0 = FGMP_OK or FGMP_ERR_TIMEOUT, copied on the stream after the kernel. */
+#define FGMP_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+fgmp_status fgmp_linear_static(const void* packed_acts, const void* packed_weights,
+                               void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                               int32_t* status_out, void* cuda_stream);
+
 /* Synchronizes the stream and returns the device-side status recorded in a workspace used
  * by fgmp_linear (FGMP_OK or FGMP_ERR_TIMEOUT). */
 fgmp_status fgmp_check(const void* workspace, void* cuda_stream);

@@ -56,6 +56,8 @@ def _load():
     L.fgmp_calibrate_tau.argtypes = [vp, i64, vp, i64, i64, _Scales, ci, f64, vp, vp, sz, vp]
     L.fgmp_linear.restype = ci
     L.fgmp_linear.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp]
+    L.fgmp_linear_static.restype = ci
+    L.fgmp_linear_static.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, vp]
     L.fgmp_check.restype = ci
     L.fgmp_check.argtypes = [vp, vp]
     L.fgmp_unpack.restype = ci
@@ -216,6 +218,24 @@ def linear(acts: PackedTensor, weights: PackedTensor, *, out_dtype=torch.float32
                       1 if out.dtype == torch.bfloat16 else 0, out.stride(0), M, N, K,
                       workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear")
     linear.last_workspace = workspace
+    return out
+
+
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+def linear_static(acts: PackedTensor, weights: PackedTensor, *, out: torch.Tensor,
+                  status_out: torch.Tensor | None = None) -> torch.Tensor:
+    """fgmp_linear_static: the decode-sized GEMM for callers that cannot allocate.  The scratch
+    lives inside the library, so nothing is allocated here either: `out` (and `status_out`,
+    int32[2], optional) must be given.  Calls must not overlap on the GPU."""
+    L = _load()
+    assert acts.K == weights.K and acts.kind == 0 and weights.kind == 1
+    assert out.dtype in (torch.float32, torch.bfloat16)
+    M, N, K = acts.rows, weights.rows, acts.K
+    _ok(L.fgmp_linear_static(acts.blob.data_ptr(), weights.blob.data_ptr(), out.data_ptr(),
+                             1 if out.dtype == torch.bfloat16 else 0, out.stride(0), M, N, K,
+                             _ptr(status_out), _stream()), "fgmp_linear_static")
     return out
 
 

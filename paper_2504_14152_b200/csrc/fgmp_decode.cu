@@ -432,3 +432,41 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     FGMP_LAUNCH(FGMP_K_DECODE, s, decode_kernel<<<d.grid, DEC_THREADS, DEC_SMEM, s>>>(tmW, tmA, p));
     return fgmp_launch_status();
 }
+
+// ------------------------------------------------------------------ allocation-free variant
+// Scratch of fgmp_linear_static: one array per GPU that loads the library, held until exit.
+static __device__ __align__(256) unsigned char g_static_scratch[FGMP_STATIC_SCRATCH_BYTES];
+
+extern "C" fgmp_status fgmp_linear_static(const void* packed_acts, const void* packed_weights,
+                                          void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                          int32_t* status_out, void* cuda_stream)
+{
+    if (!packed_acts || !packed_weights || !Y) return FGMP_ERR_INVALID_ARG;
+    if (M < 1 || N < 1 || K < 64 || (K % 64) != 0 || ldy < N) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)Y & 15) ||
+        ((uintptr_t)status_out & 3)) return FGMP_ERR_SHAPE;
+    if (!fgmp_decode_supported(M, N, K)) return FGMP_ERR_SHAPE;
+    if (fgmp_ws_decode(M, N, K) > (size_t)FGMP_STATIC_SCRATCH_BYTES) return FGMP_ERR_WORKSPACE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+
+    // The array's name is only a host-side handle; the kernel needs its device address, which
+    // differs per GPU.  Looked up once per device, with that device current.
+    static void* scratch_of_device[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
+    if (!scratch_of_device[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return FGMP_ERR_CUDA;
+        scratch_of_device[dev] = ptr;
+    }
+    void* scratch = scratch_of_device[dev];
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // fgmp_linear_decode zeroes the status word and the tile counters at the start of the
+    // scratch; the partial sums behind them are always written before they are read.
+    st = fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, scratch, s);
+    if (st != FGMP_OK) return st;
+    if (status_out && cudaMemcpyAsync(status_out, scratch, 2 * sizeof(int32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return FGMP_ERR_CUDA;
+    return FGMP_OK;
+}
