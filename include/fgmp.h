@@ -31,15 +31,17 @@
  *                   0x00 for FP8 blocks and for padding rows
  *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
  *                   1 = FP8
- *   ctptr, rowoff : (weights only) index of the FP8 list: ctptr[t*C + c] (uint32, C = ceil(K/256))
- *                   = list position of the first FP8 block of 128-row tile t and 256-element
- *                   K chunk c; rowoff[(t*C + c)*128 + r%128] (uint16) = offset of row r's
- *                   first FP8 block inside that (tile, chunk)
+ *   ctptr, kbcnt  : (weights only) index of the FP8 list.  A unit = one 128-row tile t x one
+ *                   256-element K chunk c (C = ceil(K/256) chunks per tile).
+ *                   ctptr[t*C + c] (uint32, one extra entry at the end) = list position of the
+ *                   unit's first FP8 block; kbcnt[(t*C + c)*16 + j] (uint8) = how many of the
+ *                   unit's FP8 blocks lie in its j-th block column
  *   atrue         : (activations with rows <= 16 only) fp16 copy of the quantized values
  *                   divided by the tensor scale, [K/16][16 tokens][16]; rows >= M are zero
- *   codes8        : weights: the FP8 blocks only, 16 bytes each, ordered by (tile, chunk, row,
- *                   block) (capacity max_fp8_blocks); activations: a dense rows*K byte plane
- *                   of which only the FP8 blocks are written.
+ *   codes8        : weights: the FP8 blocks only, 16 bytes each, ordered by (tile, chunk, block
+ *                   column, row) (capacity max_fp8_blocks); activations: a dense rows*K byte
+ *                   plane of which only the FP8 blocks are written.
+ *   rowid         : (weights only) capacity + 32 bytes: row inside its tile of every list entry
  */
 #ifndef FGMP_H
 #define FGMP_H
@@ -81,7 +83,7 @@ typedef struct {
 /* First 256 bytes of a packed blob (device memory). */
 typedef struct {
     uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
-    uint32_t version;        /* layout version, 1                                           */
+    uint32_t version;        /* layout version, 2                                           */
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;

@@ -10,17 +10,19 @@
 #define FGMP_BS 16
 
 // ---------------------------------------------------------------- blob layout
-// Weights keep their FP8 blocks in a compact list ordered by (128-row tile, 256-element K
-// chunk, row, block): the blocks one GEMM CTA needs for one pipeline stage are contiguous.
-//   ctptr [tiles*chunks + 1] uint32 : list index of the first FP8 block of each (tile, chunk)
-//   rowoff[tiles*chunks*128] uint16 : offset of a row's first FP8 block inside its (tile, chunk)
+// Weights keep their FP8 blocks in a compact list.  A "unit" is one 128-row tile x one chunk of
+// 16 blocks (256 K elements); the list is ordered by (tile, chunk, block, row), so all FP8
+// blocks that meet the same 16 activation elements are neighbours.
+//   ctptr [units + 1]     uint32 : list index of the first FP8 block of each unit
+//   kbcnt [units * 16]    uint8  : number of FP8 blocks of the unit in each of its 16 block columns
+//   rowid [capacity + 32] uint8  : row (inside its tile) of every list entry
 // Activations keep a dense FP8 plane (only FP8 blocks are written) and, when rows <= 16, a
 // dequantized fp16 copy `atrue` laid out [K/16 blocks][16 tokens][16 elements] whose values
 // are value / tensor scale (E2M1 x microscale, or E4M3 x 2^ratio); rows >= M are zero.
 struct PackedLayout {
     int64_t rows, K, KB, MW;          // KB = K/16 blocks per row, MW = mask words per row
     int64_t tiles, chunks;            // 128-row tiles, 16-block K chunks
-    size_t off_codes4, off_sf, off_mask, off_ctptr, off_rowoff, off_atrue, off_codes8, total;
+    size_t off_codes4, off_sf, off_mask, off_ctptr, off_kbcnt, off_rowid, off_atrue, off_codes8, total;
 };
 
 __host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
@@ -36,10 +38,12 @@ __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int
     L.off_sf = o;      o = fgmp_align1k(o + (size_t)L.tiles * (size_t)(K / 64) * 512);
     L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
     L.off_ctptr = o;   if (kind == 1) o = fgmp_align1k(o + ((size_t)L.tiles * L.chunks + 1) * 4);
-    L.off_rowoff = o;  if (kind == 1) o = fgmp_align1k(o + (size_t)L.tiles * L.chunks * 128 * 2);
+    L.off_kbcnt = o;   if (kind == 1) o = fgmp_align1k(o + (size_t)L.tiles * L.chunks * 16);
     L.off_atrue = o;   if (kind == 0 && rows <= 16) o = fgmp_align1k(o + (size_t)L.KB * 512);
+    // the variable-size sections come last so that every fixed offset is independent of capacity
     L.off_codes8 = o;
     o = fgmp_align1k(o + (kind == 1 ? (size_t)capacity * 16 : (size_t)rows * (size_t)K));
+    L.off_rowid = o;   if (kind == 1) o = fgmp_align1k(o + (size_t)capacity + 32);
     L.total = o;
     return L;
 }
@@ -52,15 +56,62 @@ __host__ __device__ inline size_t fgmp_sf_offset(int64_t r, int64_t kb, int64_t 
 }
 
 #ifdef __CUDACC__
-// list index of FP8 block (r, kb) of a packed weight tensor; `word` is the row's mask word
-// that holds kb
-__device__ __forceinline__ uint32_t fgmp_fp8_pos(const uint8_t* blob, const PackedLayout& L, int64_t r, int64_t kb, uint32_t word)
+// Where the FP8 blocks of one unit sit in the list.  Called by all 128 threads of a CTA, thread
+// i = row i of the tile, m16 = that row's 16 mask bits of the chunk (0 beyond the last row).
+// On return s_pos[row * 16 + kb] = offset of block (row, kb) from the unit's first list entry
+// (0xffff if the block is not FP8), s_cnt[kb] = FP8 blocks in column kb, and the return value
+// is their total.  s_warp is scratch of 64 words.  Ends with a __syncthreads().
+__device__ __forceinline__ uint32_t fgmp_unit_positions(uint32_t m16, uint32_t* s_warp, uint16_t* s_pos, uint32_t* s_cnt)
 {
-    const int64_t ct = (r >> 7) * L.chunks + (kb >> 4);
-    const uint32_t half = (word >> (((kb >> 4) & 1) * 16)) & 0xffffu;
-    const uint32_t* ctptr = reinterpret_cast<const uint32_t*>(blob + L.off_ctptr);
-    const uint16_t* rowoff = reinterpret_cast<const uint16_t*>(blob + L.off_rowoff);
-    return ctptr[ct] + rowoff[ct * 128 + (r & 127)] + __popc(half & ((1u << (kb & 15)) - 1u));
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t rank[16];
+#pragma unroll
+    for (int kb = 0; kb < 16; ++kb) {
+        const uint32_t bal = __ballot_sync(0xffffffffu, (m16 >> kb) & 1u);
+        rank[kb] = __popc(bal & ((1u << lane) - 1u));
+        if (lane == 0) s_warp[w * 16 + kb] = __popc(bal);
+    }
+    __syncthreads();
+    uint32_t run = 0;
+#pragma unroll
+    for (int kb = 0; kb < 16; ++kb) {
+        const uint32_t c0 = s_warp[kb], c1 = s_warp[16 + kb], c2 = s_warp[32 + kb], c3 = s_warp[48 + kb];
+        const uint32_t below = (w > 0 ? c0 : 0u) + (w > 1 ? c1 : 0u) + (w > 2 ? c2 : 0u);
+        s_pos[threadIdx.x * 16 + kb] = ((m16 >> kb) & 1u) ? (uint16_t)(run + below + rank[kb]) : (uint16_t)0xffff;
+        if (threadIdx.x == 0) s_cnt[kb] = c0 + c1 + c2 + c3;
+        run += c0 + c1 + c2 + c3;
+    }
+    __syncthreads();
+    return run;
+}
+
+// the 16 mask bits of (row r, chunk c) of a packed tensor; 0 beyond the last row
+__device__ __forceinline__ uint32_t fgmp_chunk_mask(const uint32_t* mask, const PackedLayout& L, int64_t r, int64_t c)
+{
+    if (r >= L.rows) return 0u;
+    return (mask[r * L.MW + (c >> 1)] >> ((c & 1) * 16)) & 0xffffu;
+}
+
+// Visits every FP8 block of one unit of a packed weight tensor: f(row, kb, list index, row in tile).
+// Called by all 128 threads of a CTA; consecutive threads visit consecutive blocks of one row.
+struct UnitScratch { uint32_t warp[64]; uint32_t cnt[16]; uint16_t pos[128 * 16]; };
+template <class F>
+__device__ __forceinline__ void fgmp_for_each_fp8_block(const uint8_t* blob, const PackedLayout& L, int64_t unit,
+                                                        UnitScratch& sc, F f)
+{
+    const int64_t tile = unit / L.chunks, c = unit % L.chunks;
+    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
+    fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    const uint32_t base = reinterpret_cast<const uint32_t*>(blob + L.off_ctptr)[unit];
+    const int kb = threadIdx.x & 15;
+#pragma unroll 1
+    for (int j = 0; j < 16; ++j) {
+        const int row = (threadIdx.x >> 4) + 8 * j;
+        const uint32_t pos = sc.pos[row * 16 + kb];
+        if (pos != 0xffffu) f(tile * 128 + row, c * 16 + kb, base + pos, row);
+    }
+    __syncthreads();
 }
 #endif
 

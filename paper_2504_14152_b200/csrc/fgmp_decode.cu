@@ -4,16 +4,21 @@
 //
 // Decomposition (exact).  With A4z / W4z the NVFP4 planes (zero in FP8 blocks), W8 the FP8
 // blocks of the weights and At the true activation values (fp16 copy, either format):
-//     Y = A4z.W4z^T            tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
-//                              weights are the 128-row MMA operand, the 16 tokens are N
-//       + At.W8^T              only where a weight block is FP8   } mma.sync m16n8k16 on
-//       + At[FP8 blocks].W4z^T only where an activation block is FP8 } gathered 8-row groups
+//     Y = A4z.W4z^T            (1) tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
+//                                  weights are the 128-row MMA operand, the 16 tokens are N
+//       + At.W8^T              (2) the FP8 weight blocks, which the list keeps grouped by block
+//                                  column: eight blocks that meet the same 16 activation
+//                                  elements form one mma.sync m16n8k16; results are scattered
+//                                  to their rows in a tile private to the warp
+//       + At[FP8 blocks].W4z^T (3) only block columns in which some token is FP8: the NVFP4
+//                                  weights of the stage are dequantized for mma.sync
 // Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all
 // SMs stream the same number of bytes; tiles shared by several CTAs are reduced in a fixed
-// order by the CTA that arrives last (deterministic).
+// order by the CTA that arrives last.  Every sum is taken in a fixed order: results are
+// reproducible bit for bit.
 //
 // Warp roles (320 threads): warp 0 = producer (TMA tensor + bulk copies), warp 1 = MMA issuer
-// and TMEM owner, warps 2-9 = FP8 corrections on CUDA-core-fed mma.sync, then epilogue.
+// and TMEM owner, warps 2-9 = corrections (2) and (3), then epilogue.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
@@ -28,14 +33,16 @@ constexpr uint32_t W4_BYTES = 128 * 128;        // 128 rows x 256 E2M1
 constexpr uint32_t A4_BYTES = TOK * 128;
 constexpr uint32_t SF_BYTES = 2048;             // 4 scale tiles of 512 B
 constexpr uint32_t ATRUE_BYTES = 16 * 512;      // 16 blocks x 16 tokens x 16 fp16
+constexpr uint32_t FP8_CAP_BLOCKS = 320;        // staged FP8 blocks per unit; more are read from global
+constexpr uint32_t ROWID_BYTES = FP8_CAP_BLOCKS + 16;
 constexpr uint32_t OFF_A4 = W4_BYTES, OFF_SFW = OFF_A4 + A4_BYTES, OFF_SFA = OFF_SFW + SF_BYTES,
-                   OFF_ATRUE = OFF_SFA + SF_BYTES, OFF_FP8 = OFF_ATRUE + ATRUE_BYTES;      // 30720
-constexpr uint32_t FP8_CAP_BLOCKS = 512;        // staged FP8 blocks per (tile, chunk); more are read from global
-constexpr uint32_t DEC_STAGE_BYTES = OFF_FP8 + FP8_CAP_BLOCKS * 16;                       // 38912
-constexpr int DEC_STAGES = 5;
-constexpr int CORR_LD = 17;                     // padded row of the correction tile (floats)
-constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 16 accumulator columns + 5 stages x 32 scale columns
-constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + 128 * CORR_LD * 4 + 1024 + 512;
+                   OFF_ATRUE = OFF_SFA + SF_BYTES, OFF_FP8 = OFF_ATRUE + ATRUE_BYTES,      // 30720
+                   OFF_ROWID = OFF_FP8 + FP8_CAP_BLOCKS * 16, OFF_KBCNT = OFF_ROWID + ROWID_BYTES;
+constexpr uint32_t DEC_STAGE_BYTES = (OFF_KBCNT + 16 + 1023) & ~1023u;                     // 36864
+constexpr int DEC_STAGES = 4;
+constexpr uint32_t PRIV_FLOATS = 128 * TOK;     // one [row][token] tile per correction warp
+constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 16 accumulator columns + 4 stages x 32 scale columns
+constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + DEC_CORR_WARPS * PRIV_FLOATS * 4 + 1024 + 512;
 
 // kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
 constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
@@ -54,29 +61,46 @@ struct StageMeta { uint32_t p0, cnt; };
 
 __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
 
+__device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return __dp4a(x, 0x01010101u, 0u); }
+
+// fire-and-forget add to a float in shared memory
+__device__ __forceinline__ void red_add(float* p, float v)
+{
+    asm volatile("red.shared::cta.add.f32 [%0], %1;" ::"r"(smem_u32(p)), "f"(v) : "memory");
+}
+
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, DecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    float* corr = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(corr) + 128 * CORR_LD * 4);
-    // bars: [0,S) full, [S,2S) empty, [2S,2S+2) acc_full, [2S+2,2S+4) acc_empty
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES + 4);
+    float* priv = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(priv + DEC_CORR_WARPS * PRIV_FLOATS);
+    // bars: [0,S) full, [S,2S) empty, [2S,2S+2) acc_full, [2S+2,2S+4) acc_empty, [2S+4,2S+6) segment syncs
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES + 6);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + DEC_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + DEC_STAGES);
     const uint32_t accf0 = smem_u32(bars + 2 * DEC_STAGES), acce0 = smem_u32(bars + 2 * DEC_STAGES + 2);
+    const uint32_t seg0 = smem_u32(bars + 2 * DEC_STAGES + 4);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + DEC_CORR_WARPS); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 32 * DEC_CORR_WARPS); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 32 * DEC_CORR_WARPS);
+            mbar_init(seg0 + 8 * b, 32 * DEC_CORR_WARPS);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
+    if (warp >= 2) {                                   // the private tiles start at zero
+        float4* z = reinterpret_cast<float4*>(priv + (warp - 2) * PRIV_FLOATS);
+#pragma unroll
+        for (int i = 0; i < (int)PRIV_FLOATS / 128; ++i) z[i * 32 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -86,6 +110,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     const int64_t G = gridDim.x, C = p.chunks;
     const int64_t u_begin = ((int64_t)blockIdx.x * p.total) / G, u_end = ((int64_t)(blockIdx.x + 1) * p.total) / G;
     const uint32_t* ctptr = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_ctptr);
+    const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+    // the row-id section lies behind the FP8 list, whose room the header records
+    const uint8_t* rowid_g = p.wblob + fgmp_align1k(p.LW.off_codes8 + (size_t)hw->capacity * 16);
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -95,6 +122,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
             const uint8_t* sfa = p.ablob + p.LA.off_sf;
             const uint8_t* atrue = p.ablob + p.LA.off_atrue;
             const uint8_t* fp8 = p.wblob + p.LW.off_codes8;
+            const uint8_t* kbcnt = p.wblob + p.LW.off_kbcnt;
             uint32_t nxt0 = 0, nxt1 = 0;
             if (u_begin < u_end) { nxt0 = __ldg(ctptr + u_begin); nxt1 = __ldg(ctptr + u_begin + 1); }
             for (int64_t u = u_begin; u < u_end; ++u) {
@@ -103,16 +131,22 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
                 if (u + 1 < u_end) { nxt0 = p1; nxt1 = __ldg(ctptr + u + 2); }
                 if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) break;
                 const uint32_t cnt = p1 - p0, staged = cnt < FP8_CAP_BLOCKS ? cnt : FP8_CAP_BLOCKS;
+                // row ids: whole 16-byte lines around [p0, p0 + staged)
+                const uint32_t rid_bytes = staged ? (((p0 & 15u) + staged + 15u) & ~15u) : 0u;
                 smeta[stage].p0 = p0; smeta[stage].cnt = cnt;
                 const uint32_t fb = full0 + 8 * stage;
                 const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
-                mbar_expect_tx(fb, OFF_FP8 + staged * 16);
+                mbar_expect_tx(fb, OFF_FP8 + staged * 16 + rid_bytes + 16);
                 tma_load_2d(sb, &tmW, (int32_t)(c * 128), (int32_t)(tile * 128), fb);
                 tma_load_2d(sb + OFF_A4, &tmA, (int32_t)(c * 128), 0, fb);
                 bulk_load(sb + OFF_SFW, sfw + ((size_t)tile * (p.K >> 6) + (size_t)c * 4) * 512, SF_BYTES, fb);
                 bulk_load(sb + OFF_SFA, sfa + (size_t)c * 4 * 512, SF_BYTES, fb);
                 bulk_load(sb + OFF_ATRUE, atrue + (size_t)c * ATRUE_BYTES, ATRUE_BYTES, fb);
-                if (staged) bulk_load(sb + OFF_FP8, fp8 + (size_t)p0 * 16, staged * 16, fb);
+                bulk_load(sb + OFF_KBCNT, kbcnt + (size_t)u * 16, 16, fb);
+                if (staged) {
+                    bulk_load(sb + OFF_FP8, fp8 + (size_t)p0 * 16, staged * 16, fb);
+                    bulk_load(sb + OFF_ROWID, rowid_g + (p0 & ~15u), rid_bytes, fb);
+                }
                 if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
             }
         }
@@ -155,126 +189,137 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     } else {
         // ------------------------------------------------------------ corrections + epilogue
         // A warp may read TMEM lanes [32q, 32q+32), q = warp % 4; two warps share a quadrant and
-        // each owns 16 of its rows, for the corrections and for the epilogue alike, so that the
-        // correction sums never cross warps.
-        const int q = warp & 3, h = (warp - 2) >> 2;
+        // each owns 16 of its rows for correction (3) and for the epilogue.
+        const int cw = warp - 2;                       // 0..7
+        const int q = warp & 3, h = cw >> 2;
         const int rowbase = 32 * q + 16 * h;           // first owned row inside the tile
         const int slice = 2 * q + h;                   // 0..7
         const int g = lane >> 2, t = lane & 3;
-        const uint32_t* wmask = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_mask);
-        const uint16_t* rowoff = reinterpret_cast<const uint16_t*>(p.wblob + p.LW.off_rowoff);
         const uint32_t* amask = reinterpret_cast<const uint32_t*>(p.ablob + p.LA.off_mask);
-        const uint8_t* fp8 = p.wblob + p.LW.off_codes8;
+        const uint8_t* fp8_g = p.wblob + p.LW.off_codes8;
         const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
-        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
         const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
-        const int64_t MWw = p.LW.MW, MWa = p.LA.MW;
+        const int64_t MWa = p.LA.MW;
         const bool tok0 = g < p.M, tok1 = g + 8 < p.M;
-        float* mycorr = corr + rowbase * CORR_LD;
+        float* mypriv = priv + cw * PRIV_FLOATS;
 
         int stage = 0; uint32_t phase = 0; bool ok = true;
         int seg = 0;
         for (int64_t u = u_begin; u < u_end && ok; ++seg) {
             const int64_t tile = u / C;
             const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
-            const int64_t n0 = tile * 128 + rowbase + g, n1 = n0 + 8;       // own rows (B fragments)
             float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 
-            // per-chunk metadata of the own rows / tokens, fetched one chunk ahead
-            uint32_t wm[2], ro[2], am[2];
-            auto fetch_meta = [&](int64_t uu, uint32_t (&wm_)[2], uint32_t (&ro_)[2], uint32_t (&am_)[2]) {
+            // activation mask bits of tokens g and g+8 for the chunk, fetched one unit ahead
+            uint32_t am[2];
+            auto fetch_meta = [&](int64_t uu, uint32_t (&am_)[2]) {
                 const int64_t c = uu % C;
                 const int sh = (int)(c & 1) * 16;
-                wm_[0] = n0 < p.N ? (__ldg(wmask + n0 * MWw + (c >> 1)) >> sh) & 0xffffu : 0u;
-                wm_[1] = n1 < p.N ? (__ldg(wmask + n1 * MWw + (c >> 1)) >> sh) & 0xffffu : 0u;
-                ro_[0] = __ldg(rowoff + uu * 128 + rowbase + g);
-                ro_[1] = __ldg(rowoff + uu * 128 + rowbase + 8 + g);
                 am_[0] = tok0 ? (__ldg(amask + (int64_t)g * MWa + (c >> 1)) >> sh) & 0xffffu : 0u;
                 am_[1] = tok1 ? (__ldg(amask + (int64_t)(g + 8) * MWa + (c >> 1)) >> sh) & 0xffffu : 0u;
             };
-            fetch_meta(u, wm, ro, am);
+            fetch_meta(u, am);
 
             for (; u < seg_end; ++u) {
-                uint32_t wm_n[2] = {0, 0}, ro_n[2] = {0, 0}, am_n[2] = {0, 0};
-                if (u + 1 < seg_end) fetch_meta(u + 1, wm_n, ro_n, am_n);
-                // which blocks of this chunk need work at all (any of the 8 rows / 16 tokens)
-                uint32_t ow0 = wm[0], ow1 = wm[1], oa = am[0] | am[1];
+                uint32_t am_n[2] = {0, 0};
+                if (u + 1 < seg_end) fetch_meta(u + 1, am_n);
+                uint32_t oa = am[0] | am[1];           // block columns in which any token is FP8
 #pragma unroll
-                for (int o = 4; o < 32; o <<= 1) {
-                    ow0 |= __shfl_xor_sync(0xffffffffu, ow0, o);
-                    ow1 |= __shfl_xor_sync(0xffffffffu, ow1, o);
-                    oa |= __shfl_xor_sync(0xffffffffu, oa, o);
-                }
+                for (int o = 4; o < 32; o <<= 1) oa |= __shfl_xor_sync(0xffffffffu, oa, o);
                 if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint32_t list0 = smeta[stage].p0;
-                uint32_t todo = ow0 | ow1 | oa;
+                const uint32_t shift = list0 & 15u;
+
+                // (2) FP8 weight blocks of block columns cw and cw + 8
+                const uint4 kc = *reinterpret_cast<const uint4*>(sb + OFF_KBCNT);
+                const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int kb = cw + 8 * hh, wi = kb >> 2, sh8 = (kb & 3) * 8;
+                    const uint32_t word = wi == 0 ? kc.x : (wi == 1 ? kc.y : (wi == 2 ? kc.z : kc.w));
+                    const uint32_t start = (wi > 0 ? ks0 : 0u) + (wi > 1 ? ks1 : 0u) + (wi > 2 ? ks2 : 0u)
+                                         + byte_sum(word & ((1u << sh8) - 1u));
+                    const uint32_t end = start + ((word >> sh8) & 0xffu);
+                    if (start == end) continue;
+                    const uint2 at0 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + g * 32 + t * 8);
+                    const uint2 at1 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + (g + 8) * 32 + t * 8);
+                    for (uint32_t e = start; e < end; e += 8) {
+                        const uint32_t idx = e + g;
+                        uint32_t raw = 0;
+                        if (idx < end) {
+                            if (idx < FP8_CAP_BLOCKS) raw = *reinterpret_cast<const uint32_t*>(sb + OFF_FP8 + idx * 16 + t * 4);
+                            else raw = __ldg(reinterpret_cast<const uint32_t*>(fp8_g + ((size_t)list0 + idx) * 16 + t * 4));
+                        }
+                        uint32_t h0, h1;
+                        const uint16_t lo = (uint16_t)raw, hi = (uint16_t)(raw >> 16);
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(lo));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(hi));
+                        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), rw2), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), rw2);
+                        float c[4] = {0.f, 0.f, 0.f, 0.f};
+                        mma_f16_16816(c, at0.x, at1.x, at0.y, at1.y, *reinterpret_cast<const uint32_t*>(&x0), *reinterpret_cast<const uint32_t*>(&x1));
+                        // c[0], c[2]: list entry e + 2t for tokens g, g + 8; c[1], c[3]: entry e + 2t + 1
+                        const uint32_t i0 = e + 2 * t, i1 = i0 + 1;
+                        if (i0 < end) {
+                            const uint32_t r0 = i0 < FP8_CAP_BLOCKS ? sb[OFF_ROWID + shift + i0] : __ldg(rowid_g + list0 + i0);
+                            red_add(mypriv + r0 * TOK + g, c[0]);
+                            red_add(mypriv + r0 * TOK + g + 8, c[2]);
+                        }
+                        if (i1 < end) {
+                            const uint32_t r1 = i1 < FP8_CAP_BLOCKS ? sb[OFF_ROWID + shift + i1] : __ldg(rowid_g + list0 + i1);
+                            red_add(mypriv + r1 * TOK + g, c[1]);
+                            red_add(mypriv + r1 * TOK + g + 8, c[3]);
+                        }
+                    }
+                }
+
+                // (3) FP8 activation blocks against the NVFP4 weights of the warp's 16 rows
+                uint32_t todo = oa;
                 while (todo) {
                     const int kb = __ffs(todo) - 1;
                     todo &= todo - 1;
                     const uint32_t bit = 1u << kb;
-                    // A fragment: true activation values of tokens g and g+8, elements 4t..4t+3 of block kb
                     const uint2 at0 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + g * 32 + t * 8);
                     const uint2 at1 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + (g + 8) * 32 + t * 8);
-                    // (1) FP8 weight blocks
+                    const uint32_t a0 = (am[0] & bit) ? at0.x : 0u, a2 = (am[0] & bit) ? at0.y : 0u;
+                    const uint32_t a1 = (am[1] & bit) ? at1.x : 0u, a3 = (am[1] & bit) ? at1.y : 0u;
 #pragma unroll
                     for (int rg = 0; rg < 2; ++rg) {
-                        if (!((rg ? ow1 : ow0) & bit)) continue;
-                        uint32_t b0 = 0, b1 = 0;
-                        if (wm[rg] & bit) {
-                            const uint32_t idx = ro[rg] + __popc(wm[rg] & (bit - 1u));
-                            uint32_t raw;
-                            if (idx < FP8_CAP_BLOCKS) raw = *reinterpret_cast<const uint32_t*>(sb + OFF_FP8 + idx * 16 + t * 4);
-                            else raw = __ldg(reinterpret_cast<const uint32_t*>(fp8 + ((size_t)list0 + idx) * 16 + t * 4));
-                            uint32_t h0, h1;
-                            uint16_t lo = (uint16_t)raw, hi = (uint16_t)(raw >> 16);
-                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(lo));
-                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(hi));
-                            __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), rw2), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), rw2);
-                            b0 = *reinterpret_cast<uint32_t*>(&x0); b1 = *reinterpret_cast<uint32_t*>(&x1);
-                        }
-                        mma_f16_16816(acc[rg], at0.x, at1.x, at0.y, at1.y, b0, b1);
-                    }
-                    // (2) FP8 activation blocks against the NVFP4 weights of this stage
-                    if (oa & bit) {
-                        const uint32_t a0 = (am[0] & bit) ? at0.x : 0u, a2 = (am[0] & bit) ? at0.y : 0u;
-                        const uint32_t a1 = (am[1] & bit) ? at1.x : 0u, a3 = (am[1] & bit) ? at1.y : 0u;
-#pragma unroll
-                        for (int rg = 0; rg < 2; ++rg) {
-                            const int r = rowbase + 8 * rg + g;            // row inside the tile
-                            const uint32_t codes = *reinterpret_cast<const uint16_t*>(
-                                sb + r * 128 + ((((uint32_t)kb >> 1) ^ ((uint32_t)r & 7u)) << 4) + (kb & 1) * 8 + t * 2);
-                            const uint32_t sfb = sb[OFF_SFW + (kb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)];
-                            uint32_t q0, q1, sc2;
-                            asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
-                                : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
-                            uint16_t s16 = (uint16_t)(sfb | (sfb << 8));
-                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
-                            __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&q0), *reinterpret_cast<__half2*>(&sc2));
-                            __half2 x1 = __hmul2(*reinterpret_cast<__half2*>(&q1), *reinterpret_cast<__half2*>(&sc2));
-                            mma_f16_16816(acc[rg], a0, a1, a2, a3, *reinterpret_cast<uint32_t*>(&x0), *reinterpret_cast<uint32_t*>(&x1));
-                        }
+                        const int r = rowbase + 8 * rg + g;            // row inside the tile
+                        const uint32_t codes = *reinterpret_cast<const uint16_t*>(
+                            sb + r * 128 + ((((uint32_t)kb >> 1) ^ ((uint32_t)r & 7u)) << 4) + (kb & 1) * 8 + t * 2);
+                        const uint32_t sfb = sb[OFF_SFW + (kb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)];
+                        uint32_t q0, q1, sc2;
+                        asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
+                            : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
+                        const uint16_t s16 = (uint16_t)(sfb | (sfb << 8));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
+                        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&q0), *reinterpret_cast<__half2*>(&sc2));
+                        const __half2 x1 = __hmul2(*reinterpret_cast<__half2*>(&q1), *reinterpret_cast<__half2*>(&sc2));
+                        mma_f16_16816(acc[rg], a0, a1, a2, a3, *reinterpret_cast<const uint32_t*>(&x0), *reinterpret_cast<const uint32_t*>(&x1));
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * stage);
                 if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
-                wm[0] = wm_n[0]; wm[1] = wm_n[1]; ro[0] = ro_n[0]; ro[1] = ro_n[1]; am[0] = am_n[0]; am[1] = am_n[1];
+                am[0] = am_n[0]; am[1] = am_n[1];
             }
             if (!ok) break;
 
-            // transpose the correction sums through this warp's private rows of the tile:
-            // mycorr[row][token]
+            // fold the (3) sums into the warp's own tile: acc[rg] = (token g | g+8) x (row 2t | 2t+1)
 #pragma unroll
             for (int rg = 0; rg < 2; ++rg) {
-                const int r = 8 * rg + 2 * t;
-                mycorr[r * CORR_LD + g] = acc[rg][0];
-                mycorr[(r + 1) * CORR_LD + g] = acc[rg][1];
-                mycorr[r * CORR_LD + g + 8] = acc[rg][2];
-                mycorr[(r + 1) * CORR_LD + g + 8] = acc[rg][3];
+                const int r = rowbase + 8 * rg + 2 * t;
+                red_add(mypriv + r * TOK + g, acc[rg][0]);
+                red_add(mypriv + (r + 1) * TOK + g, acc[rg][1]);
+                red_add(mypriv + r * TOK + g + 8, acc[rg][2]);
+                red_add(mypriv + (r + 1) * TOK + g + 8, acc[rg][3]);
             }
-            __syncwarp();
+            // all eight tiles are complete for this segment once every correction thread is here
+            const uint32_t seg_phase = (uint32_t)(seg & 1);
+            mbar_arrive(seg0);
+            if (!(ok = mbar_wait(seg0, seg_phase, abort_flag, p.status, 6))) break;
 
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
@@ -288,8 +333,28 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
             const int lr = lane & 15;
             float v[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]) + mycorr[lr * CORR_LD + j];
+            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
+            if (mine) {
+#pragma unroll
+                for (int w = 0; w < DEC_CORR_WARPS; ++w) {
+                    const float4* src = reinterpret_cast<const float4*>(priv + w * PRIV_FLOATS + (rowbase + lr) * TOK);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 x = src[j];
+                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
+                    }
+                }
+            }
+            // every warp has read all tiles before any tile is cleared for the next segment
+            mbar_arrive(seg0 + 8);
+            if (!(ok = mbar_wait(seg0 + 8, seg_phase, abort_flag, p.status, 7))) break;
+            {
+                float4* z = reinterpret_cast<float4*>(mypriv);
+#pragma unroll
+                for (int i = 0; i < (int)PRIV_FLOATS / 128; ++i) z[i * 32 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
             __syncwarp();
+
             const int64_t n = tile * 128 + rowbase + lr;
             const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
             bool write_out = whole;

@@ -21,6 +21,27 @@ namespace {
 
 // ------------------------------------------------------------------ expand to bf16 planes
 // plane[r, k] = e2m1 * e4m3scale (NVFP4 block) or e4m3 * 2^ratio (FP8 block); exact in bf16.
+__device__ __forceinline__ void e4m3x16_scaled(const uint4& c, float r8, float (&v)[16])
+{
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 a = e4m3x2_to_f32x2(w[i] & 0xffff), bb = e4m3x2_to_f32x2(w[i] >> 16);
+        v[4 * i] = a.x * r8; v[4 * i + 1] = a.y * r8; v[4 * i + 2] = bb.x * r8; v[4 * i + 3] = bb.y * r8;
+    }
+}
+
+// 16 values that are exact in bf16 (the low 16 bits of every float are zero) -> 32 bytes
+__device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&v)[16])
+{
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        o[i] = (__float_as_uint(v[2 * i]) >> 16) | (__float_as_uint(v[2 * i + 1]) & 0xffff0000u);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
 __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, int kind,
                                                      uint4* plane)
 {
@@ -33,18 +54,11 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
         int64_t r = b / L.KB, kb = b % L.KB;
         uint32_t word = pmask[r * L.MW + (kb >> 5)];
         bool is8 = (word >> (kb & 31)) & 1;
+        if (is8 && kind == 1) continue;        // weights: FP8 blocks come from the list (expand8_w_kernel)
         float v[16];
         if (is8) {
-            size_t src = (kind == 1)
-                ? L.off_codes8 + (size_t)fgmp_fp8_pos(blob, L, r, kb, word) * 16
-                : L.off_codes8 + (size_t)(r * K + kb * 16);
-            uint4 c = *reinterpret_cast<const uint4*>(blob + src);
-            const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float2 a = e4m3x2_to_f32x2(w[i] & 0xffff), bb = e4m3x2_to_f32x2(w[i] >> 16);
-                v[4 * i] = a.x * r8; v[4 * i + 1] = a.y * r8; v[4 * i + 2] = bb.x * r8; v[4 * i + 3] = bb.y * r8;
-            }
+            uint4 c = *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16));
+            e4m3x16_scaled(c, r8, v);
         } else {
             uint2 c = *reinterpret_cast<const uint2*>(blob + L.off_codes4 + (r * K) / 2 + kb * 8);
             float d = e4m3_to_f32(blob[L.off_sf + fgmp_sf_offset(r, kb, K)]);
@@ -55,14 +69,22 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
                 v[2 * i] = q.x * d; v[2 * i + 1] = q.y * d;
             }
         }
-        uint32_t o[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)   // exact: the low 16 bits of every value are zero
-            o[i] = (__float_as_uint(v[2 * i]) >> 16) | (__float_as_uint(v[2 * i + 1]) & 0xffff0000u);
-        uint4* dst = plane + (r * K) / 8 + kb * 2;
-        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
     }
+}
+
+// FP8 blocks of packed weights: list -> bf16 plane; one CTA of 128 threads per unit
+__global__ void __launch_bounds__(128) expand8_w_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane)
+{
+    __shared__ UnitScratch sc;
+    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
+    const PackedLayout L = fgmp_layout(rows, K, 1, h->capacity);
+    const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
+    fgmp_for_each_fp8_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, uint32_t idx, int) {
+        float v[16];
+        e4m3x16_scaled(*reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)idx * 16), r8, v);
+        store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
+    });
 }
 
 // ------------------------------------------------------------------ bf16 tcgen05 GEMM
@@ -302,6 +324,8 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
         nb = N * (K / 16);
         g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
         FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_weights, N, K, 1, reinterpret_cast<uint4*>(planeW)));
+        const PackedLayout LW = fgmp_layout(N, K, 1, 0);
+        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand8_w_kernel<<<(unsigned)(LW.tiles * LW.chunks), 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW)));
     }
     GemmParams p;
     p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K;

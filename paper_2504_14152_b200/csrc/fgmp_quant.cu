@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     if (!SCORE_ONLY) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
-            h->magic = FGMP_MAGIC; h->version = 1; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->magic = FGMP_MAGIC; h->version = 2; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }
@@ -147,19 +147,24 @@ __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
             *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) = c;
         }
         if (codes8) {
+            // weights: zero here, the FP8 blocks are filled in from the list by unpack8_w_kernel
             uint4 c = make_uint4(0, 0, 0, 0);
-            if (is8) {
-                size_t src;
-                if (kind == 1) {
-                    src = L.off_codes8 + (size_t)fgmp_fp8_pos(blob, L, r, kb, word) * 16;
-                } else {
-                    src = L.off_codes8 + (size_t)(r * K + kb * 16);
-                }
-                c = *reinterpret_cast<const uint4*>(blob + src);
-            }
+            if (is8 && kind == 0) c = *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16));
             *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) = c;
         }
     }
+}
+
+// FP8 blocks of packed weights: list -> dense plane; one CTA of 128 threads per unit
+__global__ void __launch_bounds__(128) unpack8_w_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint8_t* codes8)
+{
+    __shared__ UnitScratch sc;
+    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
+    const PackedLayout L = fgmp_layout(rows, K, 1, h->capacity);
+    fgmp_for_each_fp8_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, uint32_t idx, int) {
+        *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) =
+            *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)idx * 16);
+    });
 }
 
 fgmp_status check_act_args(const void* X, int64_t ldx, const float* fisher, int64_t M, int64_t K, fgmp_scales sc, int sm)
@@ -250,6 +255,18 @@ extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, 
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
     int64_t nblk = rows * (K / 16);
     int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);
-    FGMP_LAUNCH(FGMP_K_UNPACK, (cudaStream_t)cuda_stream, unpack_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_kernel<<<grid, 256, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
+    if (codes8) {
+        // the blob says what it is; a weight blob keeps its FP8 blocks in the compact list
+        fgmp_packed_header h;
+        if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) return FGMP_ERR_CUDA;
+        if (h.magic != FGMP_MAGIC || h.rows != rows || h.K != K) return FGMP_ERR_INVALID_ARG;
+        if (h.kind == 1) {
+            const PackedLayout L = fgmp_layout(rows, K, 1, h.capacity);
+            FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack8_w_kernel<<<(unsigned)(L.tiles * L.chunks), 128, 0, s>>>((const uint8_t*)packed, rows, K, codes8));
+        }
+    }
     return fgmp_launch_status();
 }

@@ -279,55 +279,35 @@ __global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t
     if (threadIdx.x == 0 && append_total) out[n] = (uint32_t)carry_s;
 }
 
-// per (128-row tile, 16-block K chunk): rowoff = exclusive prefix over the tile's rows of the
-// number of FP8 blocks each row has in the chunk; ctcnt = their total.  One CTA of 128 threads
-// per (tile, chunk).
-__global__ void __launch_bounds__(128) w_ctcount_kernel(const uint32_t* mask, int64_t N, int64_t MW, int64_t chunks,
-                                                        uint16_t* rowoff, uint32_t* ctcnt)
+// per unit (128-row tile x 16-block K chunk): how many FP8 blocks each of its 16 block columns
+// holds (kbcnt) and their total (ctcnt).  One CTA of 128 threads per unit.
+__global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask, PackedLayout L, uint8_t* kbcnt, uint32_t* ctcnt)
 {
-    __shared__ uint32_t wsum[4];
-    const int64_t ct = blockIdx.x;
-    const int64_t tile = ct / chunks, chunk = ct % chunks;
-    const int64_t r = tile * 128 + threadIdx.x;
-    uint32_t cnt = 0;
-    if (r < N) cnt = __popc((mask[r * MW + (chunk >> 1)] >> ((chunk & 1) * 16)) & 0xffffu);
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    uint32_t incl = cnt;
-    for (int o = 1; o < 32; o <<= 1) { uint32_t y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
-    if (lane == 31) wsum[wid] = incl;
-    __syncthreads();
-    uint32_t base = 0;
-    for (int w = 0; w < wid; ++w) base += wsum[w];
-    rowoff[ct * 128 + threadIdx.x] = (uint16_t)(base + incl - cnt);
-    if (threadIdx.x == 127) ctcnt[ct] = base + incl;
+    __shared__ UnitScratch sc;
+    const int64_t unit = blockIdx.x;
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, (unit / L.chunks) * 128 + threadIdx.x, unit % L.chunks);
+    const uint32_t total = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    if (threadIdx.x < 16) kbcnt[unit * 16 + threadIdx.x] = (uint8_t)sc.cnt[threadIdx.x];
+    if (threadIdx.x == 0) ctcnt[unit] = total;
 }
 
-__global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw8, int64_t N, int64_t K, int ratio,
+// codes4 and microscales of every block (zero for FP8 blocks)
+__global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw8, int64_t N, int64_t K,
                                                      const SelectState* st, const uint8_t* sc_in,
-                                                     uint8_t* blob, PackedLayout L, int64_t capacity)
+                                                     uint8_t* blob, PackedLayout L)
 {
     const float s4 = st->s4;
-    const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
-    const float inv8 = __fdiv_rn(1.0f, s8);
     const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
     const int64_t B = N * L.KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
         int64_t n = b / L.KB, kb = b % L.KB;
-        float v[16], f[16];
-        load_block(W, ldw8, nullptr, 0, n, kb, v, f);
         uint32_t word = mask[n * L.MW + (kb >> 5)];
         bool is8 = (word >> (kb & 31)) & 1;
         uint32_t c4[2] = {0, 0};
         uint32_t sc = 0;
-        if (is8) {
-            uint32_t c8[4];
-            float dq8[16];
-            block_fp8(v, inv8, s8, c8, dq8);
-            int64_t pos = (int64_t)fgmp_fp8_pos(blob, L, n, kb, word);
-            if (pos < capacity)
-                *reinterpret_cast<uint4*>(blob + L.off_codes8 + (size_t)pos * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
-        } else {
-            float dq4[16];
+        if (!is8) {
+            float v[16], f[16], dq4[16];
+            load_block(W, ldw8, nullptr, 0, n, kb, v, f);
             sc = sc_in[b];
             block_nvfp4(v, sc, s4, c4, dq4);
         }
@@ -341,11 +321,29 @@ __global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw
         blob[L.off_sf + fgmp_sf_offset(N + i / L.KB, i % L.KB, K)] = 0;
 }
 
+// the FP8 blocks: E4M3 codes and row ids into the list, one CTA of 128 threads per unit
+__global__ void __launch_bounds__(128) w_emit8_kernel(const uint4* W, int64_t ldw8, int ratio, const SelectState* st,
+                                                      uint8_t* blob, PackedLayout L, int64_t capacity)
+{
+    __shared__ UnitScratch sc;
+    const float s8 = __fmul_rn(st->s4, __int_as_float((127 + ratio) << 23));
+    const float inv8 = __fdiv_rn(1.0f, s8);
+    fgmp_for_each_fp8_block(blob, L, blockIdx.x, sc, [&](int64_t n, int64_t kb, uint32_t idx, int row) {
+        if ((int64_t)idx >= capacity) return;
+        float v[16], f[16], dq8[16];
+        uint32_t c8[4];
+        load_block(W, ldw8, nullptr, 0, n, kb, v, f);
+        block_fp8(v, inv8, s8, c8, dq8);
+        *reinterpret_cast<uint4*>(blob + L.off_codes8 + (size_t)idx * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
+        blob[L.off_rowid + idx] = (uint8_t)row;
+    });
+}
+
 __global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, int64_t N, int64_t K, int ratio,
                                 int64_t capacity, int fraction_mode, float tau_given, float* tau_eff_out)
 {
     if (threadIdx.x == 0) {
-        h->magic = FGMP_MAGIC; h->version = 1; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
+        h->magic = FGMP_MAGIC; h->version = 2; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
         h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = capacity;
         float teff = fraction_mode ? st->tau : tau_given;
         h->tau_eff = teff;
@@ -388,7 +386,7 @@ int64_t tmp_words(int64_t N, int64_t K)
 
 size_t ws_weights_bytes(int64_t N, int64_t K)
 {
-    int64_t KB = K / 16, MW = (KB + 31) / 32, B = N * KB;
+    int64_t KB = K / 16, B = N * KB;
     return STATE_BYTES + fgmp_align1k((size_t)B * 4) + fgmp_align1k((size_t)B) + 2 * fgmp_align1k((size_t)tmp_words(N, K) * 4);
 }
 
@@ -423,8 +421,13 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     // capacity: what the blob can hold
     const PackedLayout L0 = fgmp_layout(N, K, 1, 0);
     if (packed_bytes < L0.total) return FGMP_ERR_WORKSPACE;
-    int64_t capacity = (int64_t)((packed_bytes - L0.off_codes8) / 16);
-    if (capacity > B) capacity = B;
+    // the largest list the blob has room for (16 code bytes + 1 row id per block, sections rounded)
+    int64_t capacity = 0, cap_hi = (int64_t)((packed_bytes - L0.off_codes8) / 16);
+    if (cap_hi > B) cap_hi = B;
+    while (capacity < cap_hi) {
+        const int64_t mid = capacity + (cap_hi - capacity + 1) / 2;
+        if (fgmp_layout(N, K, 1, mid).total <= packed_bytes) capacity = mid; else cap_hi = mid - 1;
+    }
     if (fraction_mode && capacity < k) return FGMP_ERR_WORKSPACE;
     const PackedLayout L = fgmp_layout(N, K, 1, capacity);
     if (ws_bytes < ws_weights_bytes(N, K)) return FGMP_ERR_WORKSPACE;
@@ -459,7 +462,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     }
     uint32_t* mask = reinterpret_cast<uint32_t*>(blob + L.off_mask);
     uint32_t* ctptr = reinterpret_cast<uint32_t*>(blob + L.off_ctptr);
-    uint16_t* rowoff = reinterpret_cast<uint16_t*>(blob + L.off_rowoff);
+    uint8_t* kbcnt = blob + L.off_kbcnt;
     const int64_t NCT = L.tiles * L.chunks;
     const int gw = grid_for(NW * 32, 256, 8);
     if (fraction_mode && k > 0) {
@@ -471,9 +474,10 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
         FGMP_LAUNCH(FGMP_K_W_AUX, s, set_tau_kernel<<<1, 32, 0, s>>>(st, fraction_mode ? INFINITY : tau));
     }
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a));
-    FGMP_LAUNCH(FGMP_K_W_MASK, s, w_ctcount_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, N, MW, L.chunks, rowoff, tmp_a));
+    FGMP_LAUNCH(FGMP_K_W_MASK, s, w_unit_count_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, L, kbcnt, tmp_a));
     FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, ctptr, NCT, &st->n_fp8, 1));
-    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, ratio, st, sc_tmp, blob, L, capacity));
+    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, st, sc_tmp, blob, L));
+    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit8_kernel<<<(unsigned)NCT, 128, 0, s>>>(W, ldw / 8, ratio, st, blob, L, capacity));
     FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, N, K, ratio, capacity,
                                      fraction_mode ? 1 : 0, tau, tau_eff_out));
     return fgmp_launch_status();
