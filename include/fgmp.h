@@ -21,27 +21,38 @@
  *   - a packed tensor is an opaque device blob (layout below) produced by the two
  *     quantizers and consumed by fgmp_linear / fgmp_unpack; it must be 1024-byte aligned.
  *
- * Packed blob layout (all sections 1024-byte aligned, in this order)
+ * Packed blobs (sections 1024-byte aligned).  A "unit" = one tile of 128 rows x one chunk of 256
+ * K elements (16 blocks); C = ceil(K/256) chunks per tile.
+ *
+ * Activations: header | codes4 | sf | mask | arec | codes8
  *   header  256 B : fgmp_packed_header (device-written)
  *   codes4        : rows * K/2 bytes, row-major; two E2M1 codes per byte, even element in
  *                   the low nibble; all-zero for FP8 blocks
  *   sf            : E4M3 microscales in 512-byte tiles of 128 rows x 4 blocks:
  *                   byte of (row r, block kb) = ((r/128) * (K/64) + kb/4) * 512
  *                                               + (r%32)*16 + ((r%128)/32)*4 + kb%4;
- *                   0x00 for FP8 blocks and for padding rows
+ *                   0x00 for FP8 blocks
  *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
  *                   1 = FP8
- *   ctptr, kbcnt  : (weights only) index of the FP8 list.  A unit = one 128-row tile t x one
- *                   256-element K chunk c (C = ceil(K/256) chunks per tile).
- *                   ctptr[t*C + c] (uint32, one extra entry at the end) = list position of the
- *                   unit's first FP8 block; kbcnt[(t*C + c)*16 + j] (uint8) = how many of the
- *                   unit's FP8 blocks lie in its j-th block column
- *   atrue         : (activations with rows <= 16 only) fp16 copy of the quantized values
- *                   divided by the tensor scale, [K/16][16 tokens][16]; rows >= M are zero
- *   codes8        : weights: the FP8 blocks only, 16 bytes each, ordered by (tile, chunk, block
- *                   column, row) (capacity max_fp8_blocks); activations: a dense rows*K byte
- *                   plane of which only the FP8 blocks are written.
- *   rowid         : (weights only) capacity + 32 bytes: row inside its tile of every list entry
+ *   arec          : (rows <= 16 only) C records of 12416 bytes, one per chunk, holding what the
+ *                   decode-sized GEMM streams: the chunk's codes as a 16-token x 128-byte tile
+ *                   (16-byte pieces of token m XOR-swizzled with m%8), its microscales (four
+ *                   512-byte tiles), an fp16 copy [16 blocks][16 tokens][16] of the quantized
+ *                   values divided by the tensor scale, and 16 uint16 mask words; token rows
+ *                   >= rows are zero
+ *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written
+ *
+ * Weights: header | mask | uptr | records
+ *   uptr          : uint32 [units + 1]: start of unit (t, c)'s record, index t*C + c, in
+ *                   128-byte steps from the first record
+ *   record        : 16384 B E2M1 codes as a 128-row x 128-byte tile (16-byte pieces of row r
+ *                   XOR-swizzled with r%8; zero for FP8 blocks and rows beyond N)
+ *                   | 2048 B microscales (four 512-byte tiles as above)
+ *                   | 16 B: number of FP8 blocks in each of the unit's 16 block columns
+ *                   | row (inside the tile) of every FP8 block, padded to 16 bytes
+ *                   | the FP8 blocks, 16 E4M3 codes each, ordered by (block column, row);
+ *                   padded to 128 bytes
+ *                   fgmp_weights_bytes(N, K, max_fp8_blocks) leaves room for that many FP8 blocks.
  */
 #ifndef FGMP_H
 #define FGMP_H
@@ -83,14 +94,14 @@ typedef struct {
 /* First 256 bytes of a packed blob (device memory). */
 typedef struct {
     uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
-    uint32_t version;        /* layout version, 2                                           */
+    uint32_t version;        /* layout version, 3                                           */
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;
     int64_t n_fp8;           /* number of FP8 blocks                                        */
     float tau_eff;           /* weights, fraction mode: smallest selected score             */
     uint32_t kind;           /* 0 = activations, 1 = weights                                */
-    int64_t capacity;        /* weights: room for this many FP8 blocks                      */
+    int64_t capacity;        /* weights: room for records, in 128-byte steps                */
     int32_t error;           /* 0, or FGMP_ERR_CAPACITY                                     */
     int32_t reserved[49];
 } fgmp_packed_header;
@@ -112,7 +123,8 @@ size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K);
  * scores are taken in row-major block order) and tau is ignored; fp8_fraction < 0: a block
  * is FP8 iff score > tau.  The blob must have room for the result
  * (packed_bytes >= fgmp_weights_bytes(N, K, max_fp8_blocks)); if threshold mode finds
- * more FP8 blocks than that, header.error = FGMP_ERR_CAPACITY and the blob is invalid.
+ * more FP8 blocks than the blob has room for, header.error = FGMP_ERR_CAPACITY and the blob
+ * is invalid (fgmp_unpack refuses it).
  * tau_eff_out (device float, may be NULL) receives the smallest selected score. */
 fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, const float* fisher_elem, int64_t ldf,
                                   int64_t N, int64_t K, fgmp_scales sc, fgmp_score_mode sm,

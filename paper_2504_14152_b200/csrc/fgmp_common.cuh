@@ -10,57 +10,97 @@
 #define FGMP_BS 16
 
 // ---------------------------------------------------------------- blob layout
-// Weights keep their FP8 blocks in a compact list.  A "unit" is one 128-row tile x one chunk of
-// 16 blocks (256 K elements); the list is ordered by (tile, chunk, block, row), so all FP8
-// blocks that meet the same 16 activation elements are neighbours.
-//   ctptr [units + 1]     uint32 : list index of the first FP8 block of each unit
-//   kbcnt [units * 16]    uint8  : number of FP8 blocks of the unit in each of its 16 block columns
-//   rowid [capacity + 32] uint8  : row (inside its tile) of every list entry
-// Activations keep a dense FP8 plane (only FP8 blocks are written) and, when rows <= 16, a
-// dequantized fp16 copy `atrue` laid out [K/16 blocks][16 tokens][16 elements] whose values
-// are value / tensor scale (E2M1 x microscale, or E4M3 x 2^ratio); rows >= M are zero.
+// A "unit" is one 128-row tile x one chunk of 16 blocks (256 K elements).
+//
+// Weights (kind 1): header | mask | uptr | records.  Everything a GEMM needs of one unit is one
+// contiguous record, so that a unit streams from HBM with a single bulk copy:
+//   REC_W4    16384 B : E2M1 codes, row r of the tile = 128 bytes whose 16-byte pieces are
+//                       XOR-swizzled with (r & 7) -- the 128B-swizzled K-major tile tcgen05 reads;
+//                       zero in FP8 blocks and in rows beyond the tensor
+//   REC_SF     2048 B : E4M3 microscales, 4 tiles of 512 B (128 rows x 4 blocks each):
+//                       (j/4)*512 + (r%32)*16 + (r/32)*4 + j%4 for block column j of the chunk
+//   REC_KBCNT    16 B : FP8 blocks of the unit per block column
+//   REC_ROWID         : row of every FP8 block of the unit, padded to 16 bytes
+//   then              : the FP8 blocks, 16 E4M3 codes each, ordered by (block column, row) so that
+//                       blocks meeting the same 16 activation elements are neighbours
+// Records are 128-byte aligned; uptr[u] (uint32, units + 1 entries) = start of record u in
+// 128-byte steps from the first record.
+//
+// Activations (kind 0): header | codes4 | sf | mask | arec | codes8.  codes4 is row-major, sf
+// uses the same 512-byte tiles over all rows, codes8 is a dense plane of which only FP8 blocks are
+// written.  arec exists when rows <= 16: one record per chunk holding what the decode GEMM
+// needs of 16 token rows (rows >= M are zero):
+//   AREC_A4    2048 B : codes, token m = 128 bytes, swizzled like REC_W4
+//   AREC_SF    2048 B : microscales, 4 tiles of 512 B
+//   AREC_TRUE  8192 B : fp16 [16 blocks][16 tokens][16 elements] = value / tensor scale
+//                       (E2M1 x microscale, or E4M3 x 2^ratio), exact
+//   AREC_MASK    32 B : uint16 per token, bit j = block column j of the chunk is FP8
+constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_ROWID = 18448;
+constexpr uint32_t AREC_A4 = 0, AREC_SF = 2048, AREC_TRUE = 4096, AREC_MASK = 12288, AREC_BYTES = 12416;
+
 struct PackedLayout {
     int64_t rows, K, KB, MW;          // KB = K/16 blocks per row, MW = mask words per row
-    int64_t tiles, chunks;            // 128-row tiles, 16-block K chunks
-    size_t off_codes4, off_sf, off_mask, off_ctptr, off_kbcnt, off_rowid, off_atrue, off_codes8, total;
+    int64_t tiles, chunks, units;     // 128-row tiles, 16-block K chunks, tiles * chunks
+    size_t off_codes4, off_sf, off_mask, off_arec, off_codes8;   // activations (mask: both)
+    size_t off_uptr, off_rec;                                    // weights
+    size_t total;
 };
 
 __host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 
-// kind 0 = activations, 1 = weights (capacity = room for that many FP8 blocks)
-__host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int kind, int64_t capacity)
+// bytes of the record of a unit with cnt FP8 blocks
+__host__ __device__ inline uint32_t fgmp_rec_fp8_offset(uint32_t cnt) { return REC_ROWID + ((cnt + 15u) & ~15u); }
+__host__ __device__ inline uint32_t fgmp_rec_bytes(uint32_t cnt) { return (fgmp_rec_fp8_offset(cnt) + cnt * 16u + 127u) & ~127u; }
+
+// kind 0 = activations, 1 = weights (max_fp8 = room for that many FP8 blocks in the records)
+__host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int kind, int64_t max_fp8)
 {
     PackedLayout L;
     L.rows = rows; L.K = K; L.KB = K / 16; L.MW = (L.KB + 31) / 32;
-    L.tiles = (rows + 127) / 128; L.chunks = (L.KB + 15) / 16;
+    L.tiles = (rows + 127) / 128; L.chunks = (L.KB + 15) / 16; L.units = L.tiles * L.chunks;
     size_t o = 1024;                                   // header section
-    L.off_codes4 = o;  o = fgmp_align1k(o + (size_t)rows * (size_t)(K / 2));
-    L.off_sf = o;      o = fgmp_align1k(o + (size_t)L.tiles * (size_t)(K / 64) * 512);
-    L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
-    L.off_ctptr = o;   if (kind == 1) o = fgmp_align1k(o + ((size_t)L.tiles * L.chunks + 1) * 4);
-    L.off_kbcnt = o;   if (kind == 1) o = fgmp_align1k(o + (size_t)L.tiles * L.chunks * 16);
-    L.off_atrue = o;   if (kind == 0 && rows <= 16) o = fgmp_align1k(o + (size_t)L.KB * 512);
-    // the variable-size sections come last so that every fixed offset is independent of capacity
-    L.off_codes8 = o;
-    o = fgmp_align1k(o + (kind == 1 ? (size_t)capacity * 16 : (size_t)rows * (size_t)K));
-    L.off_rowid = o;   if (kind == 1) o = fgmp_align1k(o + (size_t)capacity + 32);
+    L.off_codes4 = L.off_sf = L.off_arec = L.off_codes8 = L.off_uptr = L.off_rec = 0;
+    if (kind == 0) {
+        L.off_codes4 = o;  o = fgmp_align1k(o + (size_t)rows * (size_t)(K / 2));
+        L.off_sf = o;      o = fgmp_align1k(o + (size_t)L.tiles * (size_t)(K / 64) * 512);
+        L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
+        L.off_arec = o;    if (rows <= 16) o = fgmp_align1k(o + (size_t)L.chunks * AREC_BYTES);
+        L.off_codes8 = o;  o = fgmp_align1k(o + (size_t)rows * (size_t)K);
+    } else {
+        L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
+        L.off_uptr = o;    o = fgmp_align1k(o + ((size_t)L.units + 1) * 4);
+        L.off_rec = o;
+        // a record is at most 18448 + 15 + 127 bytes plus 17 per FP8 block
+        o = fgmp_align1k(o + (size_t)L.units * 18592 + (size_t)max_fp8 * 17);
+    }
     L.total = o;
     return L;
 }
 
-// byte offset of the microscale of (row r, block kb) inside the sf section
+// byte offset of the microscale of (row r, block kb) inside the sf section of packed activations
 __host__ __device__ inline size_t fgmp_sf_offset(int64_t r, int64_t kb, int64_t K)
 {
     return ((size_t)(r >> 7) * (size_t)(K >> 6) + (size_t)(kb >> 2)) * 512
          + (size_t)(r & 31) * 16 + (size_t)((r & 127) >> 5) * 4 + (size_t)(kb & 3);
 }
 
+// inside a record (r = row in the tile, j = block column in the chunk): the 8 code bytes and
+// the microscale byte
+__host__ __device__ inline uint32_t fgmp_rec_w4_offset(uint32_t r, uint32_t j)
+{
+    return r * 128u + (((j >> 1) ^ (r & 7u)) << 4) + (j & 1u) * 8u;
+}
+__host__ __device__ inline uint32_t fgmp_rec_sf_offset(uint32_t r, uint32_t j)
+{
+    return (j >> 2) * 512u + (r & 31u) * 16u + (r >> 5) * 4u + (j & 3u);
+}
+
 #ifdef __CUDACC__
-// Where the FP8 blocks of one unit sit in the list.  Called by all 128 threads of a CTA, thread
+// Where the FP8 blocks of one unit sit in its record.  Called by all 128 threads of a CTA, thread
 // i = row i of the tile, m16 = that row's 16 mask bits of the chunk (0 beyond the last row).
-// On return s_pos[row * 16 + kb] = offset of block (row, kb) from the unit's first list entry
-// (0xffff if the block is not FP8), s_cnt[kb] = FP8 blocks in column kb, and the return value
-// is their total.  s_warp is scratch of 64 words.  Ends with a __syncthreads().
+// On return s_pos[row * 16 + j] = index of block (row, j) among the unit's FP8 blocks (0xffff if
+// the block is not FP8), s_cnt[j] = FP8 blocks in column j, and the return value is their total.
+// s_warp is scratch of 64 words.  Ends with a __syncthreads().
 __device__ __forceinline__ uint32_t fgmp_unit_positions(uint32_t m16, uint32_t* s_warp, uint16_t* s_pos, uint32_t* s_cnt)
 {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -92,24 +132,35 @@ __device__ __forceinline__ uint32_t fgmp_chunk_mask(const uint32_t* mask, const 
     return (mask[r * L.MW + (c >> 1)] >> ((c & 1) * 16)) & 0xffffu;
 }
 
-// Visits every FP8 block of one unit of a packed weight tensor: f(row, kb, list index, row in tile).
-// Called by all 128 threads of a CTA; consecutive threads visit consecutive blocks of one row.
 struct UnitScratch { uint32_t warp[64]; uint32_t cnt[16]; uint16_t pos[128 * 16]; };
+
+// record of unit u of a packed weight tensor
+__device__ __forceinline__ const uint8_t* fgmp_record(const uint8_t* blob, const PackedLayout& L, int64_t u)
+{
+    return blob + L.off_rec + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[u] * 128;
+}
+
+// Visits every block of one unit of a packed weight tensor, 128 threads per unit, consecutive
+// threads on consecutive blocks of one row: f(row, kb, row in tile, column in chunk, rec, e8) with
+// rec = the unit's record and e8 = address of the block's 16 E4M3 codes, or nullptr if NVFP4.
 template <class F>
-__device__ __forceinline__ void fgmp_for_each_fp8_block(const uint8_t* blob, const PackedLayout& L, int64_t unit,
-                                                        UnitScratch& sc, F f)
+__device__ __forceinline__ void fgmp_for_each_block(const uint8_t* blob, const PackedLayout& L, int64_t unit,
+                                                    UnitScratch& sc, F f)
 {
     const int64_t tile = unit / L.chunks, c = unit % L.chunks;
     const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
     const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
-    fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
-    const uint32_t base = reinterpret_cast<const uint32_t*>(blob + L.off_ctptr)[unit];
-    const int kb = threadIdx.x & 15;
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    const uint8_t* rec = fgmp_record(blob, L, unit);
+    const uint8_t* fp8 = rec + fgmp_rec_fp8_offset(cnt);
+    const int j = threadIdx.x & 15;
 #pragma unroll 1
-    for (int j = 0; j < 16; ++j) {
-        const int row = (threadIdx.x >> 4) + 8 * j;
-        const uint32_t pos = sc.pos[row * 16 + kb];
-        if (pos != 0xffffu) f(tile * 128 + row, c * 16 + kb, base + pos, row);
+    for (int i = 0; i < 16; ++i) {
+        const int row = (threadIdx.x >> 4) + 8 * i;
+        const int64_t r = tile * 128 + row, kb = c * 16 + j;
+        if (r >= L.rows || kb >= L.KB) continue;
+        const uint32_t pos = sc.pos[row * 16 + j];
+        f(r, kb, row, j, rec, pos != 0xffffu ? fp8 + (size_t)pos * 16 : (const uint8_t*)nullptr);
     }
     __syncthreads();
 }

@@ -6,19 +6,20 @@
 // blocks of the weights and At the true activation values (fp16 copy, either format):
 //     Y = A4z.W4z^T            (1) tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
 //                                  weights are the 128-row MMA operand, the 16 tokens are N
-//       + At.W8^T              (2) the FP8 weight blocks, which the list keeps grouped by block
-//                                  column: eight blocks that meet the same 16 activation
-//                                  elements form one mma.sync m16n8k16; results are scattered
-//                                  to their rows in a tile private to the warp
+//       + At.W8^T              (2) the FP8 weight blocks, which a record keeps grouped by block
+//                                  column: sixteen blocks that meet the same 16 activation
+//                                  elements form the M side of mma.sync m16n8k16; results are
+//                                  added to their rows in a tile private to the warp
 //       + At[FP8 blocks].W4z^T (3) only block columns in which some token is FP8: the NVFP4
 //                                  weights of the stage are dequantized for mma.sync
 // Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all
-// SMs stream the same number of bytes; tiles shared by several CTAs are reduced in a fixed
-// order by the CTA that arrives last.  Every sum is taken in a fixed order: results are
+// SMs stream the same number of bytes; a unit is two bulk copies (its weight record, the
+// activation record of its chunk).  Tiles shared by several CTAs are reduced in a fixed order
+// by the CTA that arrives last.  Every sum is taken in a fixed order: results are
 // reproducible bit for bit.
 //
-// Warp roles (320 threads): warp 0 = producer (TMA tensor + bulk copies), warp 1 = MMA issuer
-// and TMEM owner, warps 2-9 = corrections (2) and (3), then epilogue.
+// Warp roles (320 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2-9 = corrections (2) and (3), then epilogue.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
@@ -29,16 +30,10 @@ namespace {
 constexpr int DEC_THREADS = 320;
 constexpr int DEC_CORR_WARPS = 8;
 constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
-constexpr uint32_t W4_BYTES = 128 * 128;        // 128 rows x 256 E2M1
-constexpr uint32_t A4_BYTES = TOK * 128;
-constexpr uint32_t SF_BYTES = 2048;             // 4 scale tiles of 512 B
-constexpr uint32_t ATRUE_BYTES = 16 * 512;      // 16 blocks x 16 tokens x 16 fp16
-constexpr uint32_t FP8_CAP_BLOCKS = 320;        // staged FP8 blocks per unit; more are read from global
-constexpr uint32_t ROWID_BYTES = FP8_CAP_BLOCKS + 16;
-constexpr uint32_t OFF_A4 = W4_BYTES, OFF_SFW = OFF_A4 + A4_BYTES, OFF_SFA = OFF_SFW + SF_BYTES,
-                   OFF_ATRUE = OFF_SFA + SF_BYTES, OFF_FP8 = OFF_ATRUE + ATRUE_BYTES,      // 30720
-                   OFF_ROWID = OFF_FP8 + FP8_CAP_BLOCKS * 16, OFF_KBCNT = OFF_ROWID + ROWID_BYTES;
-constexpr uint32_t DEC_STAGE_BYTES = (OFF_KBCNT + 16 + 1023) & ~1023u;                     // 36864
+constexpr uint32_t FP8_CAP_BLOCKS = 320;        // FP8 blocks of a unit that fit a stage; more are read from global
+constexpr uint32_t WREC_CAP = (REC_ROWID + FP8_CAP_BLOCKS + FP8_CAP_BLOCKS * 16 + 127) & ~127u;   // 23936
+constexpr uint32_t STG_A = (WREC_CAP + 1023) & ~1023u;                                           // 24576
+constexpr uint32_t DEC_STAGE_BYTES = (STG_A + AREC_BYTES + 1023) & ~1023u;                       // 37888
 constexpr int DEC_STAGES = 4;
 constexpr uint32_t PRIV_FLOATS = 128 * TOK;     // one [row][token] tile per correction warp
 constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 16 accumulator columns + 4 stages x 32 scale columns
@@ -57,20 +52,32 @@ struct DecParams {
     int* status; uint32_t* counters; float* partials; int maxseg;
 };
 
-struct StageMeta { uint32_t p0, cnt; };
+struct StageMeta { uint32_t step, staged; };     // record start (128-byte steps), bytes of it in the stage
 
 __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
 
 __device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return __dp4a(x, 0x01010101u, 0u); }
 
-// fire-and-forget add to a float in shared memory
-__device__ __forceinline__ void red_add(float* p, float v)
+// two E4M3 pairs (4 bytes) -> two fp16 pairs, scaled by a power of two
+__device__ __forceinline__ void e4m3x4_to_h2x2(uint32_t raw, __half2 scale, uint32_t& lo, uint32_t& hi)
 {
-    asm volatile("red.shared::cta.add.f32 [%0], %1;" ::"r"(smem_u32(p)), "f"(v) : "memory");
+    uint32_t h0, h1;
+    const uint16_t l = (uint16_t)raw, h = (uint16_t)(raw >> 16);
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(l));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(h));
+    const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), scale), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), scale);
+    lo = *reinterpret_cast<const uint32_t*>(&x0); hi = *reinterpret_cast<const uint32_t*>(&x1);
+}
+
+__device__ __forceinline__ void add2(float* p, float a, float b)
+{
+    float2 v = *reinterpret_cast<float2*>(p);
+    v.x += a; v.y += b;
+    *reinterpret_cast<float2*>(p) = v;
 }
 
 __global__ void __launch_bounds__(DEC_THREADS, 1)
-decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, DecParams p)
+decode_kernel(DecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -85,6 +92,17 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + DEC_STAGES);
     const uint32_t accf0 = smem_u32(bars + 2 * DEC_STAGES), acce0 = smem_u32(bars + 2 * DEC_STAGES + 2);
     const uint32_t seg0 = smem_u32(bars + 2 * DEC_STAGES + 4);
+
+    // this CTA's span of (tile, chunk) units
+    const int64_t G = gridDim.x, C = p.chunks;
+    const int64_t u_begin = ((int64_t)blockIdx.x * p.total) / G, u_end = ((int64_t)(blockIdx.x + 1) * p.total) / G;
+    const uint32_t* uptr = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_uptr);
+    const uint8_t* recs = p.wblob + p.LW.off_rec;
+
+    // the producer's first record offsets are on their way while the CTA sets itself up
+    int64_t pf_base = u_begin;
+    uint32_t pf = 0;
+    if (warp == 0 && pf_base + lane <= p.total) pf = __ldg(uptr + pf_base + lane);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + DEC_CORR_WARPS); }
@@ -106,49 +124,33 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // this CTA's span of (tile, chunk) units
-    const int64_t G = gridDim.x, C = p.chunks;
-    const int64_t u_begin = ((int64_t)blockIdx.x * p.total) / G, u_end = ((int64_t)(blockIdx.x + 1) * p.total) / G;
-    const uint32_t* ctptr = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_ctptr);
-    const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
-    // the row-id section lies behind the FP8 list, whose room the header records
-    const uint8_t* rowid_g = p.wblob + fgmp_align1k(p.LW.off_codes8 + (size_t)hw->capacity * 16);
-
     if (warp == 0) {
-        // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0;
-            const uint8_t* sfw = p.wblob + p.LW.off_sf;
-            const uint8_t* sfa = p.ablob + p.LA.off_sf;
-            const uint8_t* atrue = p.ablob + p.LA.off_atrue;
-            const uint8_t* fp8 = p.wblob + p.LW.off_codes8;
-            const uint8_t* kbcnt = p.wblob + p.LW.off_kbcnt;
-            uint32_t nxt0 = 0, nxt1 = 0;
-            if (u_begin < u_end) { nxt0 = __ldg(ctptr + u_begin); nxt1 = __ldg(ctptr + u_begin + 1); }
-            for (int64_t u = u_begin; u < u_end; ++u) {
-                const int64_t tile = u / C, c = u % C;
-                const uint32_t p0 = nxt0, p1 = nxt1;
-                if (u + 1 < u_end) { nxt0 = p1; nxt1 = __ldg(ctptr + u + 2); }
-                if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) break;
-                const uint32_t cnt = p1 - p0, staged = cnt < FP8_CAP_BLOCKS ? cnt : FP8_CAP_BLOCKS;
-                // row ids: whole 16-byte lines around [p0, p0 + staged)
-                const uint32_t rid_bytes = staged ? (((p0 & 15u) + staged + 15u) & ~15u) : 0u;
-                smeta[stage].p0 = p0; smeta[stage].cnt = cnt;
-                const uint32_t fb = full0 + 8 * stage;
-                const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
-                mbar_expect_tx(fb, OFF_FP8 + staged * 16 + rid_bytes + 16);
-                tma_load_2d(sb, &tmW, (int32_t)(c * 128), (int32_t)(tile * 128), fb);
-                tma_load_2d(sb + OFF_A4, &tmA, (int32_t)(c * 128), 0, fb);
-                bulk_load(sb + OFF_SFW, sfw + ((size_t)tile * (p.K >> 6) + (size_t)c * 4) * 512, SF_BYTES, fb);
-                bulk_load(sb + OFF_SFA, sfa + (size_t)c * 4 * 512, SF_BYTES, fb);
-                bulk_load(sb + OFF_ATRUE, atrue + (size_t)c * ATRUE_BYTES, ATRUE_BYTES, fb);
-                bulk_load(sb + OFF_KBCNT, kbcnt + (size_t)u * 16, 16, fb);
-                if (staged) {
-                    bulk_load(sb + OFF_FP8, fp8 + (size_t)p0 * 16, staged * 16, fb);
-                    bulk_load(sb + OFF_ROWID, rowid_g + (p0 & ~15u), rid_bytes, fb);
-                }
-                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+        // ------------------------------------------------------------ producer (whole warp; lane 0 issues)
+        int stage = 0; uint32_t phase = 0;
+        const uint8_t* arec = p.ablob + p.LA.off_arec;
+        for (int64_t u = u_begin; u < u_end; ++u) {
+            if (u + 1 - pf_base > 31) {                // next 32 record offsets
+                pf_base = u;
+                pf = (pf_base + lane <= p.total) ? __ldg(uptr + pf_base + lane) : 0u;
             }
+            const uint32_t step0 = __shfl_sync(0xffffffffu, pf, (int)(u - pf_base));
+            const uint32_t step1 = __shfl_sync(0xffffffffu, pf, (int)(u + 1 - pf_base));
+            int ok = 1;
+            if (lane == 0) {
+                ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1) ? 1 : 0;
+                if (ok) {
+                    const uint32_t bytes = (step1 - step0) * 128u;
+                    const uint32_t staged = bytes < WREC_CAP ? bytes : WREC_CAP;
+                    smeta[stage].step = step0; smeta[stage].staged = staged;
+                    const uint32_t fb = full0 + 8 * stage;
+                    const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
+                    mbar_expect_tx(fb, staged + AREC_BYTES);
+                    bulk_load(sb, recs + (size_t)step0 * 128, staged, fb);
+                    bulk_load(sb + STG_A, arec + (size_t)(u % C) * AREC_BYTES, AREC_BYTES, fb);
+                }
+            }
+            if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+            if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
@@ -170,10 +172,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
                     const uint32_t sf_t = tmem_base + 32 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        tmem_cp_sf(sf_t + 4 * j, smem_desc_sf(sb + OFF_SFW + 512 * j));
-                        tmem_cp_sf(sf_t + 16 + 4 * j, smem_desc_sf(sb + OFF_SFA + 512 * j));
+                        tmem_cp_sf(sf_t + 4 * j, smem_desc_sf(sb + REC_SF + 512 * j));
+                        tmem_cp_sf(sf_t + 16 + 4 * j, smem_desc_sf(sb + STG_A + AREC_SF + 512 * j));
                     }
-                    const uint64_t adesc = smem_desc_sw128(sb), bdesc = smem_desc_sw128(sb + OFF_A4);
+                    const uint64_t adesc = smem_desc_sw128(sb + REC_W4), bdesc = smem_desc_sw128(sb + STG_A + AREC_A4);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         umma_nvf4(d_tmem, adesc + 2 * j, bdesc + 2 * j, IDESC_NVF4, sf_t + 4 * j, sf_t + 16 + 4 * j,
@@ -195,13 +197,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
         const int rowbase = 32 * q + 16 * h;           // first owned row inside the tile
         const int slice = 2 * q + h;                   // 0..7
         const int g = lane >> 2, t = lane & 3;
-        const uint32_t* amask = reinterpret_cast<const uint32_t*>(p.ablob + p.LA.off_mask);
-        const uint8_t* fp8_g = p.wblob + p.LW.off_codes8;
         const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
+        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
         const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
-        const int64_t MWa = p.LA.MW;
-        const bool tok0 = g < p.M, tok1 = g + 8 < p.M;
         float* mypriv = priv + cw * PRIV_FLOATS;
 
         int stage = 0; uint32_t phase = 0; bool ok = true;
@@ -211,30 +210,17 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
             const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
             float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 
-            // activation mask bits of tokens g and g+8 for the chunk, fetched one unit ahead
-            uint32_t am[2];
-            auto fetch_meta = [&](int64_t uu, uint32_t (&am_)[2]) {
-                const int64_t c = uu % C;
-                const int sh = (int)(c & 1) * 16;
-                am_[0] = tok0 ? (__ldg(amask + (int64_t)g * MWa + (c >> 1)) >> sh) & 0xffffu : 0u;
-                am_[1] = tok1 ? (__ldg(amask + (int64_t)(g + 8) * MWa + (c >> 1)) >> sh) & 0xffffu : 0u;
-            };
-            fetch_meta(u, am);
-
             for (; u < seg_end; ++u) {
-                uint32_t am_n[2] = {0, 0};
-                if (u + 1 < seg_end) fetch_meta(u + 1, am_n);
-                uint32_t oa = am[0] | am[1];           // block columns in which any token is FP8
-#pragma unroll
-                for (int o = 4; o < 32; o <<= 1) oa |= __shfl_xor_sync(0xffffffffu, oa, o);
                 if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-                const uint32_t list0 = smeta[stage].p0;
-                const uint32_t shift = list0 & 15u;
+                const uint8_t* sa = sb + STG_A;
+                const uint32_t staged = smeta[stage].staged;
+                const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
 
                 // (2) FP8 weight blocks of block columns cw and cw + 8
-                const uint4 kc = *reinterpret_cast<const uint4*>(sb + OFF_KBCNT);
+                const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
                 const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z);
+                const uint32_t off8 = fgmp_rec_fp8_offset(ks0 + ks1 + ks2 + byte_sum(kc.w));
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int kb = cw + 8 * hh, wi = kb >> 2, sh8 = (kb & 3) * 8;
@@ -243,53 +229,62 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
                                          + byte_sum(word & ((1u << sh8) - 1u));
                     const uint32_t end = start + ((word >> sh8) & 0xffu);
                     if (start == end) continue;
-                    const uint2 at0 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + g * 32 + t * 8);
-                    const uint2 at1 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + (g + 8) * 32 + t * 8);
-                    for (uint32_t e = start; e < end; e += 8) {
-                        const uint32_t idx = e + g;
-                        uint32_t raw = 0;
-                        if (idx < end) {
-                            if (idx < FP8_CAP_BLOCKS) raw = *reinterpret_cast<const uint32_t*>(sb + OFF_FP8 + idx * 16 + t * 4);
-                            else raw = __ldg(reinterpret_cast<const uint32_t*>(fp8_g + ((size_t)list0 + idx) * 16 + t * 4));
+                    // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of the column
+                    const uint2 bt0 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + g * 32 + t * 8);
+                    const uint2 bt1 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + (g + 8) * 32 + t * 8);
+                    for (uint32_t e = start; e < end; e += 16) {
+                        // A fragments: FP8 blocks e + g and e + g + 8, the same four elements
+                        const uint32_t iA = e + g, iB = iA + 8;
+                        uint32_t rawA = 0, rawB = 0, rowA = 0, rowB = 0;
+                        if (iA < end) {
+                            const uint32_t o = off8 + iA * 16 + t * 4;
+                            rawA = o + 4 <= staged ? *reinterpret_cast<const uint32_t*>(sb + o) : __ldg(reinterpret_cast<const uint32_t*>(rec_g + o));
+                            rowA = REC_ROWID + iA < staged ? sb[REC_ROWID + iA] : __ldg(rec_g + REC_ROWID + iA);
                         }
-                        uint32_t h0, h1;
-                        const uint16_t lo = (uint16_t)raw, hi = (uint16_t)(raw >> 16);
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(lo));
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(hi));
-                        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), rw2), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), rw2);
-                        float c[4] = {0.f, 0.f, 0.f, 0.f};
-                        mma_f16_16816(c, at0.x, at1.x, at0.y, at1.y, *reinterpret_cast<const uint32_t*>(&x0), *reinterpret_cast<const uint32_t*>(&x1));
-                        // c[0], c[2]: list entry e + 2t for tokens g, g + 8; c[1], c[3]: entry e + 2t + 1
-                        const uint32_t i0 = e + 2 * t, i1 = i0 + 1;
-                        if (i0 < end) {
-                            const uint32_t r0 = i0 < FP8_CAP_BLOCKS ? sb[OFF_ROWID + shift + i0] : __ldg(rowid_g + list0 + i0);
-                            red_add(mypriv + r0 * TOK + g, c[0]);
-                            red_add(mypriv + r0 * TOK + g + 8, c[2]);
+                        if (iB < end) {
+                            const uint32_t o = off8 + iB * 16 + t * 4;
+                            rawB = o + 4 <= staged ? *reinterpret_cast<const uint32_t*>(sb + o) : __ldg(reinterpret_cast<const uint32_t*>(rec_g + o));
+                            rowB = REC_ROWID + iB < staged ? sb[REC_ROWID + iB] : __ldg(rec_g + REC_ROWID + iB);
                         }
-                        if (i1 < end) {
-                            const uint32_t r1 = i1 < FP8_CAP_BLOCKS ? sb[OFF_ROWID + shift + i1] : __ldg(rowid_g + list0 + i1);
-                            red_add(mypriv + r1 * TOK + g, c[1]);
-                            red_add(mypriv + r1 * TOK + g + 8, c[3]);
+                        uint32_t a0, a1, a2, a3;
+                        e4m3x4_to_h2x2(rawA, rw2, a0, a2);
+                        e4m3x4_to_h2x2(rawB, rw2, a1, a3);
+                        float c[4] = {0.f, 0.f, 0.f, 0.f}, d[4] = {0.f, 0.f, 0.f, 0.f};
+                        mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);     // tokens 2t, 2t+1
+                        mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);     // tokens 8+2t, 9+2t
+                        // c[0..1] / d[0..1]: block iA, c[2..3] / d[2..3]: block iB.  Within one column every
+                        // block has its own row, so no two lanes touch the same address here.
+                        if (iA < end) {
+                            add2(mypriv + rowA * TOK + 2 * t, c[0], c[1]);
+                            add2(mypriv + rowA * TOK + 8 + 2 * t, d[0], d[1]);
                         }
+                        if (iB < end) {
+                            add2(mypriv + rowB * TOK + 2 * t, c[2], c[3]);
+                            add2(mypriv + rowB * TOK + 8 + 2 * t, d[2], d[3]);
+                        }
+                        __syncwarp();                  // the next group may add to the same rows
                     }
                 }
 
                 // (3) FP8 activation blocks against the NVFP4 weights of the warp's 16 rows
-                uint32_t todo = oa;
+                const uint32_t am0 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + g * 2);
+                const uint32_t am1 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + (g + 8) * 2);
+                uint32_t todo = am0 | am1;             // block columns in which any token is FP8
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) todo |= __shfl_xor_sync(0xffffffffu, todo, o);
                 while (todo) {
                     const int kb = __ffs(todo) - 1;
                     todo &= todo - 1;
                     const uint32_t bit = 1u << kb;
-                    const uint2 at0 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + g * 32 + t * 8);
-                    const uint2 at1 = *reinterpret_cast<const uint2*>(sb + OFF_ATRUE + kb * 512 + (g + 8) * 32 + t * 8);
-                    const uint32_t a0 = (am[0] & bit) ? at0.x : 0u, a2 = (am[0] & bit) ? at0.y : 0u;
-                    const uint32_t a1 = (am[1] & bit) ? at1.x : 0u, a3 = (am[1] & bit) ? at1.y : 0u;
+                    const uint2 at0 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + g * 32 + t * 8);
+                    const uint2 at1 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + (g + 8) * 32 + t * 8);
+                    const uint32_t a0 = (am0 & bit) ? at0.x : 0u, a2 = (am0 & bit) ? at0.y : 0u;
+                    const uint32_t a1 = (am1 & bit) ? at1.x : 0u, a3 = (am1 & bit) ? at1.y : 0u;
 #pragma unroll
                     for (int rg = 0; rg < 2; ++rg) {
-                        const int r = rowbase + 8 * rg + g;            // row inside the tile
-                        const uint32_t codes = *reinterpret_cast<const uint16_t*>(
-                            sb + r * 128 + ((((uint32_t)kb >> 1) ^ ((uint32_t)r & 7u)) << 4) + (kb & 1) * 8 + t * 2);
-                        const uint32_t sfb = sb[OFF_SFW + (kb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)];
+                        const uint32_t r = rowbase + 8 * rg + g;       // row inside the tile
+                        const uint32_t codes = *reinterpret_cast<const uint16_t*>(sb + REC_W4 + fgmp_rec_w4_offset(r, kb) + t * 2);
+                        const uint32_t sfb = sb[REC_SF + fgmp_rec_sf_offset(r, kb)];
                         uint32_t q0, q1, sc2;
                         asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
                             : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
@@ -303,7 +298,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * stage);
                 if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
-                am[0] = am_n[0]; am[1] = am_n[1];
             }
             if (!ok) break;
 
@@ -311,10 +305,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
 #pragma unroll
             for (int rg = 0; rg < 2; ++rg) {
                 const int r = rowbase + 8 * rg + 2 * t;
-                red_add(mypriv + r * TOK + g, acc[rg][0]);
-                red_add(mypriv + (r + 1) * TOK + g, acc[rg][1]);
-                red_add(mypriv + r * TOK + g + 8, acc[rg][2]);
-                red_add(mypriv + (r + 1) * TOK + g + 8, acc[rg][3]);
+                mypriv[r * TOK + g] += acc[rg][0];
+                mypriv[(r + 1) * TOK + g] += acc[rg][1];
+                mypriv[r * TOK + g + 8] += acc[rg][2];
+                mypriv[(r + 1) * TOK + g + 8] += acc[rg][3];
             }
             // all eight tiles are complete for this segment once every correction thread is here
             const uint32_t seg_phase = (uint32_t)(seg & 1);
@@ -415,30 +409,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// 2-D byte tensor [rows, row_bytes], box = [box_rows, 128 bytes], 128-byte swizzle
-bool make_tmap_u8(CUtensorMap* map, const void* base, int64_t rows, int64_t row_bytes, int box_rows)
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess) return false;
-        fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-    cuuint32_t box[2] = {128, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 struct DecPlan { int64_t tiles, chunks, total; int grid; int maxseg; };
 
 DecPlan decode_plan(int64_t N, int64_t K)
@@ -490,11 +460,8 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
             return FGMP_ERR_CUDA;
         attr_set[dev] = true;
     }
-    CUtensorMap tmW, tmA;
-    if (!make_tmap_u8(&tmW, p.wblob + p.LW.off_codes4, N, K / 2, 128) ||
-        !make_tmap_u8(&tmA, p.ablob + p.LA.off_codes4, M, K / 2, TOK)) return FGMP_ERR_CUDA;
     if (cudaMemsetAsync(ws, 0, 1024 + (size_t)d.tiles * 32, s) != cudaSuccess) return FGMP_ERR_CUDA;
-    FGMP_LAUNCH(FGMP_K_DECODE, s, decode_kernel<<<d.grid, DEC_THREADS, DEC_SMEM, s>>>(tmW, tmA, p));
+    FGMP_LAUNCH(FGMP_K_DECODE, s, decode_kernel<<<d.grid, DEC_THREADS, DEC_SMEM, s>>>(p));
     return fgmp_launch_status();
 }
 

@@ -42,11 +42,22 @@ __device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&v)[16])
     dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
-__global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, int kind,
-                                                     uint4* plane)
+__device__ __forceinline__ void nvfp4x16_scaled(const uint2& c, uint32_t scale_code, float (&v)[16])
+{
+    const float d = e4m3_to_f32(scale_code);
+    const uint32_t w[2] = {c.x, c.y};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float2 q = e2m1x2_to_f32x2((w[i >> 2] >> ((i & 3) * 8)) & 0xff);
+        v[2 * i] = q.x * d; v[2 * i + 1] = q.y * d;
+    }
+}
+
+// packed activations -> bf16 plane; one thread per block
+__global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane)
 {
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
-    const PackedLayout L = fgmp_layout(rows, K, kind, 0);
+    const PackedLayout L = fgmp_layout(rows, K, 0, 0);
     const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
     const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
     const int64_t nblk = rows * L.KB;
@@ -54,35 +65,26 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
         int64_t r = b / L.KB, kb = b % L.KB;
         uint32_t word = pmask[r * L.MW + (kb >> 5)];
         bool is8 = (word >> (kb & 31)) & 1;
-        if (is8 && kind == 1) continue;        // weights: FP8 blocks come from the list (expand8_w_kernel)
         float v[16];
-        if (is8) {
-            uint4 c = *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16));
-            e4m3x16_scaled(c, r8, v);
-        } else {
-            uint2 c = *reinterpret_cast<const uint2*>(blob + L.off_codes4 + (r * K) / 2 + kb * 8);
-            float d = e4m3_to_f32(blob[L.off_sf + fgmp_sf_offset(r, kb, K)]);
-            const uint32_t w[2] = {c.x, c.y};
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float2 q = e2m1x2_to_f32x2((w[i >> 2] >> ((i & 3) * 8)) & 0xff);
-                v[2 * i] = q.x * d; v[2 * i + 1] = q.y * d;
-            }
-        }
+        if (is8) e4m3x16_scaled(*reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16)), r8, v);
+        else nvfp4x16_scaled(*reinterpret_cast<const uint2*>(blob + L.off_codes4 + (r * K) / 2 + kb * 8),
+                             blob[L.off_sf + fgmp_sf_offset(r, kb, K)], v);
         store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
     }
 }
 
-// FP8 blocks of packed weights: list -> bf16 plane; one CTA of 128 threads per unit
-__global__ void __launch_bounds__(128) expand8_w_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane)
+// packed weights -> bf16 plane; one CTA of 128 threads per unit record
+__global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane)
 {
     __shared__ UnitScratch sc;
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
-    const PackedLayout L = fgmp_layout(rows, K, 1, h->capacity);
+    const PackedLayout L = fgmp_layout(rows, K, 1, 0);
     const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
-    fgmp_for_each_fp8_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, uint32_t idx, int) {
+    fgmp_for_each_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, int row, int j, const uint8_t* rec, const uint8_t* e8) {
         float v[16];
-        e4m3x16_scaled(*reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)idx * 16), r8, v);
+        if (e8) e4m3x16_scaled(*reinterpret_cast<const uint4*>(e8), r8, v);
+        else nvfp4x16_scaled(*reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j)),
+                             rec[REC_SF + fgmp_rec_sf_offset(row, j)], v);
         store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
     });
 }
@@ -318,14 +320,11 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     if (cudaMemsetAsync(status, 0, 256, s) != cudaSuccess) return FGMP_ERR_CUDA;
     const int sms = fgmp_sm_count();
     {
-        int64_t nb = M * (K / 16);
-        int g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
-        FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, 0, reinterpret_cast<uint4*>(planeA)));
-        nb = N * (K / 16);
-        g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
-        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_weights, N, K, 1, reinterpret_cast<uint4*>(planeW)));
+        const int64_t nb = M * (K / 16);
+        const int g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
+        FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, reinterpret_cast<uint4*>(planeA)));
         const PackedLayout LW = fgmp_layout(N, K, 1, 0);
-        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand8_w_kernel<<<(unsigned)(LW.tiles * LW.chunks), 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW)));
+        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_w_kernel<<<(unsigned)LW.units, 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW)));
     }
     GemmParams p;
     p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K;

@@ -18,7 +18,7 @@ struct ActParams {
     float s4, k6, s8, inv8, tau;
     uint8_t* codes4; uint8_t* sf; uint32_t* mask; uint8_t* codes8;   // codes8: dense plane
     float* scores;                       // optional (score-only kernel)
-    uint4* atrue;                        // optional fp16 copy [KB][16][16] (M <= 16)
+    uint8_t* arec;                       // optional per-chunk records for the decode GEMM (M <= 16)
     fgmp_packed_header* header;
     float r8;                            // 2^ratio
     int ratio;
@@ -35,15 +35,20 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     if (!SCORE_ONLY) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
-            h->magic = FGMP_MAGIC; h->version = 2; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->magic = FGMP_MAGIC; h->version = 3; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }
-        // token rows M..15 of the fp16 copy are zero (the grid covers 16 rows in that mode)
-        if (p.atrue && m0 >= p.M) {
+        // token rows M..15 of the decode records are zero (the grid covers 16 rows in that mode)
+        if (p.arec && m0 >= p.M) {
             if (active) {
-                uint4* dst = p.atrue + (kb * 16 + m0) * 2;
+                uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
+                const uint32_t j = (uint32_t)kb & 15u, m = (uint32_t)m0;
+                *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset(m, j)) = make_uint2(0, 0);
+                rec[AREC_SF + fgmp_rec_sf_offset(m, j)] = 0;
+                uint4* dst = reinterpret_cast<uint4*>(rec + AREC_TRUE + j * 512 + m * 32);
                 dst[0] = make_uint4(0, 0, 0, 0); dst[1] = make_uint4(0, 0, 0, 0);
+                if (j == 0) *reinterpret_cast<uint16_t*>(rec + AREC_MASK + m * 2) = 0;
             }
             return;
         }
@@ -93,7 +98,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                     *reinterpret_cast<uint4*>(p.codes8 + m * p.K + kb * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
                     c4[0] = 0; c4[1] = 0; sc = 0;
                 }
-                if (p.atrue) {
+                if (p.arec) {
                     // value / tensor scale, exact in fp16: E2M1 x microscale or E4M3 x 2^ratio
                     uint32_t o[8];
                     if (is8) {
@@ -112,8 +117,12 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                             o[i] = *reinterpret_cast<uint32_t*>(&h);
                         }
                     }
-                    uint4* dst = p.atrue + (kb * 16 + m) * 2;
+                    uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
+                    const uint32_t j = (uint32_t)kb & 15u;
+                    uint4* dst = reinterpret_cast<uint4*>(rec + AREC_TRUE + j * 512 + (uint32_t)m * 32);
                     dst[0] = make_uint4(o[0], o[1], o[2], o[3]); dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                    *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset((uint32_t)m, j)) = make_uint2(c4[0], c4[1]);
+                    rec[AREC_SF + fgmp_rec_sf_offset((uint32_t)m, j)] = (uint8_t)sc;
                 }
                 *reinterpret_cast<uint2*>(p.codes4 + (m * p.K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
                 p.sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)sc;
@@ -122,18 +131,23 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
         if (!SCORE_ONLY) {
             uint32_t word = __ballot_sync(0xffffffffu, is8);
             int64_t w = kb >> 5;
-            if ((threadIdx.x & 31) == 0 && w < p.MW) p.mask[m * p.MW + w] = word;
+            if ((threadIdx.x & 31) == 0 && w < p.MW) {
+                p.mask[m * p.MW + w] = word;
+                if (p.arec) {                          // the same bits per chunk: two chunks per word
+                    *reinterpret_cast<uint16_t*>(p.arec + (size_t)(2 * w) * AREC_BYTES + AREC_MASK + m * 2) = (uint16_t)word;
+                    if (2 * w + 1 < (p.KB + 15) / 16)
+                        *reinterpret_cast<uint16_t*>(p.arec + (size_t)(2 * w + 1) * AREC_BYTES + AREC_MASK + m * 2) = (uint16_t)(word >> 16);
+                }
+            }
         }
     }
 }
 
-// packed -> canonical arrays; one thread per block
+// packed activations -> canonical arrays; one thread per block
 __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
                               uint8_t* codes4, uint8_t* codes8, uint8_t* scales, uint32_t* mask)
 {
-    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
-    const int kind = (int)h->kind;
-    const PackedLayout L = fgmp_layout(rows, K, kind, kind ? h->capacity : 0);
+    const PackedLayout L = fgmp_layout(rows, K, 0, 0);
     const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
     const int64_t nblk = rows * L.KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
@@ -147,23 +161,29 @@ __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
             *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) = c;
         }
         if (codes8) {
-            // weights: zero here, the FP8 blocks are filled in from the list by unpack8_w_kernel
             uint4 c = make_uint4(0, 0, 0, 0);
-            if (is8 && kind == 0) c = *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16));
+            if (is8) c = *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16));
             *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) = c;
         }
     }
 }
 
-// FP8 blocks of packed weights: list -> dense plane; one CTA of 128 threads per unit
-__global__ void __launch_bounds__(128) unpack8_w_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint8_t* codes8)
+// packed weights -> canonical arrays; one CTA of 128 threads per unit record
+__global__ void __launch_bounds__(128) unpack_w_kernel(const uint8_t* blob, int64_t rows, int64_t K,
+                                                       uint8_t* codes4, uint8_t* codes8, uint8_t* scales, uint32_t* mask)
 {
     __shared__ UnitScratch sc;
-    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
-    const PackedLayout L = fgmp_layout(rows, K, 1, h->capacity);
-    fgmp_for_each_fp8_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, uint32_t idx, int) {
-        *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) =
-            *reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)idx * 16);
+    const PackedLayout L = fgmp_layout(rows, K, 1, 0);
+    if (mask) {
+        const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+        for (int64_t i = (int64_t)blockIdx.x * 128 + threadIdx.x; i < rows * L.MW; i += (int64_t)gridDim.x * 128) mask[i] = pmask[i];
+    }
+    fgmp_for_each_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, int row, int j, const uint8_t* rec, const uint8_t* e8) {
+        if (scales) scales[r * L.KB + kb] = rec[REC_SF + fgmp_rec_sf_offset(row, j)];
+        if (codes4) *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) =
+                        *reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j));
+        if (codes8) *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) =
+                        e8 ? *reinterpret_cast<const uint4*>(e8) : make_uint4(0, 0, 0, 0);
     });
 }
 
@@ -219,7 +239,7 @@ extern "C" fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx
     p.header = reinterpret_cast<fgmp_packed_header*>(blob);
     int64_t grid_rows = M;
     if (M <= 16) {                     // decode-sized batch: also emit the fp16 copy, 16 token rows
-        p.atrue = reinterpret_cast<uint4*>(blob + L.off_atrue);
+        p.arec = blob + L.off_arec;
         p.rows_per_cta = 1;
         grid_rows = 16;
     }
@@ -253,20 +273,19 @@ extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, 
     if (rows < 1 || K < 64 || (K % 64) != 0 || ((uintptr_t)packed & 1023)) return FGMP_ERR_SHAPE;
     fgmp_status st;
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
-    int64_t nblk = rows * (K / 16);
-    int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_kernel<<<grid, 256, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
-    if (codes8) {
-        // the blob says what it is; a weight blob keeps its FP8 blocks in the compact list
-        fgmp_packed_header h;
-        if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-            cudaStreamSynchronize(s) != cudaSuccess) return FGMP_ERR_CUDA;
-        if (h.magic != FGMP_MAGIC || h.rows != rows || h.K != K) return FGMP_ERR_INVALID_ARG;
-        if (h.kind == 1) {
-            const PackedLayout L = fgmp_layout(rows, K, 1, h.capacity);
-            FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack8_w_kernel<<<(unsigned)(L.tiles * L.chunks), 128, 0, s>>>((const uint8_t*)packed, rows, K, codes8));
-        }
+    // the blob says what it is: activations keep planes, weights keep unit records
+    fgmp_packed_header h;
+    if (cudaMemcpyAsync(&h, packed, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) return FGMP_ERR_CUDA;
+    if (h.magic != FGMP_MAGIC || h.rows != rows || h.K != K || h.error != 0) return FGMP_ERR_INVALID_ARG;
+    if (h.kind == 1) {
+        const PackedLayout L = fgmp_layout(rows, K, 1, 0);
+        FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_w_kernel<<<(unsigned)L.units, 128, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
+    } else {
+        int64_t nblk = rows * (K / 16);
+        int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);
+        FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_kernel<<<grid, 256, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
     }
     return fgmp_launch_status();
 }

@@ -279,75 +279,81 @@ __global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t
     if (threadIdx.x == 0 && append_total) out[n] = (uint32_t)carry_s;
 }
 
-// per unit (128-row tile x 16-block K chunk): how many FP8 blocks each of its 16 block columns
-// holds (kbcnt) and their total (ctcnt).  One CTA of 128 threads per unit.
-__global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask, PackedLayout L, uint8_t* kbcnt, uint32_t* ctcnt)
+// per unit (128-row tile x 16-block K chunk): size of its record in 128-byte steps, and the
+// running total of FP8 blocks.  One CTA of 128 threads per unit.
+__global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask, PackedLayout L, uint32_t* rec_steps,
+                                                           SelectState* st)
 {
     __shared__ UnitScratch sc;
     const int64_t unit = blockIdx.x;
     const uint32_t m16 = fgmp_chunk_mask(mask, L, (unit / L.chunks) * 128 + threadIdx.x, unit % L.chunks);
-    const uint32_t total = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
-    if (threadIdx.x < 16) kbcnt[unit * 16 + threadIdx.x] = (uint8_t)sc.cnt[threadIdx.x];
-    if (threadIdx.x == 0) ctcnt[unit] = total;
-}
-
-// codes4 and microscales of every block (zero for FP8 blocks)
-__global__ void __launch_bounds__(256) w_emit_kernel(const uint4* W, int64_t ldw8, int64_t N, int64_t K,
-                                                     const SelectState* st, const uint8_t* sc_in,
-                                                     uint8_t* blob, PackedLayout L)
-{
-    const float s4 = st->s4;
-    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const int64_t B = N * L.KB;
-    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
-        int64_t n = b / L.KB, kb = b % L.KB;
-        uint32_t word = mask[n * L.MW + (kb >> 5)];
-        bool is8 = (word >> (kb & 31)) & 1;
-        uint32_t c4[2] = {0, 0};
-        uint32_t sc = 0;
-        if (!is8) {
-            float v[16], f[16], dq4[16];
-            load_block(W, ldw8, nullptr, 0, n, kb, v, f);
-            sc = sc_in[b];
-            block_nvfp4(v, sc, s4, c4, dq4);
-        }
-        *reinterpret_cast<uint2*>(blob + L.off_codes4 + (n * K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
-        blob[L.off_sf + fgmp_sf_offset(n, kb, K)] = (uint8_t)sc;
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    if (threadIdx.x == 0) {
+        rec_steps[unit] = fgmp_rec_bytes(cnt) / 128;
+        atomicAdd(&st->n_fp8, (unsigned long long)cnt);
     }
-    // microscales of the padding rows
-    const int64_t Npad = (N + 127) & ~(int64_t)127;
-    const int64_t npad = (Npad - N) * L.KB;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < npad; i += (int64_t)gridDim.x * blockDim.x)
-        blob[L.off_sf + fgmp_sf_offset(N + i / L.KB, i % L.KB, K)] = 0;
 }
 
-// the FP8 blocks: E4M3 codes and row ids into the list, one CTA of 128 threads per unit
-__global__ void __launch_bounds__(128) w_emit8_kernel(const uint4* W, int64_t ldw8, int ratio, const SelectState* st,
-                                                      uint8_t* blob, PackedLayout L, int64_t capacity)
+// Writes the record of one unit: codes and microscales of its NVFP4 blocks, E4M3 codes and row
+// ids of its FP8 blocks, the per-column counts.  One CTA of 128 threads per unit.
+__global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw8, int ratio, const SelectState* st,
+                                                     const uint8_t* sc_in, uint8_t* blob, PackedLayout L, int64_t room_steps)
 {
     __shared__ UnitScratch sc;
-    const float s8 = __fmul_rn(st->s4, __int_as_float((127 + ratio) << 23));
+    const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
+    const uint32_t* uptr = reinterpret_cast<const uint32_t*>(blob + L.off_uptr);
+    if ((int64_t)uptr[unit + 1] > room_steps) return;          // the blob is too small: header.error says so
+    const float s4 = st->s4;
+    const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
     const float inv8 = __fdiv_rn(1.0f, s8);
-    fgmp_for_each_fp8_block(blob, L, blockIdx.x, sc, [&](int64_t n, int64_t kb, uint32_t idx, int row) {
-        if ((int64_t)idx >= capacity) return;
-        float v[16], f[16], dq8[16];
-        uint32_t c8[4];
-        load_block(W, ldw8, nullptr, 0, n, kb, v, f);
-        block_fp8(v, inv8, s8, c8, dq8);
-        *reinterpret_cast<uint4*>(blob + L.off_codes8 + (size_t)idx * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
-        blob[L.off_rowid + idx] = (uint8_t)row;
-    });
+    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    uint8_t* rec = blob + L.off_rec + (size_t)uptr[unit] * 128;
+    uint8_t* rowid = rec + REC_ROWID;
+    uint8_t* fp8 = rec + fgmp_rec_fp8_offset(cnt);
+    if (threadIdx.x < 16) rec[REC_KBCNT + threadIdx.x] = (uint8_t)sc.cnt[threadIdx.x];
+    // padding behind the row ids and behind the last FP8 block
+    for (uint32_t i = cnt + threadIdx.x; i < ((cnt + 15u) & ~15u); i += 128) rowid[i] = 0;
+    for (uint32_t i = fgmp_rec_fp8_offset(cnt) + cnt * 16 + threadIdx.x; i < fgmp_rec_bytes(cnt); i += 128) rec[i] = 0;
+    const int j = threadIdx.x & 15;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i) {
+        const int row = (threadIdx.x >> 4) + 8 * i;
+        const int64_t n = tile * 128 + row, kb = c * 16 + j;
+        uint32_t c4[2] = {0, 0};
+        uint32_t scale = 0;
+        if (n < L.rows && kb < L.KB) {
+            float v[16], f[16];
+            load_block(W, ldw8, nullptr, 0, n, kb, v, f);
+            const uint32_t pos = sc.pos[row * 16 + j];
+            if (pos != 0xffffu) {
+                uint32_t c8[4];
+                float dq8[16];
+                block_fp8(v, inv8, s8, c8, dq8);
+                *reinterpret_cast<uint4*>(fp8 + (size_t)pos * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
+                rowid[pos] = (uint8_t)row;
+            } else {
+                float dq4[16];
+                scale = sc_in[n * L.KB + kb];
+                block_nvfp4(v, scale, s4, c4, dq4);
+            }
+        }
+        *reinterpret_cast<uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j)) = make_uint2(c4[0], c4[1]);
+        rec[REC_SF + fgmp_rec_sf_offset(row, j)] = (uint8_t)scale;
+    }
 }
 
-__global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, int64_t N, int64_t K, int ratio,
-                                int64_t capacity, int fraction_mode, float tau_given, float* tau_eff_out)
+__global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, const uint32_t* uptr, int64_t units,
+                                int64_t N, int64_t K, int ratio, int64_t room_steps, int fraction_mode, float tau_given,
+                                float* tau_eff_out)
 {
     if (threadIdx.x == 0) {
-        h->magic = FGMP_MAGIC; h->version = 2; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
-        h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = capacity;
+        h->magic = FGMP_MAGIC; h->version = 3; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
+        h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = room_steps;
         float teff = fraction_mode ? st->tau : tau_given;
         h->tau_eff = teff;
-        h->error = ((int64_t)st->n_fp8 > capacity) ? (int32_t)FGMP_ERR_CAPACITY : 0;
+        h->error = ((int64_t)uptr[units] > room_steps) ? (int32_t)FGMP_ERR_CAPACITY : 0;
         if (tau_eff_out) *tau_eff_out = teff;
     }
 }
@@ -418,18 +424,11 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
         k = (int64_t)floor(fp8_fraction * (double)B + 0.5);
         if (k > B) k = B;
     }
-    // capacity: what the blob can hold
-    const PackedLayout L0 = fgmp_layout(N, K, 1, 0);
-    if (packed_bytes < L0.total) return FGMP_ERR_WORKSPACE;
-    // the largest list the blob has room for (16 code bytes + 1 row id per block, sections rounded)
-    int64_t capacity = 0, cap_hi = (int64_t)((packed_bytes - L0.off_codes8) / 16);
-    if (cap_hi > B) cap_hi = B;
-    while (capacity < cap_hi) {
-        const int64_t mid = capacity + (cap_hi - capacity + 1) / 2;
-        if (fgmp_layout(N, K, 1, mid).total <= packed_bytes) capacity = mid; else cap_hi = mid - 1;
-    }
-    if (fraction_mode && capacity < k) return FGMP_ERR_WORKSPACE;
-    const PackedLayout L = fgmp_layout(N, K, 1, capacity);
+    // room for the unit records, in 128-byte steps
+    const PackedLayout L = fgmp_layout(N, K, 1, 0);
+    if (packed_bytes < L.total) return FGMP_ERR_WORKSPACE;
+    const int64_t room_steps = (int64_t)((packed_bytes - L.off_rec) / 128);
+    if (fraction_mode && packed_bytes < fgmp_layout(N, K, 1, k).total) return FGMP_ERR_WORKSPACE;
     if (ws_bytes < ws_weights_bytes(N, K)) return FGMP_ERR_WORKSPACE;
     fgmp_status stt;
     if ((stt = fgmp_require_sm100()) != FGMP_OK) return stt;
@@ -461,9 +460,8 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
         }
     }
     uint32_t* mask = reinterpret_cast<uint32_t*>(blob + L.off_mask);
-    uint32_t* ctptr = reinterpret_cast<uint32_t*>(blob + L.off_ctptr);
-    uint8_t* kbcnt = blob + L.off_kbcnt;
-    const int64_t NCT = L.tiles * L.chunks;
+    uint32_t* uptr = reinterpret_cast<uint32_t*>(blob + L.off_uptr);
+    const int64_t NCT = L.units;
     const int gw = grid_for(NW * 32, 256, 8);
     if (fraction_mode && k > 0) {
         run_select(scores, B, st, s);
@@ -474,12 +472,11 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
         FGMP_LAUNCH(FGMP_K_W_AUX, s, set_tau_kernel<<<1, 32, 0, s>>>(st, fraction_mode ? INFINITY : tau));
     }
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a));
-    FGMP_LAUNCH(FGMP_K_W_MASK, s, w_unit_count_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, L, kbcnt, tmp_a));
-    FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, ctptr, NCT, &st->n_fp8, 1));
-    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(W, ldw / 8, N, K, st, sc_tmp, blob, L));
-    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit8_kernel<<<(unsigned)NCT, 128, 0, s>>>(W, ldw / 8, ratio, st, blob, L, capacity));
-    FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, N, K, ratio, capacity,
-                                     fraction_mode ? 1 : 0, tau, tau_eff_out));
+    FGMP_LAUNCH(FGMP_K_W_MASK, s, w_unit_count_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, L, tmp_a, st));
+    FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, uptr, NCT, nullptr, 1));
+    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<(unsigned)NCT, 128, 0, s>>>(W, ldw / 8, ratio, st, sc_tmp, blob, L, room_steps));
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, uptr, NCT, N, K, ratio,
+                                     room_steps, fraction_mode ? 1 : 0, tau, tau_eff_out));
     return fgmp_launch_status();
 }
 
