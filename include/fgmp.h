@@ -34,7 +34,7 @@
  *                   0x00 for FP8 blocks
  *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
  *                   1 = FP8
- *   arec          : (rows <= 16 only) C records of 12416 bytes, one per chunk, holding what the
+ *   arec          : (rows <= 16 only) C records of 13312 bytes, one per chunk, holding what the
  *                   decode-sized GEMM streams: the chunk's codes as a 16-token x 128-byte tile
  *                   (16-byte pieces of token m XOR-swizzled with m%8), its microscales (four
  *                   512-byte tiles), an fp16 copy [16 blocks][16 tokens][16] of the quantized

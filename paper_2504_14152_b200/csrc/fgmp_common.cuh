@@ -32,11 +32,19 @@
 // needs of 16 token rows (rows >= M are zero):
 //   AREC_A4    2048 B : codes, token m = 128 bytes, swizzled like REC_W4
 //   AREC_SF    2048 B : microscales, 4 tiles of 512 B
-//   AREC_TRUE  8192 B : fp16 [16 blocks][16 tokens][16 elements] = value / tensor scale
-//                       (E2M1 x microscale, or E4M3 x 2^ratio), exact
 //   AREC_MASK    32 B : uint16 per token, bit j = block column j of the chunk is FP8
+//   AREC_TRUE  8192 B : fp16 value / tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact)
+//                       as four K-major tiles of 16 tokens x 64 elements, token m = 128 bytes,
+//                       16-byte pieces XOR-swizzled with (m & 7): a tcgen05 kind::f16 operand
 constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_ROWID = 18448;
-constexpr uint32_t AREC_A4 = 0, AREC_SF = 2048, AREC_TRUE = 4096, AREC_MASK = 12288, AREC_BYTES = 12416;
+constexpr uint32_t AREC_A4 = 0, AREC_SF = 2048, AREC_MASK = 4096, AREC_TRUE = 5120, AREC_BYTES = 13312;
+
+// byte offset, inside a 128-byte-swizzled K-major fp16 tile of 64 elements per row, of the first
+// (half = 0) or second (half = 1) 8 elements of block column jq (0..3) of row r
+__host__ __device__ inline uint32_t fgmp_h16_tile_offset(uint32_t r, uint32_t jq, uint32_t half)
+{
+    return r * 128u + ((((jq << 1) | half) ^ (r & 7u)) << 4);
+}
 
 struct PackedLayout {
     int64_t rows, K, KB, MW;          // KB = K/16 blocks per row, MW = mask words per row

@@ -1,25 +1,28 @@
 // fgmp_linear for decode-sized batches (M <= 16 tokens): a weight-streaming kernel that
 // reads the packed weights exactly once (Section 4.1 of the paper: the four block-pair
-// products, FP32 accumulation).
+// products, FP32 accumulation).  All arithmetic runs on the tensor cores; the CUDA cores only
+// move and convert the few blocks that need it.
 //
-// Decomposition (exact).  With A4z / W4z the NVFP4 planes (zero in FP8 blocks), W8 the FP8
-// blocks of the weights and At the true activation values (fp16 copy, either format):
-//     Y = A4z.W4z^T            (1) tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
-//                                  weights are the 128-row MMA operand, the 16 tokens are N
-//       + At.W8^T              (2) the FP8 weight blocks, which a record keeps grouped by block
-//                                  column: sixteen blocks that meet the same 16 activation
-//                                  elements form the M side of mma.sync m16n8k16; results are
-//                                  added to their rows in a tile private to the warp
-//       + At[FP8 blocks].W4z^T (3) only block columns in which some token is FP8: the NVFP4
-//                                  weights of the stage are dequantized for mma.sync
-// Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all
-// SMs stream the same number of bytes; a unit is two bulk copies (its weight record, the
-// activation record of its chunk).  Tiles shared by several CTAs are reduced in a fixed order
-// by the CTA that arrives last.  Every sum is taken in a fixed order: results are
+// Decomposition (exact).  Call a block column "hot" when at least one token has an FP8 block
+// there.  With W4z the NVFP4 weight codes (zero in FP8 blocks), A4z' the NVFP4 activation codes
+// with every hot column zeroed, At the true activation values (fp16, either format) and T the
+// fp16 tile that holds the FP8 weight blocks everywhere plus, in hot columns, the dequantized
+// NVFP4 weight blocks (so T = the true weights there):
+//     Y = A4z'.W4z^T    tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM
+//       + At.T^T        tcgen05.mma kind::f16 into the same FP32 accumulator
+// In a cold column A4z'.W4z covers NVFP4 x NVFP4 and At.T covers every pair with an FP8 weight
+// block; in a hot column At.T is the complete product.  T is mostly zero: per quarter of a unit
+// (4 block columns) it is a 128 x 64 fp16 tile that scatter threads fill from the unit's record
+// and clear again after use.
+//
+// Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all SMs
+// stream the same number of bytes; a unit is two bulk copies (its weight record, the activation
+// record of its chunk).  Tiles shared by several CTAs are reduced in a fixed order by the CTA
+// that arrives last; the accumulation order inside TMEM is the issue order: results are
 // reproducible bit for bit.
 //
-// Warp roles (320 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2-9 = corrections (2) and (3), then epilogue.
+// Warp roles (448 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2-5 = epilogue (one TMEM lane quadrant each), warps 6-13 = scatter.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
@@ -27,20 +30,23 @@
 
 namespace {
 
-constexpr int DEC_THREADS = 320;
-constexpr int DEC_CORR_WARPS = 8;
+constexpr int DEC_THREADS = 448;
+constexpr int SCAT_WARPS = 8, SCAT_THREADS = 256;
 constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
 constexpr uint32_t FP8_CAP_BLOCKS = 320;        // FP8 blocks of a unit that fit a stage; more are read from global
 constexpr uint32_t WREC_CAP = (REC_ROWID + FP8_CAP_BLOCKS + FP8_CAP_BLOCKS * 16 + 127) & ~127u;   // 23936
 constexpr uint32_t STG_A = (WREC_CAP + 1023) & ~1023u;                                           // 24576
-constexpr uint32_t DEC_STAGE_BYTES = (STG_A + AREC_BYTES + 1023) & ~1023u;                       // 37888
+constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 37888
 constexpr int DEC_STAGES = 4;
-constexpr uint32_t PRIV_FLOATS = 128 * TOK;     // one [row][token] tile per correction warp
+constexpr uint32_t TQ_BYTES = 128 * 128;        // one quarter of T: 128 rows x 64 fp16, 128B-swizzled
 constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 16 accumulator columns + 4 stages x 32 scale columns
-constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + DEC_CORR_WARPS * PRIV_FLOATS * 4 + 1024 + 512;
+constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + 4 * TQ_BYTES + 1024 + 512;
+static_assert(DEC_STAGE_BYTES % 1024 == 0 && (STG_A + AREC_TRUE) % 1024 == 0, "swizzled tiles need 1 KiB alignment");
 
 // kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
 constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
+// kind::f16, D = f32, A = B = fp16, K-major operands, M = 128, N = 16, K = 16
+constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(TOK >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
 struct DecParams {
     const uint8_t* wblob; const uint8_t* ablob;
@@ -58,22 +64,41 @@ __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t tot
 
 __device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return __dp4a(x, 0x01010101u, 0u); }
 
-// two E4M3 pairs (4 bytes) -> two fp16 pairs, scaled by a power of two
-__device__ __forceinline__ void e4m3x4_to_h2x2(uint32_t raw, __half2 scale, uint32_t& lo, uint32_t& hi)
+// 16 E4M3 codes -> 16 fp16 (two 16-byte halves), scaled by a power of two
+__device__ __forceinline__ void e4m3x16_to_h16(const uint4& c, __half2 scale, uint4& lo, uint4& hi)
 {
-    uint32_t h0, h1;
-    const uint16_t l = (uint16_t)raw, h = (uint16_t)(raw >> 16);
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(l));
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(h));
-    const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), scale), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), scale);
-    lo = *reinterpret_cast<const uint32_t*>(&x0); hi = *reinterpret_cast<const uint32_t*>(&x1);
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t h0, h1;
+        const uint16_t l = (uint16_t)w[i], h = (uint16_t)(w[i] >> 16);
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(l));
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(h));
+        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), scale), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), scale);
+        o[2 * i] = *reinterpret_cast<const uint32_t*>(&x0); o[2 * i + 1] = *reinterpret_cast<const uint32_t*>(&x1);
+    }
+    lo = make_uint4(o[0], o[1], o[2], o[3]); hi = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
-__device__ __forceinline__ void add2(float* p, float a, float b)
+// 16 E2M1 codes (8 bytes) times an E4M3 microscale -> 16 fp16, exact
+__device__ __forceinline__ void nvfp4x16_to_h16(const uint2& c, uint32_t scale_code, uint4& lo, uint4& hi)
 {
-    float2 v = *reinterpret_cast<float2*>(p);
-    v.x += a; v.y += b;
-    *reinterpret_cast<float2*>(p) = v;
+    uint32_t sc2;
+    const uint16_t s16 = (uint16_t)(scale_code | (scale_code << 8));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
+    const __half2 sc = *reinterpret_cast<__half2*>(&sc2);
+    const uint32_t w[2] = {c.x, c.y};
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t q;
+        const uint32_t byte = (w[i >> 2] >> ((i & 3) * 8)) & 0xffu;
+        asm("{\n\t.reg .b8 t;\n\tcvt.u8.u32 t, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, t;\n\t}" : "=r"(q) : "r"(byte));
+        const __half2 x = __hmul2(*reinterpret_cast<__half2*>(&q), sc);
+        o[i] = *reinterpret_cast<const uint32_t*>(&x);
+    }
+    lo = make_uint4(o[0], o[1], o[2], o[3]); hi = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
 __global__ void __launch_bounds__(DEC_THREADS, 1)
@@ -81,17 +106,18 @@ decode_kernel(DecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    float* priv = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(priv + DEC_CORR_WARPS * PRIV_FLOATS);
-    // bars: [0,S) full, [S,2S) empty, [2S,2S+2) acc_full, [2S+2,2S+4) acc_empty, [2S+4,2S+6) segment syncs
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES + 6);
+    uint8_t* tq = smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES;                 // four quarter tiles of T
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tq + 4 * TQ_BYTES);
+    // bars (S = stages): [0,S) full, [S,2S) empty, [2S,3S) a4 ready, then per T quarter [0,4) full,
+    // [4,8) done, [8,12) cleared, then acc_full[2], acc_empty[2]
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * DEC_STAGES + 16);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + DEC_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + DEC_STAGES);
-    const uint32_t accf0 = smem_u32(bars + 2 * DEC_STAGES), acce0 = smem_u32(bars + 2 * DEC_STAGES + 2);
-    const uint32_t seg0 = smem_u32(bars + 2 * DEC_STAGES + 4);
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES, a4r0 = empty0 + 8 * DEC_STAGES;
+    const uint32_t tfull0 = a4r0 + 8 * DEC_STAGES, tdone0 = tfull0 + 32, tzero0 = tdone0 + 32;
+    const uint32_t accf0 = tzero0 + 32, acce0 = accf0 + 16;
 
     // this CTA's span of (tile, chunk) units
     const int64_t G = gridDim.x, C = p.chunks;
@@ -105,19 +131,21 @@ decode_kernel(DecParams p)
     if (warp == 0 && pf_base + lane <= p.total) pf = __ldg(uptr + pf_base + lane);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + DEC_CORR_WARPS); }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 32 * DEC_CORR_WARPS);
-            mbar_init(seg0 + 8 * b, 32 * DEC_CORR_WARPS);
+        for (int s = 0; s < DEC_STAGES; ++s) {
+            mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + SCAT_WARPS); mbar_init(a4r0 + 8 * s, SCAT_WARPS);
         }
+        for (int b = 0; b < 4; ++b) {
+            mbar_init(tfull0 + 8 * b, SCAT_WARPS); mbar_init(tdone0 + 8 * b, 1); mbar_init(tzero0 + 8 * b, SCAT_THREADS);
+        }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
-    if (warp >= 2) {                                   // the private tiles start at zero
-        float4* z = reinterpret_cast<float4*>(priv + (warp - 2) * PRIV_FLOATS);
-#pragma unroll
-        for (int i = 0; i < (int)PRIV_FLOATS / 128; ++i) z[i * 32 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (warp >= 6) {                                   // T starts all zero
+        uint4* z = reinterpret_cast<uint4*>(tq);
+        for (int i = (warp - 6) * 32 + lane; i < (int)(4 * TQ_BYTES / 16); i += SCAT_THREADS) z[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async();
     }
     tc_fence_before();
     __syncthreads();
@@ -156,7 +184,7 @@ decode_kernel(DecParams p)
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            int seg = 0;
+            int seg = 0; uint32_t useq = 0;
             for (int64_t u = u_begin; u < u_end && ok; ++seg) {
                 const int64_t tile = u / C;
                 const int64_t seg_end = min(u_end, (tile + 1) * C);
@@ -165,7 +193,7 @@ decode_kernel(DecParams p)
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
                 bool first = true;
-                for (; u < seg_end; ++u) {
+                for (; u < seg_end && ok; ++u, ++useq) {
                     if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
                     tc_fence_after();
                     const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
@@ -175,146 +203,44 @@ decode_kernel(DecParams p)
                         tmem_cp_sf(sf_t + 4 * j, smem_desc_sf(sb + REC_SF + 512 * j));
                         tmem_cp_sf(sf_t + 16 + 4 * j, smem_desc_sf(sb + STG_A + AREC_SF + 512 * j));
                     }
+                    // the scatter warps have zeroed the hot columns of the activation codes
+                    if (!(ok = mbar_wait(a4r0 + 8 * stage, phase, abort_flag, p.status, 8))) break;
+                    tc_fence_after();
                     const uint64_t adesc = smem_desc_sw128(sb + REC_W4), bdesc = smem_desc_sw128(sb + STG_A + AREC_A4);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
+                    for (int j = 0; j < 4; ++j)
                         umma_nvf4(d_tmem, adesc + 2 * j, bdesc + 2 * j, IDESC_NVF4, sf_t + 4 * j, sf_t + 16 + 4 * j,
                                   (first && j == 0) ? 0u : 1u);
-                    }
                     first = false;
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq) {
+                        if (!(ok = mbar_wait(tfull0 + 8 * qq, useq & 1u, abort_flag, p.status, 9))) break;
+                        tc_fence_after();
+                        const uint64_t ta = smem_desc_sw128(smem_u32(tq + qq * TQ_BYTES));
+                        const uint64_t tb = smem_desc_sw128(sb + STG_A + AREC_TRUE + qq * 2048);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_f16(d_tmem, ta + 2 * k, tb + 2 * k, IDESC_F16, 1u);
+                        umma_commit(tdone0 + 8 * qq);
+                    }
+                    if (!ok) break;
                     umma_commit(empty0 + 8 * stage);
                     if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (ok) umma_commit(accf0 + 8 * acc);
             }
         }
-    } else {
-        // ------------------------------------------------------------ corrections + epilogue
-        // A warp may read TMEM lanes [32q, 32q+32), q = warp % 4; two warps share a quadrant and
-        // each owns 16 of its rows for correction (3) and for the epilogue.
-        const int cw = warp - 2;                       // 0..7
-        const int q = warp & 3, h = cw >> 2;
-        const int rowbase = 32 * q + 16 * h;           // first owned row inside the tile
-        const int slice = 2 * q + h;                   // 0..7
-        const int g = lane >> 2, t = lane & 3;
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ epilogue: TMEM lane quadrant warp % 4
+        const int q = warp & 3;
         const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
-        const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
-        float* mypriv = priv + cw * PRIV_FLOATS;
-
-        int stage = 0; uint32_t phase = 0; bool ok = true;
+        bool ok = true;
         int seg = 0;
         for (int64_t u = u_begin; u < u_end && ok; ++seg) {
             const int64_t tile = u / C;
             const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
-            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-
-            for (; u < seg_end; ++u) {
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
-                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-                const uint8_t* sa = sb + STG_A;
-                const uint32_t staged = smeta[stage].staged;
-                const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
-
-                // (2) FP8 weight blocks of block columns cw and cw + 8
-                const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
-                const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z);
-                const uint32_t off8 = fgmp_rec_fp8_offset(ks0 + ks1 + ks2 + byte_sum(kc.w));
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int kb = cw + 8 * hh, wi = kb >> 2, sh8 = (kb & 3) * 8;
-                    const uint32_t word = wi == 0 ? kc.x : (wi == 1 ? kc.y : (wi == 2 ? kc.z : kc.w));
-                    const uint32_t start = (wi > 0 ? ks0 : 0u) + (wi > 1 ? ks1 : 0u) + (wi > 2 ? ks2 : 0u)
-                                         + byte_sum(word & ((1u << sh8) - 1u));
-                    const uint32_t end = start + ((word >> sh8) & 0xffu);
-                    if (start == end) continue;
-                    // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of the column
-                    const uint2 bt0 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + g * 32 + t * 8);
-                    const uint2 bt1 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + (g + 8) * 32 + t * 8);
-                    for (uint32_t e = start; e < end; e += 16) {
-                        // A fragments: FP8 blocks e + g and e + g + 8, the same four elements
-                        const uint32_t iA = e + g, iB = iA + 8;
-                        uint32_t rawA = 0, rawB = 0, rowA = 0, rowB = 0;
-                        if (iA < end) {
-                            const uint32_t o = off8 + iA * 16 + t * 4;
-                            rawA = o + 4 <= staged ? *reinterpret_cast<const uint32_t*>(sb + o) : __ldg(reinterpret_cast<const uint32_t*>(rec_g + o));
-                            rowA = REC_ROWID + iA < staged ? sb[REC_ROWID + iA] : __ldg(rec_g + REC_ROWID + iA);
-                        }
-                        if (iB < end) {
-                            const uint32_t o = off8 + iB * 16 + t * 4;
-                            rawB = o + 4 <= staged ? *reinterpret_cast<const uint32_t*>(sb + o) : __ldg(reinterpret_cast<const uint32_t*>(rec_g + o));
-                            rowB = REC_ROWID + iB < staged ? sb[REC_ROWID + iB] : __ldg(rec_g + REC_ROWID + iB);
-                        }
-                        uint32_t a0, a1, a2, a3;
-                        e4m3x4_to_h2x2(rawA, rw2, a0, a2);
-                        e4m3x4_to_h2x2(rawB, rw2, a1, a3);
-                        float c[4] = {0.f, 0.f, 0.f, 0.f}, d[4] = {0.f, 0.f, 0.f, 0.f};
-                        mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);     // tokens 2t, 2t+1
-                        mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);     // tokens 8+2t, 9+2t
-                        // c[0..1] / d[0..1]: block iA, c[2..3] / d[2..3]: block iB.  Within one column every
-                        // block has its own row, so no two lanes touch the same address here.
-                        if (iA < end) {
-                            add2(mypriv + rowA * TOK + 2 * t, c[0], c[1]);
-                            add2(mypriv + rowA * TOK + 8 + 2 * t, d[0], d[1]);
-                        }
-                        if (iB < end) {
-                            add2(mypriv + rowB * TOK + 2 * t, c[2], c[3]);
-                            add2(mypriv + rowB * TOK + 8 + 2 * t, d[2], d[3]);
-                        }
-                        __syncwarp();                  // the next group may add to the same rows
-                    }
-                }
-
-                // (3) FP8 activation blocks against the NVFP4 weights of the warp's 16 rows
-                const uint32_t am0 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + g * 2);
-                const uint32_t am1 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + (g + 8) * 2);
-                uint32_t todo = am0 | am1;             // block columns in which any token is FP8
-#pragma unroll
-                for (int o = 4; o < 32; o <<= 1) todo |= __shfl_xor_sync(0xffffffffu, todo, o);
-                while (todo) {
-                    const int kb = __ffs(todo) - 1;
-                    todo &= todo - 1;
-                    const uint32_t bit = 1u << kb;
-                    const uint2 at0 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + g * 32 + t * 8);
-                    const uint2 at1 = *reinterpret_cast<const uint2*>(sa + AREC_TRUE + kb * 512 + (g + 8) * 32 + t * 8);
-                    const uint32_t a0 = (am0 & bit) ? at0.x : 0u, a2 = (am0 & bit) ? at0.y : 0u;
-                    const uint32_t a1 = (am1 & bit) ? at1.x : 0u, a3 = (am1 & bit) ? at1.y : 0u;
-#pragma unroll
-                    for (int rg = 0; rg < 2; ++rg) {
-                        const uint32_t r = rowbase + 8 * rg + g;       // row inside the tile
-                        const uint32_t codes = *reinterpret_cast<const uint16_t*>(sb + REC_W4 + fgmp_rec_w4_offset(r, kb) + t * 2);
-                        const uint32_t sfb = sb[REC_SF + fgmp_rec_sf_offset(r, kb)];
-                        uint32_t q0, q1, sc2;
-                        asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
-                            : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
-                        const uint16_t s16 = (uint16_t)(sfb | (sfb << 8));
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
-                        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&q0), *reinterpret_cast<__half2*>(&sc2));
-                        const __half2 x1 = __hmul2(*reinterpret_cast<__half2*>(&q1), *reinterpret_cast<__half2*>(&sc2));
-                        mma_f16_16816(acc[rg], a0, a1, a2, a3, *reinterpret_cast<const uint32_t*>(&x0), *reinterpret_cast<const uint32_t*>(&x1));
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
-            }
-            if (!ok) break;
-
-            // fold the (3) sums into the warp's own tile: acc[rg] = (token g | g+8) x (row 2t | 2t+1)
-#pragma unroll
-            for (int rg = 0; rg < 2; ++rg) {
-                const int r = rowbase + 8 * rg + 2 * t;
-                mypriv[r * TOK + g] += acc[rg][0];
-                mypriv[(r + 1) * TOK + g] += acc[rg][1];
-                mypriv[r * TOK + g + 8] += acc[rg][2];
-                mypriv[(r + 1) * TOK + g + 8] += acc[rg][3];
-            }
-            // all eight tiles are complete for this segment once every correction thread is here
-            const uint32_t seg_phase = (uint32_t)(seg & 1);
-            mbar_arrive(seg0);
-            if (!(ok = mbar_wait(seg0, seg_phase, abort_flag, p.status, 6))) break;
-
+            u = seg_end;
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
@@ -322,34 +248,11 @@ decode_kernel(DecParams p)
             tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
             tc_fence_before();
             mbar_arrive(acce0 + 8 * accb);
-            // lanes 16h .. 16h+15 hold this warp's rows
-            const bool mine = (lane >> 4) == h;
-            const int lr = lane & 15;
             float v[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
-            if (mine) {
-#pragma unroll
-                for (int w = 0; w < DEC_CORR_WARPS; ++w) {
-                    const float4* src = reinterpret_cast<const float4*>(priv + w * PRIV_FLOATS + (rowbase + lr) * TOK);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float4 x = src[j];
-                        v[4 * j] += x.x; v[4 * j + 1] += x.y; v[4 * j + 2] += x.z; v[4 * j + 3] += x.w;
-                    }
-                }
-            }
-            // every warp has read all tiles before any tile is cleared for the next segment
-            mbar_arrive(seg0 + 8);
-            if (!(ok = mbar_wait(seg0 + 8, seg_phase, abort_flag, p.status, 7))) break;
-            {
-                float4* z = reinterpret_cast<float4*>(mypriv);
-#pragma unroll
-                for (int i = 0; i < (int)PRIV_FLOATS / 128; ++i) z[i * 32 + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            __syncwarp();
-
-            const int64_t n = tile * 128 + rowbase + lr;
+            const int row = 32 * q + lane;
+            const int64_t n = tile * 128 + row;
             const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
             bool write_out = whole;
             if (!whole) {
@@ -358,34 +261,46 @@ decode_kernel(DecParams p)
                 const int64_t c_last = cta_of_unit((tile + 1) * C - 1, G, p.total);
                 const int nseg = (int)(c_last - c_first + 1);
                 const int slot = (int)(blockIdx.x - c_first);
-                if (mine) {
-                    float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + rowbase + lr) * 16;
+                float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + row) * 16;
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
-                }
+                for (int j = 0; j < 16; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
                 __threadfence();
                 __syncwarp();
                 uint32_t old = 0;
-                if (lane == 0) old = atomicAdd(p.counters + tile * 8 + slice, 1u);
+                if (lane == 0) old = atomicAdd(p.counters + tile * 8 + q, 1u);
                 old = __shfl_sync(0xffffffffu, old, 0);
                 if (old == (uint32_t)(nseg - 1)) {
                     __threadfence();
+                    // all partials first (independent loads), then one sum in slot order
+                    float4 x[4][4];
+#pragma unroll
+                    for (int sgi = 0; sgi < 4; ++sgi) {
+                        const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            x[sgi][j] = sgi < nseg ? __ldcg(reinterpret_cast<const float4*>(src) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) v[j] = 0.f;
-                    if (mine) {
-                        for (int sgi = 0; sgi < nseg; ++sgi) {
-                            const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + rowbase + lr) * 16;
 #pragma unroll
-                            for (int j = 0; j < 16; j += 4) {
-                                float4 x = __ldcg(reinterpret_cast<const float4*>(src + j));
-                                v[j] += x.x; v[j + 1] += x.y; v[j + 2] += x.z; v[j + 3] += x.w;
-                            }
+                    for (int sgi = 0; sgi < 4; ++sgi) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            v[4 * j] += x[sgi][j].x; v[4 * j + 1] += x[sgi][j].y; v[4 * j + 2] += x[sgi][j].z; v[4 * j + 3] += x[sgi][j].w;
+                        }
+                    }
+                    for (int sgi = 4; sgi < nseg; ++sgi) {       // more than four contributors: rare, serial
+                        const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            const float4 y4 = __ldcg(reinterpret_cast<const float4*>(src + j));
+                            v[j] += y4.x; v[j + 1] += y4.y; v[j + 2] += y4.z; v[j + 3] += y4.w;
                         }
                     }
                     write_out = true;
                 }
             }
-            if (write_out && mine && n < p.N) {
+            if (write_out && n < p.N) {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     if (j < p.M) {
@@ -394,6 +309,119 @@ decode_kernel(DecParams p)
                     }
                 }
             }
+        }
+    } else {
+        // ------------------------------------------------------------ scatter: fill and clear T
+        const int stid = (warp - 6) * 32 + lane;       // 0..255
+        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+        const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
+        const uint32_t row = (uint32_t)stid & 127u, jh = (uint32_t)stid >> 7;     // dequant slots: columns jh and jh + 2 of a quarter
+        uint32_t mine[4][2] = {{0xffffffffu, 0xffffffffu}, {0xffffffffu, 0xffffffffu},
+                               {0xffffffffu, 0xffffffffu}, {0xffffffffu, 0xffffffffu}};  // T offsets written, two uint16 each
+
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        uint32_t useq = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++u, ++useq) {
+            if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+            uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+            uint8_t* sa = sb + STG_A;
+            const uint32_t staged = smeta[stage].staged;
+            const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
+
+            // hot columns: some token has an FP8 block there; their activation codes leave the NVFP4 product
+            const uint32_t mword = lane < 16 ? *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + lane * 2) : 0u;
+            const uint32_t hot = __reduce_or_sync(0xffffffffu, mword);
+            if ((hot >> (stid >> 4)) & 1u)
+                *reinterpret_cast<uint2*>(sa + AREC_A4 + fgmp_rec_w4_offset((uint32_t)stid & 15u, (uint32_t)stid >> 4)) = make_uint2(0, 0);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(a4r0 + 8 * stage);
+
+            const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
+            const uint32_t kcw[4] = {kc.x, kc.y, kc.z, kc.w};
+            const uint32_t ks[4] = {byte_sum(kc.x), byte_sum(kc.y), byte_sum(kc.z), byte_sum(kc.w)};
+            const uint32_t off8 = fgmp_rec_fp8_offset(ks[0] + ks[1] + ks[2] + ks[3]);
+            uint32_t qstart = 0;                       // first FP8 block of the quarter in the record's list
+#pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {
+                uint8_t* tile = tq + qq * TQ_BYTES;
+                // the previous MMAs on this quarter are done: clear what this thread wrote there
+                if (useq > 0) {
+                    if (!(ok = mbar_wait(tdone0 + 8 * qq, (useq - 1) & 1u, abort_flag, p.status, 10))) break;
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+#pragma unroll
+                        for (int hx = 0; hx < 2; ++hx) {
+                            const uint32_t o = (mine[qq][i] >> (16 * hx)) & 0xffffu;
+                            if (o != 0xffffu) {
+                                *reinterpret_cast<uint4*>(tile + o) = make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4*>(tile + (o ^ 16u)) = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+                    }
+                }
+                mbar_arrive(tzero0 + 8 * qq);
+                mine[qq][0] = 0xffffffffu; mine[qq][1] = 0xffffffffu;
+
+                // inputs of this thread's items: FP8 blocks stid and stid + 256 of the quarter, and the NVFP4
+                // blocks (row, column jh) and (row, column jh + 2) if those columns are hot
+                const uint32_t c0 = kcw[qq] & 0xffu, c1 = (kcw[qq] >> 8) & 0xffu, c2 = (kcw[qq] >> 16) & 0xffu;
+                const uint32_t n8 = ks[qq];
+                uint4 raw8[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+                uint32_t pos8[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const uint32_t it = (uint32_t)stid + 256u * i;
+                    pos8[i] = 0xffffu;
+                    if (it < n8) {
+                        const uint32_t e = qstart + it;
+                        const uint32_t o = off8 + e * 16;
+                        raw8[i] = o + 16 <= staged ? *reinterpret_cast<const uint4*>(sb + o) : __ldg(reinterpret_cast<const uint4*>(rec_g + o));
+                        const uint32_t r = REC_ROWID + e < staged ? sb[REC_ROWID + e] : __ldg(rec_g + REC_ROWID + e);
+                        const uint32_t jq = (it >= c0) + (it >= c0 + c1) + (it >= c0 + c1 + c2);
+                        pos8[i] = fgmp_h16_tile_offset(r, jq, 0);
+                    }
+                }
+                uint2 raw4[2] = {make_uint2(0, 0), make_uint2(0, 0)};
+                uint32_t sc4[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const uint32_t jq = jh + 2u * i, j = 4u * qq + jq;
+                    sc4[i] = 0;
+                    if ((hot >> j) & 1u) {
+                        sc4[i] = sb[REC_SF + fgmp_rec_sf_offset(row, j)];
+                        raw4[i] = *reinterpret_cast<const uint2*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j));
+                    }
+                }
+                // every thread has cleared its part of the quarter
+                if (!(ok = mbar_wait(tzero0 + 8 * qq, useq & 1u, abort_flag, p.status, 11))) break;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    if (pos8[i] != 0xffffu) {
+                        uint4 lo, hi;
+                        e4m3x16_to_h16(raw8[i], rw2, lo, hi);
+                        *reinterpret_cast<uint4*>(tile + pos8[i]) = lo;
+                        *reinterpret_cast<uint4*>(tile + (pos8[i] ^ 16u)) = hi;
+                        mine[qq][0] = (mine[qq][0] & ~(0xffffu << (16 * i))) | (pos8[i] << (16 * i));
+                    }
+                    if (sc4[i] != 0) {                 // microscale 0: the block is FP8 or all zero
+                        uint4 lo, hi;
+                        nvfp4x16_to_h16(raw4[i], sc4[i], lo, hi);
+                        const uint32_t o = fgmp_h16_tile_offset(row, jh + 2u * i, 0);
+                        *reinterpret_cast<uint4*>(tile + o) = lo;
+                        *reinterpret_cast<uint4*>(tile + (o ^ 16u)) = hi;
+                        mine[qq][1] = (mine[qq][1] & ~(0xffffu << (16 * i))) | (o << (16 * i));
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tfull0 + 8 * qq);
+                qstart += n8;
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+            if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
         }
     }
 

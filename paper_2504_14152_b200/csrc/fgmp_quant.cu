@@ -46,8 +46,9 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                 const uint32_t j = (uint32_t)kb & 15u, m = (uint32_t)m0;
                 *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset(m, j)) = make_uint2(0, 0);
                 rec[AREC_SF + fgmp_rec_sf_offset(m, j)] = 0;
-                uint4* dst = reinterpret_cast<uint4*>(rec + AREC_TRUE + j * 512 + m * 32);
-                dst[0] = make_uint4(0, 0, 0, 0); dst[1] = make_uint4(0, 0, 0, 0);
+                uint8_t* tile = rec + AREC_TRUE + (j >> 2) * 2048;
+                *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset(m, j & 3, 0)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset(m, j & 3, 1)) = make_uint4(0, 0, 0, 0);
                 if (j == 0) *reinterpret_cast<uint16_t*>(rec + AREC_MASK + m * 2) = 0;
             }
             return;
@@ -119,8 +120,9 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                     }
                     uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
                     const uint32_t j = (uint32_t)kb & 15u;
-                    uint4* dst = reinterpret_cast<uint4*>(rec + AREC_TRUE + j * 512 + (uint32_t)m * 32);
-                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]); dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                    uint8_t* tile = rec + AREC_TRUE + (j >> 2) * 2048;
+                    *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset((uint32_t)m, j & 3, 0)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset((uint32_t)m, j & 3, 1)) = make_uint4(o[4], o[5], o[6], o[7]);
                     *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset((uint32_t)m, j)) = make_uint2(c4[0], c4[1]);
                     rec[AREC_SF + fgmp_rec_sf_offset((uint32_t)m, j)] = (uint8_t)sc;
                 }
