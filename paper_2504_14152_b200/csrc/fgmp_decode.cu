@@ -21,8 +21,8 @@
 // that arrives last; the accumulation order inside TMEM is the issue order: results are
 // reproducible bit for bit.
 //
-// Warp roles (448 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2-5 = epilogue (one TMEM lane quadrant each), warps 6-13 = scatter.
+// Warp roles (704 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2-5 = epilogue (one TMEM lane quadrant each), warps 6-21 = scatter (eight groups of two).
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
@@ -30,8 +30,8 @@
 
 namespace {
 
-constexpr int DEC_THREADS = 448;
-constexpr int SCAT_WARPS = 8, SCAT_THREADS = 256;
+constexpr int DEC_THREADS = 704;
+constexpr int SCAT_THREADS = 512, GRP_WARPS = 2, GRP_THREADS = 64;   // eight groups: (quarter of T, unit parity)
 constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
 constexpr uint32_t FP8_CAP_BLOCKS = 320;        // FP8 blocks of a unit that fit a stage; more are read from global
 constexpr uint32_t WREC_CAP = (REC_ROWID + FP8_CAP_BLOCKS + FP8_CAP_BLOCKS * 16 + 127) & ~127u;   // 23936
@@ -39,14 +39,27 @@ constexpr uint32_t STG_A = (WREC_CAP + 1023) & ~1023u;                          
 constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 37888
 constexpr int DEC_STAGES = 4;
 constexpr uint32_t TQ_BYTES = 128 * 128;        // one quarter of T: 128 rows x 64 fp16, 128B-swizzled
-constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 16 accumulator columns + 4 stages x 32 scale columns
-constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + 4 * TQ_BYTES + 1024 + 512;
+constexpr int NACC = 4;                         // independent accumulators per tile: back-to-back MMAs into one
+                                                // accumulator wait for each other, so the MMAs of a unit rotate over four
+constexpr uint32_t ACC_COLS = NACC * TOK;       // columns of one accumulator buffer
+constexpr uint32_t SF_COL0 = 2 * ACC_COLS;      // scale columns start behind the two accumulator buffers
+constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 64 accumulator columns + 4 stages x 32 scale columns
+constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + 4 * TQ_BYTES + 1024 /*alignment*/ + 512 /*barriers*/ + 8192 /*lists*/;
 static_assert(DEC_STAGE_BYTES % 1024 == 0 && (STG_A + AREC_TRUE) % 1024 == 0, "swizzled tiles need 1 KiB alignment");
 
 // kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
 constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
 // kind::f16, D = f32, A = B = fp16, K-major operands, M = 128, N = 16, K = 16
 constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(TOK >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+// shared-memory matrix descriptors as (low word | start address >> 4, constant high word)
+constexpr uint32_t SW128_LO = 1u << 16, SW128_HI = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128B swizzle, 8-row groups 1 KiB apart
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
 
 struct DecParams {
     const uint8_t* wblob; const uint8_t* ablob;
@@ -108,16 +121,20 @@ decode_kernel(DecParams p)
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* tq = smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES;                 // four quarter tiles of T
     uint64_t* bars = reinterpret_cast<uint64_t*>(tq + 4 * TQ_BYTES);
-    // bars (S = stages): [0,S) full, [S,2S) empty, [2S,3S) a4 ready, then per T quarter [0,4) full,
-    // [4,8) done, [8,12) cleared, then acc_full[2], acc_empty[2]
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * DEC_STAGES + 16);
+    // bars (S = stages): [0,S) full, [S,2S) empty, [2S,3S) a4 ready, then T quarter full [4], T quarter
+    // done [2 unit parities][4] (a parity wait can only tell two consecutive phases apart, so each of
+    // the two groups that share a quarter has a barrier of its own), scatter group sync [8],
+    // acc_full[2], acc_empty[2]
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * DEC_STAGES + 28);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + DEC_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint32_t* qcnt = tmem_slot + 2;                                            // [4 quarters]
+    uint16_t* qlist = reinterpret_cast<uint16_t*>(tq + 4 * TQ_BYTES + 512);     // [4 quarters][1024]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES, a4r0 = empty0 + 8 * DEC_STAGES;
-    const uint32_t tfull0 = a4r0 + 8 * DEC_STAGES, tdone0 = tfull0 + 32, tzero0 = tdone0 + 32;
-    const uint32_t accf0 = tzero0 + 32, acce0 = accf0 + 16;
+    const uint32_t tfull0 = a4r0 + 8 * DEC_STAGES, tdone0 = tfull0 + 32, gbar0 = tdone0 + 64;
+    const uint32_t accf0 = gbar0 + 64, acce0 = accf0 + 16;
 
     // this CTA's span of (tile, chunk) units
     const int64_t G = gridDim.x, C = p.chunks;
@@ -132,13 +149,15 @@ decode_kernel(DecParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < DEC_STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + SCAT_WARPS); mbar_init(a4r0 + 8 * s, SCAT_WARPS);
+            mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + 8); mbar_init(a4r0 + 8 * s, 8);   // 8 scatter warps serve a unit
         }
         for (int b = 0; b < 4; ++b) {
-            mbar_init(tfull0 + 8 * b, SCAT_WARPS); mbar_init(tdone0 + 8 * b, 1); mbar_init(tzero0 + 8 * b, SCAT_THREADS);
+            mbar_init(tfull0 + 8 * b, GRP_WARPS); mbar_init(tdone0 + 8 * b, 1); mbar_init(tdone0 + 32 + 8 * b, 1);
+            mbar_init(gbar0 + 8 * b, GRP_WARPS); mbar_init(gbar0 + 32 + 8 * b, GRP_WARPS);
         }
         for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
         *abort_flag = 0;
+        for (int i = 0; i < 4; ++i) qcnt[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
@@ -182,52 +201,57 @@ decode_kernel(DecParams p)
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0; bool ok = true;
-            int seg = 0; uint32_t useq = 0;
-            for (int64_t u = u_begin; u < u_end && ok; ++seg) {
-                const int64_t tile = u / C;
-                const int64_t seg_end = min(u_end, (tile + 1) * C);
-                const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
-                if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
+        // The whole warp walks the loop (its values stay warp-uniform, which keeps the descriptor
+        // arithmetic cheap); lane 0 alone issues the tcgen05 instructions, so that every commit
+        // tracks every MMA before it.
+        const uint32_t smem0 = smem_u32(smem), tq0 = smem_u32(tq);
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0; uint32_t useq = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
+            const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
+            if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)acc * ACC_COLS;
+            uint32_t accum = 0;
+            for (; u < seg_end && ok; ++u, ++useq) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
-                bool first = true;
-                for (; u < seg_end && ok; ++u, ++useq) {
-                    if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
-                    tc_fence_after();
-                    const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
-                    const uint32_t sf_t = tmem_base + 32 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        tmem_cp_sf(sf_t + 4 * j, smem_desc_sf(sb + REC_SF + 512 * j));
-                        tmem_cp_sf(sf_t + 16 + 4 * j, smem_desc_sf(sb + STG_A + AREC_SF + 512 * j));
-                    }
-                    // the scatter warps have zeroed the hot columns of the activation codes
-                    if (!(ok = mbar_wait(a4r0 + 8 * stage, phase, abort_flag, p.status, 8))) break;
-                    tc_fence_after();
-                    const uint64_t adesc = smem_desc_sw128(sb + REC_W4), bdesc = smem_desc_sw128(sb + STG_A + AREC_A4);
+                const uint32_t sb = smem0 + (uint32_t)stage * DEC_STAGE_BYTES;
+                const uint32_t sf_t = tmem_base + SF_COL0 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
+                // the scatter warps have put the microscales into TMEM and zeroed the hot columns of the
+                // activation codes
+                if (!(ok = mbar_wait(a4r0 + 8 * stage, phase, abort_flag, p.status, 8))) break;
+                tc_fence_after();
+                const uint32_t w4_lo = ((sb + REC_W4) >> 4) | SW128_LO, a4_lo = ((sb + STG_A + AREC_A4) >> 4) | SW128_LO;
+                if (lane == 0) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        umma_nvf4(d_tmem, adesc + 2 * j, bdesc + 2 * j, IDESC_NVF4, sf_t + 4 * j, sf_t + 16 + 4 * j,
-                                  (first && j == 0) ? 0u : 1u);
-                    first = false;
-#pragma unroll
-                    for (int qq = 0; qq < 4; ++qq) {
-                        if (!(ok = mbar_wait(tfull0 + 8 * qq, useq & 1u, abort_flag, p.status, 9))) break;
-                        tc_fence_after();
-                        const uint64_t ta = smem_desc_sw128(smem_u32(tq + qq * TQ_BYTES));
-                        const uint64_t tb = smem_desc_sw128(sb + STG_A + AREC_TRUE + qq * 2048);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_f16(d_tmem, ta + 2 * k, tb + 2 * k, IDESC_F16, 1u);
-                        umma_commit(tdone0 + 8 * qq);
-                    }
-                    if (!ok) break;
-                    umma_commit(empty0 + 8 * stage);
-                    if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+                        umma_nvf4(d_tmem + j * TOK, desc64(w4_lo + 2 * j, SW128_HI), desc64(a4_lo + 2 * j, SW128_HI), IDESC_NVF4,
+                                  sf_t + 4 * j, sf_t + 16 + 4 * j, accum);
                 }
-                if (ok) umma_commit(accf0 + 8 * acc);
+                accum = 1;
+                const uint32_t at_lo = ((sb + STG_A + AREC_TRUE) >> 4) | SW128_LO;
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    if (!(ok = mbar_wait(tfull0 + 8 * qq, useq & 1u, abort_flag, p.status, 9))) break;
+                    tc_fence_after();
+                    const uint32_t t_lo = ((tq0 + qq * TQ_BYTES) >> 4) | SW128_LO;
+                    if (lane == 0) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            umma_f16(d_tmem + k * TOK, desc64(t_lo + 2 * k, SW128_HI), desc64(at_lo + qq * 128 + 2 * k, SW128_HI), IDESC_F16, 1u);
+                        umma_commit(tdone0 + 32 * (useq & 1u) + 8 * qq);
+                    }
+                }
+                if (!ok) break;
+                if (lane == 0) umma_commit(empty0 + 8 * stage);
+                __syncwarp();
+                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
             }
+            if (ok && lane == 0) umma_commit(accf0 + 8 * acc);
+            __syncwarp();
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------ epilogue: TMEM lane quadrant warp % 4
@@ -244,13 +268,18 @@ decode_kernel(DecParams p)
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
-            uint32_t rr[16];
-            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
-            tc_fence_before();
-            mbar_arrive(acce0 + 8 * accb);
             float v[16];
+            {
+                // the four partial accumulators of the tile, added in a fixed order
+                uint32_t r0[16], r1[16], r2[16], r3[16];
+                const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)accb * ACC_COLS;
+                tmem_ld16(t0, r0); tmem_ld16(t0 + TOK, r1); tmem_ld16(t0 + 2 * TOK, r2); tmem_ld16(t0 + 3 * TOK, r3);
+                tc_fence_before();
+                mbar_arrive(acce0 + 8 * accb);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
+                for (int j = 0; j < 16; ++j)
+                    v[j] = ((__uint_as_float(r0[j]) + __uint_as_float(r1[j])) + __uint_as_float(r2[j])) + __uint_as_float(r3[j]);
+            }
             const int row = 32 * q + lane;
             const int64_t n = tile * 128 + row;
             const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
@@ -312,116 +341,158 @@ decode_kernel(DecParams p)
         }
     } else {
         // ------------------------------------------------------------ scatter: fill and clear T
-        const int stid = (warp - 6) * 32 + lane;       // 0..255
+        // Eight groups of two warps: group (q, h) owns quarter q of T for the units of parity h, so a
+        // group has two unit times per unit and the two groups of a quarter take turns on its tile.
+        // Per unit a group zeroes the hot columns of its quarter in the activation codes, (four of the
+        // warps) loads the microscales into TMEM, converts its blocks, and then, once the previous
+        // unit's MMAs on the quarter are done, clears what that unit left there and stores its own.
+        const int sw = warp - 6;                       // 0..15
+        const int half = sw >> 3, qq = (sw >> 1) & 3;  // unit parity served, quarter owned
+        const int grp = sw >> 1;                       // 0..7
+        const int gtid = (sw & 1) * 32 + lane;         // 0..63 inside the group
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
-        const uint32_t row = (uint32_t)stid & 127u, jh = (uint32_t)stid >> 7;     // dequant slots: columns jh and jh + 2 of a quarter
-        uint32_t mine[4][2] = {{0xffffffffu, 0xffffffffu}, {0xffffffffu, 0xffffffffu},
-                               {0xffffffffu, 0xffffffffu}, {0xffffffffu, 0xffffffffu}};  // T offsets written, two uint16 each
+        uint8_t* tile = tq + qq * TQ_BYTES;
+        uint16_t* list = qlist + qq * 1024;            // T offsets written for the last unit in this quarter (0xffff = none)
 
-        int stage = 0; uint32_t phase = 0; bool ok = true;
-        uint32_t useq = 0;
-        for (int64_t u = u_begin; u < u_end && ok; ++u, ++useq) {
-            if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+        bool ok = true;
+        uint32_t gphase = 0;
+        for (int64_t useq = half; u_begin + useq < u_end && ok; useq += 2) {
+            const int stage = (int)(useq & 3);
+            const uint32_t phase = (uint32_t)(useq >> 2) & 1u;
             uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
             uint8_t* sa = sb + STG_A;
+            if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
             const uint32_t staged = smeta[stage].staged;
             const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
 
             // hot columns: some token has an FP8 block there; their activation codes leave the NVFP4 product
             const uint32_t mword = lane < 16 ? *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + lane * 2) : 0u;
             const uint32_t hot = __reduce_or_sync(0xffffffffu, mword);
-            if ((hot >> (stid >> 4)) & 1u)
-                *reinterpret_cast<uint2*>(sa + AREC_A4 + fgmp_rec_w4_offset((uint32_t)stid & 15u, (uint32_t)stid >> 4)) = make_uint2(0, 0);
+            {
+                const uint32_t col = 4u * qq + ((uint32_t)gtid >> 4), tok = (uint32_t)gtid & 15u;
+                if ((hot >> col) & 1u) *reinterpret_cast<uint2*>(sa + AREC_A4 + fgmp_rec_w4_offset(tok, col)) = make_uint2(0, 0);
+            }
             fence_proxy_async();
+            if ((sw & 7) < 4) {
+                // Microscales of the stage into TMEM, one warp per lane quadrant (warp % 4): lane i holds,
+                // for MMA step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3,
+                // which is 16 bytes of scale tile j; the token scales follow in columns 16..31.
+                uint32_t r[16];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
+                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                }
+                const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
+                tmem_st16(sf_t, r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 x = *reinterpret_cast<const uint4*>(sa + AREC_SF + 512 * j + lane * 16);
+                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                }
+                tmem_st16(sf_t + 16, r);
+                tmem_wait_st();
+                tc_fence_before();
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(a4r0 + 8 * stage);
 
             const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
-            const uint32_t kcw[4] = {kc.x, kc.y, kc.z, kc.w};
-            const uint32_t ks[4] = {byte_sum(kc.x), byte_sum(kc.y), byte_sum(kc.z), byte_sum(kc.w)};
-            const uint32_t off8 = fgmp_rec_fp8_offset(ks[0] + ks[1] + ks[2] + ks[3]);
-            uint32_t qstart = 0;                       // first FP8 block of the quarter in the record's list
-#pragma unroll
-            for (int qq = 0; qq < 4; ++qq) {
-                uint8_t* tile = tq + qq * TQ_BYTES;
-                // the previous MMAs on this quarter are done: clear what this thread wrote there
-                if (useq > 0) {
-                    if (!(ok = mbar_wait(tdone0 + 8 * qq, (useq - 1) & 1u, abort_flag, p.status, 10))) break;
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-#pragma unroll
-                        for (int hx = 0; hx < 2; ++hx) {
-                            const uint32_t o = (mine[qq][i] >> (16 * hx)) & 0xffffu;
-                            if (o != 0xffffu) {
-                                *reinterpret_cast<uint4*>(tile + o) = make_uint4(0, 0, 0, 0);
-                                *reinterpret_cast<uint4*>(tile + (o ^ 16u)) = make_uint4(0, 0, 0, 0);
-                            }
-                        }
-                    }
-                }
-                mbar_arrive(tzero0 + 8 * qq);
-                mine[qq][0] = 0xffffffffu; mine[qq][1] = 0xffffffffu;
+            const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z), ks3 = byte_sum(kc.w);
+            const uint32_t off8 = fgmp_rec_fp8_offset(ks0 + ks1 + ks2 + ks3);
+            const uint32_t kword = qq == 0 ? kc.x : (qq == 1 ? kc.y : (qq == 2 ? kc.z : kc.w));
+            const uint32_t n8 = qq == 0 ? ks0 : (qq == 1 ? ks1 : (qq == 2 ? ks2 : ks3));
+            const uint32_t qstart = (qq > 0 ? ks0 : 0u) + (qq > 1 ? ks1 : 0u) + (qq > 2 ? ks2 : 0u);
+            const uint32_t c0 = kword & 0xffu, c1 = (kword >> 8) & 0xffu, c2 = (kword >> 16) & 0xffu;
+            const uint32_t hotq = (hot >> (4 * qq)) & 15u;
+            const uint32_t nhot = __popc(hotq);
 
-                // inputs of this thread's items: FP8 blocks stid and stid + 256 of the quarter, and the NVFP4
-                // blocks (row, column jh) and (row, column jh + 2) if those columns are hot
-                const uint32_t c0 = kcw[qq] & 0xffu, c1 = (kcw[qq] >> 8) & 0xffu, c2 = (kcw[qq] >> 16) & 0xffu;
-                const uint32_t n8 = ks[qq];
-                uint4 raw8[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                uint32_t pos8[2];
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const uint32_t it = (uint32_t)stid + 256u * i;
-                    pos8[i] = 0xffffu;
-                    if (it < n8) {
-                        const uint32_t e = qstart + it;
-                        const uint32_t o = off8 + e * 16;
-                        raw8[i] = o + 16 <= staged ? *reinterpret_cast<const uint4*>(sb + o) : __ldg(reinterpret_cast<const uint4*>(rec_g + o));
-                        const uint32_t r = REC_ROWID + e < staged ? sb[REC_ROWID + e] : __ldg(rec_g + REC_ROWID + e);
-                        const uint32_t jq = (it >= c0) + (it >= c0 + c1) + (it >= c0 + c1 + c2);
-                        pos8[i] = fgmp_h16_tile_offset(r, jq, 0);
-                    }
+            // One FP8 block of the quarter (list entries qstart .. qstart + n8, ordered by (column, row)):
+            // where it goes in T and its 16 values as fp16.
+            auto fp8_item = [&](uint32_t it, uint32_t& pos, uint4& lo, uint4& hi) {
+                const uint32_t e = qstart + it;
+                const uint32_t o = off8 + e * 16;
+                const uint4 raw = o + 16 <= staged ? *reinterpret_cast<const uint4*>(sb + o) : __ldg(reinterpret_cast<const uint4*>(rec_g + o));
+                const uint32_t r = REC_ROWID + e < staged ? sb[REC_ROWID + e] : __ldg(rec_g + REC_ROWID + e);
+                const uint32_t jq = (it >= c0) + (it >= c0 + c1) + (it >= c0 + c1 + c2);
+                pos = fgmp_h16_tile_offset(r, jq, 0);
+                e4m3x16_to_h16(raw, rw2, lo, hi);
+            };
+            // The NVFP4 block of a row in hot column jq of the quarter; pos = 0xffff when its microscale
+            // is 0 (the block is FP8 or all zero) and nothing is to be written.
+            auto hot_item = [&](uint32_t row, uint32_t jq, uint32_t& pos, uint4& lo, uint4& hi) {
+                const uint32_t j = 4u * qq + jq;
+                const uint32_t sc = sb[REC_SF + fgmp_rec_sf_offset(row, j)];
+                pos = 0xffffu;
+                if (sc != 0) {
+                    pos = fgmp_h16_tile_offset(row, jq, 0);
+                    nvfp4x16_to_h16(*reinterpret_cast<const uint2*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j)), sc, lo, hi);
                 }
-                uint2 raw4[2] = {make_uint2(0, 0), make_uint2(0, 0)};
-                uint32_t sc4[2];
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const uint32_t jq = jh + 2u * i, j = 4u * qq + jq;
-                    sc4[i] = 0;
-                    if ((hot >> j) & 1u) {
-                        sc4[i] = sb[REC_SF + fgmp_rec_sf_offset(row, j)];
-                        raw4[i] = *reinterpret_cast<const uint2*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j));
-                    }
+            };
+            auto put = [&](uint32_t slot, uint32_t pos, const uint4& lo, const uint4& hi) {
+                list[slot] = (uint16_t)pos;
+                if (pos != 0xffffu) {
+                    *reinterpret_cast<uint4*>(tile + pos) = lo;
+                    *reinterpret_cast<uint4*>(tile + (pos ^ 16u)) = hi;
                 }
-                // every thread has cleared its part of the quarter
-                if (!(ok = mbar_wait(tzero0 + 8 * qq, useq & 1u, abort_flag, p.status, 11))) break;
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    if (pos8[i] != 0xffffu) {
-                        uint4 lo, hi;
-                        e4m3x16_to_h16(raw8[i], rw2, lo, hi);
-                        *reinterpret_cast<uint4*>(tile + pos8[i]) = lo;
-                        *reinterpret_cast<uint4*>(tile + (pos8[i] ^ 16u)) = hi;
-                        mine[qq][0] = (mine[qq][0] & ~(0xffffu << (16 * i))) | (pos8[i] << (16 * i));
-                    }
-                    if (sc4[i] != 0) {                 // microscale 0: the block is FP8 or all zero
-                        uint4 lo, hi;
-                        nvfp4x16_to_h16(raw4[i], sc4[i], lo, hi);
-                        const uint32_t o = fgmp_h16_tile_offset(row, jh + 2u * i, 0);
-                        *reinterpret_cast<uint4*>(tile + o) = lo;
-                        *reinterpret_cast<uint4*>(tile + (o ^ 16u)) = hi;
-                        mine[qq][1] = (mine[qq][1] & ~(0xffffu << (16 * i))) | (o << (16 * i));
-                    }
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tfull0 + 8 * qq);
-                qstart += n8;
+            };
+
+            // converted ahead of the wait below: this thread's first FP8 block and its two rows of the first hot column
+            uint32_t posA = 0xffffu, posB = 0xffffu, posC = 0xffffu;
+            uint4 loA = make_uint4(0, 0, 0, 0), hiA = loA, loB = loA, hiB = loA, loC = loA, hiC = loA;
+            if ((uint32_t)gtid < n8) fp8_item((uint32_t)gtid, posA, loA, hiA);
+            const uint32_t jq_first = hotq ? (uint32_t)__ffs(hotq) - 1u : 0u;
+            if (hotq) {
+                hot_item((uint32_t)gtid, jq_first, posB, loB, hiB);
+                hot_item((uint32_t)gtid + 64u, jq_first, posC, loC, hiC);
             }
-            if (!ok) break;
+
+            // the previous unit's MMAs on this quarter are done: clear what was written for it
+            if (useq > 0) {
+                if (!(ok = mbar_wait(tdone0 + 32 * (uint32_t)((useq - 1) & 1) + 8 * qq, (uint32_t)((useq - 1) >> 1) & 1u,
+                                     abort_flag, p.status, 10))) break;
+                const uint32_t n_old = qcnt[qq];
+                for (uint32_t i = gtid; i < n_old; i += GRP_THREADS) {
+                    const uint32_t o = list[i];
+                    if (o != 0xffffu) {
+                        *reinterpret_cast<uint4*>(tile + o) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(tile + (o ^ 16u)) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-            if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+            if (lane == 0) mbar_arrive(gbar0 + 8 * grp);          // the whole group has cleared its share
+            if (!(ok = mbar_wait(gbar0 + 8 * grp, gphase, abort_flag, p.status, 11))) break;
+            gphase ^= 1u;
+            if (gtid == 0) qcnt[qq] = n8 + nhot * 128u;
+
+            // list slots: [0, n8) the FP8 blocks, then 128 per hot column in column order
+            if ((uint32_t)gtid < n8) put((uint32_t)gtid, posA, loA, hiA);
+            for (uint32_t it = gtid + GRP_THREADS; it < n8; it += GRP_THREADS) {
+                uint32_t pos; uint4 lo, hi;
+                fp8_item(it, pos, lo, hi);
+                put(it, pos, lo, hi);
+            }
+            if (hotq) {
+                put(n8 + (uint32_t)gtid, posB, loB, hiB);
+                put(n8 + (uint32_t)gtid + 64u, posC, loC, hiC);
+                uint32_t rest = hotq & (hotq - 1u), slot = n8 + 128u + (uint32_t)gtid;
+                while (rest) {
+                    const uint32_t jq = (uint32_t)__ffs(rest) - 1u;
+                    rest &= rest - 1u;
+#pragma unroll
+                    for (uint32_t rr = 0; rr < 2; ++rr) {
+                        uint32_t pos; uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
+                        hot_item((uint32_t)gtid + 64u * rr, jq, pos, lo, hi);
+                        put(slot + 64u * rr, pos, lo, hi);
+                    }
+                    slot += 128u;
+                }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(tfull0 + 8 * qq); mbar_arrive(empty0 + 8 * stage); }
         }
     }
 
