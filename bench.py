@@ -57,52 +57,87 @@ def algorithmic_act_bytes(M, K, p):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons of one GPU while the timed region runs.
+
+    NVML is polled from a background thread as fast as it answers (a timed region of a few
+    milliseconds still gets samples); if NVML is not importable, `nvidia-smi -lms` is used."""
+    REASONS = (("hw_slowdown", 0x8), ("sw_power_cap", 0x4), ("sw_thermal_slowdown", 0x20),
+               ("hw_thermal_slowdown", 0x40))
 
     def __init__(self, index: int):
-        self.rows, self.proc, self.index = [], None, index
+        self.index, self.sm, self.mx, self.reasons = index, [], None, set()
+        self.stop = threading.Event()
+        self.thread = None
+        self.proc = None
 
-    def __enter__(self):
+    def _poll_nvml(self):
+        import pynvml
+        pynvml.nvmlInit()
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.t = threading.Thread(target=self._read, daemon=True)
-            self.t.start()
-        except Exception:
-            self.proc = None
-        return self
+            # the visible device order may differ from NVML's: map through the PCI bus id
+            bus = torch.cuda.get_device_properties(self.index).pci_bus_id if hasattr(
+                torch.cuda.get_device_properties(self.index), "pci_bus_id") else None
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            if bus is not None:
+                for i in range(pynvml.nvmlDeviceGetCount()):
+                    hi = pynvml.nvmlDeviceGetHandleByIndex(i)
+                    if pynvml.nvmlDeviceGetPciInfo(hi).bus == bus:
+                        h = hi
+                        break
+            self.mx = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while True:
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                bits = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                for name, bit in self.REASONS:
+                    if bits & bit:
+                        self.reasons.add(name)
+                if self.stop.is_set():
+                    break
+                time.sleep(0.001)
+        finally:
+            pynvml.nvmlShutdown()
 
-    def _read(self):
+    def _poll_smi(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.sw_power_cap,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.hw_thermal_slowdown")
+        self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
+                                      "--format=csv,noheader,nounits", "-lms", "50"],
+                                     stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
-
-    def __exit__(self, *a):
-        if self.proc:
-            self.proc.terminate()
+            c = [x.strip() for x in line.split(",")]
             try:
-                self.proc.wait(timeout=5)
-            except Exception:
-                self.proc.kill()
-
-    def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-                for n, v in zip(names, r[4:8]):
+                self.sm.append(float(c[0])); self.mx = float(c[1])
+                for (name, _), v in zip(self.REASONS, c[2:6]):
                     if v.lower().startswith("active"):
-                        reasons.add(n)
+                        self.reasons.add(name)
             except Exception:
                 pass
-        if not sm:
+
+    def _run(self):
+        try:
+            self._poll_nvml()
+        except Exception:
+            try:
+                self._poll_smi()
+            except Exception:
+                pass
+
+    def __enter__(self):
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        if self.proc:
+            self.proc.terminate()
+        self.thread.join(timeout=5)
+
+    def summary(self):
+        if not self.sm:
             return None
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.mx, "reasons": sorted(self.reasons),
+                "samples": len(self.sm)}
 
 
 def dist_setup(n_gpus):
@@ -187,20 +222,50 @@ def run_ours(args, world, rank, local):
         step(i)
     fg.check(ws)
 
-    timed = ("expand_weights", "gemm_bf16_tcgen05", "decode_gemm", "quant_act")
+    # ---- the timed region: K steps, replayed from one CUDA graph when capture works (the step is
+    # launch-bound at decode sizes: two short kernels and a memset), else launched eagerly
+    graph, graph_note = None, "eager launches"
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for i in range(args.steps):
+                        step(i)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph, graph_note = g, f"one CUDA graph of {args.steps} steps"
+        except Exception as e:  # capture is an optimisation of the launch path, not of the kernels
+            graph_note = f"eager launches (graph capture failed: {type(e).__name__})"
+            torch.cuda.synchronize()
+    if graph is not None:
+        graph.replay()                                  # untimed: uploads the graph
     barrier_and_sync(world)
     with ClockSampler(local) as clk:
-        fg.profile_begin(timed)
         ev[0].record()
-        for i in range(args.steps):
-            step(i)
+        if graph is not None:
+            graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
         ev[1].record()
         barrier_and_sync(world)
-        prof = fg.profile_end()
     ms = ev[0].elapsed_time(ev[1])
     fg.check(ws)
     ms = max_over_ranks(ms, world)
     clocks = clk.summary()
+
+    # ---- the same K steps once more, launched eagerly with CUDA events around every launch of the
+    # kernels below (recorded by the library on the launch stream): launch counts and kernel durations
+    timed = ("expand_weights", "gemm_bf16_tcgen05", "decode_gemm", "quant_act")
+    fg.profile_begin(timed)
+    for i in range(args.steps):
+        step(i)
+    barrier_and_sync(world)
+    prof = fg.profile_end()
+    fg.check(ws)
 
     # ---- end to end: host buffers, H2D of the step's activations and D2H of its result inside
     x_host = x_cpu.pin_memory()
@@ -261,12 +326,14 @@ def run_ours(args, world, rank, local):
     out = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "nvfp4+e4m3 operands, f32 accumulate", "data": "synthetic",
+        "dtype": "nvfp4+fp8e4m3/f32acc", "data": "synthetic",
         "config": {"workload": args.workload, "M": M, "N": N, "K": K, "fp8_fraction_weights": p,
                    "fp8_fraction_activations": p, "score_mode": "lp_error(Eq.6)", "clip": "sw_brute(Eq.11)",
                    "l2": f"rotating {n_copies} packed weight copies ({n_copies * wbytes / 1e6:.0f} MB > 126 MB L2)"
                    if kind == "decode" else "operands + bf16 planes exceed L2",
-                   "step": "quantize_activations + linear (online path); weight packing is offline"},
+                   "step": "quantize_activations + linear (online path); weight packing is offline",
+                   "launch": graph_note,
+                   "kernel_times": "second pass of the same steps, CUDA events around each launch"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": x_cpu.numel() * 2,
                 "d2h_bytes_per_step": M * N * 4, "ms_per_step": e2e_ms / args.steps},
@@ -364,6 +431,7 @@ def main():
     ap.add_argument("--workload", default="llama2-7b-fc1-decode", choices=sorted(WORKLOADS))
     ap.add_argument("--m", type=int, default=0, help="override the token count M")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the timed steps eagerly")
     args = ap.parse_args()
 
     if args.impl == "reference":
