@@ -1,56 +1,54 @@
 // fgmp_linear for decode-sized batches (M <= 16 tokens): a weight-streaming kernel that
 // reads the packed weights exactly once (Section 4.1 of the paper: the four block-pair
-// products, FP32 accumulation).  All arithmetic runs on the tensor cores; the CUDA cores only
-// move and convert the few blocks that need it.
+// products, FP32 accumulation).
 //
-// Decomposition (exact).  Call a block column "hot" when at least one token has an FP8 block
-// there.  With W4z the NVFP4 weight codes (zero in FP8 blocks), A4z' the NVFP4 activation codes
-// with every hot column zeroed, At the true activation values (fp16, either format) and T the
-// fp16 tile that holds the FP8 weight blocks everywhere plus, in hot columns, the dequantized
-// NVFP4 weight blocks (so T = the true weights there):
-//     Y = A4z'.W4z^T    tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM
-//       + At.T^T        tcgen05.mma kind::f16 into the same FP32 accumulator
-// In a cold column A4z'.W4z covers NVFP4 x NVFP4 and At.T covers every pair with an FP8 weight
-// block; in a hot column At.T is the complete product.  T is mostly zero: per quarter of a unit
-// (4 block columns) it is a 128 x 64 fp16 tile that scatter threads fill from the unit's record
-// and clear again after use.
+// Decomposition (exact).  With A4z / W4z the NVFP4 planes (zero in FP8 blocks), W8 the FP8
+// blocks of the weights and At the true activation values (fp16 copy, either format):
+//     Y = A4z.W4z^T            (1) tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
+//                                  weights are the 128-row MMA operand, the 16 tokens are N
+//       + At.W8^T              (2) the FP8 weight blocks, which a record keeps grouped by block
+//                                  column: sixteen blocks that meet the same 16 activation
+//                                  elements form the M side of mma.sync m16n8k16; results are
+//                                  added to their rows in a tile private to the warp
+//       + At[FP8 blocks].W4z^T (3) only block columns in which some token is FP8: the NVFP4
+//                                  weights of the stage are dequantized for mma.sync
+// A tcgen05.mma of this shape costs about 50 ns whatever its size, so the tensor-core path is kept
+// to the four instructions per unit that (1) needs; the microscales reach TMEM by tcgen05.st from
+// otherwise idle warps instead of tcgen05.cp, and (2), (3) run beside it on warps of their own.
 //
 // Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all SMs
 // stream the same number of bytes; a unit is two bulk copies (its weight record, the activation
 // record of its chunk).  Tiles shared by several CTAs are reduced in a fixed order by the CTA
-// that arrives last; the accumulation order inside TMEM is the issue order: results are
-// reproducible bit for bit.
+// that arrives last.  Every sum is taken in a fixed order: results are reproducible bit for bit.
 //
-// Warp roles (704 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2-5 = epilogue (one TMEM lane quadrant each), warps 6-21 = scatter (eight groups of two).
+// Warp roles (704 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner, warps 2-5 =
+// epilogue (one TMEM lane quadrant each), warps 6-13 = (2), two block columns each, warps 14-21 =
+// (3), 16 rows each; the first four of them also load the microscales.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
 #include <cuda_fp16.h>
+#include <type_traits>
 
 namespace {
 
 constexpr int DEC_THREADS = 704;
-constexpr int SCAT_THREADS = 512, GRP_WARPS = 2, GRP_THREADS = 64;   // eight groups: (quarter of T, unit parity)
+constexpr int CORR_WARPS = 16;                  // warps 6..21
 constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
 constexpr uint32_t FP8_CAP_BLOCKS = 320;        // FP8 blocks of a unit that fit a stage; more are read from global
 constexpr uint32_t WREC_CAP = (REC_ROWID + FP8_CAP_BLOCKS + FP8_CAP_BLOCKS * 16 + 127) & ~127u;   // 23936
 constexpr uint32_t STG_A = (WREC_CAP + 1023) & ~1023u;                                           // 24576
 constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 37888
 constexpr int DEC_STAGES = 4;
-constexpr uint32_t TQ_BYTES = 128 * 128;        // one quarter of T: 128 rows x 64 fp16, 128B-swizzled
-constexpr int NACC = 4;                         // independent accumulators per tile: back-to-back MMAs into one
-                                                // accumulator wait for each other, so the MMAs of a unit rotate over four
-constexpr uint32_t ACC_COLS = NACC * TOK;       // columns of one accumulator buffer
-constexpr uint32_t SF_COL0 = 2 * ACC_COLS;      // scale columns start behind the two accumulator buffers
-constexpr uint32_t DEC_TMEM_COLS = 256;         // 2 x 64 accumulator columns + 4 stages x 32 scale columns
-constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + 4 * TQ_BYTES + 1024 /*alignment*/ + 512 /*barriers*/ + 8192 /*lists*/;
-static_assert(DEC_STAGE_BYTES % 1024 == 0 && (STG_A + AREC_TRUE) % 1024 == 0, "swizzled tiles need 1 KiB alignment");
+constexpr int NTILES = 9;                       // [row][token] fp32 tiles: one per (2) warp, one shared by the (3) warps
+constexpr uint32_t TILE_FLOATS = 128 * TOK;
+constexpr uint32_t SF_COL0 = 32;                // TMEM: 2 x 16 accumulator columns, then 32 scale columns per stage
+constexpr uint32_t DEC_TMEM_COLS = 256;
+constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + NTILES * TILE_FLOATS * 4 + 1024 /*alignment*/ + 512 /*barriers*/;
+static_assert(DEC_STAGE_BYTES % 1024 == 0, "swizzled tiles need 1 KiB alignment");
 
 // kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
 constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
-// kind::f16, D = f32, A = B = fp16, K-major operands, M = 128, N = 16, K = 16
-constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(TOK >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
 // shared-memory matrix descriptors as (low word | start address >> 4, constant high word)
 constexpr uint32_t SW128_LO = 1u << 16, SW128_HI = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128B swizzle, 8-row groups 1 KiB apart
@@ -77,41 +75,12 @@ __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t tot
 
 __device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return __dp4a(x, 0x01010101u, 0u); }
 
-// 16 E4M3 codes -> 16 fp16 (two 16-byte halves), scaled by a power of two
-__device__ __forceinline__ void e4m3x16_to_h16(const uint4& c, __half2 scale, uint4& lo, uint4& hi)
+// A correction tile holds [128 rows][16 tokens] fp32, a row = 64 bytes = four 16-byte pieces of
+// four tokens; piece index is XOR-ed with (row >> 1) & 3 so that 32 lanes reading one piece of 32
+// consecutive rows (the epilogue) do not collide on banks.  Float index of (row, token):
+__device__ __forceinline__ uint32_t tile_idx(uint32_t row, uint32_t token)
 {
-    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-    uint32_t o[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        uint32_t h0, h1;
-        const uint16_t l = (uint16_t)w[i], h = (uint16_t)(w[i] >> 16);
-        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h0) : "h"(l));
-        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h1) : "h"(h));
-        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&h0), scale), x1 = __hmul2(*reinterpret_cast<__half2*>(&h1), scale);
-        o[2 * i] = *reinterpret_cast<const uint32_t*>(&x0); o[2 * i + 1] = *reinterpret_cast<const uint32_t*>(&x1);
-    }
-    lo = make_uint4(o[0], o[1], o[2], o[3]); hi = make_uint4(o[4], o[5], o[6], o[7]);
-}
-
-// 16 E2M1 codes (8 bytes) times an E4M3 microscale -> 16 fp16, exact
-__device__ __forceinline__ void nvfp4x16_to_h16(const uint2& c, uint32_t scale_code, uint4& lo, uint4& hi)
-{
-    uint32_t sc2;
-    const uint16_t s16 = (uint16_t)(scale_code | (scale_code << 8));
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
-    const __half2 sc = *reinterpret_cast<__half2*>(&sc2);
-    const uint32_t w[2] = {c.x, c.y};
-    uint32_t o[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        uint32_t q;
-        const uint32_t byte = (w[i >> 2] >> ((i & 3) * 8)) & 0xffu;
-        asm("{\n\t.reg .b8 t;\n\tcvt.u8.u32 t, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, t;\n\t}" : "=r"(q) : "r"(byte));
-        const __half2 x = __hmul2(*reinterpret_cast<__half2*>(&q), sc);
-        o[i] = *reinterpret_cast<const uint32_t*>(&x);
-    }
-    lo = make_uint4(o[0], o[1], o[2], o[3]); hi = make_uint4(o[4], o[5], o[6], o[7]);
+    return row * 16u + ((((token >> 2) ^ (row >> 1)) & 3u) << 2) + (token & 3u);
 }
 
 __global__ void __launch_bounds__(DEC_THREADS, 1)
@@ -119,22 +88,17 @@ decode_kernel(DecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t* tq = smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES;                 // four quarter tiles of T
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tq + 4 * TQ_BYTES);
-    // bars (S = stages): [0,S) full, [S,2S) empty, [2S,3S) a4 ready, then T quarter full [4], T quarter
-    // done [2 unit parities][4] (a parity wait can only tell two consecutive phases apart, so each of
-    // the two groups that share a quarter has a barrier of its own), scatter group sync [8],
-    // acc_full[2], acc_empty[2]
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * DEC_STAGES + 28);
+    float* tiles = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NTILES * TILE_FLOATS);
+    // bars (S = stages): [0,S) full, [S,2S) empty, [2S,3S) scales in TMEM, then acc_full[2], acc_empty[2],
+    // corrections of a segment done [2], tiles free [1]
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * DEC_STAGES + 8);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + DEC_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    uint32_t* qcnt = tmem_slot + 2;                                            // [4 quarters]
-    uint16_t* qlist = reinterpret_cast<uint16_t*>(tq + 4 * TQ_BYTES + 512);     // [4 quarters][1024]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES, a4r0 = empty0 + 8 * DEC_STAGES;
-    const uint32_t tfull0 = a4r0 + 8 * DEC_STAGES, tdone0 = tfull0 + 32, gbar0 = tdone0 + 64;
-    const uint32_t accf0 = gbar0 + 64, acce0 = accf0 + 16;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES, sfr0 = empty0 + 8 * DEC_STAGES;
+    const uint32_t accf0 = sfr0 + 8 * DEC_STAGES, acce0 = accf0 + 16, cdone0 = acce0 + 16, tfree = cdone0 + 16;
 
     // this CTA's span of (tile, chunk) units
     const int64_t G = gridDim.x, C = p.chunks;
@@ -149,22 +113,19 @@ decode_kernel(DecParams p)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < DEC_STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + 8); mbar_init(a4r0 + 8 * s, 8);   // 8 scatter warps serve a unit
+            mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + CORR_WARPS); mbar_init(sfr0 + 8 * s, 4);
         }
-        for (int b = 0; b < 4; ++b) {
-            mbar_init(tfull0 + 8 * b, GRP_WARPS); mbar_init(tdone0 + 8 * b, 1); mbar_init(tdone0 + 32 + 8 * b, 1);
-            mbar_init(gbar0 + 8 * b, GRP_WARPS); mbar_init(gbar0 + 32 + 8 * b, GRP_WARPS);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); mbar_init(cdone0 + 8 * b, CORR_WARPS);
         }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
+        mbar_init(tfree, 4);
         *abort_flag = 0;
-        for (int i = 0; i < 4; ++i) qcnt[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
-    if (warp >= 6) {                                   // T starts all zero
-        uint4* z = reinterpret_cast<uint4*>(tq);
-        for (int i = (warp - 6) * 32 + lane; i < (int)(4 * TQ_BYTES / 16); i += SCAT_THREADS) z[i] = make_uint4(0, 0, 0, 0);
-        fence_proxy_async();
+    if (warp >= 6) {                                   // the tiles start at zero
+        float4* z = reinterpret_cast<float4*>(tiles);
+        for (int i = (warp - 6) * 32 + lane; i < (int)(NTILES * TILE_FLOATS / 4); i += CORR_WARPS * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     tc_fence_before();
     __syncthreads();
@@ -201,52 +162,36 @@ decode_kernel(DecParams p)
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        // The whole warp walks the loop (its values stay warp-uniform, which keeps the descriptor
-        // arithmetic cheap); lane 0 alone issues the tcgen05 instructions, so that every commit
-        // tracks every MMA before it.
-        const uint32_t smem0 = smem_u32(smem), tq0 = smem_u32(tq);
+        // The whole warp walks the loop; lane 0 alone issues the tcgen05 instructions, so that every
+        // commit tracks every MMA before it.
+        const uint32_t smem0 = smem_u32(smem);
         int stage = 0; uint32_t phase = 0; bool ok = true;
-        int seg = 0; uint32_t useq = 0;
+        int seg = 0;
         for (int64_t u = u_begin; u < u_end && ok; ++seg) {
             const int64_t tile = u / C;
             const int64_t seg_end = min(u_end, (tile + 1) * C);
             const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)acc * ACC_COLS;
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
             uint32_t accum = 0;
-            for (; u < seg_end && ok; ++u, ++useq) {
+            for (; u < seg_end && ok; ++u) {
                 if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
+                if (!(ok = mbar_wait(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;   // microscales are in TMEM
                 tc_fence_after();
                 const uint32_t sb = smem0 + (uint32_t)stage * DEC_STAGE_BYTES;
                 const uint32_t sf_t = tmem_base + SF_COL0 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
-                // the scatter warps have put the microscales into TMEM and zeroed the hot columns of the
-                // activation codes
-                if (!(ok = mbar_wait(a4r0 + 8 * stage, phase, abort_flag, p.status, 8))) break;
-                tc_fence_after();
                 const uint32_t w4_lo = ((sb + REC_W4) >> 4) | SW128_LO, a4_lo = ((sb + STG_A + AREC_A4) >> 4) | SW128_LO;
                 if (lane == 0) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        umma_nvf4(d_tmem + j * TOK, desc64(w4_lo + 2 * j, SW128_HI), desc64(a4_lo + 2 * j, SW128_HI), IDESC_NVF4,
+                    for (int j = 0; j < 4; ++j) {
+                        umma_nvf4(d_tmem, desc64(w4_lo + 2 * j, SW128_HI), desc64(a4_lo + 2 * j, SW128_HI), IDESC_NVF4,
                                   sf_t + 4 * j, sf_t + 16 + 4 * j, accum);
+                        accum = 1;
+                    }
+                    umma_commit(empty0 + 8 * stage);
                 }
                 accum = 1;
-                const uint32_t at_lo = ((sb + STG_A + AREC_TRUE) >> 4) | SW128_LO;
-#pragma unroll
-                for (int qq = 0; qq < 4; ++qq) {
-                    if (!(ok = mbar_wait(tfull0 + 8 * qq, useq & 1u, abort_flag, p.status, 9))) break;
-                    tc_fence_after();
-                    const uint32_t t_lo = ((tq0 + qq * TQ_BYTES) >> 4) | SW128_LO;
-                    if (lane == 0) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_f16(d_tmem + k * TOK, desc64(t_lo + 2 * k, SW128_HI), desc64(at_lo + qq * 128 + 2 * k, SW128_HI), IDESC_F16, 1u);
-                        umma_commit(tdone0 + 32 * (useq & 1u) + 8 * qq);
-                    }
-                }
-                if (!ok) break;
-                if (lane == 0) umma_commit(empty0 + 8 * stage);
                 __syncwarp();
                 if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
             }
@@ -259,6 +204,8 @@ decode_kernel(DecParams p)
         const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
+        const float r8 = __int_as_float((127 + hw->fp8_log2_ratio) << 23);     // FP8 tensor scale / NVFP4 tensor scale of the weights
+        const int row = 32 * q + lane;
         bool ok = true;
         int seg = 0;
         for (int64_t u = u_begin; u < u_end && ok; ++seg) {
@@ -268,19 +215,37 @@ decode_kernel(DecParams p)
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
+            uint32_t rr[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
+            tc_fence_before();
+            mbar_arrive(acce0 + 8 * accb);
             float v[16];
-            {
-                // the four partial accumulators of the tile, added in a fixed order
-                uint32_t r0[16], r1[16], r2[16], r3[16];
-                const uint32_t t0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)accb * ACC_COLS;
-                tmem_ld16(t0, r0); tmem_ld16(t0 + TOK, r1); tmem_ld16(t0 + 2 * TOK, r2); tmem_ld16(t0 + 3 * TOK, r3);
-                tc_fence_before();
-                mbar_arrive(acce0 + 8 * accb);
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    v[j] = ((__uint_as_float(r0[j]) + __uint_as_float(r1[j])) + __uint_as_float(r2[j])) + __uint_as_float(r3[j]);
+            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
+            // corrections (2) and (3) of the segment: this row of every tile, in tile order; the row is
+            // cleared for the next segment on the way
+            if (!(ok = mbar_wait(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 6))) break;
+            float c2[16];                              // (2): sums of the FP8 weight codes, still without 2^ratio
+#pragma unroll
+            for (int j = 0; j < 16; ++j) c2[j] = 0.f;
+#pragma unroll
+            for (int w = 0; w < NTILES; ++w) {
+                float4* src = reinterpret_cast<float4*>(tiles + w * TILE_FLOATS + row * TOK);
+                float4 x[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) x[j] = src[(j ^ (row >> 1)) & 3];       // tokens 4j .. 4j+3
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (w < 8) { c2[4 * j] += x[j].x; c2[4 * j + 1] += x[j].y; c2[4 * j + 2] += x[j].z; c2[4 * j + 3] += x[j].w; }
+                    else       { v[4 * j] += x[j].x; v[4 * j + 1] += x[j].y; v[4 * j + 2] += x[j].z; v[4 * j + 3] += x[j].w; }
+                    src[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
             }
-            const int row = 32 * q + lane;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] += c2[j] * r8;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tfree);
+
             const int64_t n = tile * 128 + row;
             const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
             bool write_out = whole;
@@ -339,160 +304,230 @@ decode_kernel(DecParams p)
                 }
             }
         }
+    } else if (warp < 14) {
+        // ------------------------------------------------------------ (2): FP8 weight blocks of block columns cw, cw + 8
+        // The E4M3 codes go into the MMA as they are; the factor 2^ratio between the FP8 and NVFP4
+        // tensor scales is applied once to the tile sums in the epilogue.
+        const int cw = warp - 6;
+        const uint32_t g = lane >> 2, t = lane & 3;
+        float* mytile = tiles + cw * TILE_FLOATS;
+        // where this lane's activation fragments of the two columns sit in an activation record
+        uint32_t boff[2];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const uint32_t j = (uint32_t)cw + 8u * hh;
+            boff[hh] = AREC_TRUE + (j >> 2) * 2048 + fgmp_h16_tile_offset(g, j & 3u, t >> 1) + (t & 1u) * 8;   // token g; token g + 8 is 1 KiB on
+        }
+        const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
+
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
+            // the epilogue has taken (and cleared) the previous segment's sums
+            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
+            for (; u < seg_end; ++u) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+                const uint8_t* sa = sb + STG_A;
+                const uint32_t staged = smeta[stage].staged;
+                const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
+                const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
+                const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z);
+                const uint32_t ntot = ks0 + ks1 + ks2 + byte_sum(kc.w);
+                const uint32_t off8 = fgmp_rec_fp8_offset(ntot);
+                uint32_t start[2], end[2];
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int kb = cw + 8 * hh, wi = kb >> 2, sh8 = (kb & 3) * 8;
+                    const uint32_t word = wi == 0 ? kc.x : (wi == 1 ? kc.y : (wi == 2 ? kc.z : kc.w));
+                    start[hh] = (wi > 0 ? ks0 : 0u) + (wi > 1 ? ks1 : 0u) + (wi > 2 ? ks2 : 0u)
+                              + byte_sum(word & ((1u << sh8) - 1u));
+                    end[hh] = start[hh] + ((word >> sh8) & 0xffu);
+                }
+                // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of each column
+                const uint2 b00 = *reinterpret_cast<const uint2*>(sa + boff[0]), b01 = *reinterpret_cast<const uint2*>(sa + boff[0] + 1024);
+                const uint2 b10 = *reinterpret_cast<const uint2*>(sa + boff[1]), b11 = *reinterpret_cast<const uint2*>(sa + boff[1] + 1024);
+
+                // ALL = every FP8 block of the unit is in the stage (the usual case); otherwise the tail of the
+                // list is read from global memory
+                auto body = [&](auto all_c) {
+                    constexpr bool ALL = decltype(all_c)::value;
+                    // One group of up to 16 blocks of one column: blocks e + g and e + g + 8 are the M side of two
+                    // mma.sync (tokens 0-7 and 8-15 as N).  c/d[0..1]: block iA, tokens 2t, 2t+1 / 8+2t, 9+2t; [2..3]: block iB.
+                    auto group_mma = [&](uint32_t e, uint32_t end_, const uint2& bt0, const uint2& bt1, float (&c)[4], float (&d)[4],
+                                         uint32_t& rowA, uint32_t& rowB) {
+                        const uint32_t iA = e + g, iB = iA + 8;
+                        uint32_t rawA = 0, rawB = 0;
+                        rowA = 0xffffffffu; rowB = 0xffffffffu;
+                        if (iA < end_) {
+                            const uint32_t o = off8 + iA * 16 + t * 4;
+                            rawA = (ALL || o + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + o) : __ldg(reinterpret_cast<const uint32_t*>(rec_g + o));
+                            rowA = (ALL || REC_ROWID + iA < staged) ? sb[REC_ROWID + iA] : __ldg(rec_g + REC_ROWID + iA);
+                        }
+                        if (iB < end_) {
+                            const uint32_t o = off8 + iB * 16 + t * 4;
+                            rawB = (ALL || o + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + o) : __ldg(reinterpret_cast<const uint32_t*>(rec_g + o));
+                            rowB = (ALL || REC_ROWID + iB < staged) ? sb[REC_ROWID + iB] : __ldg(rec_g + REC_ROWID + iB);
+                        }
+                        uint32_t a0, a1, a2, a3;
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a0) : "h"((uint16_t)rawA));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a2) : "h"((uint16_t)(rawA >> 16)));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a1) : "h"((uint16_t)rawB));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a3) : "h"((uint16_t)(rawB >> 16)));
+                        c[0] = c[1] = c[2] = c[3] = 0.f; d[0] = d[1] = d[2] = d[3] = 0.f;
+                        mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);
+                        mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);
+                    };
+                    // Within one column every block has its own row, so the four read-modify-writes of a group touch
+                    // distinct addresses in every lane and across lanes: all loads first, then all stores.
+                    auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t rowA, uint32_t rowB) {
+                        float2 *pA = nullptr, *pB = nullptr;    // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on (piece ^ 2)
+                        float2 vA0 = make_float2(0.f, 0.f), vA1 = vA0, vB0 = vA0, vB1 = vA0;
+                        if (rowA != 0xffffffffu) {
+                            pA = reinterpret_cast<float2*>(mytile + rowA * 16u + (((tpiece ^ (rowA >> 1)) & 3u) << 2) + tcol);
+                            vA0 = pA[0]; vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
+                        }
+                        if (rowB != 0xffffffffu) {
+                            pB = reinterpret_cast<float2*>(mytile + rowB * 16u + (((tpiece ^ (rowB >> 1)) & 3u) << 2) + tcol);
+                            vB0 = pB[0]; vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
+                        }
+                        if (rowA != 0xffffffffu) {
+                            pA[0] = make_float2(vA0.x + c[0], vA0.y + c[1]);
+                            *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(vA1.x + d[0], vA1.y + d[1]);
+                        }
+                        if (rowB != 0xffffffffu) {
+                            pB[0] = make_float2(vB0.x + c[2], vB0.y + c[3]);
+                            *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(vB1.x + d[2], vB1.y + d[3]);
+                        }
+                        __syncwarp();                  // a later group may add to the same rows
+                    };
+                    // the first group of both columns side by side (their MMAs are independent), then their sums in order
+                    {
+                        float c0[4], d0[4], c1[4], d1[4];
+                        uint32_t rA0, rB0, rA1, rB1;
+                        group_mma(start[0], end[0], b00, b01, c0, d0, rA0, rB0);
+                        group_mma(start[1], end[1], b10, b11, c1, d1, rA1, rB1);
+                        group_add(c0, d0, rA0, rB0);
+                        group_add(c1, d1, rA1, rB1);
+                    }
+                    // columns with more than 16 FP8 blocks
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        for (uint32_t e = start[hh] + 16; e < end[hh]; e += 16) {
+                            float c[4], d[4];
+                            uint32_t rA, rB;
+                            group_mma(e, end[hh], hh ? b10 : b00, hh ? b11 : b01, c, d, rA, rB);
+                            group_add(c, d, rA, rB);
+                        }
+                    }
+                };
+                if (off8 + ntot * 16 <= staged) body(std::true_type{}); else body(std::false_type{});
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
+        }
     } else {
-        // ------------------------------------------------------------ scatter: fill and clear T
-        // Eight groups of two warps: group (q, h) owns quarter q of T for the units of parity h, so a
-        // group has two unit times per unit and the two groups of a quarter take turns on its tile.
-        // Per unit a group zeroes the hot columns of its quarter in the activation codes, (four of the
-        // warps) loads the microscales into TMEM, converts its blocks, and then, once the previous
-        // unit's MMAs on the quarter are done, clears what that unit left there and stores its own.
-        const int sw = warp - 6;                       // 0..15
-        const int half = sw >> 3, qq = (sw >> 1) & 3;  // unit parity served, quarter owned
-        const int grp = sw >> 1;                       // 0..7
-        const int gtid = (sw & 1) * 32 + lane;         // 0..63 inside the group
-        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
-        const __half2 rw2 = __float2half2_rn(__int_as_float((127 + hw->fp8_log2_ratio) << 23));
-        uint8_t* tile = tq + qq * TQ_BYTES;
-        uint16_t* list = qlist + qq * 1024;            // T offsets written for the last unit in this quarter (0xffff = none)
-
-        bool ok = true;
-        uint32_t gphase = 0;
-        for (int64_t useq = half; u_begin + useq < u_end && ok; useq += 2) {
-            const int stage = (int)(useq & 3);
-            const uint32_t phase = (uint32_t)(useq >> 2) & 1u;
-            uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-            uint8_t* sa = sb + STG_A;
-            if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
-            const uint32_t staged = smeta[stage].staged;
-            const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
-
-            // hot columns: some token has an FP8 block there; their activation codes leave the NVFP4 product
-            const uint32_t mword = lane < 16 ? *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + lane * 2) : 0u;
-            const uint32_t hot = __reduce_or_sync(0xffffffffu, mword);
-            {
-                const uint32_t col = 4u * qq + ((uint32_t)gtid >> 4), tok = (uint32_t)gtid & 15u;
-                if ((hot >> col) & 1u) *reinterpret_cast<uint2*>(sa + AREC_A4 + fgmp_rec_w4_offset(tok, col)) = make_uint2(0, 0);
-            }
-            fence_proxy_async();
-            if ((sw & 7) < 4) {
-                // Microscales of the stage into TMEM, one warp per lane quadrant (warp % 4): lane i holds,
-                // for MMA step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3,
-                // which is 16 bytes of scale tile j; the token scales follow in columns 16..31.
-                uint32_t r[16];
+        // ------------------------------------------------------------ (3): FP8 activation blocks x NVFP4 weights, 16 rows per warp
+        const int tw = warp - 14;
+        const int rowbase = 16 * tw;
+        const uint32_t g = lane >> 2, t = lane & 3;
+        float* tile3 = tiles + 8 * TILE_FLOATS;
+        // per-lane constants of the record addressing: rows rowbase + g and rowbase + 8 + g (the same r & 7 = g)
+        uint32_t w4_base[2], sf_base[2];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
-                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
-                }
-                const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
-                tmem_st16(sf_t, r);
+        for (int rg = 0; rg < 2; ++rg) {
+            const uint32_t r = (uint32_t)rowbase + 8u * rg + g;
+            w4_base[rg] = REC_W4 + r * 128 + t * 2;
+            sf_base[rg] = REC_SF + (r & 31u) * 16 + (r >> 5) * 4;
+        }
+        const uint32_t at_base = AREC_TRUE + g * 128 + (t & 1u) * 8;
+
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
+            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            for (; u < seg_end; ++u) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+                const uint8_t* sa = sb + STG_A;
+                if (tw < 4) {
+                    // Microscales of the stage into TMEM, one warp per lane quadrant (warp % 4): lane i holds,
+                    // for MMA step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3,
+                    // which is 16 bytes of scale tile j; the token scales follow in columns 16..31.
+                    uint32_t r[16];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 x = *reinterpret_cast<const uint4*>(sa + AREC_SF + 512 * j + lane * 16);
-                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
+                        r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                    }
+                    const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
+                    tmem_st16(sf_t, r);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(sa + AREC_SF + 512 * j + lane * 16);
+                        r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                    }
+                    tmem_st16(sf_t + 16, r);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
                 }
-                tmem_st16(sf_t + 16, r);
-                tmem_wait_st();
-                tc_fence_before();
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(a4r0 + 8 * stage);
-
-            const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
-            const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z), ks3 = byte_sum(kc.w);
-            const uint32_t off8 = fgmp_rec_fp8_offset(ks0 + ks1 + ks2 + ks3);
-            const uint32_t kword = qq == 0 ? kc.x : (qq == 1 ? kc.y : (qq == 2 ? kc.z : kc.w));
-            const uint32_t n8 = qq == 0 ? ks0 : (qq == 1 ? ks1 : (qq == 2 ? ks2 : ks3));
-            const uint32_t qstart = (qq > 0 ? ks0 : 0u) + (qq > 1 ? ks1 : 0u) + (qq > 2 ? ks2 : 0u);
-            const uint32_t c0 = kword & 0xffu, c1 = (kword >> 8) & 0xffu, c2 = (kword >> 16) & 0xffu;
-            const uint32_t hotq = (hot >> (4 * qq)) & 15u;
-            const uint32_t nhot = __popc(hotq);
-
-            // One FP8 block of the quarter (list entries qstart .. qstart + n8, ordered by (column, row)):
-            // where it goes in T and its 16 values as fp16.
-            auto fp8_item = [&](uint32_t it, uint32_t& pos, uint4& lo, uint4& hi) {
-                const uint32_t e = qstart + it;
-                const uint32_t o = off8 + e * 16;
-                const uint4 raw = o + 16 <= staged ? *reinterpret_cast<const uint4*>(sb + o) : __ldg(reinterpret_cast<const uint4*>(rec_g + o));
-                const uint32_t r = REC_ROWID + e < staged ? sb[REC_ROWID + e] : __ldg(rec_g + REC_ROWID + e);
-                const uint32_t jq = (it >= c0) + (it >= c0 + c1) + (it >= c0 + c1 + c2);
-                pos = fgmp_h16_tile_offset(r, jq, 0);
-                e4m3x16_to_h16(raw, rw2, lo, hi);
-            };
-            // The NVFP4 block of a row in hot column jq of the quarter; pos = 0xffff when its microscale
-            // is 0 (the block is FP8 or all zero) and nothing is to be written.
-            auto hot_item = [&](uint32_t row, uint32_t jq, uint32_t& pos, uint4& lo, uint4& hi) {
-                const uint32_t j = 4u * qq + jq;
-                const uint32_t sc = sb[REC_SF + fgmp_rec_sf_offset(row, j)];
-                pos = 0xffffu;
-                if (sc != 0) {
-                    pos = fgmp_h16_tile_offset(row, jq, 0);
-                    nvfp4x16_to_h16(*reinterpret_cast<const uint2*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j)), sc, lo, hi);
-                }
-            };
-            auto put = [&](uint32_t slot, uint32_t pos, const uint4& lo, const uint4& hi) {
-                list[slot] = (uint16_t)pos;
-                if (pos != 0xffffu) {
-                    *reinterpret_cast<uint4*>(tile + pos) = lo;
-                    *reinterpret_cast<uint4*>(tile + (pos ^ 16u)) = hi;
-                }
-            };
-
-            // converted ahead of the wait below: this thread's first FP8 block and its two rows of the first hot column
-            uint32_t posA = 0xffffu, posB = 0xffffu, posC = 0xffffu;
-            uint4 loA = make_uint4(0, 0, 0, 0), hiA = loA, loB = loA, hiB = loA, loC = loA, hiC = loA;
-            if ((uint32_t)gtid < n8) fp8_item((uint32_t)gtid, posA, loA, hiA);
-            const uint32_t jq_first = hotq ? (uint32_t)__ffs(hotq) - 1u : 0u;
-            if (hotq) {
-                hot_item((uint32_t)gtid, jq_first, posB, loB, hiB);
-                hot_item((uint32_t)gtid + 64u, jq_first, posC, loC, hiC);
-            }
-
-            // the previous unit's MMAs on this quarter are done: clear what was written for it
-            if (useq > 0) {
-                if (!(ok = mbar_wait(tdone0 + 32 * (uint32_t)((useq - 1) & 1) + 8 * qq, (uint32_t)((useq - 1) >> 1) & 1u,
-                                     abort_flag, p.status, 10))) break;
-                const uint32_t n_old = qcnt[qq];
-                for (uint32_t i = gtid; i < n_old; i += GRP_THREADS) {
-                    const uint32_t o = list[i];
-                    if (o != 0xffffu) {
-                        *reinterpret_cast<uint4*>(tile + o) = make_uint4(0, 0, 0, 0);
-                        *reinterpret_cast<uint4*>(tile + (o ^ 16u)) = make_uint4(0, 0, 0, 0);
+                const uint32_t am0 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + g * 2);
+                const uint32_t am1 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + (g + 8) * 2);
+                uint32_t todo = am0 | am1;             // block columns in which any token is FP8
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) todo |= __shfl_xor_sync(0xffffffffu, todo, o);
+                while (todo) {
+                    const uint32_t kb = (uint32_t)__ffs(todo) - 1u;
+                    todo &= todo - 1;
+                    const uint32_t bit = 1u << kb;
+                    // true activation values of tokens g and g + 8 (1 KiB apart), elements 4t..4t+3 of column kb
+                    const uint8_t* ap = sa + at_base + (kb >> 2) * 2048 + (((((kb & 3u) << 1) | (t >> 1)) ^ g) << 4);
+                    const uint2 at0 = *reinterpret_cast<const uint2*>(ap), at1 = *reinterpret_cast<const uint2*>(ap + 1024);
+                    const uint32_t a0 = (am0 & bit) ? at0.x : 0u, a2 = (am0 & bit) ? at0.y : 0u;
+                    const uint32_t a1 = (am1 & bit) ? at1.x : 0u, a3 = (am1 & bit) ? at1.y : 0u;
+                    const uint32_t wcol = ((((kb >> 1) ^ g) & 7u) << 4) + (kb & 1u) * 8, scol = (kb >> 2) * 512 + (kb & 3u);
+#pragma unroll
+                    for (int rg = 0; rg < 2; ++rg) {
+                        const uint32_t codes = *reinterpret_cast<const uint16_t*>(sb + w4_base[rg] + wcol);
+                        const uint32_t sfb = sb[sf_base[rg] + scol];
+                        uint32_t q0, q1, sc2;
+                        asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
+                            : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
+                        const uint16_t s16 = (uint16_t)(sfb | (sfb << 8));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
+                        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&q0), *reinterpret_cast<__half2*>(&sc2));
+                        const __half2 x1 = __hmul2(*reinterpret_cast<__half2*>(&q1), *reinterpret_cast<__half2*>(&sc2));
+                        mma_f16_16816(acc[rg], a0, a1, a2, a3, *reinterpret_cast<const uint32_t*>(&x0), *reinterpret_cast<const uint32_t*>(&x1));
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(gbar0 + 8 * grp);          // the whole group has cleared its share
-            if (!(ok = mbar_wait(gbar0 + 8 * grp, gphase, abort_flag, p.status, 11))) break;
-            gphase ^= 1u;
-            if (gtid == 0) qcnt[qq] = n8 + nhot * 128u;
-
-            // list slots: [0, n8) the FP8 blocks, then 128 per hot column in column order
-            if ((uint32_t)gtid < n8) put((uint32_t)gtid, posA, loA, hiA);
-            for (uint32_t it = gtid + GRP_THREADS; it < n8; it += GRP_THREADS) {
-                uint32_t pos; uint4 lo, hi;
-                fp8_item(it, pos, lo, hi);
-                put(it, pos, lo, hi);
-            }
-            if (hotq) {
-                put(n8 + (uint32_t)gtid, posB, loB, hiB);
-                put(n8 + (uint32_t)gtid + 64u, posC, loC, hiC);
-                uint32_t rest = hotq & (hotq - 1u), slot = n8 + 128u + (uint32_t)gtid;
-                while (rest) {
-                    const uint32_t jq = (uint32_t)__ffs(rest) - 1u;
-                    rest &= rest - 1u;
+            if (!ok) break;
+            // the epilogue has taken (and cleared) the previous segment's sums; now this segment's go in:
+            // acc[rg] = (token g | g+8) x (row 2t | 2t+1) of the warp's row group rg
+            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
 #pragma unroll
-                    for (uint32_t rr = 0; rr < 2; ++rr) {
-                        uint32_t pos; uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
-                        hot_item((uint32_t)gtid + 64u * rr, jq, pos, lo, hi);
-                        put(slot + 64u * rr, pos, lo, hi);
-                    }
-                    slot += 128u;
-                }
+            for (int rg = 0; rg < 2; ++rg) {
+                const uint32_t r = (uint32_t)(rowbase + 8 * rg + 2 * t);
+                tile3[tile_idx(r, g)] = acc[rg][0];
+                tile3[tile_idx(r + 1, g)] = acc[rg][1];
+                tile3[tile_idx(r, g + 8)] = acc[rg][2];
+                tile3[tile_idx(r + 1, g + 8)] = acc[rg][3];
             }
-            fence_proxy_async();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(tfull0 + 8 * qq); mbar_arrive(empty0 + 8 * stage); }
+            if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
         }
     }
 
