@@ -170,6 +170,7 @@ def max_over_ranks(x: float, world: int) -> float:
 WORKLOADS = {
     # name: (M, N, K, fp8 fraction, kind)
     "llama2-7b-fc1-decode": (16, 11008, 4096, 0.10, "decode"),
+    "llama2-70b-fc1-decode": (16, 28672, 8192, 0.10, "decode"),
     "llama2-7b-qkvo-prefill": (4096, 4096, 4096, 0.10, "prefill"),
     "llama2-7b-fc1-prefill": (4096, 11008, 4096, 0.10, "prefill"),
     "llama2-7b-fc2-prefill": (4096, 4096, 11008, 0.10, "prefill"),
