@@ -102,6 +102,19 @@ constexpr size_t GEMM_SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment sla
 // instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=BN, M=BM
 constexpr uint32_t IDESC_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
+// Tile order: bands of RASTER_M tile rows, all tile columns of a band before the next band, tile rows
+// fastest inside a band.  The CTAs that run together then share few A and B panels, which the
+// 126 MB L2 keeps between their reads.
+constexpr int RASTER_M = 8;
+__device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int64_t tiles_n, int64_t& tm, int64_t& tn)
+{
+    const int64_t per_band = (int64_t)RASTER_M * tiles_n;
+    const int64_t band = t / per_band, r = t % per_band;
+    const int64_t rows = min((int64_t)RASTER_M, tiles_m - band * RASTER_M);
+    tm = band * RASTER_M + r % rows;
+    tn = r / rows;
+}
+
 struct GemmParams {
     void* Y; int64_t ldy; int y_is_bf16;
     int64_t M, N, K;
@@ -143,7 +156,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-                const int32_t m0 = (int32_t)((t % tiles_m) * BM), n0 = (int32_t)((t / tiles_m) * BN);
+                int64_t tm, tn;
+                tile_coords(t, tiles_m, tiles_n, tm, tn);
+                const int32_t m0 = (int32_t)(tm * BM), n0 = (int32_t)(tn * BN);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1))) break;
                     const uint32_t fb = full0 + 8 * stage;
@@ -186,7 +201,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         int64_t it = 0;
         for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
             const int acc = (int)(it & 1); const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
-            const int64_t m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+            int64_t tm, tn;
+            tile_coords(t, tiles_m, tiles_n, tm, tn);
+            const int64_t m0 = tm * BM, n0 = tn * BN;
             if (!(ok = mbar_wait(accf0 + 8 * acc, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
             const int64_t row = m0 + q * 32 + lane;
