@@ -90,8 +90,8 @@ __global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* blob, int6
 }
 
 // ------------------------------------------------------------------ bf16 tcgen05 GEMM
-constexpr int BM = 128, BN = 128, BK = 64;          // BK bf16 = one 128-byte swizzle row
-constexpr int STAGES = 6;
+constexpr int BM = 128, BN = 256, BK = 64;          // BK bf16 = one 128-byte swizzle row
+constexpr int STAGES = 4;
 constexpr int UMMA_K = 16;
 constexpr int GEMM_THREADS = 192;
 constexpr uint32_t A_TILE_BYTES = BM * BK * 2, B_TILE_BYTES = BN * BK * 2;
