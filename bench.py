@@ -320,10 +320,17 @@ def run_ours(args, world, rank, local):
         else:
             ach = flops / avg_s / 1e12
             pk = peaks["bf16_tflops_sustained"]
+            # other readings of the roofline for the same launch: the mix at FP4/FP8 rates (nominal 4x / 2x
+            # of the measured bf16 rate; those peaks are not measured on this machine), and FP8 only
+            pa = pw = p
+            f4 = (1 - pa) * (1 - pw)
+            blended_s = flops * (f4 / (4 * pk) + (1 - f4) / (2 * pk)) / 1e12
             roofline = {"kernel": name, "bound": "tensor", "achieved": ach, "peak": pk, "unit": "TFLOP/s",
                         "frac": ach / pk, "traffic": load_traffic(name, args.workload),
                         "peak_source": peaks["source"] + " bf16 sustained (common-container path runs at the f16 rate)",
-                        "avg_kernel_us": avg_s * 1e6}
+                        "avg_kernel_us": avg_s * 1e6,
+                        "frac_of_blended_fp4_fp8_roofline": blended_s / avg_s,
+                        "frac_of_fp8_roofline": (flops / (2 * pk) / 1e12) / avg_s}
     out = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
