@@ -209,7 +209,7 @@ def run_ours(args, world, rank, local):
     tau = float(fg.calibrate_tau(x_dev, fx, scale_fp4=s4, fp8_fraction=p).item())
 
     acts_buf = fg.binding._alloc_aligned(fg.acts_bytes(M, K), dev)
-    ws = fg.binding._alloc_aligned(fg.workspace_bytes(fg.binding.OP_LINEAR, M, N, K), dev)
+    ws = fg.alloc_workspace(fg.binding.OP_LINEAR, M, N, K, dev)
     y = torch.empty(M, N, dtype=torch.float32, device=dev)
     # distinct activation copies as well (small at decode, > L2 in total at prefill with the planes)
     n_x = 4

@@ -152,11 +152,24 @@ fgmp_status fgmp_calibrate_tau(const void* X_bf16, int64_t ldx, const float* fis
                                double fp8_fraction, float* tau_out,
                                void* workspace, size_t ws_bytes, void* cuda_stream);
 
+/* ---- workspace of fgmp_linear ----
+ * The first FGMP_WS_CONTROL_BYTES of a workspace hold the status word that fgmp_check reads and,
+ * for decode-sized batches, the counters of tiles that several thread blocks share.  They must be
+ * zero when fgmp_linear first uses the workspace: clear them once with this call (a memset on the
+ * stream; workspace 1024-byte aligned).  Every fgmp_linear that ends without a device-side error
+ * leaves them zero again, so that a decode step needs no clearing pass of its own; after an error
+ * reported by fgmp_check, clear the workspace again before reusing it. */
+#define FGMP_WS_CONTROL_BYTES 65536
+fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_stream);
+
 /* ---- the mixed-precision GEMM (Section 4.1) ----
  * Y[m, n] = sum over blocks of dot16(A[m, kb], W[n, kb]) with each block pair multiplied in
  * its own formats (FP4xFP4, FP4xFP8, FP8xFP4, FP8xFP8), microscales and tensor scales
- * applied, accumulated in FP32.  Y is fp32 (y_is_bf16 = 0) or bf16 [M, ldy].  The first
- * 256 bytes of the workspace hold a status word that fgmp_check reads. */
+ * applied, accumulated in FP32.  Y is fp32 (y_is_bf16 = 0) or bf16 [M, ldy].  The workspace
+ * must have been cleared once with fgmp_workspace_init.  For 1 <= M <= 16, K % 256 == 0 and
+ * N <= 258048 the weight-streaming kernel runs, launched as a programmatic dependent of the kernel
+ * before it in the stream (its set-up overlaps that kernel's end; it reads the packed activations
+ * and the workspace only after that kernel has completed). */
 fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
                         void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                         void* workspace, size_t ws_bytes, void* cuda_stream);
@@ -172,7 +185,7 @@ fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
  *   - Inputs and outputs are passed as for fgmp_linear; results are bit-identical to it.
  *   - Shapes whose scratch need (fgmp_workspace_bytes(FGMP_OP_LINEAR, M, N, K)) exceeds
  *     FGMP_STATIC_SCRATCH_BYTES return FGMP_ERR_WORKSPACE; M > 16 or K % 256 != 0 returns
- *     FGMP_ERR_SHAPE.  Llama-2-70B FC1/FC2 (28672 x 8192) needs 3.5 MiB and fits.
+ *     FGMP_ERR_SHAPE.  Llama-2-70B FC1/FC2 (28672 x 8192) needs 3.6 MiB and fits; N > 258048 is not a decode shape.
  *   - The first call on each device looks up the array's device address (a host-side query,
  *     made with that device current); make that first call outside any stream capture.
  *   - All calls on one GPU share the array and each call starts by clearing the part that

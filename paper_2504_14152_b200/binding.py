@@ -60,6 +60,8 @@ def _load():
     L.fgmp_linear_static.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, vp]
     L.fgmp_check.restype = ci
     L.fgmp_check.argtypes = [vp, vp]
+    L.fgmp_workspace_init.restype = ci
+    L.fgmp_workspace_init.argtypes = [vp, sz, vp]
     L.fgmp_unpack.restype = ci
     L.fgmp_unpack.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp]
     L.fgmp_activation_scores.restype = ci
@@ -115,6 +117,17 @@ def weights_bytes(N: int, K: int, max_fp8_blocks: int) -> int:
 
 def workspace_bytes(op: int, M: int, N: int, K: int) -> int:
     return _load().fgmp_workspace_bytes(op, M, N, K)
+
+
+def workspace_init(workspace: torch.Tensor) -> torch.Tensor:
+    """Clear the control area of a workspace (once, before fgmp_linear first uses it)."""
+    _ok(_load().fgmp_workspace_init(workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_workspace_init")
+    return workspace
+
+
+def alloc_workspace(op: int, M: int, N: int, K: int, device) -> torch.Tensor:
+    """A cleared, 1024-byte aligned workspace for `op` on `device`."""
+    return workspace_init(_alloc_aligned(workspace_bytes(op, M, N, K), device))
 
 
 @dataclass
@@ -213,7 +226,7 @@ def linear(acts: PackedTensor, weights: PackedTensor, *, out_dtype=torch.float32
         out = torch.empty(M, N, dtype=out_dtype, device=acts.blob.device)
     assert out.dtype in (torch.float32, torch.bfloat16)
     if workspace is None:
-        workspace = _alloc_aligned(L.fgmp_workspace_bytes(OP_LINEAR, M, N, K), acts.blob.device)
+        workspace = alloc_workspace(OP_LINEAR, M, N, K, acts.blob.device)
     _ok(L.fgmp_linear(acts.blob.data_ptr(), weights.blob.data_ptr(), out.data_ptr(),
                       1 if out.dtype == torch.bfloat16 else 0, out.stride(0), M, N, K,
                       workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear")

@@ -127,16 +127,46 @@ decode_kernel(DecParams p)
         float4* z = reinterpret_cast<float4*>(tiles);
         for (int i = (warp - 6) * 32 + lane; i < (int)(NTILES * TILE_FLOATS / 4); i += CORR_WARPS * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    // One unit's two copies into a stage (lane 0 of the producer warp): the weight record, then the
+    // activation record of the unit's chunk
+    const uint8_t* arec = p.ablob + p.LA.off_arec;
+    auto issue_w = [&](int stage, uint32_t step0, uint32_t step1) {
+        const uint32_t bytes = (step1 - step0) * 128u;
+        const uint32_t staged = bytes < WREC_CAP ? bytes : WREC_CAP;
+        smeta[stage].step = step0; smeta[stage].staged = staged;
+        const uint32_t fb = full0 + 8 * stage;
+        mbar_expect_tx(fb, staged + AREC_BYTES);
+        bulk_load(smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES), recs + (size_t)step0 * 128, staged, fb);
+    };
+    auto issue_a = [&](int64_t u, int stage) {
+        bulk_load(smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES) + STG_A, arec + (size_t)(u % C) * AREC_BYTES, AREC_BYTES, full0 + 8 * stage);
+    };
+    // The first stages need no consumer to have freed them, and the packed weights are not written by
+    // whatever runs before this kernel: their copies start before the CTA has finished setting itself
+    // up (thread 0, which initialised the barriers, issues them) and before the wait below.
+    int pre = 0;
+    if (warp == 0) {
+        pre = (int)min((int64_t)DEC_STAGES, u_end - u_begin);
+        for (int s = 0; s < pre; ++s) {
+            const uint32_t step0 = __shfl_sync(0xffffffffu, pf, s), step1 = __shfl_sync(0xffffffffu, pf, s + 1);
+            if (lane == 0) issue_w(s, step0, step1);
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched as a programmatic dependent of the preceding kernel in the stream (normally the
+    // activation quantizer), this kernel may have started before that one finished: everything above
+    // touches neither its output nor the workspace.  From here on both are read.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer (whole warp; lane 0 issues)
-        int stage = 0; uint32_t phase = 0;
-        const uint8_t* arec = p.ablob + p.LA.off_arec;
-        for (int64_t u = u_begin; u < u_end; ++u) {
+        if (lane == 0)
+            for (int s = 0; s < pre; ++s) issue_a(u_begin + s, s);
+        int stage = pre % DEC_STAGES; uint32_t phase = (uint32_t)(pre / DEC_STAGES) & 1u;
+        for (int64_t u = u_begin + pre; u < u_end; ++u) {
             if (u + 1 - pf_base > 31) {                // next 32 record offsets
                 pf_base = u;
                 pf = (pf_base + lane <= p.total) ? __ldg(uptr + pf_base + lane) : 0u;
@@ -146,16 +176,7 @@ decode_kernel(DecParams p)
             int ok = 1;
             if (lane == 0) {
                 ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1) ? 1 : 0;
-                if (ok) {
-                    const uint32_t bytes = (step1 - step0) * 128u;
-                    const uint32_t staged = bytes < WREC_CAP ? bytes : WREC_CAP;
-                    smeta[stage].step = step0; smeta[stage].staged = staged;
-                    const uint32_t fb = full0 + 8 * stage;
-                    const uint32_t sb = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
-                    mbar_expect_tx(fb, staged + AREC_BYTES);
-                    bulk_load(sb, recs + (size_t)step0 * 128, staged, fb);
-                    bulk_load(sb + STG_A, arec + (size_t)(u % C) * AREC_BYTES, AREC_BYTES, fb);
-                }
+                if (ok) { issue_w(stage, step0, step1); issue_a(u, stage); }
             }
             if (!__shfl_sync(0xffffffffu, ok, 0)) break;
             if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
@@ -215,6 +236,18 @@ decode_kernel(DecParams p)
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
+            // a tile shared with other CTAs: how many of them have handed in their sums already (the answer is
+            // needed only after this CTA's own sums are complete, so the load costs nothing)
+            const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
+            int nseg = 1, slot = 0;
+            uint32_t seen = 0;
+            if (!whole) {
+                const int64_t c_first = cta_of_unit(tile * C, G, p.total);
+                const int64_t c_last = cta_of_unit((tile + 1) * C - 1, G, p.total);
+                nseg = (int)(c_last - c_first + 1);
+                slot = (int)(blockIdx.x - c_first);
+                if (lane == 0) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile * 8 + q) : "memory");
+            }
             uint32_t rr[16];
             tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
             tc_fence_before();
@@ -247,22 +280,24 @@ decode_kernel(DecParams p)
             if (lane == 0) mbar_arrive(tfree);
 
             const int64_t n = tile * 128 + row;
-            const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
             bool write_out = whole;
             if (!whole) {
-                // partial tile: publish, and let the warp that arrives last add everything up
-                const int64_t c_first = cta_of_unit(tile * C, G, p.total);
-                const int64_t c_last = cta_of_unit((tile + 1) * C - 1, G, p.total);
-                const int nseg = (int)(c_last - c_first + 1);
-                const int slot = (int)(blockIdx.x - c_first);
+                // partial tile: publish, and let the warp that arrives last add everything up.  When all the
+                // others were seen to have arrived, this warp is the last without asking and skips the counter.
                 float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + row) * 16;
 #pragma unroll
                 for (int j = 0; j < 16; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
-                __threadfence();
-                __syncwarp();
-                uint32_t old = 0;
-                if (lane == 0) old = atomicAdd(p.counters + tile * 8 + q, 1u);
-                old = __shfl_sync(0xffffffffu, old, 0);
+                // The counter wraps to zero with the last arrival (or is put back by the warp that skipped
+                // it), so the workspace is ready for the next call without being cleared.
+                uint32_t old = __shfl_sync(0xffffffffu, seen, 0);
+                if (old != (uint32_t)(nseg - 1)) {
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) old = atomicInc(p.counters + tile * 8 + q, (uint32_t)(nseg - 1));
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                } else if (lane == 0) {
+                    p.counters[tile * 8 + q] = 0u;
+                }
                 if (old == (uint32_t)(nseg - 1)) {
                     __threadfence();
                     // all partials first (independent loads), then one sum in slot order
@@ -559,20 +594,26 @@ DecPlan decode_plan(int64_t N, int64_t K)
 
 }  // namespace
 
+// Workspace of the decode path: status word at 0, stream-K tile counters at 1024 (32 bytes per
+// tile), both inside the control area that must be zero before a call; partial sums behind it.
 bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K)
 {
-    return M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0;
+    return M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0 &&
+           1024 + ((N + 127) / 128) * 32 <= (int64_t)FGMP_WS_CONTROL_BYTES;
 }
 
 size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K)
 {
     if (!fgmp_decode_supported(M, N, K)) return 0;
     const DecPlan d = decode_plan(N, K);
-    return 1024 + fgmp_align1k((size_t)d.tiles * 32) + (size_t)d.tiles * d.maxseg * 128 * 16 * 4;
+    return (size_t)FGMP_WS_CONTROL_BYTES + (size_t)d.tiles * d.maxseg * 128 * 16 * 4;
 }
 
+// clear_first: zero the control area on the stream before the kernel (for scratch whose state the
+// caller cannot vouch for); otherwise the kernel is launched as a programmatic dependent of the
+// kernel before it in the stream, so that its set-up and first weight copies overlap that kernel's end.
 fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
-                               int64_t M, int64_t N, int64_t K, void* workspace, cudaStream_t s)
+                               int64_t M, int64_t N, int64_t K, void* workspace, bool clear_first, cudaStream_t s)
 {
     const DecPlan d = decode_plan(N, K);
     uint8_t* ws = (uint8_t*)workspace;
@@ -583,7 +624,7 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     p.M = M; p.N = N; p.K = K; p.total = d.total; p.chunks = d.chunks;
     p.status = reinterpret_cast<int*>(ws);
     p.counters = reinterpret_cast<uint32_t*>(ws + 1024);
-    p.partials = reinterpret_cast<float*>(ws + 1024 + fgmp_align1k((size_t)d.tiles * 32));
+    p.partials = reinterpret_cast<float*>(ws + FGMP_WS_CONTROL_BYTES);
     p.maxseg = d.maxseg;
 
     static bool attr_set[64] = {};
@@ -594,8 +635,14 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
             return FGMP_ERR_CUDA;
         attr_set[dev] = true;
     }
-    if (cudaMemsetAsync(ws, 0, 1024 + (size_t)d.tiles * 32, s) != cudaSuccess) return FGMP_ERR_CUDA;
-    FGMP_LAUNCH(FGMP_K_DECODE, s, decode_kernel<<<d.grid, DEC_THREADS, DEC_SMEM, s>>>(p));
+    if (clear_first && cudaMemsetAsync(ws, 0, 1024 + (size_t)d.tiles * 32, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = DEC_SMEM; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = clear_first ? 0 : 1;
+    FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel, p));
     return fgmp_launch_status();
 }
 
@@ -628,9 +675,9 @@ extern "C" fgmp_status fgmp_linear_static(const void* packed_acts, const void* p
     }
     void* scratch = scratch_of_device[dev];
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    // fgmp_linear_decode zeroes the status word and the tile counters at the start of the
-    // scratch; the partial sums behind them are always written before they are read.
-    st = fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, scratch, s);
+    // the status word and the tile counters at the start of the scratch are zeroed first; the
+    // partial sums behind them are always written before they are read
+    st = fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, scratch, true, s);
     if (st != FGMP_OK) return st;
     if (status_out && cudaMemcpyAsync(status_out, scratch, 2 * sizeof(int32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
         return FGMP_ERR_CUDA;

@@ -317,7 +317,7 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     if (fgmp_decode_supported(M, N, K))
-        return fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, s);
+        return fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, false, s);
     uint8_t* ws = (uint8_t*)workspace;
     int* status = reinterpret_cast<int*>(ws);
     uint8_t* planeA = ws + 1024;
@@ -352,6 +352,14 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     const int grid = (int)(tiles < sms ? tiles : sms);
     FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(tmA, tmB, p));
     return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!workspace || ((uintptr_t)workspace & 1023)) return FGMP_ERR_INVALID_ARG;
+    const size_t n = ws_bytes < (size_t)FGMP_WS_CONTROL_BYTES ? ws_bytes : (size_t)FGMP_WS_CONTROL_BYTES;
+    if (n && cudaMemsetAsync(workspace, 0, n, (cudaStream_t)cuda_stream) != cudaSuccess) return FGMP_ERR_CUDA;
+    return FGMP_OK;
 }
 
 extern "C" fgmp_status fgmp_check(const void* workspace, void* cuda_stream)

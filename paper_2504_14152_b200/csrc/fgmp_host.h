@@ -17,7 +17,7 @@ size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K);
 bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K);
 size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K);
 fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
-                               int64_t M, int64_t N, int64_t K, void* workspace, cudaStream_t s);
+                               int64_t M, int64_t N, int64_t K, void* workspace, bool clear_first, cudaStream_t s);
 
 // ---- launch accounting (see fgmp_profile_begin in fgmp.h) ----
 enum FgmpKernelId {

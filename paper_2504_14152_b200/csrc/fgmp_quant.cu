@@ -28,6 +28,9 @@ struct ActParams {
 template <int MODE, bool SCORE_ONLY>
 __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
 {
+    // A kernel launched behind this one as a programmatic dependent (the decode-sized GEMM) may
+    // start setting itself up now; it waits for this grid to complete before it reads the result.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t kb = (int64_t)blockIdx.x * QA_THREADS + threadIdx.x;
     const bool active = kb < p.KB;
     const int64_t m0 = (int64_t)blockIdx.y * p.rows_per_cta;

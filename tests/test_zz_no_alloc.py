@@ -67,7 +67,7 @@ def test_static_scratch_variant_rejects_what_does_not_fit():
     assert L.fgmp_linear_static(fake, fake, fake, 0, 4096, 17, 4096, 4096, None, None) == -2
     assert L.fgmp_linear_static(fake, fake, fake, 0, 4096, 16, 4096, 4096 + 64, None, None) == -2
     # a shape whose scratch need exceeds the built-in array
-    N, K = 400000, 4096
+    N, K = 200000, 4096
     assert fg.workspace_bytes(b.OP_LINEAR, 16, N, K) > fg.STATIC_SCRATCH_BYTES
     assert L.fgmp_linear_static(fake, fake, fake, 0, N, 16, N, K, None, None) == -3
     # Llama-2-70B FC1 fits
