@@ -320,17 +320,20 @@ def run_ours(args, world, rank, local):
         else:
             ach = flops / avg_s / 1e12
             pk = peaks["bf16_tflops_sustained"]
-            # other readings of the roofline for the same launch: the mix at FP4/FP8 rates (nominal 4x / 2x
-            # of the measured bf16 rate; those peaks are not measured on this machine), and FP8 only
+            # other readings of the roofline for the same launch: the mix at the FP4/FP8 rates measured
+            # here with an MMA-only loop, and FP8 only
             pa = pw = p
             f4 = (1 - pa) * (1 - pw)
-            blended_s = flops * (f4 / (4 * pk) + (1 - f4) / (2 * pk)) / 1e12
+            tp = tensor_peaks(fg, dev)
+            p4, p8 = tp["nvfp4_sustained"], tp["e4m3_sustained"]
+            blended_s = flops * (f4 / p4 + (1 - f4) / p8) / 1e12
             roofline = {"kernel": name, "bound": "tensor", "achieved": ach, "peak": pk, "unit": "TFLOP/s",
                         "frac": ach / pk, "traffic": load_traffic(name, args.workload),
                         "peak_source": peaks["source"] + " bf16 sustained (common-container path runs at the f16 rate)",
                         "avg_kernel_us": avg_s * 1e6,
                         "frac_of_blended_fp4_fp8_roofline": blended_s / avg_s,
-                        "frac_of_fp8_roofline": (flops / (2 * pk) / 1e12) / avg_s}
+                        "frac_of_fp8_roofline": (flops / p8 / 1e12) / avg_s,
+                        "tensor_peaks_tflops": tp}
     out = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -360,7 +363,8 @@ def run_ours(args, world, rank, local):
 # DRAM bytes (read + write) per launch from the committed ncu captures (profiles/*.md).  An entry is
 # removed when its kernel changes after the capture.
 NCU_TRAFFIC = {
-    ("llama2-7b-fc1-decode", "decode_gemm"): 30555392,     # profiles/decode_kernel_llama2-7b-fc1-decode.md
+    ("llama2-7b-fc1-decode", "decode_gemm"): 30564096,          # profiles/decode_kernel_llama2-7b-fc1-decode.md
+    ("llama2-7b-fc2-prefill", "gemm_bf16_tcgen05"): 527098112,   # profiles/gemm_bf16_kernel_llama2-7b-fc2-prefill.md
 }
 
 
@@ -428,6 +432,28 @@ def run_reference(args, world, rank):
         "e2e": {"value": cb["value"], "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
+
+
+def tensor_peaks(fg, dev):
+    """TFLOP/s of an MMA-only tcgen05 loop (operands in shared memory, M = 128, N = 256, one CTA per SM)
+    per operand kind: a burst of about 20 ms and a run of about 0.3 s."""
+    ws = fg.binding._alloc_aligned(1024, dev)
+    ws.zero_()
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    out = {"method": "MMA-only tcgen05 loop, M128 N256, operands in shared memory, one CTA per SM"}
+    for kind, (nm, k) in enumerate((("bf16", 16), ("e4m3", 32), ("nvfp4", 64))):
+        fg.tensor_peak(kind, 2000, ws)
+        for tag, n in (("burst", 200_000), ("sustained", 3_000_000)):
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            fg.tensor_peak(kind, n, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            out[f"{nm}_{tag}"] = 2.0 * 128 * 256 * k * n * sms / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    fg.check(ws)
+    return out
 
 
 def main():

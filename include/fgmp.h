@@ -210,6 +210,15 @@ fgmp_status fgmp_check(const void* workspace, void* cuda_stream);
 fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, uint8_t* codes4, uint8_t* codes8,
                         uint8_t* scales, uint32_t* mask, void* cuda_stream);
 
+/* ---- measurement support: tensor-core rate per operand kind ----
+ * Runs, on every SM, mma_per_cta tcgen05 instructions of M = 128, N = 256 on operands resident in
+ * shared memory (nothing is loaded or stored): kind 0 = bf16 (K = 16 per instruction), 1 = FP8 E4M3
+ * (K = 32), 2 = NVFP4 with E4M3 block scales (K = 64).  The caller times the call on the stream;
+ * flops = 2 * 128 * 256 * K * mma_per_cta * (number of SMs).  These are the rates the block-pair
+ * products of Section 4.1 can run at at best, i.e. the denominators of the prefill roofline.
+ * workspace: >= 256 bytes, zeroed, 256-byte aligned (status word, read by fgmp_check). */
+fgmp_status fgmp_tensor_peak(int kind, int64_t mma_per_cta, void* workspace, size_t ws_bytes, void* cuda_stream);
+
 /* Block scores only (parity support and calibration): scores [M*K/16] fp32, activations. */
 fgmp_status fgmp_activation_scores(const void* X_bf16, int64_t ldx, const float* fisher_chan,
                                    int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,

@@ -60,6 +60,8 @@ def _load():
     L.fgmp_linear_static.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, vp]
     L.fgmp_check.restype = ci
     L.fgmp_check.argtypes = [vp, vp]
+    L.fgmp_tensor_peak.restype = ci
+    L.fgmp_tensor_peak.argtypes = [ci, i64, vp, sz, vp]
     L.fgmp_workspace_init.restype = ci
     L.fgmp_workspace_init.argtypes = [vp, sz, vp]
     L.fgmp_unpack.restype = ci
@@ -250,6 +252,11 @@ def linear_static(acts: PackedTensor, weights: PackedTensor, *, out: torch.Tenso
                              1 if out.dtype == torch.bfloat16 else 0, out.stride(0), M, N, K,
                              _ptr(status_out), _stream()), "fgmp_linear_static")
     return out
+
+
+def tensor_peak(kind: int, mma_per_cta: int, workspace: torch.Tensor) -> None:
+    """Launch the MMA-only loop of fgmp_tensor_peak (kind 0 bf16, 1 E4M3, 2 NVFP4); the caller times it."""
+    _ok(_load().fgmp_tensor_peak(kind, mma_per_cta, workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_tensor_peak")
 
 
 def check(workspace: torch.Tensor) -> None:
