@@ -89,29 +89,35 @@ __global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* blob, int6
     });
 }
 
-// ------------------------------------------------------------------ bf16 tcgen05 GEMM
-constexpr int BM = 128, BN = 256, BK = 64;          // BK bf16 = one 128-byte swizzle row
-constexpr int STAGES = 4;
+// ------------------------------------------------------------------ bf16 tcgen05 GEMM on CTA pairs
+// Two CTAs of a cluster share one 256 x 256 output tile: each loads its 128 rows of A and its half
+// (128 rows) of B, the pair's leader issues tcgen05.mma cta_group::2 (M = 256), which reads both
+// halves of B from the two shared memories, and each CTA's TMEM holds the accumulators of its own
+// 128 rows.  B is fetched once per pair: a stage is 32 KiB per CTA for 256 x 256 x 64 of math (a single
+// CTA with a 128 x 256 tile needs 48 KiB for half of that), which is what the L2 -> shared-memory path can
+// sustain.  No TMA multicast.  Persistent: warp 0 = TMA producer, warp 1 = MMA issuer (leader CTA
+// only) and TMEM owner, warps 2-5 = epilogue; two accumulator buffers of 256 TMEM columns.
+constexpr int BK = 64;                              // BK bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int GEMM_THREADS = 192;
-constexpr uint32_t A_TILE_BYTES = BM * BK * 2, B_TILE_BYTES = BN * BK * 2;
-constexpr uint32_t STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
-constexpr uint32_t TMEM_COLS = 2 * BN;              // two accumulator buffers
-constexpr size_t GEMM_SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int P_BM = 256, P_BN = 256;               // per pair
+constexpr int P_STAGES = 6;
+constexpr uint32_t P_A_BYTES = 128 * BK * 2, P_B_BYTES = 128 * BK * 2, P_STAGE_BYTES = P_A_BYTES + P_B_BYTES;
+constexpr uint32_t TMEM_COLS = 2 * P_BN;            // two accumulator buffers
+constexpr size_t PAIR_SMEM = (size_t)P_STAGES * P_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=256, M=256
+constexpr uint32_t IDESC_BF16_PAIR = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P_BN >> 3) << 17) | ((uint32_t)(P_BM >> 4) << 24);
 
-// instruction descriptor, kind::f16: D=f32, A=B=bf16, both K-major, N=BN, M=BM
-constexpr uint32_t IDESC_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-
-// Tile order: bands of RASTER_M tile rows, all tile columns of a band before the next band, tile rows
-// fastest inside a band.  The CTAs that run together then share few A and B panels, which the
+// Tile order: bands of P_RASTER_M tile rows, all tile columns of a band before the next band, tile rows
+// fastest inside a band.  The pairs that run together then share few A and B panels, which the
 // 126 MB L2 keeps between their reads.
-constexpr int RASTER_M = 8;
-__device__ __forceinline__ void tile_coords(int64_t t, int64_t tiles_m, int64_t tiles_n, int64_t& tm, int64_t& tn)
+constexpr int P_RASTER_M = 4;
+__device__ __forceinline__ void pair_tile_coords(int64_t t, int64_t tiles_m, int64_t tiles_n, int64_t& tm, int64_t& tn)
 {
-    const int64_t per_band = (int64_t)RASTER_M * tiles_n;
+    const int64_t per_band = (int64_t)P_RASTER_M * tiles_n;
     const int64_t band = t / per_band, r = t % per_band;
-    const int64_t rows = min((int64_t)RASTER_M, tiles_m - band * RASTER_M);
-    tm = band * RASTER_M + r % rows;
+    const int64_t rows = min((int64_t)P_RASTER_M, tiles_m - band * P_RASTER_M);
+    tm = band * P_RASTER_M + r % rows;
     tn = r / rows;
 }
 
@@ -122,76 +128,116 @@ struct GemmParams {
     int* status;
 };
 
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p)
+// one row of 32 accumulator columns -> Y (scaled by the product of the tensor scales)
+__device__ __forceinline__ void store_chunk32(const GemmParams& p, int64_t row, int64_t col0, const uint32_t (&r)[32], float alpha)
+{
+    if (row >= p.M) return;
+    if (p.y_is_bf16) {
+        __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
+        if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+                uint32_t o[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * u]) * alpha,
+                                                             __uint_as_float(r[j + 2 * u + 1]) * alpha);
+                    o[u] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(y + j) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        } else {
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) y[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
+        }
+    } else {
+        float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
+        if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
+                                                                __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
+        } else {
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) y[j] = __uint_as_float(r[j]) * alpha;
+        }
+    }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
-    // bars[0..S) full, [S..2S) empty, [2S..2S+2) acc_full, [2S+2..2S+4) acc_empty
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)P_STAGES * P_STAGE_BYTES);
+    // bars[0..S) full (used in the leader), [S..2S) empty, [2S..2S+2) acc_full, [2S+2..2S+4) acc_empty (leader)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * P_STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
-    const uint32_t accf0 = smem_u32(bars + 2 * STAGES), acce0 = smem_u32(bars + 2 * STAGES + 2);
+    const uint32_t rank = cluster_ctarank();           // 0 = leader
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + P_STAGES);
+    const uint32_t accf0 = smem_u32(bars + 2 * P_STAGES), acce0 = smem_u32(bars + 2 * P_STAGES + 2);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); }
+        for (int s = 0; s < P_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 8); }   // 4 epilogue warps x 2 CTAs
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                                     // the other CTA's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int64_t tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const int64_t tiles_m = (p.M + P_BM - 1) / P_BM, tiles_n = (p.N + P_BN - 1) / P_BN;
     const int64_t num_tiles = tiles_m * tiles_n;
+    const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_kb = (int)(p.K / BK);
 
     if (warp == 0) {
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
-            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            for (int64_t t = pair; t < num_tiles && ok; t += num_pairs) {
                 int64_t tm, tn;
-                tile_coords(t, tiles_m, tiles_n, tm, tn);
-                const int32_t m0 = (int32_t)(tm * BM), n0 = (int32_t)(tn * BN);
+                pair_tile_coords(t, tiles_m, tiles_n, tm, tn);
+                const int32_t m0 = (int32_t)(tm * P_BM + 128 * rank), n0 = (int32_t)(tn * P_BN + 128 * rank);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1))) break;
-                    const uint32_t fb = full0 + 8 * stage;
-                    mbar_expect_tx(fb, STAGE_BYTES);
-                    const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-                    tma_load_2d(sa, &tmA, kb * BK, m0, fb);
-                    tma_load_2d(sa + A_TILE_BYTES, &tmB, kb * BK, n0, fb);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    // the leader's barrier counts the bytes of both CTAs
+                    if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * P_STAGE_BYTES);
+                    const uint32_t fb = cluster_map(full0 + 8 * stage, 0);
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * P_STAGE_BYTES);
+                    tma_load_2d_pair(sa, &tmA, kb * BK, m0, fb);
+                    tma_load_2d_pair(sa + P_A_BYTES, &tmB, kb * BK, n0, fb);
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             int stage = 0; uint32_t phase = 0; bool ok = true;
             int64_t it = 0;
-            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+            for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
                 const int acc = (int)(it & 1); const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
                 if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * P_BN);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-                    const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sa + A_TILE_BYTES);
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * P_STAGE_BYTES);
+                    const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sa + P_A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_f16(d_tmem, adesc + (uint64_t)(k * UMMA_K * 2 / 16), bdesc + (uint64_t)(k * UMMA_K * 2 / 16),
-                                 IDESC_BF16, (kb | k) ? 1u : 0u);
-                    umma_commit(empty0 + 8 * stage);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                        umma_f16_pair(d_tmem, adesc + (uint64_t)(k * UMMA_K * 2 / 16), bdesc + (uint64_t)(k * UMMA_K * 2 / 16),
+                                      IDESC_BF16_PAIR, (kb | k) ? 1u : 0u);
+                    umma_commit_pair(empty0 + 8 * stage, 3);          // the stage is free in both CTAs
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit(accf0 + 8 * acc);
+                if (ok) umma_commit_pair(accf0 + 8 * acc, 3);         // both epilogues may read their halves
             }
         }
     } else {
@@ -199,68 +245,36 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const float alpha = __fmul_rn(p.ha->scale_fp4, p.hw->scale_fp4);
         bool ok = true;
         int64_t it = 0;
-        for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+        for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
             const int acc = (int)(it & 1); const uint32_t acc_phase = (uint32_t)((it >> 1) & 1);
             int64_t tm, tn;
-            tile_coords(t, tiles_m, tiles_n, tm, tn);
-            const int64_t m0 = tm * BM, n0 = tn * BN;
+            pair_tile_coords(t, tiles_m, tiles_n, tm, tn);
+            const int64_t m0 = tm * P_BM + 128 * rank, n0 = tn * P_BN;
             if (!(ok = mbar_wait(accf0 + 8 * acc, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
             const int64_t row = m0 + q * 32 + lane;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < P_BN / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
-                const int64_t col0 = n0 + c * 32;
-                if (row < p.M) {
-                    if (p.y_is_bf16) {
-                        __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
-                        if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                uint32_t o[4];
-#pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * u]) * alpha,
-                                                                             __uint_as_float(r[j + 2 * u + 1]) * alpha);
-                                    o[u] = *reinterpret_cast<uint32_t*>(&h);
-                                }
-                                *reinterpret_cast<uint4*>(y + j) = make_uint4(o[0], o[1], o[2], o[3]);
-                            }
-                        } else {
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) y[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
-                        }
-                    } else {
-                        float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
-                        if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
-                                                                                __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
-                        } else {
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) y[j] = __uint_as_float(r[j]) * alpha;
-                        }
-                    }
-                }
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * P_BN + c * 32), r);
+                store_chunk32(p, row, n0 + c * 32, r, alpha);
             }
             tc_fence_before();
-            mbar_arrive(acce0 + 8 * acc);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(cluster_map(acce0 + 8 * acc, 0));
         }
     }
 
     __syncthreads();
     if (*abort_flag) {
-        // give copies and MMAs that may still be in flight time to land before the CTA's
-        // shared memory and TMEM are released
         const unsigned long long t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
         __syncthreads();
     }
+    cluster_sync();                                     // neither CTA leaves while the other may still read its memory
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
@@ -323,16 +337,22 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     uint8_t* planeA = ws + 1024;
     uint8_t* planeW = planeA + fgmp_align1k((size_t)M * K * 2);
 
-    static bool attr_set[64] = {};
+    // CTA pairs that can be resident at once on this device (a pair needs two SMs of one cluster domain)
+    static int pairs_of_device[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM) != cudaSuccess)
+    if (dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
+    if (!pairs_of_device[dev]) {
+        if (cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PAIR_SMEM) != cudaSuccess)
             return FGMP_ERR_CUDA;
-        attr_set[dev] = true;
+        cudaLaunchConfig_t qc = {};
+        qc.gridDim = dim3((unsigned)(fgmp_sm_count() & ~1)); qc.blockDim = dim3(GEMM_THREADS); qc.dynamicSmemBytes = PAIR_SMEM;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_bf16_pair_kernel, &qc) != cudaSuccess || n < 1) return FGMP_ERR_CUDA;
+        pairs_of_device[dev] = n;
     }
     CUtensorMap tmA, tmB;
-    if (!make_tmap_bf16(&tmA, planeA, M, K, BM) || !make_tmap_bf16(&tmB, planeW, N, K, BN)) return FGMP_ERR_CUDA;
+    if (!make_tmap_bf16(&tmA, planeA, M, K, 128) || !make_tmap_bf16(&tmB, planeW, N, K, 128)) return FGMP_ERR_CUDA;
 
     if (cudaMemsetAsync(status, 0, 256, s) != cudaSuccess) return FGMP_ERR_CUDA;
     const int sms = fgmp_sm_count();
@@ -348,9 +368,9 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     p.ha = reinterpret_cast<const fgmp_packed_header*>(packed_acts);
     p.hw = reinterpret_cast<const fgmp_packed_header*>(packed_weights);
     p.status = status;
-    const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    const int grid = (int)(tiles < sms ? tiles : sms);
-    FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, s>>>(tmA, tmB, p));
+    const int64_t tiles = ((M + P_BM - 1) / P_BM) * ((N + P_BN - 1) / P_BN);
+    const int pairs = (int)(tiles < pairs_of_device[dev] ? tiles : pairs_of_device[dev]);
+    FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_pair_kernel<<<2 * pairs, GEMM_THREADS, PAIR_SMEM, s>>>(tmA, tmB, p));
     return fgmp_launch_status();
 }
 
