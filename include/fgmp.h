@@ -107,7 +107,8 @@ typedef struct {
 } fgmp_packed_header;
 
 enum { FGMP_OP_QUANTIZE_WEIGHTS = 0, FGMP_OP_QUANTIZE_ACTIVATIONS = 1, FGMP_OP_LINEAR = 2,
-       FGMP_OP_CALIBRATE_TAU = 3 };
+       FGMP_OP_CALIBRATE_TAU = 3,
+       FGMP_OP_GLOBAL_TAU = 4       /* M = total number of scores; N, K ignored */ };
 
 /* ---- sizes (pure host functions; return 0 for invalid shapes) ---- */
 size_t fgmp_weights_bytes(int64_t N, int64_t K, int64_t max_fp8_blocks);
@@ -151,6 +152,37 @@ fgmp_status fgmp_calibrate_tau(const void* X_bf16, int64_t ldx, const float* fis
                                int64_t M, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
                                double fp8_fraction, float* tau_out,
                                void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- offline: one threshold for several tensors (Eq. 10, global threshold) ----
+ * Section 3.2 prefers a single threshold per tensor kind over per-layer ones: the blocks of all
+ * layers compete for the FP8 budget, so sensitive layers end up with a larger FP8 share.
+ * fgmp_weight_scores writes the block scores of one weight tensor (the scores fgmp_quantize_weights
+ * ranks: under the clipped microscale if cm = FGMP_CLIP_SW_BRUTE; scores[n * K/16 + kb], device,
+ * 16-byte aligned; workspace as for fgmp_quantize_weights); fgmp_activation_scores does the same
+ * for a calibration batch.  fgmp_global_tau then takes the scores of n_tensors tensors
+ * (score_arrays: HOST array of device pointers, counts: HOST array of lengths) and writes to tau_out
+ * (device float) the value midway (in fp32) between the k-th and (k+1)-th largest of their union,
+ * k = floor(fraction * total + 0.5): exactly k blocks exceed it unless scores tie (k = 0 gives +inf,
+ * k = total gives -1).  Pass it as `tau` with fp8_fraction < 0 to fgmp_quantize_weights, or as the
+ * activation threshold.  workspace: fgmp_workspace_bytes(FGMP_OP_GLOBAL_TAU, total, 0, 0). */
+fgmp_status fgmp_weight_scores(const void* W_bf16, int64_t ldw, const float* fisher_elem, int64_t ldf,
+                               int64_t N, int64_t K, fgmp_scales sc, fgmp_score_mode sm, fgmp_clip_mode cm,
+                               float* scores, void* workspace, size_t ws_bytes, void* cuda_stream);
+fgmp_status fgmp_global_tau(const float* const* score_arrays, const int64_t* counts, int n_tensors,
+                            double fp8_fraction, float* tau_out,
+                            void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- offline: the baseline policies of Section 3.4 ----
+ * The "Quantization Error" policy (Eq. 12) is the score of Eq. 8 with every sensitivity weight equal to
+ * one: pass a vector (activations) or matrix (weights) of ones as the Fisher argument, with
+ * FGMP_SCORE_HP_TO_LP.  The "Output Error" policy (Eq. 13) weights element i by the average squared
+ * magnitude of input channel i of the OTHER operand: this call computes that vector, mean_sq[c] = mean
+ * over rows of X[r, c]^2 (X bf16 [rows, K] row-major, any K >= 1, rows <= 2^24; fp32, rows added in
+ * order), for the weights' policy from a calibration batch of activations, for the activations' policy
+ * from the weight matrix; broadcast it over the rows of the weights' Fisher matrix.  Both policies use
+ * the local threshold (fraction mode / fgmp_calibrate_tau). */
+fgmp_status fgmp_channel_mean_sq(const void* X_bf16, int64_t ldx, int64_t rows, int64_t K,
+                                 float* mean_sq, void* cuda_stream);
 
 /* ---- workspace of fgmp_linear ----
  * The first FGMP_WS_CONTROL_BYTES of a workspace hold the status word that fgmp_check reads and,

@@ -204,3 +204,36 @@ def clip_objective(v: np.ndarray, f: np.ndarray, c: int, scale_fp4: float) -> fl
 
 def num_threads() -> int:
     return lib().oracle_num_threads()
+
+
+def global_threshold(score_arrays, fp8_fraction: float) -> float:
+    """Global threshold of Eq. 10 (Section 3.2): one tau for several tensors, chosen so that the
+    fraction R of the blocks of all of them together exceeds it.  The plain definition: pool the
+    scores, k = floor(R * B + 0.5), tau = the fp32 value midway between the k-th largest score and
+    the largest score strictly below it (that lower score itself if fp32 has no value between
+    them; 0 if there is none below); k = 0 gives +inf, k = B gives -1 (scores are >= 0)."""
+    pooled = np.concatenate([np.asarray(a, dtype=np.float32).ravel() for a in score_arrays])
+    B = pooled.size
+    k = int(np.floor(fp8_fraction * B + 0.5))
+    if k <= 0:
+        return float("inf")
+    if k >= B:
+        return -1.0
+    s = np.sort(pooled)[::-1]
+    hi = s[k - 1]
+    below = s[s < hi]
+    lo = below.max() if below.size else np.float32(0.0)
+    t = np.float32(0.5) * np.float32(hi + lo)
+    return float(t) if (lo <= t < hi) else float(lo)
+
+
+def channel_mean_sq(x_bf16_bits: np.ndarray) -> np.ndarray:
+    """Weights of the "Output Error" policy (Eq. 13): the average squared magnitude of every input
+    channel of the other operand.  x_bf16_bits: uint16 [rows, K]; float32 [K]: rows added in order,
+    one fp32 multiply and one fp32 add per element, one division by the row count."""
+    x = (np.ascontiguousarray(x_bf16_bits).astype(np.uint32) << 16).view(np.float32)
+    s = np.zeros(x.shape[1], np.float32)
+    for r in range(x.shape[0]):
+        s = (s + (x[r] * x[r]).astype(np.float32)).astype(np.float32)
+    return (s / np.float32(x.shape[0])).astype(np.float32)
+

@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libfgmp.so")
 
 SCORE_LP_ERROR, SCORE_HP_TO_LP = 0, 1
 CLIP_NONE, CLIP_SW_BRUTE = 0, 1
-OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU = 0, 1, 2, 3
+OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU = 0, 1, 2, 3, 4
 
 
 class FgmpError(RuntimeError):
@@ -60,6 +60,12 @@ def _load():
     L.fgmp_linear_static.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, vp]
     L.fgmp_check.restype = ci
     L.fgmp_check.argtypes = [vp, vp]
+    L.fgmp_channel_mean_sq.restype = ci
+    L.fgmp_channel_mean_sq.argtypes = [vp, i64, i64, i64, vp, vp]
+    L.fgmp_weight_scores.restype = ci
+    L.fgmp_weight_scores.argtypes = [vp, i64, vp, i64, i64, i64, _Scales, ci, ci, vp, vp, sz, vp]
+    L.fgmp_global_tau.restype = ci
+    L.fgmp_global_tau.argtypes = [vp, vp, ci, ctypes.c_double, vp, vp, sz, vp]
     L.fgmp_tensor_peak.restype = ci
     L.fgmp_tensor_peak.argtypes = [ci, i64, vp, sz, vp]
     L.fgmp_workspace_init.restype = ci
@@ -205,6 +211,46 @@ def calibrate_tau(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ra
     _ok(L.fgmp_calibrate_tau(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio),
                              score_mode, float(fp8_fraction), tau.data_ptr(), workspace.data_ptr(),
                              workspace.numel(), _stream()), "fgmp_calibrate_tau")
+    return tau
+
+
+def channel_mean_sq(X: torch.Tensor) -> torch.Tensor:
+    """fp32 [K]: mean over the rows of X (bf16 [rows, K]) of X[r, c]^2 -- the weights of the Output Error policy."""
+    L = _load()
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    rows, K = X.shape
+    out = torch.empty(K, dtype=torch.float32, device=X.device)
+    _ok(L.fgmp_channel_mean_sq(X.data_ptr(), X.stride(0), rows, K, out.data_ptr(), _stream()), "fgmp_channel_mean_sq")
+    return out
+
+
+def weight_scores(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float = 0.0, ratio: int = 3,
+                  score_mode: int = SCORE_LP_ERROR, clip_mode: int = CLIP_SW_BRUTE) -> torch.Tensor:
+    """Block scores [N, K/16] of a weight tensor, as fgmp_quantize_weights ranks them."""
+    L = _load()
+    N, K = W.shape
+    scores = torch.empty(N, K // 16, dtype=torch.float32, device=W.device)
+    workspace = _alloc_aligned(L.fgmp_workspace_bytes(OP_QUANTIZE_WEIGHTS, 0, N, K), W.device)
+    _ok(L.fgmp_weight_scores(W.data_ptr(), W.stride(0), fisher.data_ptr(), fisher.stride(0), N, K,
+                             _Scales(scale_fp4, ratio), score_mode, clip_mode, scores.data_ptr(),
+                             workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_weight_scores")
+    return scores
+
+
+def global_tau(score_tensors, fp8_fraction: float) -> torch.Tensor:
+    """One threshold for several tensors (Eq. 10): a 1-element fp32 device tensor such that the given
+    fraction of all blocks of `score_tensors` (fp32 device tensors of block scores) exceeds it."""
+    L = _load()
+    ts = [t.contiguous() for t in score_tensors]
+    n = len(ts)
+    ptrs = (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+    counts = (ctypes.c_int64 * n)(*[t.numel() for t in ts])
+    total = sum(t.numel() for t in ts)
+    dev = ts[0].device
+    tau = torch.empty(1, dtype=torch.float32, device=dev)
+    workspace = _alloc_aligned(L.fgmp_workspace_bytes(OP_GLOBAL_TAU, total, 0, 0), dev)
+    _ok(L.fgmp_global_tau(ptrs, counts, n, float(fp8_fraction), tau.data_ptr(), workspace.data_ptr(),
+                          workspace.numel(), _stream()), "fgmp_global_tau")
     return tau
 
 

@@ -394,6 +394,7 @@ extern "C" fgmp_status fgmp_check(const void* workspace, void* cuda_stream)
 
 extern "C" size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K)
 {
+    if (op == FGMP_OP_GLOBAL_TAU) return M >= 1 ? fgmp_ws_global_tau(M) : 0;
     if (K < 64 || (K % 64) != 0) return 0;
     switch (op) {
         case FGMP_OP_QUANTIZE_WEIGHTS: return N >= 1 ? fgmp_ws_quantize_weights(N, K) : 0;

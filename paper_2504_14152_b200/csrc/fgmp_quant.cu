@@ -6,6 +6,7 @@
 // consecutive blocks of one row = one mask word, produced with a ballot.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
+#include <cuda_bf16.h>
 
 namespace {
 
@@ -192,6 +193,20 @@ __global__ void __launch_bounds__(128) unpack_w_kernel(const uint8_t* blob, int6
     });
 }
 
+// mean of squares per column of a bf16 matrix; thread per column, rows in order (one fp32 multiply
+// and one fp32 add per element, then one division): reproducible bit for bit
+__global__ void channel_mean_sq_kernel(const __nv_bfloat16* X, int64_t ld, int64_t rows, int64_t K, float* out)
+{
+    const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= K) return;
+    float s = 0.f;
+    for (int64_t r = 0; r < rows; ++r) {
+        const float v = __bfloat162float(X[r * ld + c]);
+        s = __fadd_rn(s, __fmul_rn(v, v));
+    }
+    out[c] = __fdiv_rn(s, (float)rows);
+}
+
 fgmp_status check_act_args(const void* X, int64_t ldx, const float* fisher, int64_t M, int64_t K, fgmp_scales sc, int sm)
 {
     if (!X || !fisher) return FGMP_ERR_INVALID_ARG;
@@ -292,5 +307,18 @@ extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, 
         int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);
         FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_kernel<<<grid, 256, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
     }
+    return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_channel_mean_sq(const void* X_bf16, int64_t ldx, int64_t rows, int64_t K,
+                                            float* mean_sq, void* cuda_stream)
+{
+    if (!X_bf16 || !mean_sq) return FGMP_ERR_INVALID_ARG;
+    if (rows < 1 || rows > ((int64_t)1 << 24) || K < 1 || ldx < K) return FGMP_ERR_SHAPE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    FGMP_LAUNCH(FGMP_K_ACT_AUX, s, channel_mean_sq_kernel<<<(unsigned)((K + 127) / 128), 128, 0, s>>>(
+        reinterpret_cast<const __nv_bfloat16*>(X_bf16), ldx, rows, K, mean_sq));
     return fgmp_launch_status();
 }

@@ -509,3 +509,83 @@ extern "C" fgmp_status fgmp_calibrate_tau(const void* X_bf16, int64_t ldx, const
     }
     return fgmp_launch_status();
 }
+
+extern "C" fgmp_status fgmp_weight_scores(const void* W_bf16, int64_t ldw, const float* fisher_elem, int64_t ldf,
+                                          int64_t N, int64_t K, fgmp_scales sc, fgmp_score_mode sm, fgmp_clip_mode cm,
+                                          float* scores, void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!W_bf16 || !fisher_elem || !scores || !workspace) return FGMP_ERR_INVALID_ARG;
+    if ((int)sm < 0 || (int)sm > 1 || (int)cm < 0 || (int)cm > 1) return FGMP_ERR_INVALID_ARG;
+    if (!(sc.scale_fp4 >= 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
+    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    if (N < 1 || K < 64 || (K % 64) != 0 || ldw < K || (ldw % 8) != 0 || ldf < K || (ldf % 4) != 0) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)W_bf16 & 15) || ((uintptr_t)fisher_elem & 15) || ((uintptr_t)scores & 15) || ((uintptr_t)workspace & 255))
+        return FGMP_ERR_SHAPE;
+    const int64_t KB = K / 16, B = N * KB;
+    if (B >= ((int64_t)1 << 32)) return FGMP_ERR_SHAPE;
+    if (ws_bytes < ws_weights_bytes(N, K)) return FGMP_ERR_WORKSPACE;
+    fgmp_status stt;
+    if ((stt = fgmp_require_sm100()) != FGMP_OK) return stt;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    SelectState* st = reinterpret_cast<SelectState*>(ws);
+    uint8_t* sc_tmp = ws + STATE_BYTES + fgmp_align1k((size_t)B * 4);
+    const uint4* W = reinterpret_cast<const uint4*>(W_bf16);
+    const int ratio = sc.fp8_log2_ratio;
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, 0ull));
+    if (sc.scale_fp4 == 0.f) {
+        FGMP_LAUNCH(FGMP_K_W_AMAX, s, w_amax_kernel<<<grid_for(N * (K / 8), 256, 8), 256, 0, s>>>(W, ldw / 8, N, K / 8, st));
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, w_scale_kernel<<<1, 32, 0, s>>>(st));
+    }
+    const int g = grid_for(B, 256, 4);
+    if (sm == FGMP_SCORE_LP_ERROR) {
+        if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+        else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+    } else {
+        if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+        else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+    }
+    return fgmp_launch_status();
+}
+
+size_t fgmp_ws_global_tau(int64_t total) { return STATE_BYTES + fgmp_align1k((size_t)total * 4); }
+
+extern "C" fgmp_status fgmp_global_tau(const float* const* score_arrays, const int64_t* counts, int n_tensors,
+                                       double fp8_fraction, float* tau_out,
+                                       void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!score_arrays || !counts || n_tensors < 1 || !tau_out || !workspace) return FGMP_ERR_INVALID_ARG;
+    if (!(fp8_fraction >= 0.0) || fp8_fraction > 1.0) return FGMP_ERR_INVALID_ARG;
+    if ((uintptr_t)workspace & 255) return FGMP_ERR_SHAPE;
+    int64_t B = 0;
+    for (int i = 0; i < n_tensors; ++i) {
+        if (!score_arrays[i] || counts[i] < 1) return FGMP_ERR_INVALID_ARG;
+        B += counts[i];
+    }
+    if (B >= ((int64_t)1 << 32)) return FGMP_ERR_SHAPE;
+    if (ws_bytes < fgmp_ws_global_tau(B)) return FGMP_ERR_WORKSPACE;
+    fgmp_status stt;
+    if ((stt = fgmp_require_sm100()) != FGMP_OK) return stt;
+    uint8_t* ws = (uint8_t*)workspace;
+    SelectState* st = reinterpret_cast<SelectState*>(ws);
+    float* scores = reinterpret_cast<float*>(ws + STATE_BYTES);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // all scores side by side: the threshold is a rank statistic of their union
+    int64_t off = 0;
+    for (int i = 0; i < n_tensors; ++i) {
+        if (cudaMemcpyAsync(scores + off, score_arrays[i], (size_t)counts[i] * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+            return FGMP_ERR_CUDA;
+        off += counts[i];
+    }
+    int64_t k = (int64_t)floor(fp8_fraction * (double)B + 0.5);
+    if (k > B) k = B;
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, state_init_kernel<<<1, 256, 0, s>>>(st, 1.0f, (unsigned long long)k));
+    if (k == 0 || k == B) {
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, k == 0 ? 1 : 2));
+    } else {
+        run_select(scores, B, st, s);
+        FGMP_LAUNCH(FGMP_K_SELECT, s, next_below_kernel<<<grid_for(B, 256, 8), 256, 0, s>>>(scores, B, st));
+        FGMP_LAUNCH(FGMP_K_W_AUX, s, calib_finish_kernel<<<1, 32, 0, s>>>(st, tau_out, 0));
+    }
+    return fgmp_launch_status();
+}

@@ -382,3 +382,80 @@ def test_decode_llama2_70b_fc2_sampled(fg):
     """The K of Llama-2-70B FC2 (28672: 112 chunks per tile, every tile shared by several thread blocks) with
     1024 of its 8192 output rows."""
     _sampled_linear_check(fg, gi.llama("fc2_70b", 16, 1024, 28672, seed=7), 0.1, 4000, 4)
+
+
+# ------------------------------------------------------------ global threshold (Eq. 10)
+
+def test_global_threshold_over_several_tensors(fg):
+    """One tau for two weight tensors and one for two activation batches: GPU scores equal the oracle's bit
+    for bit, the pooled threshold equals the oracle's, and packing with it gives each tensor exactly the
+    blocks whose score exceeds it (their total is the budget; the per-tensor shares differ)."""
+    wls = [gi.llama("g0", 48, 384, 1024, seed=31), gi.llama("g1", 32, 256, 2048, seed=32)]
+    frac = 0.1
+    # weights
+    ws_gpu, ws_cpu, fws = [], [], []
+    for i, wl in enumerate(wls):
+        w, fw = wl.w(), wl.fw() * (1.0 if i == 0 else 6.0)          # the second tensor is the more sensitive one
+        fws.append(fw)
+        ws_gpu.append(fg.weight_scores(w.cuda(), fw.cuda(), clip_mode=1))
+        q = oracle.quantize_weights(gi.bf16_bits(w), fw.numpy(), clip=True, mode=0, fp8_fraction=0.0)
+        ws_cpu.append(q.scores)
+        assert np.array_equal(ws_gpu[-1].cpu().numpy().ravel().view(np.uint32), q.scores.view(np.uint32))
+    tau_w = oracle.global_threshold(ws_cpu, frac)
+    tau_w_gpu = float(fg.global_tau(ws_gpu, frac).item())
+    assert np.float32(tau_w_gpu) == np.float32(tau_w)
+    total8 = 0
+    shares = []
+    for wl, fw, sc in zip(wls, fws, ws_cpu):
+        w = wl.w()
+        q = oracle.quantize_weights(gi.bf16_bits(w), fw.numpy(), clip=True, mode=0, fp8_fraction=-1.0, tau=tau_w)
+        pw = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=1, fp8_fraction=-1.0, tau=tau_w_gpu)
+        compare_packed(fg, pw, q, tau=tau_w, what=wl.name)
+        n8 = int(q.mask_bits().sum())
+        assert n8 == int((sc > np.float32(tau_w)).sum())
+        total8 += n8
+        shares.append(n8 / sc.size)
+    B = sum(s.size for s in ws_cpu)
+    assert total8 == int(np.floor(frac * B + 0.5))
+    assert shares[1] > frac > shares[0]
+    # activations
+    xs_gpu, xs_cpu = [], []
+    for wl in wls:
+        x, fx = wl.x(), wl.fx()
+        s4 = gi.tensor_scale(x)
+        xs_gpu.append(fg.activation_scores(x.cuda(), fx.cuda(), scale_fp4=s4))
+        xs_cpu.append(oracle.quantize_activations(gi.bf16_bits(x), fx.numpy(), s4, tau=np.inf).scores)
+    tau_a = oracle.global_threshold(xs_cpu, frac)
+    assert np.float32(float(fg.global_tau(xs_gpu, frac).item())) == np.float32(tau_a)
+    for f, want in ((0.0, float("inf")), (1.0, -1.0)):
+        assert float(fg.global_tau(xs_gpu, f).item()) == want
+
+
+# ------------------------------------------------------------ baseline policies (Eq. 12, 13)
+
+def test_baseline_policies_as_weight_substitutions(fg):
+    """Quantization Error (ones as sensitivity weights) and Output Error (mean squared channel magnitude of
+    the other operand, computed on the GPU) run through the same kernels: packed tensors equal the oracle's."""
+    wl = gi.llama("pol", 40, 256, 1024, seed=41)
+    x, w = wl.x(), wl.w()
+    xb, wb = gi.bf16_bits(x), gi.bf16_bits(w)
+    s4 = gi.tensor_scale(x)
+    # Output Error weights: bit-exact against the oracle
+    ax_cpu, aw_cpu = oracle.channel_mean_sq(xb), oracle.channel_mean_sq(wb)
+    ax_gpu, aw_gpu = fg.channel_mean_sq(x.cuda()), fg.channel_mean_sq(w.cuda())
+    assert np.array_equal(ax_gpu.cpu().numpy().view(np.uint32), ax_cpu.view(np.uint32))
+    assert np.array_equal(aw_gpu.cpu().numpy().view(np.uint32), aw_cpu.view(np.uint32))
+    ones_k = torch.ones(wl.K, dtype=torch.float32)
+    for name, fa, fwv in (("QE", ones_k, ones_k), ("OE", torch.from_numpy(aw_cpu), torch.from_numpy(ax_cpu))):
+        fwm = fwv.expand(wl.N, wl.K).contiguous()
+        # weights: local threshold = fraction mode
+        qw = oracle.quantize_weights(wb, fwm.numpy(), clip=False, mode=1, fp8_fraction=0.1)
+        pw = fg.quantize_weights(w.cuda(), fwm.cuda(), clip_mode=0, score_mode=1, fp8_fraction=0.1)
+        compare_packed(fg, pw, qw, what=name + " weights")
+        # activations: threshold from this batch's own scores
+        scores = oracle.quantize_activations(xb, fa.numpy(), s4, tau=np.inf, mode=1).scores
+        tau = tau_for_fraction(scores, 0.1)
+        qa = oracle.quantize_activations(xb, fa.numpy(), s4, tau=tau, mode=1)
+        pa = fg.quantize_activations(x.cuda(), fa.cuda(), scale_fp4=s4, score_mode=1, tau=tau)
+        compare_packed(fg, pa, qa, tau=tau, what=name + " activations")
+        assert qa.mask_bits().sum() == int(np.floor(0.1 * scores.size + 0.5))

@@ -327,3 +327,50 @@ def test_decoded_values_follow_the_format_definitions():
         v4 = E2M1[_unpack4(q)] * e4[sc] * s4
         v8 = e4[q.codes8.reshape(q.rows, q.K)] * s4 * 2.0 ** q.ratio
         assert np.array_equal(oracle.decode(q), np.where(mb, v8, v4))
+
+
+# ------------------------------------------------------------------ global threshold (Eq. 10)
+
+def test_global_threshold_counts_and_layer_shares():
+    """Pins of oracle.global_threshold: against a brute-force rank count on small pools; exactly k blocks
+    of the pool exceed it; with one tensor it is the local threshold of Eq. 9; a tensor with uniformly
+    larger scores takes a larger share of the FP8 budget than its size (the point of Eq. 10)."""
+    rng = np.random.default_rng(5)
+    a = rng.lognormal(0.0, 1.0, 300).astype(np.float32)
+    b = (4.0 * rng.lognormal(0.0, 1.0, 100)).astype(np.float32)
+    for frac in (0.05, 0.1, 0.25, 0.5):
+        tau = oracle.global_threshold([a, b], frac)
+        pool = np.concatenate([a, b])
+        k = int(np.floor(frac * pool.size + 0.5))
+        assert int((pool > np.float32(tau)).sum()) == k
+        # brute force: tau lies strictly below exactly k pooled scores and at or above all others
+        assert sum(1 for v in pool if v > np.float32(tau)) == k
+        assert np.float32(tau) in (np.float32(tau),) and np.sort(pool)[::-1][k] <= np.float32(tau) < np.sort(pool)[::-1][k - 1]
+        # the sensitive tensor gets more than its proportional share
+        share_b = (b > np.float32(tau)).mean()
+        share_a = (a > np.float32(tau)).mean()
+        assert share_b > frac > share_a
+    # one tensor: the same value as sorting that tensor alone
+    s = np.sort(a)[::-1]
+    k = int(np.floor(0.1 * a.size + 0.5))
+    assert oracle.global_threshold([a], 0.1) == float(np.float32(0.5) * (s[k - 1] + s[k]))
+    # extremes and ties
+    assert oracle.global_threshold([a, b], 0.0) == float("inf")
+    assert oracle.global_threshold([a, b], 1.0) == -1.0
+    t = np.array([3, 3, 3, 1, 1], np.float32)
+    assert oracle.global_threshold([t], 0.4) == 2.0       # k = 2 falls inside the tie at 3: next distinct value below is 1
+    assert (t > 2.0).sum() == 3                            # ties across the boundary all go to FP8
+
+
+def test_channel_mean_sq_against_float64():
+    """Pins of oracle.channel_mean_sq: exact on small integers, within fp32 rounding of the fp64 mean of
+    squares on random data, and a transposed or unsquared version fails."""
+    xi = torch.tensor([[1, -2, 3], [3, 2, -1], [2, 2, 2], [0, 4, 1]], dtype=torch.float32).to(torch.bfloat16)
+    got = oracle.channel_mean_sq(gi.bf16_bits(xi))
+    assert got.tolist() == [14 / 4, 28 / 4, 15 / 4]
+    x = gi.activations(200, 64, 3, 0.05, 30.0)
+    ref = (x.double() ** 2).mean(0).numpy()
+    got = oracle.channel_mean_sq(gi.bf16_bits(x))
+    assert got.shape == (64,)
+    assert np.all(np.abs(got - ref) <= 200 * 2.0 ** -24 * ref)
+    assert not np.allclose((x.double().abs()).mean(0).numpy(), ref)
