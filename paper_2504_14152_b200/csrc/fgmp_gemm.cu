@@ -73,20 +73,48 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
     }
 }
 
-// packed weights -> bf16 plane; one CTA of 128 threads per unit record
-__global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane)
+// packed weights -> bf16 plane; one CTA of 128 threads per unit record, consecutive threads on
+// consecutive blocks of one row, four blocks per thread in flight at a time
+__global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* __restrict__ blob, int64_t rows, int64_t K, uint4* __restrict__ plane)
 {
     __shared__ UnitScratch sc;
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
     const PackedLayout L = fgmp_layout(rows, K, 1, 0);
     const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
-    fgmp_for_each_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, int row, int j, const uint8_t* rec, const uint8_t* e8) {
-        float v[16];
-        if (e8) e4m3x16_scaled(*reinterpret_cast<const uint4*>(e8), r8, v);
-        else nvfp4x16_scaled(*reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j)),
-                             rec[REC_SF + fgmp_rec_sf_offset(row, j)], v);
-        store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
-    });
+    const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
+    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    const uint8_t* rec = fgmp_record(blob, L, unit);
+    const uint8_t* fp8 = rec + fgmp_rec_fp8_offset(cnt);
+    const int j = threadIdx.x & 15;
+    const int64_t kb = c * 16 + j;
+    if (kb >= L.KB) return;
+#pragma unroll 1
+    for (int i0 = 0; i0 < 16; i0 += 4) {
+        uint2 c4[4];
+        uint4 c8[4];
+        uint32_t sfb[4], pos[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = (threadIdx.x >> 4) + 8 * (i0 + i);
+            pos[i] = sc.pos[row * 16 + j];
+            c4[i] = __ldg(reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j)));
+            sfb[i] = __ldg(rec + REC_SF + fgmp_rec_sf_offset(row, j));
+            c8[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (pos[i] != 0xffffu) c8[i] = __ldg(reinterpret_cast<const uint4*>(fp8 + (size_t)pos[i] * 16));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = (threadIdx.x >> 4) + 8 * (i0 + i);
+            const int64_t r = tile * 128 + row;
+            if (r >= L.rows) continue;
+            float v[16];
+            if (pos[i] != 0xffffu) e4m3x16_scaled(c8[i], r8, v);
+            else nvfp4x16_scaled(c4[i], sfb[i], v);
+            store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
+        }
+    }
 }
 
 // ------------------------------------------------------------------ bf16 tcgen05 GEMM on CTA pairs
