@@ -206,6 +206,22 @@ fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
                         void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                         void* workspace, size_t ws_bytes, void* cuda_stream);
 
+/* ---- fgmp_linear with the next layer's activation quantizer in its epilogue (Section 4.2) ----
+ * The paper's post-processing unit quantizes the output activations of a layer, block by block, to
+ * FP4 or FP8 from the FP32 partial sums, so that they reach memory only in packed form.  This call is
+ * fgmp_linear with a bf16 output followed by fgmp_quantize_activations on that output -- the packed
+ * result is the same bit for bit -- without the bf16 tensor ever being written or read: every
+ * accumulator is scaled, rounded to bf16 and quantized in registers by the GEMM's epilogue.
+ * packed_out is a packed activation tensor of M rows and N columns (N is the next layer's K; size from
+ * fgmp_acts_bytes(M, N)); fisher_chan_next [N], sc_next, sm and tau_next are the arguments
+ * fgmp_quantize_activations would get.  Needs M > 16 and N % 64 == 0 (decode-sized batches: call the
+ * two functions one after the other); workspace as for fgmp_linear. */
+fgmp_status fgmp_linear_quantize(const void* packed_acts, const void* packed_weights,
+                                 int64_t M, int64_t N, int64_t K,
+                                 const float* fisher_chan_next, fgmp_scales sc_next, fgmp_score_mode sm,
+                                 float tau_next, void* packed_out, size_t packed_bytes,
+                                 void* workspace, size_t ws_bytes, void* cuda_stream);
+
 /* ---- fgmp_linear for callers that cannot allocate (the paper has no counterpart) ----
  * Some callers have no way to hand the library a workspace: code that runs where cudaMalloc is
  * forbidden (inside a region that must not touch the allocator, a host that pre-sized its

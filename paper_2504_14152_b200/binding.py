@@ -60,6 +60,8 @@ def _load():
     L.fgmp_linear_static.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, vp]
     L.fgmp_check.restype = ci
     L.fgmp_check.argtypes = [vp, vp]
+    L.fgmp_linear_quantize.restype = ci
+    L.fgmp_linear_quantize.argtypes = [vp, vp, i64, i64, i64, vp, _Scales, ci, ctypes.c_float, vp, sz, vp, sz, vp]
     L.fgmp_channel_mean_sq.restype = ci
     L.fgmp_channel_mean_sq.argtypes = [vp, i64, i64, i64, vp, vp]
     L.fgmp_weight_scores.restype = ci
@@ -280,6 +282,25 @@ def linear(acts: PackedTensor, weights: PackedTensor, *, out_dtype=torch.float32
                       workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear")
     linear.last_workspace = workspace
     return out
+
+
+def linear_quantize(acts: PackedTensor, weights: PackedTensor, fisher_next: torch.Tensor, *, scale_fp4: float,
+                    ratio: int = 3, score_mode: int = SCORE_LP_ERROR, tau: float,
+                    workspace: torch.Tensor | None = None) -> PackedTensor:
+    """acts x weights^T, quantized for the next layer in the GEMM's epilogue: the packed activations
+    [M, N] that quantize_activations(linear(..., bf16), fisher_next, ...) would give."""
+    L = _load()
+    assert acts.K == weights.K and acts.kind == 0 and weights.kind == 1
+    M, N, K = acts.rows, weights.rows, acts.K
+    dev = acts.blob.device
+    out = _alloc_aligned(L.fgmp_acts_bytes(M, N), dev)
+    if workspace is None:
+        workspace = alloc_workspace(OP_LINEAR, M, N, K, dev)
+    _ok(L.fgmp_linear_quantize(acts.blob.data_ptr(), weights.blob.data_ptr(), M, N, K, fisher_next.data_ptr(),
+                               _Scales(scale_fp4, ratio), score_mode, tau, out.data_ptr(), out.numel(),
+                               workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear_quantize")
+    linear.last_workspace = workspace
+    return PackedTensor(out, M, N, 0)
 
 
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024

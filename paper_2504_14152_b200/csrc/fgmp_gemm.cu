@@ -149,12 +149,72 @@ __device__ __forceinline__ void pair_tile_coords(int64_t t, int64_t tiles_m, int
     tn = r / rows;
 }
 
+// The activation quantizer of the NEXT layer, run on the accumulators in the epilogue (Section 4.2:
+// the post-processing unit quantizes each output block to FP4 or FP8 from the FP32 partial sums).
+// codes4 == nullptr: off.  The output row of length N is the next layer's K.
+struct QuantNext {
+    const float* fisher;                 // [N] per-channel sensitivity of the next layer's input
+    float s4, k6, s8, inv8, tau;
+    int mode, ratio;
+    uint8_t* codes4; uint8_t* sf; uint32_t* mask; uint8_t* codes8;
+    fgmp_packed_header* header;
+    int64_t MW;                          // mask words per output row
+};
+
 struct GemmParams {
     void* Y; int64_t ldy; int y_is_bf16;
     int64_t M, N, K;
     const fgmp_packed_header* ha; const fgmp_packed_header* hw;
     int* status;
+    QuantNext q;
 };
+
+// One row of 32 accumulator columns = two blocks of the next layer's activations: round to bf16 (what an
+// unfused fgmp_linear would have stored), then the quantizer's steps in its order.  Returns the two mask bits.
+__device__ __forceinline__ uint32_t quantize_chunk32(const GemmParams& p, int64_t row, int64_t col0, const uint32_t (&r)[32], float alpha)
+{
+    const QuantNext& q = p.q;
+    uint32_t bits = 0;
+    if (row >= p.M) return 0u;
+#pragma unroll
+    for (int hb = 0; hb < 2; ++hb) {
+        const int64_t col = col0 + 16 * hb;
+        if (col + 16 > p.N) break;
+        const int64_t kb = col >> 4;
+        float v[16], f[16], dq4[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __bfloat162float(__float2bfloat16_rn(__uint_as_float(r[16 * hb + i]) * alpha));
+        const float4* fp = reinterpret_cast<const float4*>(q.fisher + col);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 t = __ldg(fp + i);
+            f[4 * i] = t.x; f[4 * i + 1] = t.y; f[4 * i + 2] = t.z; f[4 * i + 3] = t.w;
+        }
+        uint32_t sc = block_dynamic_scale(v, q.k6);
+        uint32_t c4[2], c8[4];
+        block_nvfp4(v, sc, q.s4, c4, dq4);
+        float score;
+        if (q.mode == 0) {
+            score = weighted_sq_sum(v, dq4, f);
+        } else {
+            float dq8[16];
+            block_fp8(v, q.inv8, q.s8, c8, dq8);
+            score = weighted_sq_sum(dq4, dq8, f);
+        }
+        if (score > q.tau) {
+            if (q.mode == 0) {
+                float dq8[16];
+                block_fp8(v, q.inv8, q.s8, c8, dq8);
+            }
+            *reinterpret_cast<uint4*>(q.codes8 + row * p.N + kb * 16) = make_uint4(c8[0], c8[1], c8[2], c8[3]);
+            c4[0] = 0; c4[1] = 0; sc = 0;
+            bits |= 1u << hb;
+        }
+        *reinterpret_cast<uint2*>(q.codes4 + (row * p.N) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
+        q.sf[fgmp_sf_offset(row, kb, p.N)] = (uint8_t)sc;
+    }
+    return bits;
+}
 
 // one row of 32 accumulator columns -> Y (scaled by the product of the tensor scales)
 __device__ __forceinline__ void store_chunk32(const GemmParams& p, int64_t row, int64_t col0, const uint32_t (&r)[32], float alpha)
@@ -220,6 +280,12 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    if (p.q.codes4 && blockIdx.x == 0 && threadIdx.x == 0) {
+        fgmp_packed_header* h = p.q.header;
+        h->magic = FGMP_MAGIC; h->version = 3; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
+        h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+        h->error = 0;
+    }
     const int64_t tiles_m = (p.M + P_BM - 1) / P_BM, tiles_n = (p.N + P_BN - 1) / P_BN;
     const int64_t num_tiles = tiles_m * tiles_n;
     const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
@@ -281,11 +347,19 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (!(ok = mbar_wait(accf0 + 8 * acc, acc_phase, abort_flag, p.status, 4))) break;
             tc_fence_after();
             const int64_t row = m0 + q * 32 + lane;
+            uint32_t mbits = 0;                        // FP8 flags of this row's 16 output blocks in the tile
 #pragma unroll 1
             for (int c = 0; c < P_BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * P_BN + c * 32), r);
-                store_chunk32(p, row, n0 + c * 32, r, alpha);
+                if (p.q.codes4) mbits |= quantize_chunk32(p, row, n0 + c * 32, r, alpha) << (2 * c);
+                else store_chunk32(p, row, n0 + c * 32, r, alpha);
+            }
+            if (p.q.codes4 && row < p.M) {
+                // a 256-column tile is half a mask word of the row
+                uint16_t* mw = reinterpret_cast<uint16_t*>(p.q.mask + row * p.q.MW + (tn >> 1));
+                mw[tn & 1] = (uint16_t)mbits;
+                if ((tn & 1) == 0 && (tn + 1) * P_BN >= p.N) mw[1] = 0;      // no tile behind this one
             }
             tc_fence_before();
             __syncwarp();
@@ -346,20 +420,10 @@ size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K)
     return 1024 + fgmp_align1k((size_t)M * K * 2) + fgmp_align1k((size_t)N * K * 2);
 }
 
-extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
-                                   void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
-                                   void* workspace, size_t ws_bytes, void* cuda_stream)
+// expand both operands and run the pair GEMM (M > 16 or a shape the weight-streaming kernel does not take)
+static fgmp_status launch_prefill(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
+                                  int64_t M, int64_t N, int64_t K, void* workspace, const QuantNext& qn, cudaStream_t s)
 {
-    if (!packed_acts || !packed_weights || !Y || !workspace) return FGMP_ERR_INVALID_ARG;
-    if (M < 1 || N < 1 || K < 64 || (K % 64) != 0 || ldy < N) return FGMP_ERR_SHAPE;
-    if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
-        ((uintptr_t)Y & 15)) return FGMP_ERR_SHAPE;
-    if (ws_bytes < fgmp_ws_linear(M, N, K)) return FGMP_ERR_WORKSPACE;
-    fgmp_status st;
-    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
-    cudaStream_t s = (cudaStream_t)cuda_stream;
-    if (fgmp_decode_supported(M, N, K))
-        return fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, false, s);
     uint8_t* ws = (uint8_t*)workspace;
     int* status = reinterpret_cast<int*>(ws);
     uint8_t* planeA = ws + 1024;
@@ -396,10 +460,64 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     p.ha = reinterpret_cast<const fgmp_packed_header*>(packed_acts);
     p.hw = reinterpret_cast<const fgmp_packed_header*>(packed_weights);
     p.status = status;
+    p.q = qn;
     const int64_t tiles = ((M + P_BM - 1) / P_BM) * ((N + P_BN - 1) / P_BN);
     const int pairs = (int)(tiles < pairs_of_device[dev] ? tiles : pairs_of_device[dev]);
     FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_pair_kernel<<<2 * pairs, GEMM_THREADS, PAIR_SMEM, s>>>(tmA, tmB, p));
     return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
+                                   void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                   void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!packed_acts || !packed_weights || !Y || !workspace) return FGMP_ERR_INVALID_ARG;
+    if (M < 1 || N < 1 || K < 64 || (K % 64) != 0 || ldy < N) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
+        ((uintptr_t)Y & 15)) return FGMP_ERR_SHAPE;
+    if (ws_bytes < fgmp_ws_linear(M, N, K)) return FGMP_ERR_WORKSPACE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (fgmp_decode_supported(M, N, K))
+        return fgmp_linear_decode(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, false, s);
+    QuantNext off{};
+    return launch_prefill(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, off, s);
+}
+
+extern "C" fgmp_status fgmp_linear_quantize(const void* packed_acts, const void* packed_weights,
+                                            int64_t M, int64_t N, int64_t K,
+                                            const float* fisher_chan_next, fgmp_scales sc_next, fgmp_score_mode sm,
+                                            float tau_next, void* packed_out, size_t packed_bytes,
+                                            void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!packed_acts || !packed_weights || !fisher_chan_next || !packed_out || !workspace) return FGMP_ERR_INVALID_ARG;
+    if ((int)sm < 0 || (int)sm > 1 || tau_next != tau_next) return FGMP_ERR_INVALID_ARG;
+    if (!(sc_next.scale_fp4 > 0.f) || !isfinite(sc_next.scale_fp4)) return FGMP_ERR_INVALID_ARG;
+    if (sc_next.fp8_log2_ratio < -7 || sc_next.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    // the output is a packed activation tensor [M, N]: N is the next layer's K
+    if (M <= 16 || N < 64 || (N % 64) != 0 || K < 64 || (K % 64) != 0) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
+        ((uintptr_t)packed_out & 1023) || ((uintptr_t)fisher_chan_next & 15)) return FGMP_ERR_SHAPE;
+    if (ws_bytes < fgmp_ws_linear(M, N, K)) return FGMP_ERR_WORKSPACE;
+    const PackedLayout L = fgmp_layout(M, N, 0, 0);
+    if (packed_bytes < L.total) return FGMP_ERR_WORKSPACE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    uint8_t* blob = (uint8_t*)packed_out;
+    QuantNext q{};
+    q.fisher = fisher_chan_next;
+    // the same scalars, computed the same way, as fgmp_quantize_activations uses
+    q.s4 = sc_next.scale_fp4;
+    q.k6 = 1.0f / (6.0f * sc_next.scale_fp4);
+    q.s8 = ldexpf(sc_next.scale_fp4, sc_next.fp8_log2_ratio);
+    q.inv8 = 1.0f / q.s8;
+    q.tau = tau_next; q.mode = (int)sm; q.ratio = sc_next.fp8_log2_ratio;
+    q.codes4 = blob + L.off_codes4; q.sf = blob + L.off_sf;
+    q.mask = reinterpret_cast<uint32_t*>(blob + L.off_mask); q.codes8 = blob + L.off_codes8;
+    q.header = reinterpret_cast<fgmp_packed_header*>(blob);
+    q.MW = L.MW;
+    return launch_prefill(packed_acts, packed_weights, nullptr, 0, N, M, N, K, workspace, q, (cudaStream_t)cuda_stream);
 }
 
 extern "C" fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_stream)

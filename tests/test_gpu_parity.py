@@ -459,3 +459,36 @@ def test_baseline_policies_as_weight_substitutions(fg):
         pa = fg.quantize_activations(x.cuda(), fa.cuda(), scale_fp4=s4, score_mode=1, tau=tau)
         compare_packed(fg, pa, qa, tau=tau, what=name + " activations")
         assert qa.mask_bits().sum() == int(np.floor(0.1 * scores.size + 0.5))
+
+
+# ------------------------------------------------------------ quantizer in the GEMM's epilogue (Section 4.2)
+
+@pytest.mark.parametrize("M,N,K,mode", [(300, 1024, 512, 0), (4096, 4096, 1024, 0), (77, 320, 256, 1), (2048, 11008, 256, 0)])
+def test_linear_with_next_layer_quantizer_in_the_epilogue(fg, M, N, K, mode):
+    """fgmp_linear_quantize against the two calls it fuses (bit for bit) and against the oracle's quantizer
+    run on the same bf16 outputs; the bf16 outputs themselves against the oracle's GEMM."""
+    wl = gi.llama("fuse", M, N, K, seed=51)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    y16 = fg.linear(pa, pw, out_dtype=torch.bfloat16)
+    fg.check(fg.linear.last_workspace)
+    # next layer's calibrated constants: sensitivity per output channel, tensor scale, threshold for 10 % FP8
+    g = torch.Generator().manual_seed(7)
+    f_next = torch.exp(1.5 * torch.randn(N, generator=g)).float()
+    s4n = gi.tensor_scale(y16.float().cpu())
+    yb = gi.bf16_bits(y16.cpu())
+    scores = oracle.quantize_activations(yb, f_next.numpy(), s4n, tau=np.inf, mode=mode).scores
+    tau = tau_for_fraction(scores, 0.1)
+    q_ref = oracle.quantize_activations(yb, f_next.numpy(), s4n, tau=tau, mode=mode)
+    fused = fg.linear_quantize(pa, pw, f_next.cuda(), scale_fp4=s4n, score_mode=mode, tau=tau)
+    fg.check(fg.linear.last_workspace)
+    two_step = fg.quantize_activations(y16, f_next.cuda(), scale_fp4=s4n, score_mode=mode, tau=tau)
+    for a, b in zip(fg.unpack(fused), fg.unpack(two_step)):
+        assert torch.equal(a, b), "the fused epilogue and the two separate calls must agree bit for bit"
+    compare_packed(fg, fused, q_ref, tau=tau, what="epilogue quantizer")
+    assert int(q_ref.mask_bits().sum()) == int(np.floor(0.1 * scores.size + 0.5))
+    # and the GEMM outputs that were quantized are the oracle's, within the bar (bf16 output)
+    rng = np.random.default_rng(3)
+    ms, nn = rng.integers(0, M, 2000), rng.integers(0, N, 2000)
+    Y, S = oracle.linear_sampled(qa, qw, ms, nn)
+    got = y16.float().cpu().numpy().astype(np.float64)[ms, nn]
+    assert (np.abs(got - Y) <= GEMM_TOL * S + np.abs(Y) * 2.0 ** -8 + 1e-30).all()
