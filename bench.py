@@ -174,6 +174,12 @@ WORKLOADS = {
     "llama2-7b-qkvo-prefill": (4096, 4096, 4096, 0.10, "prefill"),
     "llama2-7b-fc1-prefill": (4096, 11008, 4096, 0.10, "prefill"),
     "llama2-7b-fc2-prefill": (4096, 4096, 11008, 0.10, "prefill"),
+    # Section 5.1's other model sizes: Llama-2-13B (config 4: M = 2048) and Llama-2-70B (config 5)
+    "llama2-13b-fc1-prefill": (2048, 13824, 5120, 0.10, "prefill"),
+    "llama2-13b-fc2-prefill": (2048, 5120, 13824, 0.10, "prefill"),
+    "llama2-70b-fc1-prefill": (8192, 28672, 8192, 0.10, "prefill"),
+    "llama2-70b-fc2-decode": (16, 8192, 28672, 0.10, "decode"),
+    "llama2-13b-fc1-decode": (16, 13824, 5120, 0.10, "decode"),
     "tiny": (64, 256, 256, 0.10, "decode"),
 }
 
