@@ -322,7 +322,11 @@ def run_ours(args, world, rank, local):
             roofline = {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": ach / peaks["hbm_gbs"], "traffic": load_traffic(name, args.workload),
                         "peak_source": peaks["source"], "avg_kernel_us": avg_s * 1e6,
-                        "algorithmic_bytes_per_launch": alg}
+                        "algorithmic_bytes_per_launch": alg,
+                        # the graph-timed step (quantizer + this kernel, overlapped where the launch allows)
+                        # is shorter than the event-timed launch alone: the same bytes over the whole step
+                        "step_us": ms / args.steps * 1e3,
+                        "frac_over_step_time": alg / (ms / args.steps / 1e3) / 1e9 / peaks["hbm_gbs"]}
         else:
             ach = flops / avg_s / 1e12
             pk = peaks["bf16_tflops_sustained"]
