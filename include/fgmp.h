@@ -200,8 +200,12 @@ fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_str
  * applied, accumulated in FP32.  Y is fp32 (y_is_bf16 = 0) or bf16 [M, ldy].  The workspace
  * must have been cleared once with fgmp_workspace_init.  For 1 <= M <= 16, K % 256 == 0 and
  * N <= 258048 the weight-streaming kernel runs, launched as a programmatic dependent of the kernel
- * before it in the stream (its set-up overlaps that kernel's end; it reads the packed activations
- * and the workspace only after that kernel has completed). */
+ * before it in the stream (its set-up and its first reads of packed_weights overlap that kernel's
+ * end; it reads the packed activations and the workspace only after that kernel has completed).  So
+ * packed_weights must be complete before the kernel that precedes this call in the stream starts --
+ * always true for weights packed by fgmp_quantize_weights, whose last kernel writes only header fields
+ * that are read late; a caller who fills or copies a weight blob with a kernel of their own must not
+ * make that kernel the immediate predecessor (any other operation in between is enough). */
 fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
                         void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                         void* workspace, size_t ws_bytes, void* cuda_stream);
