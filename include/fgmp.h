@@ -49,6 +49,7 @@
  *                   XOR-swizzled with r%8; zero for FP8 blocks and rows beyond N)
  *                   | 2048 B microscales (four 512-byte tiles as above)
  *                   | 16 B: number of FP8 blocks in each of the unit's 16 block columns
+ *                   | 48 B: uint16 x 17, FP8 blocks before block column j (entry 16 = all), padded
  *                   | row (inside the tile) of every FP8 block, padded to 16 bytes
  *                   | the FP8 blocks, 16 E4M3 codes each, ordered by (block column, row);
  *                   padded to 128 bytes
@@ -94,7 +95,7 @@ typedef struct {
 /* First 256 bytes of a packed blob (device memory). */
 typedef struct {
     uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
-    uint32_t version;        /* layout version, 3                                           */
+    uint32_t version;        /* layout version, 4                                           */
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;

@@ -20,6 +20,7 @@
 //   REC_SF     2048 B : E4M3 microscales, 4 tiles of 512 B (128 rows x 4 blocks each):
 //                       (j/4)*512 + (r%32)*16 + (r/32)*4 + j%4 for block column j of the chunk
 //   REC_KBCNT    16 B : FP8 blocks of the unit per block column
+//   REC_KBSTART  48 B : uint16 x 17 (padded): FP8 blocks of the unit before block column j; entry 16 = all
 //   REC_ROWID         : row of every FP8 block of the unit, padded to 16 bytes
 //   then              : the FP8 blocks, 16 E4M3 codes each, ordered by (block column, row) so that
 //                       blocks meeting the same 16 activation elements are neighbours
@@ -36,7 +37,7 @@
 //   AREC_TRUE  8192 B : fp16 value / tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact)
 //                       as four K-major tiles of 16 tokens x 64 elements, token m = 128 bytes,
 //                       16-byte pieces XOR-swizzled with (m & 7): a tcgen05 kind::f16 operand
-constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_ROWID = 18448;
+constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_KBSTART = 18448, REC_ROWID = 18496;
 constexpr uint32_t AREC_A4 = 0, AREC_SF = 2048, AREC_MASK = 4096, AREC_TRUE = 5120, AREC_BYTES = 13312;
 
 // byte offset, inside a 128-byte-swizzled K-major fp16 tile of 64 elements per row, of the first
@@ -78,8 +79,8 @@ __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int
         L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
         L.off_uptr = o;    o = fgmp_align1k(o + ((size_t)L.units + 1) * 4);
         L.off_rec = o;
-        // a record is at most 18448 + 15 + 127 bytes plus 17 per FP8 block
-        o = fgmp_align1k(o + (size_t)L.units * 18592 + (size_t)max_fp8 * 17);
+        // a record is at most REC_ROWID + 15 + 127 bytes plus 17 per FP8 block
+        o = fgmp_align1k(o + (size_t)L.units * (REC_ROWID + 144) + (size_t)max_fp8 * 17);
     }
     L.total = o;
     return L;

@@ -73,8 +73,6 @@ struct StageMeta { uint32_t step, staged; };     // record start (128-byte steps
 
 __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
 
-__device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return __dp4a(x, 0x01010101u, 0u); }
-
 // A correction tile holds [128 rows][16 tokens] fp32, a row = 64 bytes = four 16-byte pieces of
 // four tokens; piece index is XOR-ed with (row >> 1) & 3 so that 32 lanes reading one piece of 32
 // consecutive rows (the epilogue) do not collide on banks.  Float index of (row, token):
@@ -368,19 +366,10 @@ decode_kernel(DecParams p)
                 const uint8_t* sa = sb + STG_A;
                 const uint32_t staged = smeta[stage].staged;
                 const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
-                const uint4 kc = *reinterpret_cast<const uint4*>(sb + REC_KBCNT);
-                const uint32_t ks0 = byte_sum(kc.x), ks1 = byte_sum(kc.y), ks2 = byte_sum(kc.z);
-                const uint32_t ntot = ks0 + ks1 + ks2 + byte_sum(kc.w);
+                const uint16_t* kbs = reinterpret_cast<const uint16_t*>(sb + REC_KBSTART);
+                const uint32_t ntot = kbs[16];
                 const uint32_t off8 = fgmp_rec_fp8_offset(ntot);
-                uint32_t start[2], end[2];
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int kb = cw + 8 * hh, wi = kb >> 2, sh8 = (kb & 3) * 8;
-                    const uint32_t word = wi == 0 ? kc.x : (wi == 1 ? kc.y : (wi == 2 ? kc.z : kc.w));
-                    start[hh] = (wi > 0 ? ks0 : 0u) + (wi > 1 ? ks1 : 0u) + (wi > 2 ? ks2 : 0u)
-                              + byte_sum(word & ((1u << sh8) - 1u));
-                    end[hh] = start[hh] + ((word >> sh8) & 0xffu);
-                }
+                const uint32_t start[2] = {kbs[cw], kbs[cw + 8]}, end[2] = {kbs[cw + 1], kbs[cw + 9]};
                 // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of each column
                 const uint2 b00 = *reinterpret_cast<const uint2*>(sa + boff[0]), b01 = *reinterpret_cast<const uint2*>(sa + boff[0] + 1024);
                 const uint2 b10 = *reinterpret_cast<const uint2*>(sa + boff[1]), b11 = *reinterpret_cast<const uint2*>(sa + boff[1] + 1024);

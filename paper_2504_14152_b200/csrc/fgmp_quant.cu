@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     if (!SCORE_ONLY) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
-            h->magic = FGMP_MAGIC; h->version = 3; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->magic = FGMP_MAGIC; h->version = 4; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }

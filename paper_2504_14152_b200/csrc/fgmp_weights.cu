@@ -313,6 +313,11 @@ __global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw
     uint8_t* rowid = rec + REC_ROWID;
     uint8_t* fp8 = rec + fgmp_rec_fp8_offset(cnt);
     if (threadIdx.x < 16) rec[REC_KBCNT + threadIdx.x] = (uint8_t)sc.cnt[threadIdx.x];
+    if (threadIdx.x < 24) {                                    // running sums of the counts, then padding
+        uint32_t before = 0;
+        for (int i = 0; i < 16 && i < (int)threadIdx.x; ++i) before += sc.cnt[i];
+        reinterpret_cast<uint16_t*>(rec + REC_KBSTART)[threadIdx.x] = threadIdx.x <= 16 ? (uint16_t)before : (uint16_t)0;
+    }
     // padding behind the row ids and behind the last FP8 block
     for (uint32_t i = cnt + threadIdx.x; i < ((cnt + 15u) & ~15u); i += 128) rowid[i] = 0;
     for (uint32_t i = fgmp_rec_fp8_offset(cnt) + cnt * 16 + threadIdx.x; i < fgmp_rec_bytes(cnt); i += 128) rec[i] = 0;
@@ -349,7 +354,7 @@ __global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, co
                                 float* tau_eff_out)
 {
     if (threadIdx.x == 0) {
-        h->magic = FGMP_MAGIC; h->version = 3; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
+        h->magic = FGMP_MAGIC; h->version = 4; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
         h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = room_steps;
         float teff = fraction_mode ? st->tau : tau_given;
         h->tau_eff = teff;
