@@ -109,7 +109,8 @@ typedef struct {
 
 enum { FGMP_OP_QUANTIZE_WEIGHTS = 0, FGMP_OP_QUANTIZE_ACTIVATIONS = 1, FGMP_OP_LINEAR = 2,
        FGMP_OP_CALIBRATE_TAU = 3,
-       FGMP_OP_GLOBAL_TAU = 4       /* M = total number of scores; N, K ignored */ };
+       FGMP_OP_GLOBAL_TAU = 4,      /* M = total number of scores; N, K ignored */
+       FGMP_OP_LINEAR_QUANTIZE = 5 };
 
 /* ---- sizes (pure host functions; return 0 for invalid shapes) ---- */
 size_t fgmp_weights_bytes(int64_t N, int64_t K, int64_t max_fp8_blocks);
@@ -219,8 +220,10 @@ fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
  * accumulator is scaled, rounded to bf16 and quantized in registers by the GEMM's epilogue.
  * packed_out is a packed activation tensor of M rows and N columns (N is the next layer's K; size from
  * fgmp_acts_bytes(M, N)); fisher_chan_next [N], sc_next, sm and tau_next are the arguments
- * fgmp_quantize_activations would get.  Needs M > 16 and N % 64 == 0 (decode-sized batches: call the
- * two functions one after the other); workspace as for fgmp_linear. */
+ * fgmp_quantize_activations would get.  N % 64 == 0.  Decode-sized batches (the shapes that take the
+ * weight-streaming kernel, whose threads hold output rows rather than token rows) run as the two
+ * launches, with the bf16 outputs (at most 16 x N) passing through the workspace.
+ * workspace: fgmp_workspace_bytes(FGMP_OP_LINEAR_QUANTIZE, M, N, K), cleared once like fgmp_linear's. */
 fgmp_status fgmp_linear_quantize(const void* packed_acts, const void* packed_weights,
                                  int64_t M, int64_t N, int64_t K,
                                  const float* fisher_chan_next, fgmp_scales sc_next, fgmp_score_mode sm,

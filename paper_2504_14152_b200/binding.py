@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libfgmp.so")
 
 SCORE_LP_ERROR, SCORE_HP_TO_LP = 0, 1
 CLIP_NONE, CLIP_SW_BRUTE = 0, 1
-OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU = 0, 1, 2, 3, 4
+OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU, OP_LINEAR_QUANTIZE = 0, 1, 2, 3, 4, 5
 
 
 class FgmpError(RuntimeError):
@@ -295,7 +295,7 @@ def linear_quantize(acts: PackedTensor, weights: PackedTensor, fisher_next: torc
     dev = acts.blob.device
     out = _alloc_aligned(L.fgmp_acts_bytes(M, N), dev)
     if workspace is None:
-        workspace = alloc_workspace(OP_LINEAR, M, N, K, dev)
+        workspace = alloc_workspace(OP_LINEAR_QUANTIZE, M, N, K, dev)
     _ok(L.fgmp_linear_quantize(acts.blob.data_ptr(), weights.blob.data_ptr(), M, N, K, fisher_next.data_ptr(),
                                _Scales(scale_fp4, ratio), score_mode, tau, out.data_ptr(), out.numel(),
                                workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear_quantize")

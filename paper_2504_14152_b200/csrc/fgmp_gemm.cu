@@ -414,6 +414,11 @@ bool make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t K,
 
 }  // namespace
 
+size_t fgmp_ws_linear_quantize(int64_t M, int64_t N, int64_t K)
+{
+    return fgmp_ws_linear(M, N, K) + (fgmp_decode_supported(M, N, K) ? fgmp_align1k((size_t)M * N * 2) : 0);
+}
+
 size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K)
 {
     if (fgmp_decode_supported(M, N, K)) return fgmp_ws_decode(M, N, K);
@@ -496,10 +501,19 @@ extern "C" fgmp_status fgmp_linear_quantize(const void* packed_acts, const void*
     if (!(sc_next.scale_fp4 > 0.f) || !isfinite(sc_next.scale_fp4)) return FGMP_ERR_INVALID_ARG;
     if (sc_next.fp8_log2_ratio < -7 || sc_next.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
     // the output is a packed activation tensor [M, N]: N is the next layer's K
-    if (M <= 16 || N < 64 || (N % 64) != 0 || K < 64 || (K % 64) != 0) return FGMP_ERR_SHAPE;
+    if (M < 1 || N < 64 || (N % 64) != 0 || K < 64 || (K % 64) != 0) return FGMP_ERR_SHAPE;
     if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
         ((uintptr_t)packed_out & 1023) || ((uintptr_t)fisher_chan_next & 15)) return FGMP_ERR_SHAPE;
-    if (ws_bytes < fgmp_ws_linear(M, N, K)) return FGMP_ERR_WORKSPACE;
+    if (ws_bytes < fgmp_ws_linear_quantize(M, N, K)) return FGMP_ERR_WORKSPACE;
+    if (fgmp_decode_supported(M, N, K)) {
+        // decode-sized batch: the weight-streaming kernel holds an output row per thread, not a token row, so the
+        // two steps stay two launches; the bf16 outputs (at most 16 x N) pass through the end of the workspace
+        uint8_t* ybf = (uint8_t*)workspace + fgmp_ws_linear(M, N, K);
+        fgmp_status st2 = fgmp_linear(packed_acts, packed_weights, ybf, 1, N, M, N, K, workspace, fgmp_ws_linear(M, N, K), cuda_stream);
+        if (st2 != FGMP_OK) return st2;
+        return fgmp_quantize_activations(ybf, N, fisher_chan_next, M, N, sc_next, sm, tau_next, packed_out, packed_bytes,
+                                         nullptr, 0, cuda_stream);
+    }
     const PackedLayout L = fgmp_layout(M, N, 0, 0);
     if (packed_bytes < L.total) return FGMP_ERR_WORKSPACE;
     fgmp_status st;
@@ -547,6 +561,7 @@ extern "C" size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K)
         case FGMP_OP_QUANTIZE_ACTIVATIONS: return 0;
         case FGMP_OP_LINEAR: return (M >= 1 && N >= 1) ? fgmp_ws_linear(M, N, K) : 0;
         case FGMP_OP_CALIBRATE_TAU: return M >= 1 ? fgmp_ws_calibrate(M, K) : 0;
+        case FGMP_OP_LINEAR_QUANTIZE: return (M >= 1 && N >= 1) ? fgmp_ws_linear_quantize(M, N, K) : 0;
     }
     return 0;
 }

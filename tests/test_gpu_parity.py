@@ -463,7 +463,8 @@ def test_baseline_policies_as_weight_substitutions(fg):
 
 # ------------------------------------------------------------ quantizer in the GEMM's epilogue (Section 4.2)
 
-@pytest.mark.parametrize("M,N,K,mode", [(300, 1024, 512, 0), (4096, 4096, 1024, 0), (77, 320, 256, 1), (2048, 11008, 256, 0)])
+@pytest.mark.parametrize("M,N,K,mode", [(300, 1024, 512, 0), (4096, 4096, 1024, 0), (77, 320, 256, 1), (2048, 11008, 256, 0),
+                                         (16, 1024, 512, 0), (5, 320, 256, 1), (8, 192, 320, 0)])
 def test_linear_with_next_layer_quantizer_in_the_epilogue(fg, M, N, K, mode):
     """fgmp_linear_quantize against the two calls it fuses (bit for bit) and against the oracle's quantizer
     run on the same bf16 outputs; the bf16 outputs themselves against the oracle's GEMM."""
