@@ -230,7 +230,7 @@ def run_ours(args, world, rank, local):
     fg.check(ws)
 
     # ---- the timed region: K steps, replayed from one CUDA graph when capture works (the step is
-    # launch-bound at decode sizes: two short kernels and a memset), else launched eagerly
+    # launch-bound at decode sizes: two short kernels), else launched eagerly
     graph, graph_note = None, "eager launches"
     if not args.no_graph:
         try:
