@@ -34,12 +34,12 @@
  *                   0x00 for FP8 blocks
  *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
  *                   1 = FP8
- *   arec          : (rows <= 16 only) C records of 13312 bytes, one per chunk, holding what the
- *                   decode-sized GEMM streams: the chunk's codes as a 16-token x 128-byte tile
- *                   (16-byte pieces of token m XOR-swizzled with m%8), its microscales (four
- *                   512-byte tiles), an fp16 copy [16 blocks][16 tokens][16] of the quantized
- *                   values divided by the tensor scale, and 16 uint16 mask words; token rows
- *                   >= rows are zero
+ *   arec          : (rows <= 16 only) C records of 8192 bytes, one per chunk, holding what the
+ *                   decode-sized GEMM streams: the quantized values of 16 token rows divided by
+ *                   the tensor scale, in fp16 (exact), in the order that kernel's mma.sync
+ *                   fragments take them: 16 pieces of 512 bytes, piece 2*sp + o holding, for
+ *                   lane 4g + t, elements 64t + 8sp .. 64t + 8sp + 7 of token 8o + g; token
+ *                   rows >= rows are zero
  *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written
  *
  * Weights: header | mask | uptr | records
@@ -95,7 +95,7 @@ typedef struct {
 /* First 256 bytes of a packed blob (device memory). */
 typedef struct {
     uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
-    uint32_t version;        /* layout version, 4                                           */
+    uint32_t version;        /* layout version, 5                                           */
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;

@@ -29,22 +29,19 @@
 //
 // Activations (kind 0): header | codes4 | sf | mask | arec | codes8.  codes4 is row-major, sf
 // uses the same 512-byte tiles over all rows, codes8 is a dense plane of which only FP8 blocks are
-// written.  arec exists when rows <= 16: one record per chunk holding what the decode GEMM
-// needs of 16 token rows (rows >= M are zero):
-//   AREC_A4    2048 B : codes, token m = 128 bytes, swizzled like REC_W4
-//   AREC_SF    2048 B : microscales, 4 tiles of 512 B
-//   AREC_MASK    32 B : uint16 per token, bit j = block column j of the chunk is FP8
-//   AREC_TRUE  8192 B : fp16 value / tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact)
-//                       as four K-major tiles of 16 tokens x 64 elements, token m = 128 bytes,
-//                       16-byte pieces XOR-swizzled with (m & 7): a tcgen05 kind::f16 operand
+// written.  arec exists when rows <= 16: one record of AREC_BYTES per chunk holding the fp16 value
+// over the tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact) of 16 token rows (rows >= M
+// are zero), in the order the decode GEMM's mma.sync fragments take them: 16 pieces of 512 bytes,
+// piece 2*sp + nh = MMA steps 2sp, 2sp+1 of token octet nh; in a piece lane (g, t) has 16 bytes =
+// elements 64t + 8sp .. 64t + 8sp + 7 of token 8nh + g.
 constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_KBSTART = 18448, REC_ROWID = 18496;
-constexpr uint32_t AREC_A4 = 0, AREC_SF = 2048, AREC_MASK = 4096, AREC_TRUE = 5120, AREC_BYTES = 13312;
+constexpr uint32_t AREC_BYTES = 8192;
 
-// byte offset, inside a 128-byte-swizzled K-major fp16 tile of 64 elements per row, of the first
-// (half = 0) or second (half = 1) 8 elements of block column jq (0..3) of row r
-__host__ __device__ inline uint32_t fgmp_h16_tile_offset(uint32_t r, uint32_t jq, uint32_t half)
+// byte offset, inside an activation record, of the first (half = 0) or second (half = 1) 8 elements
+// of block column j (0..15) of token row m
+__host__ __device__ inline uint32_t fgmp_arec_offset(uint32_t m, uint32_t j, uint32_t half)
 {
-    return r * 128u + ((((jq << 1) | half) ^ (r & 7u)) << 4);
+    return ((((((j & 3u) << 1) | half) << 1) | (m >> 3)) << 9) + ((((m & 7u) << 2) | (j >> 2)) << 4);
 }
 
 struct PackedLayout {

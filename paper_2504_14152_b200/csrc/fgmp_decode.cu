@@ -2,28 +2,32 @@
 // reads the packed weights exactly once (Section 4.1 of the paper: the four block-pair
 // products, FP32 accumulation).
 //
-// Decomposition (exact).  With A4z / W4z the NVFP4 planes (zero in FP8 blocks), W8 the FP8
-// blocks of the weights and At the true activation values (fp16 copy, either format):
-//     Y = A4z.W4z^T            (1) tcgen05.mma kind::mxf4nvf4, UE4M3 block scales in TMEM,
-//                                  weights are the 128-row MMA operand, the 16 tokens are N
-//       + At.W8^T              (2) the FP8 weight blocks, which a record keeps grouped by block
-//                                  column: sixteen blocks that meet the same 16 activation
-//                                  elements form the M side of mma.sync m16n8k16; results are
-//                                  added to their rows in a tile private to the warp
-//       + At[FP8 blocks].W4z^T (3) only block columns in which some token is FP8: the NVFP4
-//                                  weights of the stage are dequantized for mma.sync
-// A tcgen05.mma of this shape costs about 50 ns whatever its size, so the tensor-core path is kept
-// to the four instructions per unit that (1) needs; the microscales reach TMEM by tcgen05.st from
-// otherwise idle warps instead of tcgen05.cp, and (2), (3) run beside it on warps of their own.
+// At this size the layer is bound by the weight stream, not by arithmetic, and every block pair
+// has an exact fp16 form: an E2M1 code times its E4M3 microscale has 6 significant bits, an E4M3
+// code times the power of two between the tensor scales has 4.  So both operands go through
+// mma.sync m16n8k16 (fp16 in, fp32 accumulation) as their true values over the tensor scales, and
+// the mixing of formats costs nothing extra per pair:
+//   (1) NVFP4 weight blocks: 16 weight rows are the M side, the tokens the N side.  Lane (g, t)
+//       owns, of rows g and g + 8, the 64 elements 64t .. 64t+63 of the unit; MMA step s takes
+//       elements 64t + 4s .. 64t + 4s + 3 of every lane (the order of the contraction index is
+//       free as long as both operands agree), so a lane's codes are two 16-byte loads per row and
+//       all four codes of a step share one microscale.  Codes become fp16 with
+//       cvt.rn.f16x2.e2m1x2, times the microscale (exact).  FP8 blocks are zero in this plane.
+//   (2) FP8 weight blocks, which a record keeps grouped by block column: sixteen blocks that meet
+//       the same 16 activation elements form the M side; the sums are added to their rows in a
+//       [row][token] fp32 tile private to the warp.
+// The activation quantizer leaves the fp16 values of each 256-element chunk in the order (1)
+// reads them, 16 bytes per lane.
 //
 // Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all SMs
 // stream the same number of bytes; a unit is two bulk copies (its weight record, the activation
 // record of its chunk).  Tiles shared by several CTAs are reduced in a fixed order by the CTA
 // that arrives last.  Every sum is taken in a fixed order: results are reproducible bit for bit.
 //
-// Warp roles (704 threads): warp 0 = producer, warp 1 = MMA issuer and TMEM owner, warps 2-5 =
-// epilogue (one TMEM lane quadrant each), warps 6-13 = (2), two block columns each, warps 14-21 =
-// (3), 16 rows each; the first four of them also load the microscales.
+// Warp roles (672 threads): warp 0 = producer, warps 1-4 = epilogue (32 rows each), warps 5-12 =
+// (1): warp (jr, h) does rows 32jr .. 32jr+31, MMA steps 8h .. 8h+7, warps 13-20 = (2), two block
+// columns each.  Either kind alone keeps up with the weight stream; on warps of their own they run
+// beside each other.
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
@@ -32,32 +36,18 @@
 
 namespace {
 
-constexpr int DEC_THREADS = 704;
-constexpr int CORR_WARPS = 16;                  // warps 6..21
-constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
+constexpr int MAIN_WARPS = 8, FP8_WARPS = 8, MATH_WARPS = MAIN_WARPS + FP8_WARPS;
+constexpr int DEC_THREADS = 32 * (1 + 4 + MATH_WARPS);
+constexpr int TOK = 16;                         // token rows of a tile (zero padded)
 constexpr uint32_t FP8_CAP_BLOCKS = 320;        // FP8 blocks of a unit that fit a stage; more are read from global
 constexpr uint32_t WREC_CAP = (REC_ROWID + FP8_CAP_BLOCKS + FP8_CAP_BLOCKS * 16 + 127) & ~127u;   // 23936
 constexpr uint32_t STG_A = (WREC_CAP + 1023) & ~1023u;                                           // 24576
-constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 37888
+constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 32768
 constexpr int DEC_STAGES = 4;
-constexpr int NTILES = 9;                       // [row][token] fp32 tiles: one per (2) warp, one shared by the (3) warps
+constexpr int NTILES = FP8_WARPS + 2;           // [row][token] fp32 tiles: one per (2) warp, one per half of the MMA steps of (1)
 constexpr uint32_t TILE_FLOATS = 128 * TOK;
-constexpr uint32_t SF_COL0 = 32;                // TMEM: 2 x 16 accumulator columns, then 32 scale columns per stage
-constexpr uint32_t DEC_TMEM_COLS = 256;
 constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + NTILES * TILE_FLOATS * 4 + 1024 /*alignment*/ + 512 /*barriers*/;
-static_assert(DEC_STAGE_BYTES % 1024 == 0, "swizzled tiles need 1 KiB alignment");
-
-// kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
-constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
-
-// shared-memory matrix descriptors as (low word | start address >> 4, constant high word)
-constexpr uint32_t SW128_LO = 1u << 16, SW128_HI = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128B swizzle, 8-row groups 1 KiB apart
-__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi)
-{
-    uint64_t d;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
-    return d;
-}
+static_assert(DEC_SMEM <= 232448, "shared memory of one CTA");
 
 struct DecParams {
     const uint8_t* wblob; const uint8_t* ablob;
@@ -73,30 +63,41 @@ struct StageMeta { uint32_t step, staged; };     // record start (128-byte steps
 
 __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
 
-// A correction tile holds [128 rows][16 tokens] fp32, a row = 64 bytes = four 16-byte pieces of
-// four tokens; piece index is XOR-ed with (row >> 1) & 3 so that 32 lanes reading one piece of 32
-// consecutive rows (the epilogue) do not collide on banks.  Float index of (row, token):
-__device__ __forceinline__ uint32_t tile_idx(uint32_t row, uint32_t token)
+// A tile holds [128 rows][16 tokens] fp32, a row = 64 bytes = four 16-byte pieces of four tokens;
+// piece index is XOR-ed with (row >> 1) & 3 so that 32 lanes reading one piece of 32 consecutive
+// rows (the epilogue) do not collide on banks.
+
+// eight E2M1 codes (one word) times a microscale (both halves of sc2) -> four fp16 pairs, exact
+__device__ __forceinline__ void dq8(uint32_t c32, uint32_t sc2, uint32_t (&x)[4])
 {
-    return row * 16u + ((((token >> 2) ^ (row >> 1)) & 3u) << 2) + (token & 3u);
+    uint32_t q0, q1, q2, q3;
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\tmov.b32 {b0, b1, b2, b3}, %4;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %0, b0;\n\tcvt.rn.f16x2.e2m1x2 %1, b1;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %2, b2;\n\tcvt.rn.f16x2.e2m1x2 %3, b3;\n\t}"
+        : "=r"(q0), "=r"(q1), "=r"(q2), "=r"(q3) : "r"(c32));
+    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[0]) : "r"(q0), "r"(sc2));
+    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[1]) : "r"(q1), "r"(sc2));
+    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[2]) : "r"(q2), "r"(sc2));
+    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[3]) : "r"(q3), "r"(sc2));
 }
 
+// NH = token octets in use: 1 for M <= 8, else 2
+template <int NH>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_kernel(DecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // 1 KiB aligned; an offset from the array keeps the pointer known to be shared memory (plain ld.shared / st.shared)
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     float* tiles = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NTILES * TILE_FLOATS);
-    // bars (S = stages): [0,S) full, [S,2S) empty, [2S,3S) scales in TMEM, then acc_full[2], acc_empty[2],
-    // corrections of a segment done [2], tiles free [1]
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * DEC_STAGES + 8);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + DEC_STAGES);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // bars (S = stages): [0,S) full, [S,2S) empty, then sums of a segment in the tiles [2], tiles free [1]
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smeta + DEC_STAGES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES, sfr0 = empty0 + 8 * DEC_STAGES;
-    const uint32_t accf0 = sfr0 + 8 * DEC_STAGES, acce0 = accf0 + 16, cdone0 = acce0 + 16, tfree = cdone0 + 16;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES;
+    const uint32_t cdone0 = empty0 + 8 * DEC_STAGES, tfree = cdone0 + 16;
 
     // this CTA's span of (tile, chunk) units
     const int64_t G = gridDim.x, C = p.chunks;
@@ -110,20 +111,15 @@ decode_kernel(DecParams p)
     if (warp == 0 && pf_base + lane <= p.total) pf = __ldg(uptr + pf_base + lane);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < DEC_STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + CORR_WARPS); mbar_init(sfr0 + 8 * s, 4);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); mbar_init(cdone0 + 8 * b, CORR_WARPS);
-        }
+        for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, MATH_WARPS); }
+        for (int b = 0; b < 2; ++b) mbar_init(cdone0 + 8 * b, MATH_WARPS);
         mbar_init(tfree, 4);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
-    if (warp >= 6) {                                   // the tiles start at zero
+    if (warp >= 5) {                                   // the tiles of (2) start at zero
         float4* z = reinterpret_cast<float4*>(tiles);
-        for (int i = (warp - 6) * 32 + lane; i < (int)(NTILES * TILE_FLOATS / 4); i += CORR_WARPS * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = (warp - 5) * 32 + lane; i < (int)(FP8_WARPS * TILE_FLOATS / 4); i += MATH_WARPS * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     // One unit's two copies into a stage (lane 0 of the producer warp): the weight record, then the
     // activation record of the unit's chunk
@@ -150,10 +146,7 @@ decode_kernel(DecParams p)
             if (lane == 0) issue_w(s, step0, step1);
         }
     }
-    tc_fence_before();
     __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
     // Launched as a programmatic dependent of the preceding kernel in the stream (normally the
     // activation quantizer), this kernel may have started before that one finished: everything above
     // touches neither its output nor the workspace.  From here on both are read.
@@ -179,51 +172,12 @@ decode_kernel(DecParams p)
             if (!__shfl_sync(0xffffffffu, ok, 0)) break;
             if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        // The whole warp walks the loop; lane 0 alone issues the tcgen05 instructions, so that every
-        // commit tracks every MMA before it.
-        const uint32_t smem0 = smem_u32(smem);
-        int stage = 0; uint32_t phase = 0; bool ok = true;
-        int seg = 0;
-        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
-            const int64_t tile = u / C;
-            const int64_t seg_end = min(u_end, (tile + 1) * C);
-            const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
-            if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
-            uint32_t accum = 0;
-            for (; u < seg_end && ok; ++u) {
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
-                if (!(ok = mbar_wait(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;   // microscales are in TMEM
-                tc_fence_after();
-                const uint32_t sb = smem0 + (uint32_t)stage * DEC_STAGE_BYTES;
-                const uint32_t sf_t = tmem_base + SF_COL0 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
-                const uint32_t w4_lo = ((sb + REC_W4) >> 4) | SW128_LO, a4_lo = ((sb + STG_A + AREC_A4) >> 4) | SW128_LO;
-                if (lane == 0) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        umma_nvf4(d_tmem, desc64(w4_lo + 2 * j, SW128_HI), desc64(a4_lo + 2 * j, SW128_HI), IDESC_NVF4,
-                                  sf_t + 4 * j, sf_t + 16 + 4 * j, accum);
-                        accum = 1;
-                    }
-                    umma_commit(empty0 + 8 * stage);
-                }
-                accum = 1;
-                __syncwarp();
-                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
-            }
-            if (ok && lane == 0) umma_commit(accf0 + 8 * acc);
-            __syncwarp();
-        }
-    } else if (warp < 6) {
-        // ------------------------------------------------------------ epilogue: TMEM lane quadrant warp % 4
-        const int q = warp & 3;
+    } else if (warp < 5) {
+        // ------------------------------------------------------------ epilogue: rows 32q .. 32q + 31 of the tile
+        const int q = warp - 1;
         const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
-        const float r8 = __int_as_float((127 + hw->fp8_log2_ratio) << 23);     // FP8 tensor scale / NVFP4 tensor scale of the weights
         const int row = 32 * q + lane;
         bool ok = true;
         int seg = 0;
@@ -232,8 +186,6 @@ decode_kernel(DecParams p)
             const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
             u = seg_end;
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
-            if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 4))) break;
-            tc_fence_after();
             // a tile shared with other CTAs: how many of them have handed in their sums already (the answer is
             // needed only after this CTA's own sums are complete, so the load costs nothing)
             const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
@@ -246,34 +198,24 @@ decode_kernel(DecParams p)
                 slot = (int)(blockIdx.x - c_first);
                 if (lane == 0) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile * 8 + q) : "memory");
             }
-            uint32_t rr[16];
-            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
-            tc_fence_before();
-            mbar_arrive(acce0 + 8 * accb);
+            // the segment's sums: this row of every tile, in tile order; the rows of (2) are cleared for the
+            // next segment on the way
+            if (!(ok = mbar_wait(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 6))) break;
             float v[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
-            // corrections (2) and (3) of the segment: this row of every tile, in tile order; the row is
-            // cleared for the next segment on the way
-            if (!(ok = mbar_wait(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 6))) break;
-            float c2[16];                              // (2): sums of the FP8 weight codes, still without 2^ratio
-#pragma unroll
-            for (int j = 0; j < 16; ++j) c2[j] = 0.f;
+            for (int j = 0; j < 16; ++j) v[j] = 0.f;
 #pragma unroll
             for (int w = 0; w < NTILES; ++w) {
                 float4* src = reinterpret_cast<float4*>(tiles + w * TILE_FLOATS + row * TOK);
-                float4 x[4];
+                float4 x[2 * NH];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) x[j] = src[(j ^ (row >> 1)) & 3];       // tokens 4j .. 4j+3
+                for (int j = 0; j < 2 * NH; ++j) x[j] = src[(j ^ (row >> 1)) & 3];  // tokens 4j .. 4j+3
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (w < 8) { c2[4 * j] += x[j].x; c2[4 * j + 1] += x[j].y; c2[4 * j + 2] += x[j].z; c2[4 * j + 3] += x[j].w; }
-                    else       { v[4 * j] += x[j].x; v[4 * j + 1] += x[j].y; v[4 * j + 2] += x[j].z; v[4 * j + 3] += x[j].w; }
-                    src[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int j = 0; j < 2 * NH; ++j) {
+                    v[4 * j] += x[j].x; v[4 * j + 1] += x[j].y; v[4 * j + 2] += x[j].z; v[4 * j + 3] += x[j].w;
+                    if (w < FP8_WARPS) src[(j ^ (row >> 1)) & 3] = make_float4(0.f, 0.f, 0.f, 0.f);   // the tiles of (1) are overwritten
                 }
             }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] += c2[j] * r8;
             __syncwarp();
             if (lane == 0) mbar_arrive(tfree);
 
@@ -284,7 +226,7 @@ decode_kernel(DecParams p)
                 // others were seen to have arrived, this warp is the last without asking and skips the counter.
                 float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + row) * 16;
 #pragma unroll
-                for (int j = 0; j < 16; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+                for (int j = 0; j < 8 * NH; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
                 // The counter wraps to zero with the last arrival (or is put back by the warp that skipped
                 // it), so the workspace is ready for the next call without being cleared.
                 uint32_t old = __shfl_sync(0xffffffffu, seen, 0);
@@ -299,12 +241,12 @@ decode_kernel(DecParams p)
                 if (old == (uint32_t)(nseg - 1)) {
                     __threadfence();
                     // all partials first (independent loads), then one sum in slot order
-                    float4 x[4][4];
+                    float4 x[4][2 * NH];
 #pragma unroll
                     for (int sgi = 0; sgi < 4; ++sgi) {
                         const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16;
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)
+                        for (int j = 0; j < 2 * NH; ++j)
                             x[sgi][j] = sgi < nseg ? __ldcg(reinterpret_cast<const float4*>(src) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
 #pragma unroll
@@ -312,14 +254,14 @@ decode_kernel(DecParams p)
 #pragma unroll
                     for (int sgi = 0; sgi < 4; ++sgi) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
+                        for (int j = 0; j < 2 * NH; ++j) {
                             v[4 * j] += x[sgi][j].x; v[4 * j + 1] += x[sgi][j].y; v[4 * j + 2] += x[sgi][j].z; v[4 * j + 3] += x[sgi][j].w;
                         }
                     }
                     for (int sgi = 4; sgi < nseg; ++sgi) {       // more than four contributors: rare, serial
                         const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16;
 #pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
+                        for (int j = 0; j < 8 * NH; j += 4) {
                             const float4 y4 = __ldcg(reinterpret_cast<const float4*>(src + j));
                             v[j] += y4.x; v[j + 1] += y4.y; v[j + 2] += y4.z; v[j + 3] += y4.w;
                         }
@@ -329,7 +271,7 @@ decode_kernel(DecParams p)
             }
             if (write_out && n < p.N) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
+                for (int j = 0; j < 8 * NH; ++j) {
                     if (j < p.M) {
                         if (p.y_is_bf16) reinterpret_cast<__nv_bfloat16*>(p.Ybf)[(int64_t)j * p.ldy + n] = __float2bfloat16_rn(v[j] * alpha);
                         else p.Y[(int64_t)j * p.ldy + n] = v[j] * alpha;
@@ -337,19 +279,109 @@ decode_kernel(DecParams p)
                 }
             }
         }
-    } else if (warp < 14) {
+    } else if (warp < 5 + MAIN_WARPS) {
+        // ------------------------------------------------------------ (1): NVFP4 weight blocks
+        const int w = warp - 5;
+        const int jr = w & 3, h = w >> 2;
+        const uint32_t g = lane >> 2, t = lane & 3;
+        float* htile = tiles + (FP8_WARPS + h) * TILE_FLOATS;          // sums of a segment: rows 32jr .. 32jr+31 of the tile of this h
+        // this lane's codes and microscales of rows 32jr + 16mt + 8rh + g
+        uint32_t w4_off[2][2], sf_off[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const uint32_t r = (uint32_t)(32 * jr + 16 * mt + 8 * rh) + g;
+                w4_off[mt][rh] = REC_W4 + r * 128 + (((2 * t + (uint32_t)h) ^ g) << 4);
+                sf_off[mt][rh] = REC_SF + t * 512 + (r & 31u) * 16 + (r >> 5) * 4 + 2 * (uint32_t)h;
+            }
+        const uint32_t a_off = STG_A + (uint32_t)(8 * h) * 512 + (uint32_t)lane * 16;
+        const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
+
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
+            float acc[2][NH][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh) acc[mt][nh][0] = acc[mt][nh][1] = acc[mt][nh][2] = acc[mt][nh][3] = 0.f;
+            for (; u < seg_end; ++u) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+                uint4 cw[2][2];
+                uint32_t sc2[2][2][2];
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                    for (int rh = 0; rh < 2; ++rh) {
+                        cw[mt][rh] = *reinterpret_cast<const uint4*>(sb + w4_off[mt][rh]);
+                        const uint32_t s16 = *reinterpret_cast<const uint16_t*>(sb + sf_off[mt][rh]);
+                        const uint32_t s0 = __byte_perm(s16, 0u, 0x4400), s1 = __byte_perm(s16, 0u, 0x4411);
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2[mt][rh][0]) : "h"((uint16_t)s0));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2[mt][rh][1]) : "h"((uint16_t)s1));
+                    }
+#pragma unroll
+                for (int sp = 0; sp < 4; ++sp) {
+                    const uint4 alo = *reinterpret_cast<const uint4*>(sb + a_off + (uint32_t)sp * 1024);
+                    uint4 ahi = make_uint4(0, 0, 0, 0);
+                    if (NH == 2) ahi = *reinterpret_cast<const uint4*>(sb + a_off + (uint32_t)sp * 1024 + 512);
+                    uint32_t xg[2][4], xg8[2][4];       // rows g / g + 8 of both M tiles: steps 2sp (0, 1) and 2sp + 1 (2, 3)
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        const uint32_t wg = sp == 0 ? cw[mt][0].x : sp == 1 ? cw[mt][0].y : sp == 2 ? cw[mt][0].z : cw[mt][0].w;
+                        const uint32_t wg8 = sp == 0 ? cw[mt][1].x : sp == 1 ? cw[mt][1].y : sp == 2 ? cw[mt][1].z : cw[mt][1].w;
+                        dq8(wg, sc2[mt][0][sp >> 1], xg[mt]);
+                        dq8(wg8, sc2[mt][1][sp >> 1], xg8[mt]);
+                    }
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                        for (int mt = 0; mt < 2; ++mt) {
+                            mma_f16_16816(acc[mt][0], xg[mt][2 * half], xg8[mt][2 * half], xg[mt][2 * half + 1], xg8[mt][2 * half + 1],
+                                          half ? alo.z : alo.x, half ? alo.w : alo.y);
+                            if (NH == 2)
+                                mma_f16_16816(acc[mt][NH - 1], xg[mt][2 * half], xg8[mt][2 * half], xg[mt][2 * half + 1], xg8[mt][2 * half + 1],
+                                              half ? ahi.z : ahi.x, half ? ahi.w : ahi.y);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) break;
+            // the epilogue has taken the previous segment's sums; now this segment's go in:
+            // acc[mt][nh] = rows 32jr + 16mt + {g, g + 8} x tokens 8nh + {2t, 2t+1}
+            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int rh = 0; rh < 2; ++rh) {
+                    const uint32_t r = (uint32_t)(32 * jr + 16 * mt + 8 * rh) + g;
+                    float2* pt = reinterpret_cast<float2*>(htile + r * 16u + (((tpiece ^ (r >> 1)) & 3u) << 2) + tcol);
+                    pt[0] = make_float2(acc[mt][0][2 * rh], acc[mt][0][2 * rh + 1]);
+                    if (NH == 2)
+                        *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pt) ^ 32) = make_float2(acc[mt][NH - 1][2 * rh], acc[mt][NH - 1][2 * rh + 1]);
+                }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
+        }
+    } else {
         // ------------------------------------------------------------ (2): FP8 weight blocks of block columns cw, cw + 8
-        // The E4M3 codes go into the MMA as they are; the factor 2^ratio between the FP8 and NVFP4
-        // tensor scales is applied once to the tile sums in the epilogue.
-        const int cw = warp - 6;
+        const int cw = warp - 5 - MAIN_WARPS;
         const uint32_t g = lane >> 2, t = lane & 3;
         float* mytile = tiles + cw * TILE_FLOATS;
-        // where this lane's activation fragments of the two columns sit in an activation record
+        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+        const float r8 = __int_as_float((127 + hw->fp8_log2_ratio) << 23);     // FP8 tensor scale / NVFP4 tensor scale of the weights
+        // where this lane's activation fragments of the two columns sit (token g; token g + 8 is 512 bytes on)
         uint32_t boff[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             const uint32_t j = (uint32_t)cw + 8u * hh;
-            boff[hh] = AREC_TRUE + (j >> 2) * 2048 + fgmp_h16_tile_offset(g, j & 3u, t >> 1) + (t & 1u) * 8;   // token g; token g + 8 is 1 KiB on
+            boff[hh] = STG_A + fgmp_arec_offset(g, j, t >> 1) + (t & 1u) * 8;
         }
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
 
@@ -363,23 +395,23 @@ decode_kernel(DecParams p)
             for (; u < seg_end; ++u) {
                 if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-                const uint8_t* sa = sb + STG_A;
                 const uint32_t staged = smeta[stage].staged;
                 const uint8_t* rec_g = recs + (size_t)smeta[stage].step * 128;
                 const uint16_t* kbs = reinterpret_cast<const uint16_t*>(sb + REC_KBSTART);
                 const uint32_t ntot = kbs[16];
                 const uint32_t off8 = fgmp_rec_fp8_offset(ntot);
                 const uint32_t start[2] = {kbs[cw], kbs[cw + 8]}, end[2] = {kbs[cw + 1], kbs[cw + 9]};
-                // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of each column
-                const uint2 b00 = *reinterpret_cast<const uint2*>(sa + boff[0]), b01 = *reinterpret_cast<const uint2*>(sa + boff[0] + 1024);
-                const uint2 b10 = *reinterpret_cast<const uint2*>(sa + boff[1]), b11 = *reinterpret_cast<const uint2*>(sa + boff[1] + 1024);
+                // B fragments: activation values of tokens g and g + 8, elements 4t..4t+3 of each column
+                const uint2 b00 = *reinterpret_cast<const uint2*>(sb + boff[0]), b10 = *reinterpret_cast<const uint2*>(sb + boff[1]);
+                uint2 b01 = make_uint2(0, 0), b11 = b01;
+                if (NH == 2) { b01 = *reinterpret_cast<const uint2*>(sb + boff[0] + 512); b11 = *reinterpret_cast<const uint2*>(sb + boff[1] + 512); }
 
                 // ALL = every FP8 block of the unit is in the stage (the usual case); otherwise the tail of the
                 // list is read from global memory
                 auto body = [&](auto all_c) {
                     constexpr bool ALL = decltype(all_c)::value;
-                    // One group of up to 16 blocks of one column: blocks e + g and e + g + 8 are the M side of two
-                    // mma.sync (tokens 0-7 and 8-15 as N).  c/d[0..1]: block iA, tokens 2t, 2t+1 / 8+2t, 9+2t; [2..3]: block iB.
+                    // One group of up to 16 blocks of one column: blocks e + g and e + g + 8 are the M side.
+                    // c/d[0..1]: block iA, tokens 2t, 2t+1 / 8+2t, 9+2t; [2..3]: block iB.
                     auto group_mma = [&](uint32_t e, uint32_t end_, const uint2& bt0, const uint2& bt1, float (&c)[4], float (&d)[4],
                                          uint32_t& rowA, uint32_t& rowB) {
                         const uint32_t iA = e + g, iB = iA + 8;
@@ -402,28 +434,30 @@ decode_kernel(DecParams p)
                         asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a3) : "h"((uint16_t)(rawB >> 16)));
                         c[0] = c[1] = c[2] = c[3] = 0.f; d[0] = d[1] = d[2] = d[3] = 0.f;
                         mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);
-                        mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);
+                        if (NH == 2) mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);
                     };
-                    // Within one column every block has its own row, so the four read-modify-writes of a group touch
-                    // distinct addresses in every lane and across lanes: all loads first, then all stores.
+                    // tile[row][tokens] += 2^ratio x sums.  Within one column every block has its own row, so the
+                    // read-modify-writes of a group touch distinct addresses: all loads first, then all stores.
                     auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t rowA, uint32_t rowB) {
                         float2 *pA = nullptr, *pB = nullptr;    // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on (piece ^ 2)
                         float2 vA0 = make_float2(0.f, 0.f), vA1 = vA0, vB0 = vA0, vB1 = vA0;
                         if (rowA != 0xffffffffu) {
                             pA = reinterpret_cast<float2*>(mytile + rowA * 16u + (((tpiece ^ (rowA >> 1)) & 3u) << 2) + tcol);
-                            vA0 = pA[0]; vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
+                            vA0 = pA[0];
+                            if (NH == 2) vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
                         }
                         if (rowB != 0xffffffffu) {
                             pB = reinterpret_cast<float2*>(mytile + rowB * 16u + (((tpiece ^ (rowB >> 1)) & 3u) << 2) + tcol);
-                            vB0 = pB[0]; vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
+                            vB0 = pB[0];
+                            if (NH == 2) vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
                         }
                         if (rowA != 0xffffffffu) {
-                            pA[0] = make_float2(vA0.x + c[0], vA0.y + c[1]);
-                            *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(vA1.x + d[0], vA1.y + d[1]);
+                            pA[0] = make_float2(fmaf(c[0], r8, vA0.x), fmaf(c[1], r8, vA0.y));
+                            if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(fmaf(d[0], r8, vA1.x), fmaf(d[1], r8, vA1.y));
                         }
                         if (rowB != 0xffffffffu) {
-                            pB[0] = make_float2(vB0.x + c[2], vB0.y + c[3]);
-                            *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(vB1.x + d[2], vB1.y + d[3]);
+                            pB[0] = make_float2(fmaf(c[2], r8, vB0.x), fmaf(c[3], r8, vB0.y));
+                            if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(fmaf(d[2], r8, vB1.x), fmaf(d[3], r8, vB1.y));
                         }
                         __syncwarp();                  // a later group may add to the same rows
                     };
@@ -456,103 +490,6 @@ decode_kernel(DecParams p)
             __syncwarp();
             if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
         }
-    } else {
-        // ------------------------------------------------------------ (3): FP8 activation blocks x NVFP4 weights, 16 rows per warp
-        const int tw = warp - 14;
-        const int rowbase = 16 * tw;
-        const uint32_t g = lane >> 2, t = lane & 3;
-        float* tile3 = tiles + 8 * TILE_FLOATS;
-        // per-lane constants of the record addressing: rows rowbase + g and rowbase + 8 + g (the same r & 7 = g)
-        uint32_t w4_base[2], sf_base[2];
-#pragma unroll
-        for (int rg = 0; rg < 2; ++rg) {
-            const uint32_t r = (uint32_t)rowbase + 8u * rg + g;
-            w4_base[rg] = REC_W4 + r * 128 + t * 2;
-            sf_base[rg] = REC_SF + (r & 31u) * 16 + (r >> 5) * 4;
-        }
-        const uint32_t at_base = AREC_TRUE + g * 128 + (t & 1u) * 8;
-
-        int stage = 0; uint32_t phase = 0; bool ok = true;
-        int seg = 0;
-        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
-            const int64_t tile = u / C;
-            const int64_t seg_end = min(u_end, (tile + 1) * C);
-            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            for (; u < seg_end; ++u) {
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
-                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-                const uint8_t* sa = sb + STG_A;
-                if (tw < 4) {
-                    // Microscales of the stage into TMEM, one warp per lane quadrant (warp % 4): lane i holds,
-                    // for MMA step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3,
-                    // which is 16 bytes of scale tile j; the token scales follow in columns 16..31.
-                    uint32_t r[16];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
-                        r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
-                    }
-                    const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
-                    tmem_st16(sf_t, r);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint4 x = *reinterpret_cast<const uint4*>(sa + AREC_SF + 512 * j + lane * 16);
-                        r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
-                    }
-                    tmem_st16(sf_t + 16, r);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
-                }
-                const uint32_t am0 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + g * 2);
-                const uint32_t am1 = *reinterpret_cast<const uint16_t*>(sa + AREC_MASK + (g + 8) * 2);
-                uint32_t todo = am0 | am1;             // block columns in which any token is FP8
-#pragma unroll
-                for (int o = 4; o < 32; o <<= 1) todo |= __shfl_xor_sync(0xffffffffu, todo, o);
-                while (todo) {
-                    const uint32_t kb = (uint32_t)__ffs(todo) - 1u;
-                    todo &= todo - 1;
-                    const uint32_t bit = 1u << kb;
-                    // true activation values of tokens g and g + 8 (1 KiB apart), elements 4t..4t+3 of column kb
-                    const uint8_t* ap = sa + at_base + (kb >> 2) * 2048 + (((((kb & 3u) << 1) | (t >> 1)) ^ g) << 4);
-                    const uint2 at0 = *reinterpret_cast<const uint2*>(ap), at1 = *reinterpret_cast<const uint2*>(ap + 1024);
-                    const uint32_t a0 = (am0 & bit) ? at0.x : 0u, a2 = (am0 & bit) ? at0.y : 0u;
-                    const uint32_t a1 = (am1 & bit) ? at1.x : 0u, a3 = (am1 & bit) ? at1.y : 0u;
-                    const uint32_t wcol = ((((kb >> 1) ^ g) & 7u) << 4) + (kb & 1u) * 8, scol = (kb >> 2) * 512 + (kb & 3u);
-#pragma unroll
-                    for (int rg = 0; rg < 2; ++rg) {
-                        const uint32_t codes = *reinterpret_cast<const uint16_t*>(sb + w4_base[rg] + wcol);
-                        const uint32_t sfb = sb[sf_base[rg] + scol];
-                        uint32_t q0, q1, sc2;
-                        asm("{\n\t.reg .b8 lo, hi;\n\tmov.b16 {lo, hi}, %2;\n\tcvt.rn.f16x2.e2m1x2 %0, lo;\n\tcvt.rn.f16x2.e2m1x2 %1, hi;\n\t}"
-                            : "=r"(q0), "=r"(q1) : "h"((uint16_t)codes));
-                        const uint16_t s16 = (uint16_t)(sfb | (sfb << 8));
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"(s16));
-                        const __half2 x0 = __hmul2(*reinterpret_cast<__half2*>(&q0), *reinterpret_cast<__half2*>(&sc2));
-                        const __half2 x1 = __hmul2(*reinterpret_cast<__half2*>(&q1), *reinterpret_cast<__half2*>(&sc2));
-                        mma_f16_16816(acc[rg], a0, a1, a2, a3, *reinterpret_cast<const uint32_t*>(&x0), *reinterpret_cast<const uint32_t*>(&x1));
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
-            }
-            if (!ok) break;
-            // the epilogue has taken (and cleared) the previous segment's sums; now this segment's go in:
-            // acc[rg] = (token g | g+8) x (row 2t | 2t+1) of the warp's row group rg
-            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
-#pragma unroll
-            for (int rg = 0; rg < 2; ++rg) {
-                const uint32_t r = (uint32_t)(rowbase + 8 * rg + 2 * t);
-                tile3[tile_idx(r, g)] = acc[rg][0];
-                tile3[tile_idx(r + 1, g)] = acc[rg][1];
-                tile3[tile_idx(r, g + 8)] = acc[rg][2];
-                tile3[tile_idx(r + 1, g + 8)] = acc[rg][3];
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
-        }
     }
 
     __syncthreads();
@@ -560,10 +497,6 @@ decode_kernel(DecParams p)
         const unsigned long long t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
         __syncthreads();
-    }
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, DEC_TMEM_COLS);
     }
 }
 
@@ -620,7 +553,8 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess)
             return FGMP_ERR_CUDA;
         attr_set[dev] = true;
     }
@@ -631,7 +565,8 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = clear_first ? 0 : 1;
-    FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel, p));
+    if (M <= 8) { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<1>, p)); }
+    else        { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<2>, p)); }
     return fgmp_launch_status();
 }
 

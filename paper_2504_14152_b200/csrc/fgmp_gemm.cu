@@ -282,7 +282,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
     if (p.q.codes4 && blockIdx.x == 0 && threadIdx.x == 0) {
         fgmp_packed_header* h = p.q.header;
-        h->magic = FGMP_MAGIC; h->version = 4; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
+        h->magic = FGMP_MAGIC; h->version = 5; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
         h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
         h->error = 0;
     }

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     if (!SCORE_ONLY) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
-            h->magic = FGMP_MAGIC; h->version = 4; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->magic = FGMP_MAGIC; h->version = 5; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }
@@ -48,12 +48,8 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
             if (active) {
                 uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
                 const uint32_t j = (uint32_t)kb & 15u, m = (uint32_t)m0;
-                *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset(m, j)) = make_uint2(0, 0);
-                rec[AREC_SF + fgmp_rec_sf_offset(m, j)] = 0;
-                uint8_t* tile = rec + AREC_TRUE + (j >> 2) * 2048;
-                *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset(m, j & 3, 0)) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset(m, j & 3, 1)) = make_uint4(0, 0, 0, 0);
-                if (j == 0) *reinterpret_cast<uint16_t*>(rec + AREC_MASK + m * 2) = 0;
+                *reinterpret_cast<uint4*>(rec + fgmp_arec_offset(m, j, 0)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(rec + fgmp_arec_offset(m, j, 1)) = make_uint4(0, 0, 0, 0);
             }
             return;
         }
@@ -124,11 +120,8 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                     }
                     uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
                     const uint32_t j = (uint32_t)kb & 15u;
-                    uint8_t* tile = rec + AREC_TRUE + (j >> 2) * 2048;
-                    *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset((uint32_t)m, j & 3, 0)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    *reinterpret_cast<uint4*>(tile + fgmp_h16_tile_offset((uint32_t)m, j & 3, 1)) = make_uint4(o[4], o[5], o[6], o[7]);
-                    *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset((uint32_t)m, j)) = make_uint2(c4[0], c4[1]);
-                    rec[AREC_SF + fgmp_rec_sf_offset((uint32_t)m, j)] = (uint8_t)sc;
+                    *reinterpret_cast<uint4*>(rec + fgmp_arec_offset((uint32_t)m, j, 0)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(rec + fgmp_arec_offset((uint32_t)m, j, 1)) = make_uint4(o[4], o[5], o[6], o[7]);
                 }
                 *reinterpret_cast<uint2*>(p.codes4 + (m * p.K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
                 p.sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)sc;
@@ -139,11 +132,6 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
             int64_t w = kb >> 5;
             if ((threadIdx.x & 31) == 0 && w < p.MW) {
                 p.mask[m * p.MW + w] = word;
-                if (p.arec) {                          // the same bits per chunk: two chunks per word
-                    *reinterpret_cast<uint16_t*>(p.arec + (size_t)(2 * w) * AREC_BYTES + AREC_MASK + m * 2) = (uint16_t)word;
-                    if (2 * w + 1 < (p.KB + 15) / 16)
-                        *reinterpret_cast<uint16_t*>(p.arec + (size_t)(2 * w + 1) * AREC_BYTES + AREC_MASK + m * 2) = (uint16_t)(word >> 16);
-                }
             }
         }
     }

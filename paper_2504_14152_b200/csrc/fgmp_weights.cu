@@ -354,7 +354,7 @@ __global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, co
                                 float* tau_eff_out)
 {
     if (threadIdx.x == 0) {
-        h->magic = FGMP_MAGIC; h->version = 4; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
+        h->magic = FGMP_MAGIC; h->version = 5; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
         h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = room_steps;
         float teff = fraction_mode ? st->tau : tau_given;
         h->tau_eff = teff;
