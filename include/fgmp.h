@@ -38,8 +38,8 @@
  *                   decode-sized GEMM streams: the quantized values of 16 token rows divided by
  *                   the tensor scale, in fp16 (exact), in the order that kernel's mma.sync
  *                   fragments take them: 16 pieces of 512 bytes, piece 2*sp + o holding, for
- *                   lane 4g + t, elements 64t + 8sp .. 64t + 8sp + 7 of token 8o + g; token
- *                   rows >= rows are zero
+ *                   lane (g, t), elements 64t + 8sp .. 64t + 8sp + 7 of token 8o + g in the
+ *                   16-byte slot 4g + (t ^ (g & 3)); token rows >= rows are zero
  *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written
  *
  * Weights: header | mask | uptr | records

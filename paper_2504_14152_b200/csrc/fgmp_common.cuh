@@ -33,7 +33,8 @@
 // over the tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact) of 16 token rows (rows >= M
 // are zero), in the order the decode GEMM's mma.sync fragments take them: 16 pieces of 512 bytes,
 // piece 2*sp + nh = MMA steps 2sp, 2sp+1 of token octet nh; in a piece lane (g, t) has 16 bytes =
-// elements 64t + 8sp .. 64t + 8sp + 7 of token 8nh + g.
+// elements 64t + 8sp .. 64t + 8sp + 7 of token 8nh + g, at 16-byte slot 4g + (t ^ (g & 3)) (the
+// XOR spreads the eight tokens of one block column over more banks).
 constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_KBSTART = 18448, REC_ROWID = 18496;
 constexpr uint32_t AREC_BYTES = 8192;
 
@@ -41,7 +42,7 @@ constexpr uint32_t AREC_BYTES = 8192;
 // of block column j (0..15) of token row m
 __host__ __device__ inline uint32_t fgmp_arec_offset(uint32_t m, uint32_t j, uint32_t half)
 {
-    return ((((((j & 3u) << 1) | half) << 1) | (m >> 3)) << 9) + ((((m & 7u) << 2) | (j >> 2)) << 4);
+    return ((((((j & 3u) << 1) | half) << 1) | (m >> 3)) << 9) + ((((m & 7u) << 2) | ((j >> 2) ^ (m & 3u))) << 4);
 }
 
 struct PackedLayout {

@@ -295,7 +295,7 @@ decode_kernel(DecParams p)
                 w4_off[mt][rh] = REC_W4 + r * 128 + (((2 * t + (uint32_t)h) ^ g) << 4);
                 sf_off[mt][rh] = REC_SF + t * 512 + (r & 31u) * 16 + (r >> 5) * 4 + 2 * (uint32_t)h;
             }
-        const uint32_t a_off = STG_A + (uint32_t)(8 * h) * 512 + (uint32_t)lane * 16;
+        const uint32_t a_off = STG_A + (uint32_t)(8 * h) * 512 + ((g << 2) | (t ^ (g & 3u))) * 16;
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
 
         int stage = 0; uint32_t phase = 0; bool ok = true;
