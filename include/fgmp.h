@@ -47,7 +47,7 @@
  *                   128-byte steps from the first record
  *   record        : 16384 B E2M1 codes as a 128-row x 128-byte tile (16-byte pieces of row r
  *                   XOR-swizzled with r%8; zero for FP8 blocks and rows beyond N)
- *                   | 2048 B microscales (four 512-byte tiles as above)
+ *                   | 2048 B microscales, [128 rows][16 block columns]
  *                   | 16 B: number of FP8 blocks in each of the unit's 16 block columns
  *                   | 48 B: uint16 x 17, FP8 blocks before block column j (entry 16 = all), padded
  *                   | row (inside the tile) of every FP8 block, padded to 16 bytes

@@ -17,8 +17,8 @@
 //   REC_W4    16384 B : E2M1 codes, row r of the tile = 128 bytes whose 16-byte pieces are
 //                       XOR-swizzled with (r & 7) -- the 128B-swizzled K-major tile tcgen05 reads;
 //                       zero in FP8 blocks and in rows beyond the tensor
-//   REC_SF     2048 B : E4M3 microscales, 4 tiles of 512 B (128 rows x 4 blocks each):
-//                       (j/4)*512 + (r%32)*16 + (r/32)*4 + j%4 for block column j of the chunk
+//   REC_SF     2048 B : E4M3 microscales, [128 rows][16 block columns] (the decode GEMM reads two
+//                       neighbouring bytes per lane, rows 16 bytes apart: no bank conflicts)
 //   REC_KBCNT    16 B : FP8 blocks of the unit per block column
 //   REC_KBSTART  48 B : uint16 x 17 (padded): FP8 blocks of the unit before block column j; entry 16 = all
 //   REC_ROWID         : row of every FP8 block of the unit, padded to 16 bytes
@@ -99,7 +99,7 @@ __host__ __device__ inline uint32_t fgmp_rec_w4_offset(uint32_t r, uint32_t j)
 }
 __host__ __device__ inline uint32_t fgmp_rec_sf_offset(uint32_t r, uint32_t j)
 {
-    return (j >> 2) * 512u + (r & 31u) * 16u + (r >> 5) * 4u + (j & 3u);
+    return r * 16u + j;
 }
 
 #ifdef __CUDACC__

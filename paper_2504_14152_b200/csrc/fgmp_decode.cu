@@ -293,7 +293,7 @@ decode_kernel(DecParams p)
             for (int rh = 0; rh < 2; ++rh) {
                 const uint32_t r = (uint32_t)(32 * jr + 16 * mt + 8 * rh) + g;
                 w4_off[mt][rh] = REC_W4 + r * 128 + (((2 * t + (uint32_t)h) ^ g) << 4);
-                sf_off[mt][rh] = REC_SF + t * 512 + (r & 31u) * 16 + (r >> 5) * 4 + 2 * (uint32_t)h;
+                sf_off[mt][rh] = REC_SF + r * 16 + 4 * t + 2 * (uint32_t)h;
             }
         const uint32_t a_off = STG_A + (uint32_t)(8 * h) * 512 + ((g << 2) | (t ^ (g & 3u))) * 16;
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
