@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1)
 tensor_peak_kernel(int kind, int64_t n_mma, int* status)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // offset from the array: stays known as shared memory
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + PK_A_BYTES + PK_B_BYTES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
