@@ -43,10 +43,11 @@ constexpr uint32_t FP8_CAP_BLOCKS = 320;        // FP8 blocks of a unit that fit
 constexpr uint32_t WREC_CAP = (REC_ROWID + FP8_CAP_BLOCKS + FP8_CAP_BLOCKS * 16 + 127) & ~127u;   // 23936
 constexpr uint32_t STG_A = (WREC_CAP + 1023) & ~1023u;                                           // 24576
 constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 32768
-constexpr int DEC_STAGES = 4;
+constexpr int DEC_STAGES = 4;                   // at most; a launch uses DecParams::stages of them
 constexpr int NTILES = FP8_WARPS + 2;           // [row][token] fp32 tiles: one per (2) warp, one per half of the MMA steps of (1)
 constexpr uint32_t TILE_FLOATS = 128 * TOK;
-constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + NTILES * TILE_FLOATS * 4 + 1024 /*alignment*/ + 512 /*barriers*/;
+constexpr size_t dec_smem(int stages) { return (size_t)stages * DEC_STAGE_BYTES + NTILES * TILE_FLOATS * 4 + 1024 /*alignment*/ + 512 /*barriers*/; }
+constexpr size_t DEC_SMEM = dec_smem(DEC_STAGES);
 static_assert(DEC_SMEM <= 232448, "shared memory of one CTA");
 
 struct DecParams {
@@ -57,6 +58,7 @@ struct DecParams {
     int64_t total;            // tiles * chunks
     int64_t chunks;
     int* status; uint32_t* counters; float* partials; int maxseg;
+    int stages;               // depth of the unit ring, 2 .. DEC_STAGES
 };
 
 struct StageMeta { uint32_t step, staged; };     // record start (128-byte steps), bytes of it in the stage
@@ -89,7 +91,8 @@ decode_kernel(DecParams p)
     extern __shared__ uint8_t smem_raw[];
     // 1 KiB aligned; an offset from the array keeps the pointer known to be shared memory (plain ld.shared / st.shared)
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    float* tiles = reinterpret_cast<float*>(smem + (size_t)DEC_STAGES * DEC_STAGE_BYTES);
+    const int S = p.stages;
+    float* tiles = reinterpret_cast<float*>(smem + (size_t)S * DEC_STAGE_BYTES);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NTILES * TILE_FLOATS);
     // bars (S = stages): [0,S) full, [S,2S) empty, then sums of a segment in the tiles [2], tiles free [1]
     StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES + 4);
@@ -111,7 +114,7 @@ decode_kernel(DecParams p)
     if (warp == 0 && pf_base + lane <= p.total) pf = __ldg(uptr + pf_base + lane);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, MATH_WARPS); }
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, MATH_WARPS); }
         for (int b = 0; b < 2; ++b) mbar_init(cdone0 + 8 * b, MATH_WARPS);
         mbar_init(tfree, 4);
         *abort_flag = 0;
@@ -140,7 +143,7 @@ decode_kernel(DecParams p)
     // up (thread 0, which initialised the barriers, issues them) and before the wait below.
     int pre = 0;
     if (warp == 0) {
-        pre = (int)min((int64_t)DEC_STAGES, u_end - u_begin);
+        pre = (int)min((int64_t)S, u_end - u_begin);
         for (int s = 0; s < pre; ++s) {
             const uint32_t step0 = __shfl_sync(0xffffffffu, pf, s), step1 = __shfl_sync(0xffffffffu, pf, s + 1);
             if (lane == 0) issue_w(s, step0, step1);
@@ -156,7 +159,7 @@ decode_kernel(DecParams p)
         // ------------------------------------------------------------ producer (whole warp; lane 0 issues)
         if (lane == 0)
             for (int s = 0; s < pre; ++s) issue_a(u_begin + s, s);
-        int stage = pre % DEC_STAGES; uint32_t phase = (uint32_t)(pre / DEC_STAGES) & 1u;
+        int stage = pre % S; uint32_t phase = (uint32_t)(pre / S) & 1u;
         for (int64_t u = u_begin + pre; u < u_end; ++u) {
             if (u + 1 - pf_base > 31) {                // next 32 record offsets
                 pf_base = u;
@@ -170,7 +173,7 @@ decode_kernel(DecParams p)
                 if (ok) { issue_w(stage, step0, step1); issue_a(u, stage); }
             }
             if (!__shfl_sync(0xffffffffu, ok, 0)) break;
-            if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+            if (++stage == S) { stage = 0; phase ^= 1; }
         }
     } else if (warp < 5) {
         // ------------------------------------------------------------ epilogue: rows 32q .. 32q + 31 of the tile
@@ -350,7 +353,7 @@ decode_kernel(DecParams p)
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+                if (++stage == S) { stage = 0; phase ^= 1; }
             }
             if (!ok) break;
             // the epilogue has taken the previous segment's sums; now this segment's go in:
@@ -484,7 +487,7 @@ decode_kernel(DecParams p)
                 if (off8 + ntot * 16 <= staged) body(std::true_type{}); else body(std::false_type{});
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-                if (++stage == DEC_STAGES) { stage = 0; phase ^= 1; }
+                if (++stage == S) { stage = 0; phase ^= 1; }
             }
             if (!ok) break;
             __syncwarp();
@@ -548,6 +551,10 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     p.counters = reinterpret_cast<uint32_t*>(ws + 1024);
     p.partials = reinterpret_cast<float*>(ws + FGMP_WS_CONTROL_BYTES);
     p.maxseg = d.maxseg;
+    // Ring depth: long spans of few tokens are bound by the weight stream and want every stage; the others
+    // are bound by arithmetic or by set-up and run as fast or faster with a smaller footprint (measured on
+    // Llama-2 shapes).
+    p.stages = (d.total / d.grid >= 24 && M <= 8) ? DEC_STAGES : DEC_STAGES - 1;
 
     static bool attr_set[64] = {};
     int dev = 0;
@@ -560,7 +567,7 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     }
     if (clear_first && cudaMemsetAsync(ws, 0, 1024 + (size_t)d.tiles * 32, s) != cudaSuccess) return FGMP_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = DEC_SMEM; cfg.stream = s;
+    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = dec_smem(p.stages); cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
