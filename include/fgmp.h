@@ -37,22 +37,25 @@
  *   arec          : (rows <= 16 only) C records of 8192 bytes, one per chunk, holding what the
  *                   decode-sized GEMM streams: the quantized values of 16 token rows divided by
  *                   the tensor scale, in fp16 (exact), in the order that kernel's mma.sync
- *                   fragments take them: 16 pieces of 512 bytes, piece 2*sp + o holding, for
- *                   lane (g, t), elements 64t + 8sp .. 64t + 8sp + 7 of token 8o + g in the
- *                   16-byte slot 4g + (t ^ (g & 3)); token rows >= rows are zero
- *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written
+ *                   fragments take them: token octet m/8 in its own 4096 bytes; there piece
+ *                   2*(j%4) + h of 512 bytes holds elements 8h .. 8h+7 of block column j of the
+ *                   chunk for token m, 16 bytes at lane position 4*(m%8) + j/4; token rows >=
+ *                   rows are zero
+ *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written (the
+ *                   blob is sized for the worst case of every block being FP8)
  *
- * Weights: header | mask | uptr | records
- *   uptr          : uint32 [units + 1]: start of unit (t, c)'s record, index t*C + c, in
- *                   128-byte steps from the first record
- *   record        : 16384 B E2M1 codes as a 128-row x 128-byte tile (16-byte pieces of row r
- *                   XOR-swizzled with r%8; zero for FP8 blocks and rows beyond N)
- *                   | 2048 B microscales, [128 rows][16 block columns]
- *                   | 16 B: number of FP8 blocks in each of the unit's 16 block columns
- *                   | 48 B: uint16 x 17, FP8 blocks before block column j (entry 16 = all), padded
- *                   | row (inside the tile) of every FP8 block, padded to 16 bytes
- *                   | the FP8 blocks, 16 E4M3 codes each, ordered by (block column, row);
- *                   padded to 128 bytes
+ * Weights: header | mask | uptr | records | overflow
+ *   record        : 18560 bytes per unit, unit (t, c) at index t*C + c, in the order in which the
+ *                   decode-sized GEMM's 16 warps read it: warp w = 4*(r/32) + j%4, lane 4*(r%8) + j/4
+ *                   and slot k = (r/8)%4 hold block (row r of the tile, block column j of the chunk).
+ *                   16384 B of 8-byte slots at w*1024 + (k/2)*512 + lane*16 + (k%2)*8: the 16 E2M1
+ *                   codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block (zero beyond N)
+ *                   | 2048 B of scale bytes at w*128 + lane*4 + k: the E4M3 microscale of an NVFP4
+ *                   block (bit 7 clear), or 0x80 | E4M3(2^fp8_log2_ratio) for an FP8 block
+ *                   | 128 B: uint16 x 17, FP8 blocks of the unit before warp w's; entry 16 = all
+ *   overflow      : E4M3 codes 8..15 of the FP8 blocks, 8 bytes each, unit by unit, inside a unit in
+ *                   (w, lane, k) order, each unit padded to 16 bytes
+ *   uptr          : uint32 [units + 1]: start of a unit's overflow entries in 16-byte steps
  *                   fgmp_weights_bytes(N, K, max_fp8_blocks) leaves room for that many FP8 blocks.
  */
 #ifndef FGMP_H
@@ -95,14 +98,14 @@ typedef struct {
 /* First 256 bytes of a packed blob (device memory). */
 typedef struct {
     uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
-    uint32_t version;        /* layout version, 5                                           */
+    uint32_t version;        /* layout version, 6                                           */
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;
     int64_t n_fp8;           /* number of FP8 blocks                                        */
     float tau_eff;           /* weights, fraction mode: smallest selected score             */
     uint32_t kind;           /* 0 = activations, 1 = weights                                */
-    int64_t capacity;        /* weights: room for records, in 128-byte steps                */
+    int64_t capacity;        /* weights: room for overflow entries, in 16-byte steps        */
     int32_t error;           /* 0, or FGMP_ERR_CAPACITY                                     */
     int32_t reserved[49];
 } fgmp_packed_header;
@@ -110,7 +113,7 @@ typedef struct {
 enum { FGMP_OP_QUANTIZE_WEIGHTS = 0, FGMP_OP_QUANTIZE_ACTIVATIONS = 1, FGMP_OP_LINEAR = 2,
        FGMP_OP_CALIBRATE_TAU = 3,
        FGMP_OP_GLOBAL_TAU = 4,      /* M = total number of scores; N, K ignored */
-       FGMP_OP_LINEAR_QUANTIZE = 5 };
+       FGMP_OP_LINEAR_QUANTIZE = 5, FGMP_OP_LINEAR_FUSED = 6 };
 
 /* ---- sizes (pure host functions; return 0 for invalid shapes) ---- */
 size_t fgmp_weights_bytes(int64_t N, int64_t K, int64_t max_fp8_blocks);
@@ -127,7 +130,9 @@ size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K);
  * is FP8 iff score > tau.  The blob must have room for the result
  * (packed_bytes >= fgmp_weights_bytes(N, K, max_fp8_blocks)); if threshold mode finds
  * more FP8 blocks than the blob has room for, header.error = FGMP_ERR_CAPACITY and the blob
- * is invalid (fgmp_unpack refuses it).
+ * is invalid: fgmp_unpack refuses it, and fgmp_linear given such a blob (or one whose header
+ * does not carry the N and K of the call) reads none of it and records FGMP_ERR_INVALID_ARG in
+ * the workspace status (fgmp_check).
  * tau_eff_out (device float, may be NULL) receives the smallest selected score. */
 fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, const float* fisher_elem, int64_t ldf,
                                   int64_t N, int64_t K, fgmp_scales sc, fgmp_score_mode sm,
@@ -191,8 +196,9 @@ fgmp_status fgmp_channel_mean_sq(const void* X_bf16, int64_t ldx, int64_t rows, 
  * for decode-sized batches, the counters of tiles that several thread blocks share.  They must be
  * zero when fgmp_linear first uses the workspace: clear them once with this call (a memset on the
  * stream; workspace 1024-byte aligned).  Every fgmp_linear that ends without a device-side error
- * leaves them zero again, so that a decode step needs no clearing pass of its own; after an error
- * reported by fgmp_check, clear the workspace again before reusing it. */
+ * leaves them as the next call needs them, whatever the shapes of the two calls (prefill-sized
+ * calls keep their scratch behind the control area), so that a decode step needs no clearing pass
+ * of its own; after an error reported by fgmp_check, clear the workspace again before reusing it. */
 #define FGMP_WS_CONTROL_BYTES 65536
 fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_stream);
 
@@ -211,6 +217,31 @@ fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_str
 fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
                         void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                         void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- one decode step in one launch: activation quantizer + GEMM (Section 4.2 into Section 4.1) ----
+ * For decode-sized batches (the shapes of fgmp_linear's weight-streaming kernel: 1 <= M <= 16,
+ * K % 256 == 0) this is fgmp_quantize_activations(X, ...) followed by fgmp_linear, as one kernel: the
+ * thread blocks first share out the quantizer's work (256-element chunks of eight token rows; four lanes
+ * per block, the same single-precision steps in the same order, so codes, scales and masks are those of
+ * fgmp_quantize_activations bit for bit), while the first weight records are already on their way, and
+ * start multiplying once every chunk has been handed in.  Y is what fgmp_linear returns for those packed
+ * activations, bit for bit.
+ *   packed_acts_out (may be NULL): receives the packed activations (size fgmp_acts_bytes(M, K)) for a
+ *     caller that wants them (fgmp_unpack, or a later fgmp_linear with other weights); if NULL only the
+ *     fp16 records the GEMM streams are kept, in the workspace.
+ *   workspace: fgmp_workspace_bytes(FGMP_OP_LINEAR_FUSED, M, N, K), cleared once with
+ *     fgmp_workspace_init.  Beside fgmp_linear's words the control area holds a call number, which
+ *     tags what the blocks publish to each other, so nothing has to be cleared between calls; after an
+ *     error reported by fgmp_check clear the workspace again.  Calls that share a workspace must not
+ *     overlap on the GPU.
+ *   The kernel is launched as a programmatic dependent like fgmp_linear's (same condition on
+ *   packed_weights); X and the workspace are read only after the preceding kernel has completed.
+ * Larger M runs the two calls (packed_acts_out is then required). */
+fgmp_status fgmp_linear_fused(const void* X_bf16, int64_t ldx, const float* fisher_chan,
+                              fgmp_scales sc, fgmp_score_mode sm, float tau, const void* packed_weights,
+                              void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                              void* packed_acts_out, size_t packed_bytes,
+                              void* workspace, size_t ws_bytes, void* cuda_stream);
 
 /* ---- fgmp_linear with the next layer's activation quantizer in its epilogue (Section 4.2) ----
  * The paper's post-processing unit quantizes the output activations of a layer, block by block, to
@@ -256,7 +287,8 @@ fgmp_status fgmp_linear_static(const void* packed_acts, const void* packed_weigh
                                int32_t* status_out, void* cuda_stream);
 
 /* Synchronizes the stream and returns the device-side status recorded in a workspace used
- * by fgmp_linear (FGMP_OK or FGMP_ERR_TIMEOUT). */
+ * by fgmp_linear (FGMP_OK, FGMP_ERR_TIMEOUT, or FGMP_ERR_INVALID_ARG for a packed tensor whose
+ * header does not match the call). */
 fgmp_status fgmp_check(const void* workspace, void* cuda_stream);
 
 /* ---- parity support: packed -> canonical arrays (device) ----

@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libfgmp.so")
 
 SCORE_LP_ERROR, SCORE_HP_TO_LP = 0, 1
 CLIP_NONE, CLIP_SW_BRUTE = 0, 1
-OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU, OP_LINEAR_QUANTIZE = 0, 1, 2, 3, 4, 5
+OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU, OP_LINEAR_QUANTIZE, OP_LINEAR_FUSED = 0, 1, 2, 3, 4, 5, 6
 
 
 class FgmpError(RuntimeError):
@@ -56,6 +56,8 @@ def _load():
     L.fgmp_calibrate_tau.argtypes = [vp, i64, vp, i64, i64, _Scales, ci, f64, vp, vp, sz, vp]
     L.fgmp_linear.restype = ci
     L.fgmp_linear.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp]
+    L.fgmp_linear_fused.restype = ci
+    L.fgmp_linear_fused.argtypes = [vp, i64, vp, _Scales, ci, f32, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp, sz, vp]
     L.fgmp_linear_static.restype = ci
     L.fgmp_linear_static.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, vp]
     L.fgmp_check.restype = ci
@@ -281,6 +283,34 @@ def linear(acts: PackedTensor, weights: PackedTensor, *, out_dtype=torch.float32
                       1 if out.dtype == torch.bfloat16 else 0, out.stride(0), M, N, K,
                       workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear")
     linear.last_workspace = workspace
+    return out
+
+
+def linear_fused(X: torch.Tensor, fisher: torch.Tensor, weights: PackedTensor, *, scale_fp4: float, ratio: int = 3,
+                 score_mode: int = SCORE_LP_ERROR, tau: float, out_dtype=torch.float32,
+                 out: torch.Tensor | None = None, packed_out: torch.Tensor | None = None, want_packed: bool = False,
+                 workspace: torch.Tensor | None = None):
+    """One decode step in one call: X bf16 [M, K] is quantized (as quantize_activations would) and
+    multiplied with the packed weights.  Returns Y, or (Y, PackedTensor) when the packed activations
+    are asked for (want_packed / packed_out)."""
+    L = _load()
+    assert X.is_cuda and X.dtype == torch.bfloat16 and fisher.dtype == torch.float32 and X.dim() == 2
+    assert weights.kind == 1 and X.shape[1] == weights.K
+    M, K = X.shape
+    N = weights.rows
+    if out is None:
+        out = torch.empty(M, N, dtype=out_dtype, device=X.device)
+    if packed_out is None and want_packed:
+        packed_out = _alloc_aligned(L.fgmp_acts_bytes(M, K), X.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_LINEAR_FUSED, M, N, K, X.device)
+    _ok(L.fgmp_linear_fused(X.data_ptr(), X.stride(0), fisher.data_ptr(), _Scales(scale_fp4, ratio), score_mode, tau,
+                            weights.blob.data_ptr(), out.data_ptr(), 1 if out.dtype == torch.bfloat16 else 0,
+                            out.stride(0), M, N, K, _ptr(packed_out), 0 if packed_out is None else packed_out.numel(),
+                            workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear_fused")
+    linear.last_workspace = workspace
+    if packed_out is not None:
+        return out, PackedTensor(packed_out, M, K, 0)
     return out
 
 

@@ -12,61 +12,60 @@
 // ---------------------------------------------------------------- blob layout
 // A "unit" is one 128-row tile x one chunk of 16 blocks (256 K elements).
 //
-// Weights (kind 1): header | mask | uptr | records.  Everything a GEMM needs of one unit is one
-// contiguous record, so that a unit streams from HBM with a single bulk copy:
-//   REC_W4    16384 B : E2M1 codes, row r of the tile = 128 bytes whose 16-byte pieces are
-//                       XOR-swizzled with (r & 7) -- the 128B-swizzled K-major tile tcgen05 reads;
-//                       zero in FP8 blocks and in rows beyond the tensor
-//   REC_SF     2048 B : E4M3 microscales, [128 rows][16 block columns] (the decode GEMM reads two
-//                       neighbouring bytes per lane, rows 16 bytes apart: no bank conflicts)
-//   REC_KBCNT    16 B : FP8 blocks of the unit per block column
-//   REC_KBSTART  48 B : uint16 x 17 (padded): FP8 blocks of the unit before block column j; entry 16 = all
-//   REC_ROWID         : row of every FP8 block of the unit, padded to 16 bytes
-//   then              : the FP8 blocks, 16 E4M3 codes each, ordered by (block column, row) so that
-//                       blocks meeting the same 16 activation elements are neighbours
-// Records are 128-byte aligned; uptr[u] (uint32, units + 1 entries) = start of record u in
-// 128-byte steps from the first record.
+// Weights (kind 1): header | mask | uptr | records | overflow.  A unit's record has a fixed size and
+// sits at a fixed place, so that it streams from HBM with one bulk copy whose address needs no
+// look-up; what does not fit the fixed part (the second half of every FP8 block) follows in the
+// overflow section, found through uptr.  Inside a record the blocks are in the order in which the
+// decode GEMM's warps take them: warp w = 4*(r/32) + j%4 owns rows 32*(r/32) .. +31 and the block
+// columns j with j%4 == w%4; its lane 4*(r%8) + j/4 holds, as slot k = (r/8)%4, block (r, j).
+//   REC_W4    16384 B : one 8-byte slot per block at w*1024 + (k/2)*512 + lane*16 + (k%2)*8: the 16 E2M1
+//                       codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block
+//   REC_SF     2048 B : one byte per block at w*128 + lane*4 + k: the E4M3 microscale (bit 7 clear) of an
+//                       NVFP4 block; for an FP8 block 0x80 | E4M3(2^fp8_log2_ratio), i.e. bit 7 is the
+//                       block's precision flag and the low bits the factor between the tensor scales
+//   REC_WSTART  128 B : uint16 x 17: FP8 blocks of the unit that precede warp w's in (w, lane, k)
+//                       order; entry 16 = all of them
+// Overflow of a unit: E4M3 codes 8..15 of its FP8 blocks, 8 bytes each, in (w, lane, k) order, padded
+// to 16 bytes; uptr[u] (uint32, units + 1 entries) = its start in 16-byte steps from off_ovf.
 //
 // Activations (kind 0): header | codes4 | sf | mask | arec | codes8.  codes4 is row-major, sf
-// uses the same 512-byte tiles over all rows, codes8 is a dense plane of which only FP8 blocks are
+// uses 512-byte tiles over all rows, codes8 is a dense plane of which only FP8 blocks are
 // written.  arec exists when rows <= 16: one record of AREC_BYTES per chunk holding the fp16 value
 // over the tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact) of 16 token rows (rows >= M
-// are zero), in the order the decode GEMM's mma.sync fragments take them: 16 pieces of 512 bytes,
-// piece 2*sp + nh = MMA steps 2sp, 2sp+1 of token octet nh; in a piece lane (g, t) has 16 bytes =
-// elements 64t + 8sp .. 64t + 8sp + 7 of token 8nh + g, at 16-byte slot 4g + (t ^ (g & 3)) (the
-// XOR spreads the eight tokens of one block column over more banks).
-constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBCNT = 18432, REC_KBSTART = 18448, REC_ROWID = 18496;
+// are zero), in the order the decode GEMM's mma.sync fragments take them: token octet o = m/8 in
+// its own half of 4096 bytes; there 8 pieces of 512 bytes, piece 2*(j%4) + half holding elements
+// 8*half .. 8*half+7 of block column j of token m for lane 4*(m%8) + j/4, 16 bytes per lane.
+constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_WSTART = 18432, REC_BYTES = 18560;
 constexpr uint32_t AREC_BYTES = 8192;
 
 // byte offset, inside an activation record, of the first (half = 0) or second (half = 1) 8 elements
 // of block column j (0..15) of token row m
 __host__ __device__ inline uint32_t fgmp_arec_offset(uint32_t m, uint32_t j, uint32_t half)
 {
-    return ((((((j & 3u) << 1) | half) << 1) | (m >> 3)) << 9) + ((((m & 7u) << 2) | ((j >> 2) ^ (m & 3u))) << 4);
+    return ((m >> 3) << 12) + (((((j & 3u) << 1) | half)) << 9) + ((((m & 7u) << 2) | (j >> 2)) << 4);
 }
 
 struct PackedLayout {
     int64_t rows, K, KB, MW;          // KB = K/16 blocks per row, MW = mask words per row
     int64_t tiles, chunks, units;     // 128-row tiles, 16-block K chunks, tiles * chunks
     size_t off_codes4, off_sf, off_mask, off_arec, off_codes8;   // activations (mask: both)
-    size_t off_uptr, off_rec;                                    // weights
+    size_t off_uptr, off_rec, off_ovf;                           // weights
     size_t total;
 };
 
 __host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 
-// bytes of the record of a unit with cnt FP8 blocks
-__host__ __device__ inline uint32_t fgmp_rec_fp8_offset(uint32_t cnt) { return REC_ROWID + ((cnt + 15u) & ~15u); }
-__host__ __device__ inline uint32_t fgmp_rec_bytes(uint32_t cnt) { return (fgmp_rec_fp8_offset(cnt) + cnt * 16u + 127u) & ~127u; }
+// overflow of a unit with cnt FP8 blocks, in 16-byte steps
+__host__ __device__ inline uint32_t fgmp_ovf_steps(uint32_t cnt) { return (cnt + 1u) >> 1; }
 
-// kind 0 = activations, 1 = weights (max_fp8 = room for that many FP8 blocks in the records)
+// kind 0 = activations, 1 = weights (max_fp8 = room for that many FP8 blocks in the overflow section)
 __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int kind, int64_t max_fp8)
 {
     PackedLayout L;
     L.rows = rows; L.K = K; L.KB = K / 16; L.MW = (L.KB + 31) / 32;
     L.tiles = (rows + 127) / 128; L.chunks = (L.KB + 15) / 16; L.units = L.tiles * L.chunks;
     size_t o = 1024;                                   // header section
-    L.off_codes4 = L.off_sf = L.off_arec = L.off_codes8 = L.off_uptr = L.off_rec = 0;
+    L.off_codes4 = L.off_sf = L.off_arec = L.off_codes8 = L.off_uptr = L.off_rec = L.off_ovf = 0;
     if (kind == 0) {
         L.off_codes4 = o;  o = fgmp_align1k(o + (size_t)rows * (size_t)(K / 2));
         L.off_sf = o;      o = fgmp_align1k(o + (size_t)L.tiles * (size_t)(K / 64) * 512);
@@ -76,9 +75,9 @@ __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int
     } else {
         L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
         L.off_uptr = o;    o = fgmp_align1k(o + ((size_t)L.units + 1) * 4);
-        L.off_rec = o;
-        // a record is at most REC_ROWID + 15 + 127 bytes plus 17 per FP8 block
-        o = fgmp_align1k(o + (size_t)L.units * (REC_ROWID + 144) + (size_t)max_fp8 * 17);
+        L.off_rec = o;     o = fgmp_align1k(o + (size_t)L.units * REC_BYTES);
+        // 8 bytes per FP8 block, and up to 8 bytes of padding per unit
+        L.off_ovf = o;     o = fgmp_align1k(o + (size_t)max_fp8 * 8 + (size_t)L.units * 8);
     }
     L.total = o;
     return L;
@@ -91,47 +90,32 @@ __host__ __device__ inline size_t fgmp_sf_offset(int64_t r, int64_t kb, int64_t 
          + (size_t)(r & 31) * 16 + (size_t)((r & 127) >> 5) * 4 + (size_t)(kb & 3);
 }
 
-// inside a record (r = row in the tile, j = block column in the chunk): the 8 code bytes and
-// the microscale byte
+// inside a record (r = row in the tile, j = block column in the chunk): who holds the block ...
+__host__ __device__ inline uint32_t fgmp_rec_warp(uint32_t r, uint32_t j) { return ((r >> 5) << 2) | (j & 3u); }
+__host__ __device__ inline uint32_t fgmp_rec_lane(uint32_t r, uint32_t j) { return ((r & 7u) << 2) | (j >> 2); }
+__host__ __device__ inline uint32_t fgmp_rec_slot(uint32_t r, uint32_t j) { (void)j; return (r >> 3) & 3u; }
+// ... where its 8-byte slot and its scale byte sit, and its rank in the order of the overflow entries
 __host__ __device__ inline uint32_t fgmp_rec_w4_offset(uint32_t r, uint32_t j)
 {
-    return r * 128u + (((j >> 1) ^ (r & 7u)) << 4) + (j & 1u) * 8u;
+    const uint32_t k = fgmp_rec_slot(r, j);
+    return fgmp_rec_warp(r, j) * 1024u + (k >> 1) * 512u + fgmp_rec_lane(r, j) * 16u + (k & 1u) * 8u;
 }
 __host__ __device__ inline uint32_t fgmp_rec_sf_offset(uint32_t r, uint32_t j)
 {
-    return r * 16u + j;
+    return fgmp_rec_warp(r, j) * 128u + fgmp_rec_lane(r, j) * 4u + fgmp_rec_slot(r, j);
 }
+__host__ __device__ inline uint32_t fgmp_rec_order(uint32_t r, uint32_t j)
+{
+    return ((fgmp_rec_warp(r, j) * 32u + fgmp_rec_lane(r, j)) << 2) | fgmp_rec_slot(r, j);
+}
+// the inverse: row and block column of slot k of lane `lane` of warp w
+__host__ __device__ inline uint32_t fgmp_rec_row(uint32_t w, uint32_t lane, uint32_t k) { return ((w >> 2) << 5) + (k << 3) + (lane >> 2); }
+__host__ __device__ inline uint32_t fgmp_rec_col(uint32_t w, uint32_t lane) { return ((lane & 3u) << 2) | (w & 3u); }
+
+// E4M3 code of 2^ratio, -7 <= ratio <= 7 (2^-7 is subnormal)
+__host__ __device__ inline uint32_t fgmp_pow2_e4m3(int ratio) { return ratio >= -6 ? (uint32_t)(ratio + 7) << 3 : 0x04u; }
 
 #ifdef __CUDACC__
-// Where the FP8 blocks of one unit sit in its record.  Called by all 128 threads of a CTA, thread
-// i = row i of the tile, m16 = that row's 16 mask bits of the chunk (0 beyond the last row).
-// On return s_pos[row * 16 + j] = index of block (row, j) among the unit's FP8 blocks (0xffff if
-// the block is not FP8), s_cnt[j] = FP8 blocks in column j, and the return value is their total.
-// s_warp is scratch of 64 words.  Ends with a __syncthreads().
-__device__ __forceinline__ uint32_t fgmp_unit_positions(uint32_t m16, uint32_t* s_warp, uint16_t* s_pos, uint32_t* s_cnt)
-{
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    uint32_t rank[16];
-#pragma unroll
-    for (int kb = 0; kb < 16; ++kb) {
-        const uint32_t bal = __ballot_sync(0xffffffffu, (m16 >> kb) & 1u);
-        rank[kb] = __popc(bal & ((1u << lane) - 1u));
-        if (lane == 0) s_warp[w * 16 + kb] = __popc(bal);
-    }
-    __syncthreads();
-    uint32_t run = 0;
-#pragma unroll
-    for (int kb = 0; kb < 16; ++kb) {
-        const uint32_t c0 = s_warp[kb], c1 = s_warp[16 + kb], c2 = s_warp[32 + kb], c3 = s_warp[48 + kb];
-        const uint32_t below = (w > 0 ? c0 : 0u) + (w > 1 ? c1 : 0u) + (w > 2 ? c2 : 0u);
-        s_pos[threadIdx.x * 16 + kb] = ((m16 >> kb) & 1u) ? (uint16_t)(run + below + rank[kb]) : (uint16_t)0xffff;
-        if (threadIdx.x == 0) s_cnt[kb] = c0 + c1 + c2 + c3;
-        run += c0 + c1 + c2 + c3;
-    }
-    __syncthreads();
-    return run;
-}
-
 // the 16 mask bits of (row r, chunk c) of a packed tensor; 0 beyond the last row
 __device__ __forceinline__ uint32_t fgmp_chunk_mask(const uint32_t* mask, const PackedLayout& L, int64_t r, int64_t c)
 {
@@ -139,37 +123,38 @@ __device__ __forceinline__ uint32_t fgmp_chunk_mask(const uint32_t* mask, const 
     return (mask[r * L.MW + (c >> 1)] >> ((c & 1) * 16)) & 0xffffu;
 }
 
-struct UnitScratch { uint32_t warp[64]; uint32_t cnt[16]; uint16_t pos[128 * 16]; };
-
-// record of unit u of a packed weight tensor
-__device__ __forceinline__ const uint8_t* fgmp_record(const uint8_t* blob, const PackedLayout& L, int64_t u)
+// Kernels that walk a unit in record order run 512 threads per unit: thread = (warp w, lane), four
+// slots each.  Exclusive prefix over the lanes of a warp of the number of flagged slots (flags = the
+// bits 0x80808080 of the lane's four scale bytes, or any word with one bit per flagged slot).
+__device__ __forceinline__ uint32_t fgmp_warp_excl_count(uint32_t flags, uint32_t& warp_total)
 {
-    return blob + L.off_rec + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[u] * 128;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t cnt = __popc(flags);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= (uint32_t)o) incl += y;
+    }
+    warp_total = __shfl_sync(0xffffffffu, incl, 31);
+    return incl - cnt;
 }
 
-// Visits every block of one unit of a packed weight tensor, 128 threads per unit, consecutive
-// threads on consecutive blocks of one row: f(row, kb, row in tile, column in chunk, rec, e8) with
-// rec = the unit's record and e8 = address of the block's 16 E4M3 codes, or nullptr if NVFP4.
-template <class F>
-__device__ __forceinline__ void fgmp_for_each_block(const uint8_t* blob, const PackedLayout& L, int64_t unit,
-                                                    UnitScratch& sc, F f)
+// What thread (w, lane) of a 512-thread CTA needs to read its four blocks of one unit of a packed
+// weight tensor: the record, the unit's overflow entries, the lane's four scale bytes and the index
+// of the overflow entry of its first FP8 block (its further FP8 blocks follow, in slot order).
+struct UnitLaneView { const uint8_t* rec; const uint8_t* ovf; uint32_t sc4, idx; };
+__device__ __forceinline__ UnitLaneView fgmp_unit_lane(const uint8_t* blob, const PackedLayout& L, int64_t unit)
 {
-    const int64_t tile = unit / L.chunks, c = unit % L.chunks;
-    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
-    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
-    const uint8_t* rec = fgmp_record(blob, L, unit);
-    const uint8_t* fp8 = rec + fgmp_rec_fp8_offset(cnt);
-    const int j = threadIdx.x & 15;
-#pragma unroll 1
-    for (int i = 0; i < 16; ++i) {
-        const int row = (threadIdx.x >> 4) + 8 * i;
-        const int64_t r = tile * 128 + row, kb = c * 16 + j;
-        if (r >= L.rows || kb >= L.KB) continue;
-        const uint32_t pos = sc.pos[row * 16 + j];
-        f(r, kb, row, j, rec, pos != 0xffffu ? fp8 + (size_t)pos * 16 : (const uint8_t*)nullptr);
-    }
-    __syncthreads();
+    UnitLaneView v;
+    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    v.rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
+    v.ovf = blob + L.off_ovf + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[unit] * 16;
+    v.sc4 = *reinterpret_cast<const uint32_t*>(v.rec + REC_SF + w * 128u + lane * 4u);
+    uint32_t total;
+    const uint32_t excl = fgmp_warp_excl_count(v.sc4 & 0x80808080u, total);
+    v.idx = reinterpret_cast<const uint16_t*>(v.rec + REC_WSTART)[w] + excl;
+    return v;
 }
 #endif
 

@@ -14,6 +14,7 @@ size_t fgmp_ws_quantize_weights(int64_t N, int64_t K);
 size_t fgmp_ws_calibrate(int64_t M, int64_t K);
 size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K);
 size_t fgmp_ws_linear_quantize(int64_t M, int64_t N, int64_t K);
+size_t fgmp_ws_linear_fused(int64_t M, int64_t N, int64_t K);
 size_t fgmp_ws_global_tau(int64_t total_scores);
 // weight-streaming kernel for M <= 16 tokens and K % 256 == 0
 bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K);

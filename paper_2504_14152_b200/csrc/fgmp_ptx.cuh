@@ -36,16 +36,18 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
     return t;
 }
 
-// Bounded wait: gives up after ~2 s (or when another thread of the CTA already gave up),
+// Bounded wait: gives up after limit_ns (or when another thread of the CTA already gave up),
 // records the failure and returns false.  `abort_flag` lives in shared memory.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+constexpr unsigned long long MBAR_WAIT_LIMIT_NS = 2000000000ull;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where,
+                                            unsigned long long limit_ns)
 {
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > 2000000000ull) {
+        if (globaltimer_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             atomicCAS(status, 0, (int)FGMP_ERR_TIMEOUT);
             atomicExch(status + 1, where);
@@ -54,10 +56,11 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         __nanosleep(64);
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where,
+                                          unsigned long long limit_ns = MBAR_WAIT_LIMIT_NS)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, where);
+    return mbar_wait_slow(bar, parity, abort_flag, status, where, limit_ns);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar)

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     if (!SCORE_ONLY) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
-            h->magic = FGMP_MAGIC; h->version = 5; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->magic = FGMP_MAGIC; h->version = 6; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }
@@ -162,23 +162,33 @@ __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
     }
 }
 
-// packed weights -> canonical arrays; one CTA of 128 threads per unit record
-__global__ void __launch_bounds__(128) unpack_w_kernel(const uint8_t* blob, int64_t rows, int64_t K,
+// packed weights -> canonical arrays; one CTA of 512 threads per unit, in record order
+__global__ void __launch_bounds__(512) unpack_w_kernel(const uint8_t* blob, int64_t rows, int64_t K,
                                                        uint8_t* codes4, uint8_t* codes8, uint8_t* scales, uint32_t* mask)
 {
-    __shared__ UnitScratch sc;
     const PackedLayout L = fgmp_layout(rows, K, 1, 0);
     if (mask) {
         const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-        for (int64_t i = (int64_t)blockIdx.x * 128 + threadIdx.x; i < rows * L.MW; i += (int64_t)gridDim.x * 128) mask[i] = pmask[i];
+        for (int64_t i = (int64_t)blockIdx.x * 512 + threadIdx.x; i < rows * L.MW; i += (int64_t)gridDim.x * 512) mask[i] = pmask[i];
     }
-    fgmp_for_each_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, int row, int j, const uint8_t* rec, const uint8_t* e8) {
-        if (scales) scales[r * L.KB + kb] = rec[REC_SF + fgmp_rec_sf_offset(row, j)];
-        if (codes4) *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) =
-                        *reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j));
-        if (codes8) *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) =
-                        e8 ? *reinterpret_cast<const uint4*>(e8) : make_uint4(0, 0, 0, 0);
-    });
+    const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
+    const UnitLaneView u = fgmp_unit_lane(blob, L, unit);
+    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    const int64_t kb = c * 16 + fgmp_rec_col(w, lane);
+    uint32_t idx = u.idx;
+#pragma unroll 1
+    for (uint32_t k = 0; k < 4; ++k) {
+        const int64_t r = tile * 128 + fgmp_rec_row(w, lane, k);
+        const uint32_t sb = (u.sc4 >> (8 * k)) & 0xffu;
+        const uint2 slot = *reinterpret_cast<const uint2*>(u.rec + REC_W4 + w * 1024u + (k >> 1) * 512u + lane * 16u + (k & 1u) * 8u);
+        uint2 hi = make_uint2(0u, 0u);
+        const bool is8 = (sb & 0x80u) != 0;
+        if (is8) hi = *reinterpret_cast<const uint2*>(u.ovf + (size_t)(idx++) * 8);
+        if (r >= L.rows || kb >= L.KB) continue;
+        if (scales) scales[r * L.KB + kb] = is8 ? (uint8_t)0 : (uint8_t)sb;
+        if (codes4) *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) = is8 ? make_uint2(0u, 0u) : slot;
+        if (codes8) *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) = is8 ? make_uint4(slot.x, slot.y, hi.x, hi.y) : make_uint4(0, 0, 0, 0);
+    }
 }
 
 // mean of squares per column of a bf16 matrix; thread per column, rows in order (one fp32 multiply
@@ -289,7 +299,7 @@ extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, 
     if (h.magic != FGMP_MAGIC || h.rows != rows || h.K != K || h.error != 0) return FGMP_ERR_INVALID_ARG;
     if (h.kind == 1) {
         const PackedLayout L = fgmp_layout(rows, K, 1, 0);
-        FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_w_kernel<<<(unsigned)L.units, 128, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
+        FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_w_kernel<<<(unsigned)L.units, 512, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
     } else {
         int64_t nblk = rows * (K / 16);
         int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);

@@ -330,6 +330,98 @@ def test_decode_workspace_is_left_clear_for_the_next_call(fg):
     assert int(ws[: 1024 + 32 * 16].to(torch.int32).abs().sum().item()) == 0
 
 
+def test_prefill_call_between_decode_calls_on_one_workspace(fg):
+    """A prefill-shaped call keeps its scratch behind the control area, so decode-shaped calls before and
+    after it on the same workspace (cleared once) still find their tile counters at zero."""
+    shapes = [(16, 640, 1024), (77, 300, 1024), (16, 640, 1024), (200, 256, 512), (3, 1408, 512)]
+    big = max(fg.workspace_bytes(fg.binding.OP_LINEAR, M, N, K) for M, N, K in shapes)
+    ws = fg.workspace_init(fg.binding._alloc_aligned(big, torch.device("cuda")))
+    for i, (M, N, K) in enumerate(shapes):
+        wl = gi.llama("d", M, N, K, seed=40 + i)
+        qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+        Y, S = oracle.linear(qa, qw)
+        y_shared = fg.linear(pa, pw, workspace=ws)
+        fg.check(ws)
+        assert torch.equal(y_shared, fg.linear(pa, pw)), f"call {i}: a reused workspace changed the result"
+        err = np.abs(y_shared.cpu().numpy().astype(np.float64) - Y)
+        assert (err <= 1e-5 * S + 1e-30).all(), f"call {i}"
+    assert int(ws[: 65536].to(torch.int32).abs().sum().item()) == 0
+
+
+# ------------------------------------------------------------ quantizer + GEMM in one launch
+
+@pytest.mark.parametrize("M,N,K,mode", [(16, 640, 1024, 0), (5, 1408, 512, 1), (1, 300, 2048, 0), (9, 129, 256, 0),
+                                        (16, 11008, 4096, 0), (8, 4096, 11008, 1), (16, 1000, 7424, 0)])
+def test_fused_decode_step_equals_the_two_calls_and_the_oracle(fg, M, N, K, mode):
+    """fgmp_linear_fused: packed activations bit-equal to the oracle's (and so to fgmp_quantize_activations'),
+    Y bit-equal to fgmp_linear on them and within the bar of the oracle; twice on one workspace."""
+    wl = gi.llama("f", M, N, K, seed=60 + M)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, mode=mode, clip=False)
+    x, fx = wl.x(), wl.fx()
+    s4 = gi.tensor_scale(x)
+    tau = tau_for_fraction(qa.scores, 0.1)
+    ws = fg.alloc_workspace(fg.binding.OP_LINEAR_FUSED, M, N, K, torch.device("cuda"))
+    y_two = fg.linear(pa, pw)
+    for rep in range(2):
+        y, pf = fg.linear_fused(x.cuda(), fx.cuda(), pw, scale_fp4=s4, score_mode=mode, tau=tau, want_packed=True, workspace=ws)
+        fg.check(ws)
+        compare_packed(fg, pf, qa, tau, f"fused rep {rep}")
+        assert torch.equal(y, y_two), f"rep {rep}: fused Y differs from the two calls"
+    # without the packed output (records in the workspace only)
+    y3 = fg.linear_fused(x.cuda(), fx.cuda(), pw, scale_fp4=s4, score_mode=mode, tau=tau, workspace=ws)
+    fg.check(ws)
+    assert torch.equal(y3, y_two)
+    rng = np.random.default_rng(0)
+    ms = np.r_[rng.integers(0, M, 3000), [0, M - 1, 0, M - 1]]
+    nn = np.r_[rng.integers(0, N, 3000), [0, N - 1, N - 1, 0]]
+    Y, S = oracle.linear_sampled(qa, qw, ms, nn)
+    err = np.abs(y3.cpu().numpy().astype(np.float64)[ms, nn] - Y)
+    assert (err <= 1e-5 * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    # a plain fgmp_linear on the same workspace afterwards still works (control area as it expects)
+    assert torch.equal(fg.linear(pa, pw, workspace=ws), y_two)
+    fg.check(ws)
+
+
+def test_fused_step_for_a_prefill_sized_batch_runs_the_two_calls(fg):
+    wl = gi.llama("f", 40, 300, 512, seed=70)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    x, fx = wl.x(), wl.fx()
+    s4 = gi.tensor_scale(x)
+    tau = tau_for_fraction(qa.scores, 0.1)
+    y, pf = fg.linear_fused(x.cuda(), fx.cuda(), pw, scale_fp4=s4, tau=tau, want_packed=True)
+    compare_packed(fg, pf, qa, tau, "fused prefill-sized")
+    assert torch.equal(y, fg.linear(pa, pw))
+
+
+def test_weight_blob_that_does_not_match_the_call_is_refused_on_the_device(fg):
+    """Threshold mode with too little room: the packer flags the blob, fgmp_unpack refuses it, and fgmp_linear
+    reads none of it (status FGMP_ERR_INVALID_ARG) -- on both GEMM paths.  So does a blob of another shape."""
+    wl = gi.llama("cap", 16, 640, 1024, seed=5)
+    w, fw = wl.w(), wl.fw()
+    qa, qw, pa, pw_ok = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    pw = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=0, fp8_fraction=-1.0, tau=0.0, max_fp8_blocks=100)
+    assert pw.header()["error"] == -7
+    with pytest.raises(fg.FgmpError):
+        fg.unpack(pw)
+    y = fg.linear(pa, pw)
+    with pytest.raises(fg.FgmpError) as e:
+        fg.check(fg.linear.last_workspace)
+    assert e.value.code == -1
+    # a blob packed for another N
+    other = fg.quantize_weights(wl.w()[:512].contiguous().cuda(), fw[:512].contiguous().cuda(), clip_mode=0, fp8_fraction=0.1)
+    other.rows = 640                                           # the caller claims a shape the blob does not have
+    big = fg.binding._alloc_aligned(pw_ok.blob.numel(), torch.device("cuda"))
+    big[: other.blob.numel()] = other.blob                     # inside an allocation large enough for the claimed shape
+    other.blob = big
+    fg.linear(pa, other)
+    with pytest.raises(fg.FgmpError) as e:
+        fg.check(fg.linear.last_workspace)
+    assert e.value.code == -1
+    # the good blob still works afterwards
+    y = fg.linear(pa, pw_ok)
+    fg.check(fg.linear.last_workspace)
+
+
 @pytest.mark.parametrize("kind", [0, 1, 2])
 def test_tensor_peak_loop_runs(fg, kind):
     ws = fg.binding._alloc_aligned(1024, torch.device("cuda"))
