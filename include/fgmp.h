@@ -50,7 +50,7 @@
  *                   and slot k = (r/8)%4 hold block (row r of the tile, block column j of the chunk).
  *                   16384 B of 8-byte slots at w*1024 + (k/2)*512 + lane*16 + (k%2)*8: the 16 E2M1
  *                   codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block (zero beyond N)
- *                   | 2048 B of scale bytes at w*128 + lane*4 + k: the E4M3 microscale of an NVFP4
+ *                   | 2048 B of scale bytes at (w/4)*512 + lane*16 + (w%4)*4 + k: the E4M3 microscale of an NVFP4
  *                   block (bit 7 clear), or 0x80 | E4M3(2^fp8_log2_ratio) for an FP8 block
  *                   | 128 B: uint16 x 17, FP8 blocks of the unit before warp w's; entry 16 = all
  *   overflow      : E4M3 codes 8..15 of the FP8 blocks, 8 bytes each, unit by unit, inside a unit in

@@ -20,7 +20,8 @@
 // columns j with j%4 == w%4; its lane 4*(r%8) + j/4 holds, as slot k = (r/8)%4, block (r, j).
 //   REC_W4    16384 B : one 8-byte slot per block at w*1024 + (k/2)*512 + lane*16 + (k%2)*8: the 16 E2M1
 //                       codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block
-//   REC_SF     2048 B : one byte per block at w*128 + lane*4 + k: the E4M3 microscale (bit 7 clear) of an
+//   REC_SF     2048 B : one byte per block at (w/4)*512 + lane*16 + (w%4)*4 + k (the sixteen blocks of one
+//                       lane of the four warps of a row group side by side): the E4M3 microscale (bit 7 clear) of an
 //                       NVFP4 block; for an FP8 block 0x80 | E4M3(2^fp8_log2_ratio), i.e. bit 7 is the
 //                       block's precision flag and the low bits the factor between the tensor scales
 //   REC_WSTART  128 B : uint16 x 17: FP8 blocks of the unit that precede warp w's in (w, lane, k)
@@ -102,7 +103,8 @@ __host__ __device__ inline uint32_t fgmp_rec_w4_offset(uint32_t r, uint32_t j)
 }
 __host__ __device__ inline uint32_t fgmp_rec_sf_offset(uint32_t r, uint32_t j)
 {
-    return fgmp_rec_warp(r, j) * 128u + fgmp_rec_lane(r, j) * 4u + fgmp_rec_slot(r, j);
+    const uint32_t w = fgmp_rec_warp(r, j);
+    return (w >> 2) * 512u + fgmp_rec_lane(r, j) * 16u + (w & 3u) * 4u + fgmp_rec_slot(r, j);
 }
 __host__ __device__ inline uint32_t fgmp_rec_order(uint32_t r, uint32_t j)
 {
@@ -150,7 +152,7 @@ __device__ __forceinline__ UnitLaneView fgmp_unit_lane(const uint8_t* blob, cons
     const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
     v.rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
     v.ovf = blob + L.off_ovf + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[unit] * 16;
-    v.sc4 = *reinterpret_cast<const uint32_t*>(v.rec + REC_SF + w * 128u + lane * 4u);
+    v.sc4 = *reinterpret_cast<const uint32_t*>(v.rec + REC_SF + (w >> 2) * 512u + lane * 16u + (w & 3u) * 4u);
     uint32_t total;
     const uint32_t excl = fgmp_warp_excl_count(v.sc4 & 0x80808080u, total);
     v.idx = reinterpret_cast<const uint16_t*>(v.rec + REC_WSTART)[w] + excl;

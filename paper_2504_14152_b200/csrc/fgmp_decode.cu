@@ -9,7 +9,7 @@
 // mma.sync m16n8k16 (fp16 in, fp32 accumulation) as their true values over the tensor scales.
 // 16 weight rows are the M side of an MMA, a token octet the N side.  The order of the contraction
 // index is free as long as both operands agree, so an MMA step takes four consecutive elements of
-// one block per lane: lane (g, t) of warp (jr, hq) owns block column 4t + hq of rows 32jr + 8k + g,
+// one block per lane: lane (g, t) owns, for hq = 0..3, block column 4t + hq of rows 32jr + 8k + g,
 // k = 0..3, of the unit, and its four MMA steps per 16-row tile walk through that block.  A lane
 // therefore meets whole blocks, and the format of a block is a per-lane choice between two
 // conversion instructions (cvt e2m1x2 / cvt e4m3x2, predicated on the block's flag) followed by the
@@ -21,10 +21,12 @@
 // Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all SMs
 // stream the same number of bytes; a unit is up to three bulk copies (its fixed-size record, the
 // second halves of its FP8 blocks, the activation record of its chunk) into a ring of stages.
-// Tiles shared by several CTAs are reduced in a fixed order by the CTA that arrives last.  Every
-// sum is taken in a fixed order: results are reproducible bit for bit.
-//
-// Warp roles (544 threads): warps 0-15 = arithmetic, warp 16 = producer.
+// The 16 warps form four groups; consecutive units of a CTA go to consecutive groups, so four units
+// are being multiplied at any time and the latencies of one (barrier, shared-memory loads, the
+// dependent MMAs) hide behind the others.  Inside a group warp jr takes rows 32jr .. 32jr+31.  There
+// is no producer warp: the warp that is last to finish a unit refills its stage.  Tiles shared by
+// several CTAs are reduced in a fixed order by the CTA that arrives last.  Every sum is taken in a
+// fixed order: results are reproducible bit for bit.
 #include "fgmp_common.cuh"
 #include "fgmp_actq.cuh"
 #include "fgmp_host.h"
@@ -36,17 +38,16 @@
 namespace {
 
 constexpr int MATH_WARPS = 16, MATH_THREADS = 32 * MATH_WARPS;
-constexpr int PRODUCER_WARP = MATH_WARPS;
-constexpr int DEC_THREADS = 32 * (MATH_WARPS + 1);
-constexpr uint32_t OVF_CAP = 5632;              // overflow bytes of a unit that fit a stage (704 FP8 blocks); more are read from global
+constexpr int DEC_THREADS = MATH_THREADS;
+constexpr uint32_t OVF_CAP = 2560;              // overflow bytes of a unit that fit a stage (320 FP8 blocks); more are read from global
 constexpr uint32_t STG_OVF = REC_BYTES;
-constexpr uint32_t STG_A = STG_OVF + OVF_CAP;                                                    // 24192
-constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 32384
-constexpr int DEC_STAGES = 5;                   // at most; a launch uses DecParams::stages of them
-constexpr uint32_t EPI_FLOATS = 4 * 128 * 16;   // [hq][row][token] fp32: the four column classes of a tile
-constexpr size_t dec_smem(int stages) { return (size_t)stages * DEC_STAGE_BYTES + EPI_FLOATS * 4 + 1024 /*alignment*/ + 512 /*barriers*/; }
-constexpr size_t DEC_SMEM = dec_smem(DEC_STAGES);
-static_assert(DEC_SMEM <= 232448, "shared memory of one CTA");
+constexpr uint32_t STG_A = STG_OVF + OVF_CAP;                                                    // 21120
+constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 29312
+constexpr int DEC_STAGES = 6;                   // at most; a launch uses DecParams::stages of them
+constexpr uint32_t EPI_FLOATS = 4 * 128 * 16;   // [warp / 4][row][token] fp32: the partial sums of a tile
+constexpr int MAX_SPAN = 8192;                  // units of one CTA whose overflow starts fit the shared-memory table
+constexpr size_t dec_smem(int stages, int64_t span) { return (size_t)stages * DEC_STAGE_BYTES + EPI_FLOATS * 4 + ((size_t)(span + 1) * 4 + 15) / 16 * 16 + 1024 /*alignment*/ + 512 /*barriers*/; }
+static_assert(dec_smem(DEC_STAGES, 64) <= 232448, "shared memory of one CTA");
 static_assert((STG_A % 128) == 0 && (DEC_STAGE_BYTES % 128) == 0, "bulk-copy alignment");
 
 // control words of the workspace (int32, from byte 256): see fgmp_linear_fused
@@ -70,7 +71,18 @@ struct DecParams {
     uint32_t* cw;                         // control words
 };
 
-struct StageMeta { uint32_t step, staged; };     // overflow start (16-byte steps), bytes of it in the stage
+struct StageMeta { uint32_t step, staged; };
+
+// Profiling builds (-DFGMP_TIMELINE) stamp the global timer at the phases of every CTA into a buffer
+// registered with fgmp_debug_timeline (16 x uint64 per CTA); ordinary builds contain none of this.
+#ifdef FGMP_TIMELINE
+__device__ unsigned long long* g_timeline = nullptr;
+#define FGMP_STAMP(slot) do { if (g_timeline && threadIdx.x == 0) g_timeline[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
+#define FGMP_STAMP_ANY(slot) do { if (g_timeline) g_timeline[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
+#else
+#define FGMP_STAMP(slot) do { } while (0)
+#define FGMP_STAMP_ANY(slot) do { } while (0)
+#endif     // overflow start (16-byte steps), bytes of it in the stage
 
 __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
 
@@ -164,8 +176,15 @@ __device__ __forceinline__ void quantize_item(const DecParams& p, int64_t c, int
     }
 }
 
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
 // NH = token octets in use: 1 for M <= 8, else 2.  FUSED: the activation quantizer runs in the prologue.
-template <int NH, bool FUSED>
+// NG = groups of 16 / NG warps that work on different units at the same time; a warp takes rows 32jr .. 32jr+31
+// and NG of the four classes of block columns (j % 4).
+template <int NH, bool FUSED, int NG>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_kernel(DecParams p)
 {
@@ -174,76 +193,73 @@ decode_kernel(DecParams p)
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int S = p.stages;
     float* epi = reinterpret_cast<float*>(smem + (size_t)S * DEC_STAGE_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(epi + EPI_FLOATS);
-    // bars: [0, DEC_STAGES) full, [DEC_STAGES, 2 DEC_STAGES) empty
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 2 * DEC_STAGES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(epi + EPI_FLOATS);             // full[DEC_STAGES]
+    uint32_t* done = reinterpret_cast<uint32_t*>(bars + DEC_STAGES);            // warps that have finished with a stage
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(done + DEC_STAGES + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smeta + DEC_STAGES);
     volatile uint32_t* s_misc = reinterpret_cast<volatile uint32_t*>(abort_flag + 1);   // [0] tag, [1..2] claimed item, [3] last-arrival flag
+    uint32_t* table = const_cast<uint32_t*>(s_misc + 8);                        // overflow starts of this CTA's units (+ 1)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * DEC_STAGES;
+    const uint32_t full0 = smem_u32(bars);
+    FGMP_STAMP(0);
     constexpr uint32_t A_BYTES = NH == 2 ? AREC_BYTES : AREC_BYTES / 2;
 
     // this CTA's span of (tile, chunk) units
     const int64_t G = gridDim.x, C = p.chunks;
     const int64_t u_begin = ((int64_t)blockIdx.x * p.total) / G, u_end = ((int64_t)(blockIdx.x + 1) * p.total) / G;
+    const int n_units = (int)(u_end - u_begin);
     const uint32_t* uptr = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_uptr);
     const uint8_t* recs = p.wblob + p.LW.off_rec;
     const uint8_t* ovfs = p.wblob + p.LW.off_ovf;
     const uint8_t* arec = FUSED ? p.arec : p.ablob + p.LA.off_arec;
 
-    // One unit's copies into a stage (lane 0 of the producer warp): record and overflow, then the
-    // activation record of the unit's chunk
-    auto issue_w = [&](int64_t u, int stage, uint32_t step0, uint32_t step1) {
-        const uint32_t bytes = (step1 - step0) * 16u;
+    // the copies of unit i (index inside the span) into its stage, by one thread
+    auto stage_dst = [&](int stage) { return smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES); };
+    auto issue_rec = [&](int i, int stage) { bulk_load(stage_dst(stage), recs + (size_t)(u_begin + i) * REC_BYTES, REC_BYTES, full0 + 8 * stage); };
+    auto issue_ovf = [&](int i, int stage, bool expect) {
+        const uint32_t step0 = table[i], bytes = (table[i + 1] - step0) * 16u;
         const uint32_t staged = bytes < OVF_CAP ? bytes : OVF_CAP;
         smeta[stage].step = step0; smeta[stage].staged = staged;
-        const uint32_t fb = full0 + 8 * stage;
-        const uint32_t dst = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
-        mbar_expect_tx(fb, REC_BYTES + staged + A_BYTES);
-        bulk_load(dst, recs + (size_t)u * REC_BYTES, REC_BYTES, fb);
-        if (staged) bulk_load(dst + STG_OVF, ovfs + (size_t)step0 * 16, staged, fb);
+        if (expect && staged) mbar_expect_tx_only(full0 + 8 * stage, staged);
+        if (staged) bulk_load(stage_dst(stage) + STG_OVF, ovfs + (size_t)step0 * 16, staged, full0 + 8 * stage);
+        return staged;
     };
-    auto issue_a = [&](int64_t u, int stage) {
-        bulk_load(smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES) + STG_A, arec + (size_t)(u % C) * AREC_BYTES, A_BYTES, full0 + 8 * stage);
+    auto issue_a = [&](int i, int stage) {
+        bulk_load(stage_dst(stage) + STG_A, arec + (size_t)((u_begin + i) % C) * AREC_BYTES, A_BYTES, full0 + 8 * stage);
     };
 
-    // ------------------------------------------------------------ set-up (producer warp): barriers, the weight
-    // blob's header, and the first stages' weight copies.  The packed weights are not written by whatever runs
-    // before this kernel, so all of this may overlap the end of that kernel (programmatic dependent launch).
-    int64_t pf_base = u_begin;
-    uint32_t pf = 0;
-    int pre = 0;
-    if (warp == PRODUCER_WARP) {
-        if (lane == 0) {
-            for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, MATH_WARPS); }
-            *abort_flag = 0;
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
+    // ------------------------------------------------------------ set-up: barriers, the weight blob's header, and the
+    // first stages' weight copies.  The packed weights are not written by whatever runs before this kernel, so all
+    // of this may overlap the end of that kernel (programmatic dependent launch).
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); done[s] = 0; }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         // nothing is read through the blob's tables before its header has been seen to describe this call
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
-        int okh = 1;
-        if (lane == 0) {
-            const uint2 mv = __ldg(reinterpret_cast<const uint2*>(hw));
-            okh = mv.x == FGMP_MAGIC && mv.y == 6u && __ldg(&hw->rows) == p.N && __ldg(&hw->K) == p.K &&
-                  __ldg(&hw->kind) == 1u && __ldg(&hw->error) == 0;
-            if (!okh) { *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 9); }
-        }
-        okh = __shfl_sync(0xffffffffu, okh, 0);
-        if (okh) {
-            if (pf_base + lane <= p.total) pf = __ldg(uptr + pf_base + lane);
-            pre = (int)min((int64_t)S, u_end - u_begin);
-            for (int s = 0; s < pre; ++s) {
-                const uint32_t step0 = __shfl_sync(0xffffffffu, pf, s), step1 = __shfl_sync(0xffffffffu, pf, s + 1);
-                if (lane == 0) issue_w(u_begin + s, s, step0, step1);
-            }
-        }
+        const uint2 mv = __ldg(reinterpret_cast<const uint2*>(hw));
+        const bool okh = mv.x == FGMP_MAGIC && mv.y == 6u && __ldg(&hw->rows) == p.N && __ldg(&hw->K) == p.K &&
+                         __ldg(&hw->kind) == 1u && __ldg(&hw->error) == 0;
+        if (!okh) { *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 9); }
     }
     __syncthreads();
+    FGMP_STAMP(1);
+    const int pre = min(S, n_units);
+    if (!*abort_flag) {
+        for (int i = threadIdx.x; i <= n_units; i += DEC_THREADS) table[i] = __ldg(uptr + u_begin + i);
+        if (threadIdx.x == 0)
+            for (int s = 0; s < pre; ++s) { mbar_expect_tx_only(full0 + 8 * s, REC_BYTES + A_BYTES); issue_rec(s, s); }
+    }
+    __syncthreads();
+    if (!*abort_flag && threadIdx.x == 0)
+        for (int s = 0; s < pre; ++s) issue_ovf(s, s, true);
+    FGMP_STAMP(2);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // Launched as a programmatic dependent of the preceding kernel in the stream, this kernel may have
     // started before that one finished: everything above touches neither its output nor the workspace.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    FGMP_STAMP(3);
     if (FUSED) {
         if (threadIdx.x == 0) {
             uint32_t e;
@@ -254,45 +270,7 @@ decode_kernel(DecParams p)
     }
     const uint32_t tag = FUSED ? s_misc[0] : 0u;
 
-    if (*abort_flag) {
-        // the weight blob does not belong to this call: nothing else is read
-    } else if (warp == PRODUCER_WARP) {
-        // ------------------------------------------------------------ producer (whole warp; lane 0 issues)
-        int ok = 1;
-        if (lane == 0) {
-            if (FUSED) {
-                // every chunk's record is in place once the last work item of the quantizer has been handed in
-                ok = wait_global_equals(p.cw + CW_QREADY, tag, abort_flag, p.status, 8) ? 1 : 0;
-                asm volatile("fence.proxy.async;" ::: "memory");   // records were written with ordinary stores, the bulk copy reads them
-            } else {
-                const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
-                const uint2 mv = __ldg(reinterpret_cast<const uint2*>(ha));
-                if (!(mv.x == FGMP_MAGIC && mv.y == 6u && __ldg(&ha->rows) == p.M && __ldg(&ha->K) == p.K && __ldg(&ha->kind) == 0u)) {
-                    *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 10);
-                    ok = 0;
-                }
-            }
-            if (ok) for (int s = 0; s < pre; ++s) issue_a(u_begin + s, s);
-        }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        int stage = pre % S; uint32_t phase = (uint32_t)(pre / S) & 1u;
-        for (int64_t u = u_begin + pre; u < u_end && ok; ++u) {
-            if (u + 1 - pf_base > 31) {                // next 32 overflow starts
-                pf_base = u;
-                pf = (pf_base + lane <= p.total) ? __ldg(uptr + pf_base + lane) : 0u;
-            }
-            const uint32_t step0 = __shfl_sync(0xffffffffu, pf, (int)(u - pf_base));
-            const uint32_t step1 = __shfl_sync(0xffffffffu, pf, (int)(u + 1 - pf_base));
-            if (lane == 0) {
-                ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1) ? 1 : 0;
-                if (ok) { issue_w(u, stage, step0, step1); issue_a(u, stage); }
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (++stage == S) { stage = 0; phase ^= 1; }
-        }
-    } else {
-        // ------------------------------------------------------------ arithmetic warps
-        bool ok = true;
+    if (!*abort_flag) {
         if (FUSED) {
             // The quantizer's work items are handed out through a counter, so that every item is taken by a CTA
             // that is running: no CTA ever waits for one that has not started.  The counter and the count of
@@ -318,117 +296,173 @@ decode_kernel(DecParams p)
                     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(tag) : "memory");
             }
         }
+        // the activation records of the first stages; their barriers' one arrival comes last
+        FGMP_STAMP(4);
+        if (threadIdx.x == 0) {
+            bool oka = true;
+            if (FUSED) {
+                // every chunk's record is in place once the last work item of the quantizer has been handed in
+                oka = wait_global_equals(p.cw + CW_QREADY, tag, abort_flag, p.status, 8);
+                asm volatile("fence.proxy.async;" ::: "memory");   // records were written with ordinary stores, the bulk copy reads them
+            } else {
+                const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
+                const uint2 mv = __ldg(reinterpret_cast<const uint2*>(ha));
+                if (!(mv.x == FGMP_MAGIC && mv.y == 6u && __ldg(&ha->rows) == p.M && __ldg(&ha->K) == p.K && __ldg(&ha->kind) == 0u)) {
+                    *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 10);
+                    oka = false;
+                }
+            }
+            if (oka) for (int s = 0; s < pre; ++s) { issue_a(s, s); mbar_arrive(full0 + 8 * s); }
+        }
+        FGMP_STAMP(5);
 
-        const uint32_t w = (uint32_t)warp, jr = w >> 2, hq = w & 3u;
+        // ------------------------------------------------------------ the units of this CTA, group by group
+        constexpr int GROUPS = NG, GROUP_WARPS = MATH_WARPS / NG;
+        const uint32_t part = (uint32_t)warp >> 2, jr = (uint32_t)warp & 3u;      // part: which partial tile this warp's sums go to
+        const uint32_t gq = part * NG / 4u;                                       // group
+        const int hq0 = NG == 4 ? 0 : (NG == 2 ? 2 * (int)(part & 1u) : (int)part);
         const uint32_t g = (uint32_t)lane >> 2, t = (uint32_t)lane & 3u;
-        const uint32_t w4_off = REC_W4 + w * 1024u + (uint32_t)lane * 16u;
-        const uint32_t sf_off = REC_SF + w * 128u + (uint32_t)lane * 4u;
-        const uint32_t a_off = STG_A + (hq * 2u) * 512u + (uint32_t)lane * 16u;
+        const uint32_t sf_off = REC_SF + jr * 512u + (uint32_t)lane * 16u;
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
         const float alpha = FUSED ? __fmul_rn(p.q.s4, __ldg(&reinterpret_cast<const fgmp_packed_header*>(p.wblob)->scale_fp4))
                                   : __fmul_rn(__ldg(&reinterpret_cast<const fgmp_packed_header*>(p.ablob)->scale_fp4),
                                               __ldg(&reinterpret_cast<const fgmp_packed_header*>(p.wblob)->scale_fp4));
-
-        int stage = 0; uint32_t phase = 0;
-        for (int64_t u = u_begin; u < u_end && ok;) {
-            const int64_t tile = u / C;
-            const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
-            // acc[mt][nh] = rows 32jr + 16mt + {g, g + 8} x tokens 8nh + {2t, 2t+1}, block columns == hq (mod 4)
+        bool ok = true;
+        for (int sbeg = 0; sbeg < n_units;) {
+            const int64_t tile = (u_begin + sbeg) / C;
+            const int send = (int)min((int64_t)n_units, (tile + 1) * C - u_begin);
+            // acc[mt][nh] = rows 32jr + 16mt + {g, g + 8} x tokens 8nh + {2t, 2t+1}, this group's units of the tile
             float acc[2][NH][4];
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) acc[mt][nh][0] = acc[mt][nh][1] = acc[mt][nh][2] = acc[mt][nh][3] = 0.f;
-            for (; u < seg_end; ++u) {
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+            for (int i = sbeg + (int)((gq - (uint32_t)sbeg) & (uint32_t)(NG - 1)); i < send; i += GROUPS) {
+                const int stage = i % S; const uint32_t phase = (uint32_t)(i / S) & 1u;
+                if (ok) ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5);
+                if (!ok) break;
+                if (i == 0) FGMP_STAMP(6);
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-                const uint32_t sc4 = *reinterpret_cast<const uint32_t*>(sb + sf_off);
-                const uint4 s01 = *reinterpret_cast<const uint4*>(sb + w4_off);
-                const uint4 s23 = *reinterpret_cast<const uint4*>(sb + w4_off + 512);
-                // scale pairs: byte k of sc4 (flag bit cleared) in both halves, E4M3 -> fp16
-                uint32_t sc2[4];
-                {
-                    const uint32_t s7 = sc4 & 0x7f7f7f7fu;
+                const uint4 scv = *reinterpret_cast<const uint4*>(sb + sf_off);
+                const bool any8 = __any_sync(0xffffffffu, ((scv.x | scv.y | scv.z | scv.w) & 0x80808080u) != 0u);
+                // where this lane's overflow entries start, per hq (only with FP8 blocks in the unit)
+                uint32_t idx4 = 0;
+                if (any8) {
+                    const uint32_t pack = __popc(scv.x & 0x80808080u) | (__popc(scv.y & 0x80808080u) << 8) |
+                                          (__popc(scv.z & 0x80808080u) << 16) | (__popc(scv.w & 0x80808080u) << 24);
+                    uint32_t incl = pack;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint32_t two = __byte_perm(s7, 0u, 0x4400u | (uint32_t)(k << 4) | (uint32_t)k);
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2[k]) : "h"((uint16_t)two));
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += y;
                     }
+                    idx4 = incl - pack;
                 }
-                const uint32_t slot[4][2] = {{s01.x, s01.y}, {s01.z, s01.w}, {s23.x, s23.y}, {s23.z, s23.w}};
-                const uint32_t flags = sc4 & 0x80808080u;
-                // the MMAs of one half (elements 8h .. 8h+7 of every block): x[k] = four fp16 pairs of slot k
-                auto half_mma = [&](int h, const uint32_t (&x)[4][4]) {
-                    uint4 b[NH];
+                const uint32_t staged = smeta[stage].staged;
+                const uint8_t* ovf_g = ovfs + (size_t)smeta[stage].step * 16;
+#pragma unroll 1
+                for (int hq = hq0; hq < hq0 + NG; ++hq) {
+                    const uint32_t w = 4 * jr + (uint32_t)hq;
+                    const uint32_t sc4 = *reinterpret_cast<const uint32_t*>(sb + sf_off + 4 * hq);
+                    const uint4 s01 = *reinterpret_cast<const uint4*>(sb + REC_W4 + w * 1024u + (uint32_t)lane * 16u);
+                    const uint4 s23 = *reinterpret_cast<const uint4*>(sb + REC_W4 + w * 1024u + 512u + (uint32_t)lane * 16u);
+                    const uint32_t a_off = STG_A + (uint32_t)(hq * 2) * 512u + (uint32_t)lane * 16u;
+                    // scale pairs: byte k of sc4 (flag bit cleared) in both halves, E4M3 -> fp16
+                    uint32_t sc2[4];
+                    {
+                        const uint32_t s7 = sc4 & 0x7f7f7f7fu;
 #pragma unroll
-                    for (int nh = 0; nh < NH; ++nh) b[nh] = *reinterpret_cast<const uint4*>(sb + a_off + nh * 4096 + h * 512);
-#pragma unroll
-                    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                        for (int sl = 0; sl < 2; ++sl)
-#pragma unroll
-                            for (int nh = 0; nh < NH; ++nh)
-                                mma_f16_16816(acc[mt][nh], x[2 * mt][2 * sl], x[2 * mt + 1][2 * sl], x[2 * mt][2 * sl + 1], x[2 * mt + 1][2 * sl + 1],
-                                              sl ? b[nh].z : b[nh].x, sl ? b[nh].w : b[nh].y);
-                };
-                if (!__any_sync(0xffffffffu, flags != 0u)) {
-                    // no FP8 block among the warp's 128: every slot holds sixteen E2M1 codes
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t x[4][4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) dq_nvfp4(slot[k][h], sc2[k], x[k]);
-                        half_mma(h, x);
-                    }
-                } else {
-                    // second halves of this lane's FP8 blocks: consecutive entries of the unit's overflow list
-                    uint32_t wtot;
-                    uint32_t idx = fgmp_warp_excl_count(flags, wtot) + *reinterpret_cast<const uint16_t*>(sb + REC_WSTART + 2 * w);
-                    const uint32_t staged = smeta[stage].staged;
-                    const uint8_t* ovf_g = ovfs + (size_t)smeta[stage].step * 16;
-                    uint2 hi8[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        hi8[k] = make_uint2(0u, 0u);
-                        if (flags & (0x80u << (8 * k))) {
-                            hi8[k] = (idx * 8u + 8u <= staged) ? *reinterpret_cast<const uint2*>(sb + STG_OVF + idx * 8u)
-                                                               : __ldg(reinterpret_cast<const uint2*>(ovf_g + (size_t)idx * 8));
-                            ++idx;
+                        for (int k = 0; k < 4; ++k) {
+                            const uint32_t two = __byte_perm(s7, 0u, 0x4400u | (uint32_t)(k << 4) | (uint32_t)k);
+                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2[k]) : "h"((uint16_t)two));
                         }
                     }
-                    // NVFP4: codes 0..7 in slot word 0, 8..15 in word 1; FP8: codes 0..3, 4..7 in the slot, 8..11, 12..15 in the overflow entry
-                    {
-                        uint32_t x[4][4];
+                    const uint32_t slot[4][2] = {{s01.x, s01.y}, {s01.z, s01.w}, {s23.x, s23.y}, {s23.z, s23.w}};
+                    // the MMAs of one half (elements 8h .. 8h+7 of every block): x[k] = four fp16 pairs of slot k
+                    auto half_mma = [&](int h, const uint32_t (&x)[4][4]) {
+                        uint4 b[NH];
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) dq_mixed(slot[k][0], slot[k][0], slot[k][1], flags & (0x80u << (8 * k)), sc2[k], x[k]);
-                        half_mma(0, x);
-                    }
-                    {
-                        uint32_t x[4][4];
+                        for (int nh = 0; nh < NH; ++nh) b[nh] = *reinterpret_cast<const uint4*>(sb + a_off + nh * 4096 + h * 512);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) dq_mixed(slot[k][1], hi8[k].x, hi8[k].y, flags & (0x80u << (8 * k)), sc2[k], x[k]);
-                        half_mma(1, x);
+                        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                            for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+                                for (int nh = 0; nh < NH; ++nh)
+                                    mma_f16_16816(acc[mt][nh], x[2 * mt][2 * sl], x[2 * mt + 1][2 * sl], x[2 * mt][2 * sl + 1], x[2 * mt + 1][2 * sl + 1],
+                                                  sl ? b[nh].z : b[nh].x, sl ? b[nh].w : b[nh].y);
+                    };
+                    if (!any8) {
+                        // no FP8 block in the warp's part of the unit: every slot holds sixteen E2M1 codes
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            uint32_t x[4][4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) dq_nvfp4(slot[k][h], sc2[k], x[k]);
+                            half_mma(h, x);
+                        }
+                    } else {
+                        // second halves of this lane's FP8 blocks: consecutive entries of the unit's overflow list
+                        const uint32_t flags = sc4 & 0x80808080u;
+                        uint32_t idx = ((idx4 >> (8 * hq)) & 0xffu) + *reinterpret_cast<const uint16_t*>(sb + REC_WSTART + 2 * w);
+                        uint2 hi8[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            hi8[k] = make_uint2(0u, 0u);
+                            if (flags & (0x80u << (8 * k))) {
+                                hi8[k] = (idx * 8u + 8u <= staged) ? *reinterpret_cast<const uint2*>(sb + STG_OVF + idx * 8u)
+                                                                   : __ldg(reinterpret_cast<const uint2*>(ovf_g + (size_t)idx * 8));
+                                ++idx;
+                            }
+                        }
+                        // NVFP4: codes 0..7 in slot word 0, 8..15 in word 1; FP8: codes 0..3, 4..7 in the slot, 8..11, 12..15 in the overflow entry
+                        {
+                            uint32_t x[4][4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) dq_mixed(slot[k][0], slot[k][0], slot[k][1], flags & (0x80u << (8 * k)), sc2[k], x[k]);
+                            half_mma(0, x);
+                        }
+                        {
+                            uint32_t x[4][4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) dq_mixed(slot[k][1], hi8[k].x, hi8[k].y, flags & (0x80u << (8 * k)), sc2[k], x[k]);
+                            half_mma(1, x);
+                        }
                     }
                 }
+                // this warp is done with the stage; the group's last warp to say so refills it with the unit S further on
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-                if (++stage == S) { stage = 0; phase ^= 1; }
+                if (lane == 0) {
+                    uint32_t old;
+                    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(smem_u32(done + stage)) : "memory");
+                    if (old == GROUP_WARPS - 1) {
+                        done[stage] = 0;
+                        const int nxt = i + S;
+                        if (nxt < n_units) {
+                            const uint32_t step0 = table[nxt], bytes = (table[nxt + 1] - step0) * 16u;
+                            mbar_expect_tx(full0 + 8 * stage, REC_BYTES + A_BYTES + (bytes < OVF_CAP ? bytes : OVF_CAP));
+                            issue_rec(nxt, stage); issue_ovf(nxt, stage, false); issue_a(nxt, stage);
+                        }
+                    }
+                }
             }
-            if (!ok) break;
 
-            // ---- end of a segment (this CTA's units of one tile): the four column classes are added, then the
-            // tile is written or, if other CTAs share it, handed in; the last CTA to arrive adds the parts in order
+            // ---- end of a segment (this CTA's units of one tile): the groups' sums are added, then the tile is
+            // written or, if other CTAs share it, handed in; the last CTA to arrive adds the parts in order.
+            // (After a failed wait the barriers below are still passed by everyone; nothing is written.)
+            if (send == n_units) { FGMP_STAMP(7); if (threadIdx.x == DEC_THREADS - 32) FGMP_STAMP_ANY(8); }
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
                 for (int rh = 0; rh < 2; ++rh) {
                     const uint32_t r = 32 * jr + 16 * (uint32_t)mt + 8 * (uint32_t)rh + g;
-                    float2* pt = reinterpret_cast<float2*>(epi + hq * 2048u + r * 16u + (((tpiece ^ (r >> 1)) & 3u) << 2) + tcol);
+                    float2* pt = reinterpret_cast<float2*>(epi + part * 2048u + r * 16u + (((tpiece ^ (r >> 1)) & 3u) << 2) + tcol);
                     pt[0] = make_float2(acc[mt][0][2 * rh], acc[mt][0][2 * rh + 1]);
                     if (NH == 2)
                         *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pt) ^ 32) = make_float2(acc[mt][NH - 1][2 * rh], acc[mt][NH - 1][2 * rh + 1]);
                 }
             math_bar();
+            const bool good = !*abort_flag;
             const uint32_t row = threadIdx.x >> 2, tq = threadIdx.x & 3u;      // this thread: tokens 4tq .. 4tq+3 of one row
             const bool live = tq < 2u * NH;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -439,18 +473,19 @@ decode_kernel(DecParams p)
                     v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
                 }
             }
-            const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
+            const bool whole = (u_begin + sbeg == tile * C) && (u_begin + send == (tile + 1) * C);
             bool write_out = whole;
             if (!whole) {
                 const int64_t c_first = cta_of_unit(tile * C, G, p.total);
                 const int64_t c_last = cta_of_unit((tile + 1) * C - 1, G, p.total);
                 const int nseg = (int)(c_last - c_first + 1), slot_i = (int)(blockIdx.x - c_first);
-                if (live) __stcg(reinterpret_cast<float4*>(p.partials + (((size_t)tile * p.maxseg + slot_i) * 128 + row) * 16 + 4 * tq), v);
+                if (live && good) __stcg(reinterpret_cast<float4*>(p.partials + (((size_t)tile * p.maxseg + slot_i) * 128 + row) * 16 + 4 * tq), v);
                 __threadfence();
                 math_bar();
                 // the counter wraps to zero with the last arrival, so the workspace is ready for the next call
-                if (threadIdx.x == 0) s_misc[3] = atomicInc(p.counters + tile, (uint32_t)(nseg - 1)) == (uint32_t)(nseg - 1) ? 1u : 0u;
+                if (threadIdx.x == 0) s_misc[3] = (good && atomicInc(p.counters + tile, (uint32_t)(nseg - 1)) == (uint32_t)(nseg - 1)) ? 1u : 0u;
                 math_bar();
+                write_out = false;
                 if (s_misc[3]) {
                     __threadfence();
                     v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -463,7 +498,7 @@ decode_kernel(DecParams p)
                 }
             }
             const int64_t n = tile * 128 + row;
-            if (write_out && live && n < p.N) {
+            if (write_out && good && live && n < p.N) {
                 const float y[4] = {v.x * alpha, v.y * alpha, v.z * alpha, v.w * alpha};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -475,10 +510,12 @@ decode_kernel(DecParams p)
                 }
             }
             math_bar();                                // the next segment's sums overwrite the tile
+            sbeg = send;
         }
     }
 
     __syncthreads();
+    FGMP_STAMP(9);
     if (*abort_flag) {
         const unsigned long long t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
@@ -490,7 +527,7 @@ decode_kernel(DecParams p)
     }
 }
 
-struct DecPlan { int64_t tiles, chunks, total; int grid; int maxseg; };
+struct DecPlan { int64_t tiles, chunks, total; int grid; int maxseg; int64_t span; };
 
 DecPlan decode_plan(int64_t N, int64_t K)
 {
@@ -501,6 +538,7 @@ DecPlan decode_plan(int64_t N, int64_t K)
     // a tile of `chunks` units meets at most this many CTA spans of >= floor(total/grid) units
     const int64_t span = d.total / d.grid;
     d.maxseg = (int)((d.chunks + span - 1) / span + 1);
+    d.span = (d.total + d.grid - 1) / d.grid;           // the longest span of a CTA
     return d;
 }
 
@@ -513,11 +551,15 @@ fgmp_status set_attrs_once()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
     std::lock_guard<std::mutex> lk(g_dec_mu);
     if (!g_attr_set[dev]) {
-        if (cudaFuncSetAttribute(decode_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(decode_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess)
+        const int most = 232448;
+#define FGMP_SET(NG_) \
+        if (cudaFuncSetAttribute(decode_kernel<1, false, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess || \
+            cudaFuncSetAttribute(decode_kernel<2, false, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess || \
+            cudaFuncSetAttribute(decode_kernel<1, true, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess || \
+            cudaFuncSetAttribute(decode_kernel<2, true, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess) \
             return FGMP_ERR_CUDA;
+        FGMP_SET(1) FGMP_SET(2) FGMP_SET(4)
+#undef FGMP_SET
         g_attr_set[dev] = true;
     }
     return FGMP_OK;
@@ -543,7 +585,8 @@ DecParams base_params(const void* packed_weights, void* Y, int y_is_bf16, int64_
     p.maxseg = d.maxseg;
     // Ring depth: long spans are bound by the weight stream and want every stage; short ones are bound by
     // set-up, which a smaller footprint shortens.
-    p.stages = (d.total / d.grid >= 24) ? DEC_STAGES : DEC_STAGES - 1;
+    p.stages = DEC_STAGES;
+    while (p.stages > 2 && dec_smem(p.stages, d.span) > 232448) --p.stages;      // very long spans: their table takes the room of a stage
     return p;
 }
 
@@ -551,13 +594,17 @@ template <bool FUSED>
 fgmp_status launch_decode(const DecParams& p, const DecPlan& d, bool programmatic, cudaStream_t s)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = dec_smem(p.stages); cfg.stream = s;
+    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = dec_smem(p.stages, d.span); cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = programmatic ? 1 : 0;
-    if (p.M <= 8) { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<1, FUSED>, p)); }
-    else          { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<2, FUSED>, p)); }
+    const int ng = 4;       // measured on Llama-2 shapes: four groups of four warps are the fastest split
+#define FGMP_GO(NG_) \
+    if (p.M <= 8) { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<1, FUSED, NG_>, p)); } \
+    else          { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<2, FUSED, NG_>, p)); }
+    if (ng == 1) { FGMP_GO(1) } else if (ng == 4) { FGMP_GO(4) } else { FGMP_GO(2) }
+#undef FGMP_GO
     return fgmp_launch_status();
 }
 
@@ -565,8 +612,11 @@ fgmp_status launch_decode(const DecParams& p, const DecPlan& d, bool programmati
 
 bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K)
 {
-    return M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0 &&
-           1024 + ((N + 127) / 128) * 4 <= (int64_t)FGMP_WS_CONTROL_BYTES;
+    if (!(M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0 &&
+          1024 + ((N + 127) / 128) * 4 <= (int64_t)FGMP_WS_CONTROL_BYTES)) return false;
+    const int64_t total = ((N + 127) / 128) * (K / 256);
+    const int sms = fgmp_sm_count();
+    return (total + sms - 1) / sms <= MAX_SPAN;
 }
 
 size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K)
@@ -643,6 +693,13 @@ extern "C" fgmp_status fgmp_linear_fused(const void* X_bf16, int64_t ldx, const 
     }
     return launch_decode<true>(p, d, true, (cudaStream_t)cuda_stream);
 }
+
+#ifdef FGMP_TIMELINE
+extern "C" int fgmp_debug_timeline(unsigned long long* buffer)
+{
+    return cudaMemcpyToSymbol(g_timeline, &buffer, sizeof(buffer)) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 // ------------------------------------------------------------------ allocation-free variant
 // Scratch of fgmp_linear_static: one array per GPU that loads the library, held until exit.

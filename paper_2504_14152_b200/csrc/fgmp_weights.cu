@@ -361,7 +361,7 @@ __global__ void __launch_bounds__(512) w_emit_kernel(const uint4* W, int64_t ldw
         *reinterpret_cast<uint2*>(rec + REC_W4 + w * 1024u + (k >> 1) * 512u + lane * 16u + (k & 1u) * 8u) = slot;
         sc4 |= scale << (8 * k);
     }
-    *reinterpret_cast<uint32_t*>(rec + REC_SF + w * 128u + lane * 4u) = sc4;
+    *reinterpret_cast<uint32_t*>(rec + REC_SF + (w >> 2) * 512u + lane * 16u + (w & 3u) * 4u) = sc4;
 }
 
 // With too little room the starts of the overflow entries are pulled back inside the blob, so that a

@@ -62,7 +62,7 @@ def test_weight_record_maps_are_bijections(maps):
         assert (r_back, j_back) == (r, j)
         # a warp's slots: 1 KiB, two 512-byte halves (k // 2) of 16 bytes per lane (two slots side by side)
         assert o4 == w * 1024 + (k // 2) * 512 + lane * 16 + (k % 2) * 8
-        assert osf == w * 128 + lane * 4 + k
+        assert osf == (w // 4) * 512 + lane * 16 + (w % 4) * 4 + k     # a lane's sixteen scale bytes of a row group: one 16-byte load
         assert order == (w * 32 + lane) * 4 + k
     # one warp-wide 16-byte load per half reads 512 contiguous bytes: no bank conflicts
     for w in range(16):
