@@ -12,38 +12,39 @@
 // ---------------------------------------------------------------- blob layout
 // A "unit" is one 128-row tile x one chunk of 16 blocks (256 K elements).
 //
-// Weights (kind 1): header | mask | uptr | records | overflow.  A unit's record has a fixed size and
+// Weights (kind 1): header | mask | uptr | records | lists.  A unit's record has a fixed size and
 // sits at a fixed place, so that it streams from HBM with one bulk copy whose address needs no
-// look-up; what does not fit the fixed part (the second half of every FP8 block) follows in the
-// overflow section, found through uptr.  Inside a record the blocks are in the order in which the
-// decode GEMM's warps take them: warp w = 4*(r/32) + j%4 owns rows 32*(r/32) .. +31 and the block
-// columns j with j%4 == w%4; its lane 4*(r%8) + j/4 holds, as slot k = (r/8)%4, block (r, j).
-//   REC_W4    16384 B : one 8-byte slot per block at w*1024 + (k/2)*512 + lane*16 + (k%2)*8: the 16 E2M1
-//                       codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block
-//   REC_SF     2048 B : one byte per block at (w/4)*512 + lane*16 + (w%4)*4 + k (the sixteen blocks of one
-//                       lane of the four warps of a row group side by side): the E4M3 microscale (bit 7 clear) of an
-//                       NVFP4 block; for an FP8 block 0x80 | E4M3(2^fp8_log2_ratio), i.e. bit 7 is the
-//                       block's precision flag and the low bits the factor between the tensor scales
-//   REC_WSTART  128 B : uint16 x 17: FP8 blocks of the unit that precede warp w's in (w, lane, k)
-//                       order; entry 16 = all of them
-// Overflow of a unit: E4M3 codes 8..15 of its FP8 blocks, 8 bytes each, in (w, lane, k) order, padded
-// to 16 bytes; uptr[u] (uint32, units + 1 entries) = its start in 16-byte steps from off_ovf.
+// look-up; the list of its FP8 blocks follows in the lists section, found through uptr.
+//   REC_W4    16384 B : one 8-byte slot per block, row r of the tile = 128 bytes whose 16-byte pieces are
+//                       XOR-swizzled with (r & 7) -- the 128B-swizzled K-major tile tcgen05 reads: the 16
+//                       E2M1 codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block (which the tensor
+//                       core ignores because the block's scale byte is zero); zero in rows beyond the tensor
+//   REC_SF     2048 B : E4M3 microscales, 0x00 for FP8 blocks, in the order the scales go to tensor
+//                       memory: four 512-byte tiles (one per MMA step of 64 elements), in a tile 16 bytes
+//                       per r % 32, there 4 bytes per r / 32, there one byte per block of the step
+//   REC_KBSTART 128 B : uint16 x 17 (padded): FP8 blocks of the unit before block column j; entry 16 = all
+// List of a unit with cnt FP8 blocks, ordered by (block column, row) so that blocks meeting the same 16
+// activation elements are neighbours: the row of every block (cnt bytes, padded to 16), then E4M3 codes
+// 8..15 of every block (8 bytes each, padded to 16).  uptr[u] (uint32, units + 1 entries) = start of
+// unit u's list in 16-byte steps from off_ovf.
 //
 // Activations (kind 0): header | codes4 | sf | mask | arec | codes8.  codes4 is row-major, sf
 // uses 512-byte tiles over all rows, codes8 is a dense plane of which only FP8 blocks are
-// written.  arec exists when rows <= 16: one record of AREC_BYTES per chunk holding the fp16 value
-// over the tensor scale (E2M1 x microscale, or E4M3 x 2^ratio; exact) of 16 token rows (rows >= M
-// are zero), in the order the decode GEMM's mma.sync fragments take them: token octet o = m/8 in
-// its own half of 4096 bytes; there 8 pieces of 512 bytes, piece 2*(j%4) + half holding elements
-// 8*half .. 8*half+7 of block column j of token m for lane 4*(m%8) + j/4, 16 bytes per lane.
-constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_WSTART = 18432, REC_BYTES = 18560;
-constexpr uint32_t AREC_BYTES = 8192;
+// written.  arec exists when rows <= 16: one record of AREC_BYTES per chunk for the decode GEMM, 16
+// token rows (rows >= M are zero):
+//   AREC_A4   2048 B : the E2M1 codes as a 16-row x 128-byte tile, swizzled like REC_W4 (zero in FP8 blocks)
+//   AREC_SF    256 B : E4M3 microscales, [token][block column], 0x00 for FP8 blocks
+//   AREC_HOT    16 B : uint32: bit j set if block column j of some token is FP8 ("hot" column), then padding
+//   AREC_AT   8192 B : the value over the tensor scale of every element in fp16 (E2M1 x microscale, or E4M3 x
+//                      2^ratio; exact): token octet m / 8 in its own 4096 bytes, there 256 bytes per block
+//                      column, there 32 bytes per token -- what a warp reads for one column is contiguous
+constexpr uint32_t REC_W4 = 0, REC_SF = 16384, REC_KBSTART = 18432, REC_BYTES = 18560;
+constexpr uint32_t AREC_A4 = 0, AREC_SF = 2048, AREC_HOT = 2304, AREC_AT = 2560, AREC_BYTES = 10752;
 
-// byte offset, inside an activation record, of the first (half = 0) or second (half = 1) 8 elements
-// of block column j (0..15) of token row m
-__host__ __device__ inline uint32_t fgmp_arec_offset(uint32_t m, uint32_t j, uint32_t half)
+// byte offset, inside an activation record, of the fp16 values of block column j (0..15) of token row m
+__host__ __device__ inline uint32_t fgmp_arec_at_offset(uint32_t m, uint32_t j)
 {
-    return ((m >> 3) << 12) + (((((j & 3u) << 1) | half)) << 9) + ((((m & 7u) << 2) | (j >> 2)) << 4);
+    return AREC_AT + ((m >> 3) << 12) + (j << 8) + ((m & 7u) << 5);
 }
 
 struct PackedLayout {
@@ -56,10 +57,11 @@ struct PackedLayout {
 
 __host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 
-// overflow of a unit with cnt FP8 blocks, in 16-byte steps
-__host__ __device__ inline uint32_t fgmp_ovf_steps(uint32_t cnt) { return (cnt + 1u) >> 1; }
+// list of a unit with cnt FP8 blocks: where the second halves start, and its size in 16-byte steps
+__host__ __device__ inline uint32_t fgmp_list_halves_offset(uint32_t cnt) { return (cnt + 15u) & ~15u; }
+__host__ __device__ inline uint32_t fgmp_list_steps(uint32_t cnt) { return (fgmp_list_halves_offset(cnt) + ((cnt * 8u + 15u) & ~15u)) >> 4; }
 
-// kind 0 = activations, 1 = weights (max_fp8 = room for that many FP8 blocks in the overflow section)
+// kind 0 = activations, 1 = weights (max_fp8 = room for that many FP8 blocks in the lists section)
 __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int kind, int64_t max_fp8)
 {
     PackedLayout L;
@@ -77,8 +79,8 @@ __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int
         L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
         L.off_uptr = o;    o = fgmp_align1k(o + ((size_t)L.units + 1) * 4);
         L.off_rec = o;     o = fgmp_align1k(o + (size_t)L.units * REC_BYTES);
-        // 8 bytes per FP8 block, and up to 8 bytes of padding per unit
-        L.off_ovf = o;     o = fgmp_align1k(o + (size_t)max_fp8 * 8 + (size_t)L.units * 8);
+        // 9 bytes per FP8 block, and up to 30 bytes of padding per unit
+        L.off_ovf = o;     o = fgmp_align1k(o + (size_t)max_fp8 * 9 + (size_t)L.units * 32);
     }
     L.total = o;
     return L;
@@ -91,33 +93,47 @@ __host__ __device__ inline size_t fgmp_sf_offset(int64_t r, int64_t kb, int64_t 
          + (size_t)(r & 31) * 16 + (size_t)((r & 127) >> 5) * 4 + (size_t)(kb & 3);
 }
 
-// inside a record (r = row in the tile, j = block column in the chunk): who holds the block ...
-__host__ __device__ inline uint32_t fgmp_rec_warp(uint32_t r, uint32_t j) { return ((r >> 5) << 2) | (j & 3u); }
-__host__ __device__ inline uint32_t fgmp_rec_lane(uint32_t r, uint32_t j) { return ((r & 7u) << 2) | (j >> 2); }
-__host__ __device__ inline uint32_t fgmp_rec_slot(uint32_t r, uint32_t j) { (void)j; return (r >> 3) & 3u; }
-// ... where its 8-byte slot and its scale byte sit, and its rank in the order of the overflow entries
+// inside a record or the A4 tile of an activation record (r = row in the tile, j = block column in the
+// chunk): the 8-byte slot and the scale byte
 __host__ __device__ inline uint32_t fgmp_rec_w4_offset(uint32_t r, uint32_t j)
 {
-    const uint32_t k = fgmp_rec_slot(r, j);
-    return fgmp_rec_warp(r, j) * 1024u + (k >> 1) * 512u + fgmp_rec_lane(r, j) * 16u + (k & 1u) * 8u;
+    return r * 128u + (((j >> 1) ^ (r & 7u)) << 4) + (j & 1u) * 8u;
 }
 __host__ __device__ inline uint32_t fgmp_rec_sf_offset(uint32_t r, uint32_t j)
 {
-    const uint32_t w = fgmp_rec_warp(r, j);
-    return (w >> 2) * 512u + fgmp_rec_lane(r, j) * 16u + (w & 3u) * 4u + fgmp_rec_slot(r, j);
+    return (j >> 2) * 512u + (r & 31u) * 16u + (r >> 5) * 4u + (j & 3u);
 }
-__host__ __device__ inline uint32_t fgmp_rec_order(uint32_t r, uint32_t j)
-{
-    return ((fgmp_rec_warp(r, j) * 32u + fgmp_rec_lane(r, j)) << 2) | fgmp_rec_slot(r, j);
-}
-// the inverse: row and block column of slot k of lane `lane` of warp w
-__host__ __device__ inline uint32_t fgmp_rec_row(uint32_t w, uint32_t lane, uint32_t k) { return ((w >> 2) << 5) + (k << 3) + (lane >> 2); }
-__host__ __device__ inline uint32_t fgmp_rec_col(uint32_t w, uint32_t lane) { return ((lane & 3u) << 2) | (w & 3u); }
-
-// E4M3 code of 2^ratio, -7 <= ratio <= 7 (2^-7 is subnormal)
-__host__ __device__ inline uint32_t fgmp_pow2_e4m3(int ratio) { return ratio >= -6 ? (uint32_t)(ratio + 7) << 3 : 0x04u; }
 
 #ifdef __CUDACC__
+// Where the FP8 blocks of one unit sit in its list.  Called by all 128 threads of a CTA, thread
+// i = row i of the tile, m16 = that row's 16 mask bits of the chunk (0 beyond the last row).
+// On return s_pos[row * 16 + j] = index of block (row, j) among the unit's FP8 blocks in (column, row)
+// order (0xffff if the block is not FP8), s_cnt[j] = FP8 blocks in column j, and the return value is
+// their total.  s_warp is scratch of 64 words.  Ends with a __syncthreads().
+__device__ __forceinline__ uint32_t fgmp_unit_positions(uint32_t m16, uint32_t* s_warp, uint16_t* s_pos, uint32_t* s_cnt)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t rank[16];
+#pragma unroll
+    for (int kb = 0; kb < 16; ++kb) {
+        const uint32_t bal = __ballot_sync(0xffffffffu, (m16 >> kb) & 1u);
+        rank[kb] = __popc(bal & ((1u << lane) - 1u));
+        if (lane == 0) s_warp[w * 16 + kb] = __popc(bal);
+    }
+    __syncthreads();
+    uint32_t run = 0;
+#pragma unroll
+    for (int kb = 0; kb < 16; ++kb) {
+        const uint32_t c0 = s_warp[kb], c1 = s_warp[16 + kb], c2 = s_warp[32 + kb], c3 = s_warp[48 + kb];
+        const uint32_t below = (w > 0 ? c0 : 0u) + (w > 1 ? c1 : 0u) + (w > 2 ? c2 : 0u);
+        s_pos[threadIdx.x * 16 + kb] = ((m16 >> kb) & 1u) ? (uint16_t)(run + below + rank[kb]) : (uint16_t)0xffff;
+        if (threadIdx.x == 0) s_cnt[kb] = c0 + c1 + c2 + c3;
+        run += c0 + c1 + c2 + c3;
+    }
+    __syncthreads();
+    return run;
+}
+
 // the 16 mask bits of (row r, chunk c) of a packed tensor; 0 beyond the last row
 __device__ __forceinline__ uint32_t fgmp_chunk_mask(const uint32_t* mask, const PackedLayout& L, int64_t r, int64_t c)
 {
@@ -125,38 +141,32 @@ __device__ __forceinline__ uint32_t fgmp_chunk_mask(const uint32_t* mask, const 
     return (mask[r * L.MW + (c >> 1)] >> ((c & 1) * 16)) & 0xffffu;
 }
 
-// Kernels that walk a unit in record order run 512 threads per unit: thread = (warp w, lane), four
-// slots each.  Exclusive prefix over the lanes of a warp of the number of flagged slots (flags = the
-// bits 0x80808080 of the lane's four scale bytes, or any word with one bit per flagged slot).
-__device__ __forceinline__ uint32_t fgmp_warp_excl_count(uint32_t flags, uint32_t& warp_total)
-{
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t cnt = __popc(flags);
-    uint32_t incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= (uint32_t)o) incl += y;
-    }
-    warp_total = __shfl_sync(0xffffffffu, incl, 31);
-    return incl - cnt;
-}
+struct UnitScratch { uint32_t warp[64]; uint32_t cnt[16]; uint16_t pos[128 * 16]; };
 
-// What thread (w, lane) of a 512-thread CTA needs to read its four blocks of one unit of a packed
-// weight tensor: the record, the unit's overflow entries, the lane's four scale bytes and the index
-// of the overflow entry of its first FP8 block (its further FP8 blocks follow, in slot order).
-struct UnitLaneView { const uint8_t* rec; const uint8_t* ovf; uint32_t sc4, idx; };
-__device__ __forceinline__ UnitLaneView fgmp_unit_lane(const uint8_t* blob, const PackedLayout& L, int64_t unit)
+// Visits every block of one unit of a packed weight tensor, 128 threads per unit, consecutive
+// threads on consecutive blocks of one row: f(row, kb, row in tile, column in chunk, rec, hi) with
+// rec = the unit's record and hi = address of E4M3 codes 8..15 of an FP8 block (codes 0..7 are in its
+// slot), or nullptr if the block is NVFP4.
+template <class F>
+__device__ __forceinline__ void fgmp_for_each_block(const uint8_t* blob, const PackedLayout& L, int64_t unit,
+                                                    UnitScratch& sc, F f)
 {
-    UnitLaneView v;
-    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    v.rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
-    v.ovf = blob + L.off_ovf + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[unit] * 16;
-    v.sc4 = *reinterpret_cast<const uint32_t*>(v.rec + REC_SF + (w >> 2) * 512u + lane * 16u + (w & 3u) * 4u);
-    uint32_t total;
-    const uint32_t excl = fgmp_warp_excl_count(v.sc4 & 0x80808080u, total);
-    v.idx = reinterpret_cast<const uint16_t*>(v.rec + REC_WSTART)[w] + excl;
-    return v;
+    const int64_t tile = unit / L.chunks, c = unit % L.chunks;
+    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    const uint8_t* rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
+    const uint8_t* halves = blob + L.off_ovf + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[unit] * 16 + fgmp_list_halves_offset(cnt);
+    const int j = threadIdx.x & 15;
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i) {
+        const int row = (threadIdx.x >> 4) + 8 * i;
+        const int64_t r = tile * 128 + row, kb = c * 16 + j;
+        if (r >= L.rows || kb >= L.KB) continue;
+        const uint32_t pos = sc.pos[row * 16 + j];
+        f(r, kb, row, j, rec, pos != 0xffffu ? halves + (size_t)pos * 8 : (const uint8_t*)nullptr);
+    }
+    __syncthreads();
 }
 #endif
 

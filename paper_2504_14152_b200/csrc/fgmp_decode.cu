@@ -3,52 +3,76 @@
 // products, FP32 accumulation), optionally with the activation quantizer of Section 4.2 in
 // its prologue (fgmp_linear_fused).
 //
-// At this size the layer is bound by the weight stream, not by arithmetic, and every block pair
-// has an exact fp16 form: an E2M1 code times its E4M3 microscale has 6 significant bits, an E4M3
-// code times the power of two between the tensor scales has 4.  So both operands go through
-// mma.sync m16n8k16 (fp16 in, fp32 accumulation) as their true values over the tensor scales.
-// 16 weight rows are the M side of an MMA, a token octet the N side.  The order of the contraction
-// index is free as long as both operands agree, so an MMA step takes four consecutive elements of
-// one block per lane: lane (g, t) owns, for hq = 0..3, block column 4t + hq of rows 32jr + 8k + g,
-// k = 0..3, of the unit, and its four MMA steps per 16-row tile walk through that block.  A lane
-// therefore meets whole blocks, and the format of a block is a per-lane choice between two
-// conversion instructions (cvt e2m1x2 / cvt e4m3x2, predicated on the block's flag) followed by the
-// same multiply with the block's scale byte (the microscale, or 2^ratio for an FP8 block): the
-// mixing of formats costs conversions, not extra MMAs, and all sums stay in registers.
-// The record of a unit is stored in exactly this order (fgmp_common.cuh), so every shared-memory read
-// of a warp is one contiguous, conflict-free piece; the activation record of a chunk likewise.
+// At this size the layer is bound by the weight stream.  Converting packed codes to a common number
+// format in the SIMT pipes costs more instructions per byte than the stream leaves time for (an E2M1
+// pair takes a byte extraction, a conversion and a scale multiply), so the bulk of the products must
+// not be converted at all.  Decomposition (exact), with the FP8 blocks as the exceptions:
+//   (1) NVFP4 weight block x NVFP4 activation block: tcgen05.mma kind::mxf4nvf4 straight from the
+//       packed codes, E4M3 block scales in tensor memory, FP32 accumulation there; weights are the
+//       128-row operand, the 16 tokens are N.  A block that must not take part gets a zero scale: the
+//       record stores scale 0 for FP8 weight blocks, the activation record for FP8 activation blocks,
+//       and the scales of every token are zeroed in "hot" block columns (those in which some token of
+//       the batch is FP8), which are left to (3) as a whole.
+//   (2) FP8 weight block x any activation block: mma.sync m16n8k16 on exact fp16 values (an E4M3 code
+//       has 4 significant bits; the activation record holds every activation over its tensor scale in
+//       fp16, exact for either format).  A record lists its FP8 blocks by block column, so sixteen
+//       blocks that meet the same 16 activation elements form the M side; the sums are added to their
+//       rows in a [row][token] tile private to the warp.
+//   (3) NVFP4 weight block x any activation block in a hot column: the column's weights are dequantized
+//       in registers (exact in fp16: 6 significant bits) for mma.sync, 32 rows per warp, sums in registers.
+// Every block pair is in exactly one of the three.  With 10 % FP8 blocks that concentrate in few block
+// columns (outlier channels) (2) and (3) are small; with unstructured activation masks (3) grows towards
+// the whole tensor and the kernel is as fast as its SIMT conversions allow.
 //
 // Work is split stream-K style over (128-row tile, 256-element K chunk) units so that all SMs
-// stream the same number of bytes; a unit is up to three bulk copies (its fixed-size record, the
-// second halves of its FP8 blocks, the activation record of its chunk) into a ring of stages.
-// The 16 warps form four groups; consecutive units of a CTA go to consecutive groups, so four units
-// are being multiplied at any time and the latencies of one (barrier, shared-memory loads, the
-// dependent MMAs) hide behind the others.  Inside a group warp jr takes rows 32jr .. 32jr+31.  There
-// is no producer warp: the warp that is last to finish a unit refills its stage.  Tiles shared by
-// several CTAs are reduced in a fixed order by the CTA that arrives last.  Every sum is taken in a
-// fixed order: results are reproducible bit for bit.
+// stream the same number of bytes; a unit is three bulk copies (its fixed-size record, the list of
+// its FP8 blocks, the activation record of its chunk) into a ring of stages.  Tiles shared by several
+// CTAs are reduced in a fixed order by the CTA that arrives last.  Every sum is taken in a fixed
+// order: results are reproducible bit for bit.
+//
+// Warp roles (576 threads): warp 0 = producer, warp 1 = MMA issuer and owner of the tensor memory,
+// warps 2-5 = block scales into tensor memory (one lane quadrant each), warps 6-9 = (2), four block
+// columns each, warps 10-13 = (3), 32 rows each, warps 14-17 = epilogue (one lane quadrant each).
 #include "fgmp_common.cuh"
 #include "fgmp_actq.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
 #include <cuda_fp16.h>
+#include <cstdio>
 #include <mutex>
 #include <type_traits>
 
 namespace {
 
-constexpr int MATH_WARPS = 16, MATH_THREADS = 32 * MATH_WARPS;
-constexpr int DEC_THREADS = MATH_THREADS;
-constexpr uint32_t OVF_CAP = 2560;              // overflow bytes of a unit that fit a stage (320 FP8 blocks); more are read from global
-constexpr uint32_t STG_OVF = REC_BYTES;
-constexpr uint32_t STG_A = STG_OVF + OVF_CAP;                                                    // 21120
-constexpr uint32_t DEC_STAGE_BYTES = STG_A + AREC_BYTES;                                         // 29312
-constexpr int DEC_STAGES = 6;                   // at most; a launch uses DecParams::stages of them
-constexpr uint32_t EPI_FLOATS = 4 * 128 * 16;   // [warp / 4][row][token] fp32: the partial sums of a tile
-constexpr int MAX_SPAN = 8192;                  // units of one CTA whose overflow starts fit the shared-memory table
-constexpr size_t dec_smem(int stages, int64_t span) { return (size_t)stages * DEC_STAGE_BYTES + EPI_FLOATS * 4 + ((size_t)(span + 1) * 4 + 15) / 16 * 16 + 1024 /*alignment*/ + 512 /*barriers*/; }
-static_assert(dec_smem(DEC_STAGES, 64) <= 232448, "shared memory of one CTA");
-static_assert((STG_A % 128) == 0 && (DEC_STAGE_BYTES % 128) == 0, "bulk-copy alignment");
+constexpr int DEC_WARPS = 18, DEC_THREADS = 32 * DEC_WARPS;
+constexpr int W_PROD = 0, W_MMA = 1, W_SCALE = 2, W_FP8 = 6, W_HOT = 10, W_EPI = 14;
+constexpr int Q_THREADS = 32 * 16;              // warps 2..17 share out the prologue quantizer
+constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
+constexpr uint32_t LIST_CAP = 2944;             // bytes of a unit's FP8 list that fit a stage (about 320 blocks); more is read from global
+constexpr uint32_t STG_LIST = REC_BYTES;                                                         // 18560
+constexpr uint32_t STG_A = STG_LIST + LIST_CAP;                                                  // 21504, 1 KiB aligned
+constexpr uint32_t DEC_STAGE_BYTES = 32768;
+constexpr int DEC_STAGES = 5;
+constexpr int NTILES = 5;                       // [row][token] fp32 tiles: one per (2) warp, one shared by the (3) warps
+constexpr uint32_t TILE_FLOATS = 128 * TOK;
+constexpr uint32_t SF_COL0 = 32;                // tensor memory: 2 x 16 accumulator columns, then 32 scale columns per stage
+constexpr uint32_t DEC_TMEM_COLS = 256;
+constexpr size_t DEC_SMEM = (size_t)DEC_STAGES * DEC_STAGE_BYTES + NTILES * TILE_FLOATS * 4 + 1024 /*alignment*/ + 512 /*barriers*/;
+static_assert(STG_A % 1024 == 0 && STG_A + AREC_BYTES <= DEC_STAGE_BYTES, "stage layout");
+static_assert(DEC_SMEM <= 232448, "shared memory of one CTA");
+static_assert(SF_COL0 + 32 * DEC_STAGES <= DEC_TMEM_COLS, "tensor memory columns");
+
+// kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, N = 16, dense K = 64
+constexpr uint32_t IDESC_NVF4 = (1u << 7) | (1u << 10) | ((uint32_t)(TOK >> 3) << 17) | (0u << 23) | ((uint32_t)(128 >> 4) << 24);
+
+// shared-memory matrix descriptors as (low word | start address >> 4, constant high word)
+constexpr uint32_t SW128_LO = 1u << 16, SW128_HI = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128B swizzle, 8-row groups 1 KiB apart
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
 
 // control words of the workspace (int32, from byte 256): see fgmp_linear_fused
 enum { CW_EPOCH = 0, CW_DONE = 1, CW_CLAIM = 2, CW_QCOUNT = 3, CW_QREADY = 4 };
@@ -61,64 +85,36 @@ struct DecParams {
     int64_t total;            // tiles * chunks
     int64_t chunks;
     int* status; uint32_t* counters; float* partials; int maxseg;
-    int stages;               // depth of the unit ring, 2 .. DEC_STAGES
     // activation quantizer in the prologue (fused launches only)
     const uint8_t* X; int64_t ldx;        // bf16 [M, ldx]
     const float* fisher;
     ActQuantScalars q; int q_mode;        // q_mode: fgmp_score_mode
-    uint8_t* arec;                        // where the fp16 records of the chunks go (and are streamed from)
+    uint8_t* arec;                        // where the records of the chunks go (and are streamed from)
     uint8_t* q_codes4; uint8_t* q_sf; uint8_t* q_mask; uint8_t* q_codes8; fgmp_packed_header* q_header;   // optional packed output
     uint32_t* cw;                         // control words
 };
 
-struct StageMeta { uint32_t step, staged; };
+struct StageMeta { uint32_t step, staged; };     // list start (16-byte steps), bytes of it in the stage
 
 // Profiling builds (-DFGMP_TIMELINE) stamp the global timer at the phases of every CTA into a buffer
 // registered with fgmp_debug_timeline (16 x uint64 per CTA); ordinary builds contain none of this.
 #ifdef FGMP_TIMELINE
 __device__ unsigned long long* g_timeline = nullptr;
-#define FGMP_STAMP(slot) do { if (g_timeline && threadIdx.x == 0) g_timeline[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
 #define FGMP_STAMP_ANY(slot) do { if (g_timeline) g_timeline[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
 #else
-#define FGMP_STAMP(slot) do { } while (0)
 #define FGMP_STAMP_ANY(slot) do { } while (0)
-#endif     // overflow start (16-byte steps), bytes of it in the stage
+#endif
 
 __device__ __forceinline__ int64_t cta_of_unit(int64_t i, int64_t G, int64_t total) { return ((i + 1) * G - 1) / total; }
 
-__device__ __forceinline__ void math_bar() { asm volatile("bar.sync 1, %0;" ::"n"(MATH_THREADS) : "memory"); }
+__device__ __forceinline__ void quant_bar() { asm volatile("bar.sync 1, %0;" ::"n"(Q_THREADS) : "memory"); }
 
-// eight E2M1 codes (one word) times a scale (both halves of sc2) -> four fp16 pairs, exact
-__device__ __forceinline__ void dq_nvfp4(uint32_t c32, uint32_t sc2, uint32_t (&x)[4])
+// A correction tile holds [128 rows][16 tokens] fp32, a row = 64 bytes = four 16-byte pieces of
+// four tokens; piece index is XOR-ed with (row >> 1) & 3 so that 32 lanes reading one piece of 32
+// consecutive rows (the epilogue) do not collide on banks.  Float index of (row, token):
+__device__ __forceinline__ uint32_t tile_idx(uint32_t row, uint32_t token)
 {
-    uint32_t q0, q1, q2, q3;
-    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\tmov.b32 {b0, b1, b2, b3}, %4;\n\t"
-        "cvt.rn.f16x2.e2m1x2 %0, b0;\n\tcvt.rn.f16x2.e2m1x2 %1, b1;\n\t"
-        "cvt.rn.f16x2.e2m1x2 %2, b2;\n\tcvt.rn.f16x2.e2m1x2 %3, b3;\n\t}"
-        : "=r"(q0), "=r"(q1), "=r"(q2), "=r"(q3) : "r"(c32));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[0]) : "r"(q0), "r"(sc2));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[1]) : "r"(q1), "r"(sc2));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[2]) : "r"(q2), "r"(sc2));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[3]) : "r"(q3), "r"(sc2));
-}
-
-// The same eight elements of a block that is NVFP4 (codes in c32) or, if is8 != 0, FP8 (E4M3 codes in e8a,
-// e8b): the lane's flag picks the conversion, the multiply with the block's scale pair is common.
-__device__ __forceinline__ void dq_mixed(uint32_t c32, uint32_t e8a, uint32_t e8b, uint32_t is8, uint32_t sc2, uint32_t (&x)[4])
-{
-    uint32_t q0, q1, q2, q3;
-    asm("{\n\t.reg .pred p;\n\t.reg .b8 b0, b1, b2, b3;\n\t.reg .b16 h0, h1, h2, h3;\n\t"
-        "setp.ne.u32 p, %7, 0;\n\t"
-        "mov.b32 {b0, b1, b2, b3}, %4;\n\tmov.b32 {h0, h1}, %5;\n\tmov.b32 {h2, h3}, %6;\n\t"
-        "@!p cvt.rn.f16x2.e2m1x2 %0, b0;\n\t@p cvt.rn.f16x2.e4m3x2 %0, h0;\n\t"
-        "@!p cvt.rn.f16x2.e2m1x2 %1, b1;\n\t@p cvt.rn.f16x2.e4m3x2 %1, h1;\n\t"
-        "@!p cvt.rn.f16x2.e2m1x2 %2, b2;\n\t@p cvt.rn.f16x2.e4m3x2 %2, h2;\n\t"
-        "@!p cvt.rn.f16x2.e2m1x2 %3, b3;\n\t@p cvt.rn.f16x2.e4m3x2 %3, h3;\n\t}"
-        : "=&r"(q0), "=&r"(q1), "=&r"(q2), "=&r"(q3) : "r"(c32), "r"(e8a), "r"(e8b), "r"(is8));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[0]) : "r"(q0), "r"(sc2));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[1]) : "r"(q1), "r"(sc2));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[2]) : "r"(q2), "r"(sc2));
-    asm("mul.f16x2 %0, %1, %2;" : "=r"(x[3]) : "r"(q3), "r"(sc2));
+    return row * 16u + ((((token >> 2) ^ (row >> 1)) & 3u) << 2) + (token & 3u);
 }
 
 // Bounded wait for a word in global memory to take a value that another CTA publishes.
@@ -140,126 +136,155 @@ __device__ __noinline__ bool wait_global_equals(const uint32_t* addr, uint32_t v
     }
 }
 
-// One work item of the prologue quantizer: chunk c (256 elements), token octet o: warp w takes token
-// 8o + w/2 and the eight blocks 16c + 8(w%2) .. +7, four lanes per block.
+// One work item of the prologue quantizer: chunk c (256 elements) of every token row.  Run by the 16
+// warps 2..17: warp wq takes, per token octet o, token 8o + wq/2 and the eight blocks 8(wq%2) .. +7 of
+// the chunk, four lanes per block.  s_hot: one word of shared memory.
 template <int MODE>
-__device__ __forceinline__ void quantize_item(const DecParams& p, int64_t c, int o)
+__device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, uint32_t* s_hot)
 {
-    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u, li = lane & 3u;
-    const int64_t m = 8 * o + (int64_t)(w >> 1);
-    const uint32_t j = 8u * (w & 1u) + (lane >> 2);
+    const uint32_t tq = threadIdx.x - 64u;                 // index among the quantizer's threads
+    const uint32_t wq = tq >> 5, lane = tq & 31u, li = lane & 3u;
+    const uint32_t j = 8u * (wq & 1u) + (lane >> 2);
     const int64_t kb = 16 * c + j;
-    uint8_t* dst = p.arec + (size_t)c * AREC_BYTES + fgmp_arec_offset((uint32_t)m, j, li >> 1) + (li & 1u) * 8u;
-    if (m >= p.M) {                                   // token rows beyond the batch are zero
-        *reinterpret_cast<uint2*>(dst) = make_uint2(0u, 0u);
-        return;
-    }
-    const uint2 x = __ldg(reinterpret_cast<const uint2*>(p.X + ((size_t)m * p.ldx + (size_t)kb * 16 + 4 * li) * 2));
-    const float4 f = __ldg(reinterpret_cast<const float4*>(p.fisher + kb * 16 + 4 * li));
-    const BlockQuarter r = quantize_block_quarter<MODE>(x, f, p.q);
-    *reinterpret_cast<uint2*>(dst) = r.h;
-    if (p.q_codes4) {
-        const int64_t MW = p.LA.MW;
-        *reinterpret_cast<uint16_t*>(p.q_codes4 + (m * p.K) / 2 + kb * 8 + li * 2) = (uint16_t)r.c4;
-        if (li == 0) p.q_sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)r.sc;
-        if (r.is8) *reinterpret_cast<uint32_t*>(p.q_codes8 + m * p.K + kb * 16 + 4 * li) = r.c8;
+    uint8_t* rec = p.arec + (size_t)c * AREC_BYTES;
+    if (tq == 0) *s_hot = 0u;
+    quant_bar();
+    const int octets = p.M > 8 ? 2 : 1;
+    for (int o = 0; o < 2; ++o) {
+        const uint32_t m = 8u * (uint32_t)o + (wq >> 1);
+        uint8_t* a4 = rec + AREC_A4 + fgmp_rec_w4_offset(m, j) + 2u * li;
+        uint8_t* at = rec + fgmp_arec_at_offset(m, j) + 8u * li;
+        if (o >= octets || (int64_t)m >= p.M) {             // token rows beyond the batch are zero
+            *reinterpret_cast<uint16_t*>(a4) = 0;
+            *reinterpret_cast<uint2*>(at) = make_uint2(0u, 0u);
+            if (li == 0) rec[AREC_SF + m * 16u + j] = 0;
+            continue;
+        }
+        const uint2 x = __ldg(reinterpret_cast<const uint2*>(p.X + ((size_t)m * p.ldx + (size_t)kb * 16 + 4 * li) * 2));
+        const float4 f = __ldg(reinterpret_cast<const float4*>(p.fisher + kb * 16 + 4 * li));
+        const BlockQuarter r = quantize_block_quarter<MODE>(x, f, p.q);
+        *reinterpret_cast<uint16_t*>(a4) = (uint16_t)r.c4;
+        *reinterpret_cast<uint2*>(at) = r.h;
+        if (li == 0) rec[AREC_SF + m * 16u + j] = (uint8_t)r.sc;
         const uint32_t bal = __ballot_sync(0xffffffffu, r.is8 && li == 0);
-        if (lane == 0) {
-            uint32_t byte = 0;
+        uint32_t byte = 0;
 #pragma unroll
-            for (int b = 0; b < 8; ++b) byte |= ((bal >> (4 * b)) & 1u) << b;
-            const int64_t kb0 = kb;                   // lane 0: first block of the warp's eight
-            uint8_t* mb = p.q_mask + (size_t)m * MW * 4 + (kb0 >> 3);
-            mb[0] = (uint8_t)byte;
-            if (kb0 + 8 == p.LA.KB && (p.LA.KB & 31) != 0) { mb[1] = 0; mb[2] = 0; }   // rest of the row's last mask word
+        for (int b = 0; b < 8; ++b) byte |= ((bal >> (4 * b)) & 1u) << b;
+        if (lane == 0 && byte) atomicOr(s_hot, byte << (8u * (wq & 1u)));
+        if (p.q_codes4) {
+            const int64_t MW = p.LA.MW;
+            *reinterpret_cast<uint16_t*>(p.q_codes4 + ((int64_t)m * p.K) / 2 + kb * 8 + li * 2) = (uint16_t)r.c4;
+            if (li == 0) p.q_sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)r.sc;
+            if (r.is8) *reinterpret_cast<uint32_t*>(p.q_codes8 + (int64_t)m * p.K + kb * 16 + 4 * li) = r.c8;
+            if (lane == 0) {
+                uint8_t* mb = p.q_mask + (size_t)m * MW * 4 + (kb >> 3);    // lane 0: first block of the warp's eight
+                mb[0] = (uint8_t)byte;
+                if (kb + 8 == p.LA.KB && (p.LA.KB & 31) != 0) { mb[1] = 0; mb[2] = 0; }   // rest of the row's last mask word
+            }
         }
     }
-}
-
-__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    quant_bar();
+    if (tq == 0) *reinterpret_cast<uint32_t*>(rec + AREC_HOT) = *s_hot;
 }
 
 // NH = token octets in use: 1 for M <= 8, else 2.  FUSED: the activation quantizer runs in the prologue.
-// NG = groups of 16 / NG warps that work on different units at the same time; a warp takes rows 32jr .. 32jr+31
-// and NG of the four classes of block columns (j % 4).
-template <int NH, bool FUSED, int NG>
+template <int NH, bool FUSED>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_kernel(DecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     // 1 KiB aligned; an offset from the array keeps the pointer known to be shared memory (plain ld.shared / st.shared)
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    const int S = p.stages;
-    float* epi = reinterpret_cast<float*>(smem + (size_t)S * DEC_STAGE_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(epi + EPI_FLOATS);             // full[DEC_STAGES]
-    uint32_t* done = reinterpret_cast<uint32_t*>(bars + DEC_STAGES);            // warps that have finished with a stage
-    StageMeta* smeta = reinterpret_cast<StageMeta*>(done + DEC_STAGES + 1);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smeta + DEC_STAGES);
-    volatile uint32_t* s_misc = reinterpret_cast<volatile uint32_t*>(abort_flag + 1);   // [0] tag, [1..2] claimed item, [3] last-arrival flag
-    uint32_t* table = const_cast<uint32_t*>(s_misc + 8);                        // overflow starts of this CTA's units (+ 1)
+    constexpr int S = DEC_STAGES;
+    float* tiles = reinterpret_cast<float*>(smem + (size_t)S * DEC_STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + NTILES * TILE_FLOATS);
+    // bars: [0,S) full, [S,2S) empty, [2S,3S) scales in tensor memory, then acc_full[2], acc_empty[2],
+    // corrections of a segment done [2], tiles free [1]
+    StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * S + 8);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + S);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile uint32_t* s_misc = reinterpret_cast<volatile uint32_t*>(abort_flag + 1);   // [0] tag, [1..2] claimed item, [3] hot columns of a chunk
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars);
-    FGMP_STAMP(0);
-    constexpr uint32_t A_BYTES = NH == 2 ? AREC_BYTES : AREC_BYTES / 2;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, sfr0 = empty0 + 8 * S;
+    const uint32_t accf0 = sfr0 + 8 * S, acce0 = accf0 + 16, cdone0 = acce0 + 16, tfree = cdone0 + 16;
+    constexpr uint32_t A_BYTES = NH == 2 ? AREC_BYTES : AREC_AT + 4096u;
 
     // this CTA's span of (tile, chunk) units
     const int64_t G = gridDim.x, C = p.chunks;
     const int64_t u_begin = ((int64_t)blockIdx.x * p.total) / G, u_end = ((int64_t)(blockIdx.x + 1) * p.total) / G;
-    const int n_units = (int)(u_end - u_begin);
     const uint32_t* uptr = reinterpret_cast<const uint32_t*>(p.wblob + p.LW.off_uptr);
     const uint8_t* recs = p.wblob + p.LW.off_rec;
-    const uint8_t* ovfs = p.wblob + p.LW.off_ovf;
+    const uint8_t* lists = p.wblob + p.LW.off_ovf;
     const uint8_t* arec = FUSED ? p.arec : p.ablob + p.LA.off_arec;
 
-    // the copies of unit i (index inside the span) into its stage, by one thread
-    auto stage_dst = [&](int stage) { return smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES); };
-    auto issue_rec = [&](int i, int stage) { bulk_load(stage_dst(stage), recs + (size_t)(u_begin + i) * REC_BYTES, REC_BYTES, full0 + 8 * stage); };
-    auto issue_ovf = [&](int i, int stage, bool expect) {
-        const uint32_t step0 = table[i], bytes = (table[i + 1] - step0) * 16u;
-        const uint32_t staged = bytes < OVF_CAP ? bytes : OVF_CAP;
+    // One unit's copies into a stage (lane 0 of the producer warp): record and list, then the
+    // activation record of the unit's chunk
+    auto issue_w = [&](int64_t u, int stage, uint32_t step0, uint32_t step1) {
+        const uint32_t bytes = (step1 - step0) * 16u;
+        const uint32_t staged = bytes < LIST_CAP ? bytes : LIST_CAP;
         smeta[stage].step = step0; smeta[stage].staged = staged;
-        if (expect && staged) mbar_expect_tx_only(full0 + 8 * stage, staged);
-        if (staged) bulk_load(stage_dst(stage) + STG_OVF, ovfs + (size_t)step0 * 16, staged, full0 + 8 * stage);
-        return staged;
+        const uint32_t fb = full0 + 8 * stage;
+        const uint32_t dst = smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES);
+        mbar_expect_tx(fb, REC_BYTES + staged + A_BYTES);
+        bulk_load(dst, recs + (size_t)u * REC_BYTES, REC_BYTES, fb);
+        if (staged) bulk_load(dst + STG_LIST, lists + (size_t)step0 * 16, staged, fb);
     };
-    auto issue_a = [&](int i, int stage) {
-        bulk_load(stage_dst(stage) + STG_A, arec + (size_t)((u_begin + i) % C) * AREC_BYTES, A_BYTES, full0 + 8 * stage);
+    auto issue_a = [&](int64_t u, int stage) {
+        bulk_load(smem_u32(smem + (size_t)stage * DEC_STAGE_BYTES) + STG_A, arec + (size_t)(u % C) * AREC_BYTES, A_BYTES, full0 + 8 * stage);
     };
 
-    // ------------------------------------------------------------ set-up: barriers, the weight blob's header, and the
-    // first stages' weight copies.  The packed weights are not written by whatever runs before this kernel, so all
-    // of this may overlap the end of that kernel (programmatic dependent launch).
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); done[s] = 0; }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // ------------------------------------------------------------ set-up.  The packed weights are not written by
+    // whatever runs before this kernel, so the producer's part (barriers, the weight blob's header, the first
+    // stages' weight copies) may overlap the end of that kernel (programmatic dependent launch).
+    int64_t pf_base = u_begin;
+    uint32_t pf = 0;
+    int pre = 0;
+    if (warp == W_PROD) {
+        if (lane == 0) {
+            for (int s = 0; s < S; ++s) {
+                mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + 8); mbar_init(sfr0 + 8 * s, 4);
+            }
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); mbar_init(cdone0 + 8 * b, 8);
+            }
+            mbar_init(tfree, 4);
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
         // nothing is read through the blob's tables before its header has been seen to describe this call
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
-        const uint2 mv = __ldg(reinterpret_cast<const uint2*>(hw));
-        const bool okh = mv.x == FGMP_MAGIC && mv.y == 6u && __ldg(&hw->rows) == p.N && __ldg(&hw->K) == p.K &&
-                         __ldg(&hw->kind) == 1u && __ldg(&hw->error) == 0;
-        if (!okh) { *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 9); }
+        int okh = 1;
+        if (lane == 0) {
+            const uint2 mv = __ldg(reinterpret_cast<const uint2*>(hw));
+            okh = mv.x == FGMP_MAGIC && mv.y == 7u && __ldg(&hw->rows) == p.N && __ldg(&hw->K) == p.K &&
+                  __ldg(&hw->kind) == 1u && __ldg(&hw->error) == 0;
+            if (!okh) { *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 9); }
+        }
+        okh = __shfl_sync(0xffffffffu, okh, 0);
+        if (okh) {
+            if (pf_base + lane <= p.total) pf = __ldg(uptr + pf_base + lane);
+            pre = (int)min((int64_t)S, u_end - u_begin);
+            for (int s = 0; s < pre; ++s) {
+                const uint32_t step0 = __shfl_sync(0xffffffffu, pf, s), step1 = __shfl_sync(0xffffffffu, pf, s + 1);
+                if (lane == 0) issue_w(u_begin + s, s, step0, step1);
+            }
+        }
     }
-    __syncthreads();
-    FGMP_STAMP(1);
-    const int pre = min(S, n_units);
-    if (!*abort_flag) {
-        for (int i = threadIdx.x; i <= n_units; i += DEC_THREADS) table[i] = __ldg(uptr + u_begin + i);
-        if (threadIdx.x == 0)
-            for (int s = 0; s < pre; ++s) { mbar_expect_tx_only(full0 + 8 * s, REC_BYTES + A_BYTES); issue_rec(s, s); }
+    if (warp == W_MMA) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
+    if (warp >= W_FP8 && warp < W_EPI) {               // the tiles start at zero
+        float4* z = reinterpret_cast<float4*>(tiles);
+        for (int i = (warp - W_FP8) * 32 + lane; i < (int)(NTILES * TILE_FLOATS / 4); i += 8 * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    tc_fence_before();
     __syncthreads();
-    if (!*abort_flag && threadIdx.x == 0)
-        for (int s = 0; s < pre; ++s) issue_ovf(s, s, true);
-    FGMP_STAMP(2);
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    FGMP_STAMP_ANY(warp == 0 && lane == 0 ? 1 : 15);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // Launched as a programmatic dependent of the preceding kernel in the stream, this kernel may have
     // started before that one finished: everything above touches neither its output nor the workspace.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    FGMP_STAMP(3);
     if (FUSED) {
         if (threadIdx.x == 0) {
             uint32_t e;
@@ -269,253 +294,456 @@ decode_kernel(DecParams p)
         __syncthreads();
     }
     const uint32_t tag = FUSED ? s_misc[0] : 0u;
+    const bool dead = *abort_flag != 0;                // the weight blob does not belong to this call: nothing else is read
 
-    if (!*abort_flag) {
-        if (FUSED) {
-            // The quantizer's work items are handed out through a counter, so that every item is taken by a CTA
-            // that is running: no CTA ever waits for one that has not started.  The counter and the count of
-            // finished items wrap to zero with the call's last access.
-            const uint32_t octets = p.M > 8 ? 2u : 1u;
-            const uint32_t n_items = (uint32_t)C * octets;
-            for (uint32_t it = 0;; ++it) {
-                if (threadIdx.x == 0) s_misc[1 + (it & 1u)] = atomicInc(p.cw + CW_CLAIM, n_items + (uint32_t)G - 1u);
-                math_bar();
-                const uint32_t item = s_misc[1 + (it & 1u)];
-                if (item >= n_items) break;
-                if (item == 0 && threadIdx.x == 0 && p.q_header) {
-                    fgmp_packed_header* h = p.q_header;
-                    h->magic = FGMP_MAGIC; h->version = 6; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.q.s4;
-                    h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
-                    h->error = 0;
-                }
-                if (p.q_mode == 0) quantize_item<0>(p, (int64_t)(item / octets), (int)(item % octets));
-                else               quantize_item<1>(p, (int64_t)(item / octets), (int)(item % octets));
-                __threadfence();
-                math_bar();
-                if (threadIdx.x == 0 && atomicInc(p.cw + CW_QCOUNT, n_items - 1u) == n_items - 1u)
-                    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(tag) : "memory");
+    if (FUSED && !dead && warp >= W_SCALE) {
+        // The quantizer's work items (chunks) are handed out through a counter, so that every item is taken by
+        // a CTA that is running: no CTA ever waits for one that has not started.  The counter and the count of
+        // finished items wrap to zero with the call's last access.
+        const uint32_t n_items = (uint32_t)C;
+        for (uint32_t it = 0;; ++it) {
+            if (threadIdx.x == 64) s_misc[1 + (it & 1u)] = atomicInc(p.cw + CW_CLAIM, n_items + (uint32_t)G - 1u);
+            quant_bar();
+            const uint32_t item = s_misc[1 + (it & 1u)];
+            if (item >= n_items) break;
+            if (item == 0 && threadIdx.x == 64 && p.q_header) {
+                fgmp_packed_header* h = p.q_header;
+                h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.q.s4;
+                h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+                h->error = 0;
             }
+            if (p.q_mode == 0) quantize_chunk<0>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
+            else               quantize_chunk<1>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
+            __threadfence();
+            quant_bar();
+            if (threadIdx.x == 64 && atomicInc(p.cw + CW_QCOUNT, n_items - 1u) == n_items - 1u)
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(tag) : "memory");
         }
-        // the activation records of the first stages; their barriers' one arrival comes last
-        FGMP_STAMP(4);
-        if (threadIdx.x == 0) {
-            bool oka = true;
+    }
+
+    if (dead) {
+    } else if (warp == W_PROD) {
+        // ------------------------------------------------------------ producer (whole warp; lane 0 issues)
+        int ok = 1;
+        if (lane == 0) {
             if (FUSED) {
                 // every chunk's record is in place once the last work item of the quantizer has been handed in
-                oka = wait_global_equals(p.cw + CW_QREADY, tag, abort_flag, p.status, 8);
+                ok = wait_global_equals(p.cw + CW_QREADY, tag, abort_flag, p.status, 8) ? 1 : 0;
                 asm volatile("fence.proxy.async;" ::: "memory");   // records were written with ordinary stores, the bulk copy reads them
             } else {
                 const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
                 const uint2 mv = __ldg(reinterpret_cast<const uint2*>(ha));
-                if (!(mv.x == FGMP_MAGIC && mv.y == 6u && __ldg(&ha->rows) == p.M && __ldg(&ha->K) == p.K && __ldg(&ha->kind) == 0u)) {
+                if (!(mv.x == FGMP_MAGIC && mv.y == 7u && __ldg(&ha->rows) == p.M && __ldg(&ha->K) == p.K && __ldg(&ha->kind) == 0u)) {
                     *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 10);
-                    oka = false;
+                    ok = 0;
                 }
             }
-            if (oka) for (int s = 0; s < pre; ++s) { issue_a(s, s); mbar_arrive(full0 + 8 * s); }
+            if (ok) for (int s = 0; s < pre; ++s) issue_a(u_begin + s, s);
         }
-        FGMP_STAMP(5);
-
-        // ------------------------------------------------------------ the units of this CTA, group by group
-        constexpr int GROUPS = NG, GROUP_WARPS = MATH_WARPS / NG;
-        const uint32_t part = (uint32_t)warp >> 2, jr = (uint32_t)warp & 3u;      // part: which partial tile this warp's sums go to
-        const uint32_t gq = part * NG / 4u;                                       // group
-        const int hq0 = NG == 4 ? 0 : (NG == 2 ? 2 * (int)(part & 1u) : (int)part);
-        const uint32_t g = (uint32_t)lane >> 2, t = (uint32_t)lane & 3u;
-        const uint32_t sf_off = REC_SF + jr * 512u + (uint32_t)lane * 16u;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        int stage = pre % S; uint32_t phase = (uint32_t)(pre / S) & 1u;
+        for (int64_t u = u_begin + pre; u < u_end && ok; ++u) {
+            if (u + 1 - pf_base > 31) {                // next 32 list starts
+                pf_base = u;
+                pf = (pf_base + lane <= p.total) ? __ldg(uptr + pf_base + lane) : 0u;
+            }
+            const uint32_t step0 = __shfl_sync(0xffffffffu, pf, (int)(u - pf_base));
+            const uint32_t step1 = __shfl_sync(0xffffffffu, pf, (int)(u + 1 - pf_base));
+            if (lane == 0) {
+                ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1) ? 1 : 0;
+                if (ok) { issue_w(u, stage, step0, step1); issue_a(u, stage); }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+    } else if (warp == W_MMA) {
+        // ------------------------------------------------------------ MMA issuer
+        // The whole warp walks the loop; lane 0 alone issues the tcgen05 instructions, so that every
+        // commit tracks every MMA before it.
+        const uint32_t smem0 = smem_u32(smem);
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
+            const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
+            if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
+            uint32_t accum = 0;
+            for (; u < seg_end && ok; ++u) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
+                if (!(ok = mbar_wait(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;   // the scales are in tensor memory
+                tc_fence_after();
+                const uint32_t sb = smem0 + (uint32_t)stage * DEC_STAGE_BYTES;
+                const uint32_t sf_t = tmem_base + SF_COL0 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
+                const uint32_t w4_lo = ((sb + REC_W4) >> 4) | SW128_LO, a4_lo = ((sb + STG_A + AREC_A4) >> 4) | SW128_LO;
+                if (lane == 0) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        umma_nvf4(d_tmem, desc64(w4_lo + 2 * j, SW128_HI), desc64(a4_lo + 2 * j, SW128_HI), IDESC_NVF4,
+                                  sf_t + 4 * j, sf_t + 16 + 4 * j, accum);
+                        accum = 1;
+                    }
+                    umma_commit(empty0 + 8 * stage);
+                }
+                accum = 1;
+                __syncwarp();
+                if (++stage == S) { stage = 0; phase ^= 1; }
+            }
+            if (ok && lane == 0) umma_commit(accf0 + 8 * acc);
+            __syncwarp();
+        }
+    } else if (warp < W_FP8) {
+        // ------------------------------------------------------------ block scales into tensor memory, lane quadrant warp % 4
+        // Lane i holds, for MMA step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3 --
+        // 16 bytes of scale tile j of the record; the token scales follow in columns 16..31 (16 tokens: lanes
+        // 0..15, first column of every step), zeroed in the chunk's hot block columns.
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        for (int64_t u = u_begin; u < u_end && ok; ++u) {
+            if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 4))) break;
+            const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+            const uint8_t* sa = sb + STG_A;
+            uint32_t r[16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
+                r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+            }
+            const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
+            tmem_st16(sf_t, r);
+            const uint32_t cold = ~*reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
+            const uint4 ts = *reinterpret_cast<const uint4*>(sa + AREC_SF + (lane & 15) * 16);
+            const uint32_t tsw[4] = {ts.x, ts.y, ts.z, ts.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                // bits 4j .. 4j+3 of `cold` spread to the four bytes of the step's scale word
+                const uint32_t keep = ((((cold >> (4 * j)) & 0xfu) * 0x00204081u) & 0x01010101u) * 0xffu;
+                r[4 * j] = lane < 16 ? (tsw[j] & keep) : 0u;
+                r[4 * j + 1] = 0u; r[4 * j + 2] = 0u; r[4 * j + 3] = 0u;
+            }
+            tmem_st16(sf_t + 16, r);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
+            if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+    } else if (warp < W_HOT) {
+        // ------------------------------------------------------------ (2): FP8 weight blocks of block columns bq, bq+4, bq+8, bq+12
+        // The E4M3 codes go into the MMA as they are; the factor 2^ratio between the FP8 and NVFP4
+        // tensor scales is applied once to the tile sums in the epilogue.
+        const int bq = warp - W_FP8;
+        const uint32_t g = lane >> 2, t = lane & 3;
+        float* mytile = tiles + bq * TILE_FLOATS;
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
-        const float alpha = FUSED ? __fmul_rn(p.q.s4, __ldg(&reinterpret_cast<const fgmp_packed_header*>(p.wblob)->scale_fp4))
-                                  : __fmul_rn(__ldg(&reinterpret_cast<const fgmp_packed_header*>(p.ablob)->scale_fp4),
-                                              __ldg(&reinterpret_cast<const fgmp_packed_header*>(p.wblob)->scale_fp4));
-        bool ok = true;
-        for (int sbeg = 0; sbeg < n_units;) {
-            const int64_t tile = (u_begin + sbeg) / C;
-            const int send = (int)min((int64_t)n_units, (tile + 1) * C - u_begin);
-            // acc[mt][nh] = rows 32jr + 16mt + {g, g + 8} x tokens 8nh + {2t, 2t+1}, this group's units of the tile
+
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
+            // the epilogue has taken (and cleared) the previous segment's sums
+            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
+            for (; u < seg_end; ++u) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+                const uint8_t* sa = sb + STG_A;
+                const uint32_t staged = smeta[stage].staged;
+                const uint8_t* list_g = lists + (size_t)smeta[stage].step * 16;
+                const uint16_t* kbs = reinterpret_cast<const uint16_t*>(sb + REC_KBSTART);
+                const uint32_t ntot = kbs[16];
+                const uint32_t hoff = fgmp_list_halves_offset(ntot);
+                // ALL = the whole list of the unit is in the stage (the usual case); otherwise its tail is read
+                // from global memory
+                auto body = [&](auto all_c) {
+                    constexpr bool ALL = decltype(all_c)::value;
+                    // One group of up to 16 blocks of column j: blocks e + g and e + g + 8 are the M side of the
+                    // mma.sync (tokens 0-7 and 8-15 as N).  Lane t has elements 4t .. 4t+3 of a block: from its slot
+                    // in the record (t < 2) or from the list (t >= 2).
+                    // c/d[0..1]: block iA, tokens 2t, 2t+1 / 8+2t, 9+2t; [2..3]: block iB.
+                    auto group_mma = [&](uint32_t j, uint32_t e, uint32_t end_, const uint2& bt0, const uint2& bt1, float (&c)[4], float (&d)[4],
+                                         uint32_t& rowA, uint32_t& rowB) {
+                        const uint32_t iA = e + g, iB = iA + 8;
+                        uint32_t rawA = 0, rawB = 0;
+                        rowA = 0xffffffffu; rowB = 0xffffffffu;
+                        auto fetch = [&](uint32_t i, uint32_t& row, uint32_t& raw) {
+                            row = (ALL || i < staged) ? sb[STG_LIST + i] : __ldg(list_g + i);
+                            if (t < 2) {
+                                raw = *reinterpret_cast<const uint32_t*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j) + 4 * t);
+                            } else {
+                                const uint32_t o = hoff + i * 8 + 4 * (t - 2);
+                                raw = (ALL || o + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + o)
+                                                               : __ldg(reinterpret_cast<const uint32_t*>(list_g + o));
+                            }
+                        };
+                        if (iA < end_) fetch(iA, rowA, rawA);
+                        if (iB < end_) fetch(iB, rowB, rawB);
+                        uint32_t a0, a1, a2, a3;
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a0) : "h"((uint16_t)rawA));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a2) : "h"((uint16_t)(rawA >> 16)));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a1) : "h"((uint16_t)rawB));
+                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a3) : "h"((uint16_t)(rawB >> 16)));
+                        c[0] = c[1] = c[2] = c[3] = 0.f; d[0] = d[1] = d[2] = d[3] = 0.f;
+                        mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);
+                        if (NH == 2) mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);
+                    };
+                    // Within one column every block has its own row, so the read-modify-writes of a group touch
+                    // distinct addresses in every lane and across lanes: all loads first, then all stores.
+                    auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t rowA, uint32_t rowB) {
+                        float2 *pA = nullptr, *pB = nullptr;    // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on (piece ^ 2)
+                        float2 vA0 = make_float2(0.f, 0.f), vA1 = vA0, vB0 = vA0, vB1 = vA0;
+                        if (rowA != 0xffffffffu) {
+                            pA = reinterpret_cast<float2*>(mytile + rowA * 16u + (((tpiece ^ (rowA >> 1)) & 3u) << 2) + tcol);
+                            vA0 = pA[0];
+                            if (NH == 2) vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
+                        }
+                        if (rowB != 0xffffffffu) {
+                            pB = reinterpret_cast<float2*>(mytile + rowB * 16u + (((tpiece ^ (rowB >> 1)) & 3u) << 2) + tcol);
+                            vB0 = pB[0];
+                            if (NH == 2) vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
+                        }
+                        if (rowA != 0xffffffffu) {
+                            pA[0] = make_float2(vA0.x + c[0], vA0.y + c[1]);
+                            if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(vA1.x + d[0], vA1.y + d[1]);
+                        }
+                        if (rowB != 0xffffffffu) {
+                            pB[0] = make_float2(vB0.x + c[2], vB0.y + c[3]);
+                            if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(vB1.x + d[2], vB1.y + d[3]);
+                        }
+                        __syncwarp();                  // a later group may add to the same rows
+                    };
+#pragma unroll 1
+                    for (int cp = 0; cp < 2; ++cp) {
+                        // two block columns side by side (their MMAs are independent), then their sums in order
+                        const uint32_t j0 = (uint32_t)bq + 8u * cp, j1 = j0 + 4u;
+                        const uint32_t st0 = kbs[j0], en0 = kbs[j0 + 1], st1 = kbs[j1], en1 = kbs[j1 + 1];
+                        // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of each column
+                        const uint2 b00 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g, j0) + 8 * t);
+                        const uint2 b10 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g, j1) + 8 * t);
+                        uint2 b01 = make_uint2(0u, 0u), b11 = b01;
+                        if (NH == 2) {
+                            b01 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j0) + 8 * t);
+                            b11 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j1) + 8 * t);
+                        }
+                        {
+                            float c0[4], d0[4], c1[4], d1[4];
+                            uint32_t rA0, rB0, rA1, rB1;
+                            group_mma(j0, st0, en0, b00, b01, c0, d0, rA0, rB0);
+                            group_mma(j1, st1, en1, b10, b11, c1, d1, rA1, rB1);
+                            group_add(c0, d0, rA0, rB0);
+                            group_add(c1, d1, rA1, rB1);
+                        }
+                        // columns with more than 16 FP8 blocks
+                        for (uint32_t e = st0 + 16; e < en0; e += 16) {
+                            float c[4], d[4];
+                            uint32_t rA, rB;
+                            group_mma(j0, e, en0, b00, b01, c, d, rA, rB);
+                            group_add(c, d, rA, rB);
+                        }
+                        for (uint32_t e = st1 + 16; e < en1; e += 16) {
+                            float c[4], d[4];
+                            uint32_t rA, rB;
+                            group_mma(j1, e, en1, b10, b11, c, d, rA, rB);
+                            group_add(c, d, rA, rB);
+                        }
+                    }
+                };
+                if (ntot && hoff + ntot * 8 <= staged) body(std::true_type{}); else if (ntot) body(std::false_type{});
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+                if (++stage == S) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
+        }
+    } else if (warp < W_EPI) {
+        // ------------------------------------------------------------ (3): hot block columns, rows 32jr .. 32jr+31
+        // Lane (g, t) has elements 4t .. 4t+3 of the column's block in rows 32jr + 16mt + {g, g + 8}: two code
+        // bytes and the block's microscale (zero for an FP8 weight block, which (2) covers).
+        const uint32_t jr = (uint32_t)(warp - W_HOT);
+        const uint32_t g = lane >> 2, t = lane & 3;
+        float* tile3 = tiles + 4 * TILE_FLOATS;
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_end = min(u_end, (tile + 1) * C);
             float acc[2][NH][4];
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) acc[mt][nh][0] = acc[mt][nh][1] = acc[mt][nh][2] = acc[mt][nh][3] = 0.f;
-            for (int i = sbeg + (int)((gq - (uint32_t)sbeg) & (uint32_t)(NG - 1)); i < send; i += GROUPS) {
-                const int stage = i % S; const uint32_t phase = (uint32_t)(i / S) & 1u;
-                if (ok) ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5);
-                if (!ok) break;
-                if (i == 0) FGMP_STAMP(6);
+            for (; u < seg_end; ++u) {
+                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 6))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-                const uint4 scv = *reinterpret_cast<const uint4*>(sb + sf_off);
-                const bool any8 = __any_sync(0xffffffffu, ((scv.x | scv.y | scv.z | scv.w) & 0x80808080u) != 0u);
-                // where this lane's overflow entries start, per hq (only with FP8 blocks in the unit)
-                uint32_t idx4 = 0;
-                if (any8) {
-                    const uint32_t pack = __popc(scv.x & 0x80808080u) | (__popc(scv.y & 0x80808080u) << 8) |
-                                          (__popc(scv.z & 0x80808080u) << 16) | (__popc(scv.w & 0x80808080u) << 24);
-                    uint32_t incl = pack;
+                const uint8_t* sa = sb + STG_A;
+                uint32_t todo = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT) & 0xffffu;
+#ifdef FGMP_DEBUG_PRINT
+                if (blockIdx.x == 0 && lane == 5) printf("hot warp %d u %lld todo %x stage %d\n", warp, (long long)u, todo, stage);
+#endif
+                while (todo) {
+                    const uint32_t j = (uint32_t)__ffs(todo) - 1u;
+                    todo &= todo - 1;
+                    uint2 b[NH];
 #pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= o) incl += y;
-                    }
-                    idx4 = incl - pack;
-                }
-                const uint32_t staged = smeta[stage].staged;
-                const uint8_t* ovf_g = ovfs + (size_t)smeta[stage].step * 16;
-#pragma unroll 1
-                for (int hq = hq0; hq < hq0 + NG; ++hq) {
-                    const uint32_t w = 4 * jr + (uint32_t)hq;
-                    const uint32_t sc4 = *reinterpret_cast<const uint32_t*>(sb + sf_off + 4 * hq);
-                    const uint4 s01 = *reinterpret_cast<const uint4*>(sb + REC_W4 + w * 1024u + (uint32_t)lane * 16u);
-                    const uint4 s23 = *reinterpret_cast<const uint4*>(sb + REC_W4 + w * 1024u + 512u + (uint32_t)lane * 16u);
-                    const uint32_t a_off = STG_A + (uint32_t)(hq * 2) * 512u + (uint32_t)lane * 16u;
-                    // scale pairs: byte k of sc4 (flag bit cleared) in both halves, E4M3 -> fp16
-                    uint32_t sc2[4];
-                    {
-                        const uint32_t s7 = sc4 & 0x7f7f7f7fu;
+                    for (int nh = 0; nh < NH; ++nh) b[nh] = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8 * nh, j) + 8 * t);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const uint32_t two = __byte_perm(s7, 0u, 0x4400u | (uint32_t)(k << 4) | (uint32_t)k);
-                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2[k]) : "h"((uint16_t)two));
+                    for (int mt = 0; mt < 2; ++mt) {
+                        uint32_t x[2][2];
+#pragma unroll
+                        for (int rh = 0; rh < 2; ++rh) {
+                            const uint32_t r = 32 * jr + 16 * (uint32_t)mt + 8 * (uint32_t)rh + g;
+                            const uint32_t codes = *reinterpret_cast<const uint16_t*>(sb + REC_W4 + fgmp_rec_w4_offset(r, j) + 2 * t);
+                            const uint32_t sfb = sb[REC_SF + fgmp_rec_sf_offset(r, j)];
+                            uint32_t q0, q1, sc2;
+                            // (one byte at a time: unpacking a word into byte registers of which only some are used
+                            // gave wrong values on this toolchain)
+                            asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(q0) : "r"(codes & 0xffu));
+                            asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(q1) : "r"(codes >> 8));
+                            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sc2) : "h"((uint16_t)(sfb | (sfb << 8))));
+                            asm("mul.f16x2 %0, %1, %2;" : "=r"(x[rh][0]) : "r"(q0), "r"(sc2));
+                            asm("mul.f16x2 %0, %1, %2;" : "=r"(x[rh][1]) : "r"(q1), "r"(sc2));
                         }
-                    }
-                    const uint32_t slot[4][2] = {{s01.x, s01.y}, {s01.z, s01.w}, {s23.x, s23.y}, {s23.z, s23.w}};
-                    // the MMAs of one half (elements 8h .. 8h+7 of every block): x[k] = four fp16 pairs of slot k
-                    auto half_mma = [&](int h, const uint32_t (&x)[4][4]) {
-                        uint4 b[NH];
 #pragma unroll
-                        for (int nh = 0; nh < NH; ++nh) b[nh] = *reinterpret_cast<const uint4*>(sb + a_off + nh * 4096 + h * 512);
-#pragma unroll
-                        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                            for (int sl = 0; sl < 2; ++sl)
-#pragma unroll
-                                for (int nh = 0; nh < NH; ++nh)
-                                    mma_f16_16816(acc[mt][nh], x[2 * mt][2 * sl], x[2 * mt + 1][2 * sl], x[2 * mt][2 * sl + 1], x[2 * mt + 1][2 * sl + 1],
-                                                  sl ? b[nh].z : b[nh].x, sl ? b[nh].w : b[nh].y);
-                    };
-                    if (!any8) {
-                        // no FP8 block in the warp's part of the unit: every slot holds sixteen E2M1 codes
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            uint32_t x[4][4];
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) dq_nvfp4(slot[k][h], sc2[k], x[k]);
-                            half_mma(h, x);
-                        }
-                    } else {
-                        // second halves of this lane's FP8 blocks: consecutive entries of the unit's overflow list
-                        const uint32_t flags = sc4 & 0x80808080u;
-                        uint32_t idx = ((idx4 >> (8 * hq)) & 0xffu) + *reinterpret_cast<const uint16_t*>(sb + REC_WSTART + 2 * w);
-                        uint2 hi8[4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            hi8[k] = make_uint2(0u, 0u);
-                            if (flags & (0x80u << (8 * k))) {
-                                hi8[k] = (idx * 8u + 8u <= staged) ? *reinterpret_cast<const uint2*>(sb + STG_OVF + idx * 8u)
-                                                                   : __ldg(reinterpret_cast<const uint2*>(ovf_g + (size_t)idx * 8));
-                                ++idx;
-                            }
-                        }
-                        // NVFP4: codes 0..7 in slot word 0, 8..15 in word 1; FP8: codes 0..3, 4..7 in the slot, 8..11, 12..15 in the overflow entry
-                        {
-                            uint32_t x[4][4];
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) dq_mixed(slot[k][0], slot[k][0], slot[k][1], flags & (0x80u << (8 * k)), sc2[k], x[k]);
-                            half_mma(0, x);
-                        }
-                        {
-                            uint32_t x[4][4];
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) dq_mixed(slot[k][1], hi8[k].x, hi8[k].y, flags & (0x80u << (8 * k)), sc2[k], x[k]);
-                            half_mma(1, x);
-                        }
+                        for (int nh = 0; nh < NH; ++nh) mma_f16_16816(acc[mt][nh], x[0][0], x[1][0], x[0][1], x[1][1], b[nh].x, b[nh].y);
+#ifdef FGMP_DEBUG_PRINT
+                        if (blockIdx.x == 0 && lane == 5 && mt == 0 && j < 2) printf("  w %d j %u x %08x %08x b %08x %08x acc %f\n", warp, j, x[0][0], x[1][0], b[0].x, b[0].y, acc[0][0][0]);
+#endif
                     }
                 }
-                // this warp is done with the stage; the group's last warp to say so refills it with the unit S further on
                 __syncwarp();
-                if (lane == 0) {
-                    uint32_t old;
-                    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(smem_u32(done + stage)) : "memory");
-                    if (old == GROUP_WARPS - 1) {
-                        done[stage] = 0;
-                        const int nxt = i + S;
-                        if (nxt < n_units) {
-                            const uint32_t step0 = table[nxt], bytes = (table[nxt + 1] - step0) * 16u;
-                            mbar_expect_tx(full0 + 8 * stage, REC_BYTES + A_BYTES + (bytes < OVF_CAP ? bytes : OVF_CAP));
-                            issue_rec(nxt, stage); issue_ovf(nxt, stage, false); issue_a(nxt, stage);
-                        }
-                    }
-                }
+                if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+                if (++stage == S) { stage = 0; phase ^= 1; }
             }
-
-            // ---- end of a segment (this CTA's units of one tile): the groups' sums are added, then the tile is
-            // written or, if other CTAs share it, handed in; the last CTA to arrive adds the parts in order.
-            // (After a failed wait the barriers below are still passed by everyone; nothing is written.)
-            if (send == n_units) { FGMP_STAMP(7); if (threadIdx.x == DEC_THREADS - 32) FGMP_STAMP_ANY(8); }
+            if (!ok) break;
+            // the epilogue has taken the previous segment's sums; now this segment's go in:
+            // acc[mt][nh] = rows 32jr + 16mt + {g, g + 8} x tokens 8nh + {2t, 2t+1}
+            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-                for (int rh = 0; rh < 2; ++rh) {
-                    const uint32_t r = 32 * jr + 16 * (uint32_t)mt + 8 * (uint32_t)rh + g;
-                    float2* pt = reinterpret_cast<float2*>(epi + part * 2048u + r * 16u + (((tpiece ^ (r >> 1)) & 3u) << 2) + tcol);
-                    pt[0] = make_float2(acc[mt][0][2 * rh], acc[mt][0][2 * rh + 1]);
-                    if (NH == 2)
-                        *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pt) ^ 32) = make_float2(acc[mt][NH - 1][2 * rh], acc[mt][NH - 1][2 * rh + 1]);
+                for (int nh = 0; nh < NH; ++nh) {
+                    const uint32_t r = 32 * jr + 16 * (uint32_t)mt + g, m = 8 * (uint32_t)nh + 2 * t;
+                    tile3[tile_idx(r, m)] = acc[mt][nh][0];
+                    tile3[tile_idx(r, m + 1)] = acc[mt][nh][1];
+                    tile3[tile_idx(r + 8, m)] = acc[mt][nh][2];
+                    tile3[tile_idx(r + 8, m + 1)] = acc[mt][nh][3];
                 }
-            math_bar();
-            const bool good = !*abort_flag;
-            const uint32_t row = threadIdx.x >> 2, tq = threadIdx.x & 3u;      // this thread: tokens 4tq .. 4tq+3 of one row
-            const bool live = tq < 2u * NH;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (live) {
-#pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    const float4 x = *reinterpret_cast<const float4*>(epi + h * 2048 + row * 16u + (((tq ^ (row >> 1)) & 3u) << 2));
-                    v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
-                }
-            }
-            const bool whole = (u_begin + sbeg == tile * C) && (u_begin + send == (tile + 1) * C);
-            bool write_out = whole;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: tensor-memory lane quadrant warp % 4
+        const int q = warp & 3;
+        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+        const float s4a = FUSED ? p.q.s4 : __ldg(&reinterpret_cast<const fgmp_packed_header*>(p.ablob)->scale_fp4);
+        const float alpha = __fmul_rn(s4a, __ldg(&hw->scale_fp4));
+        const float r8 = __int_as_float((127 + __ldg(&hw->fp8_log2_ratio)) << 23);     // FP8 tensor scale / NVFP4 tensor scale of the weights
+        const int row = 32 * q + lane;
+        bool ok = true;
+        int seg = 0;
+        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
+            const int64_t tile = u / C;
+            const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
+            u = seg_end;
+            const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
+            if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 11))) break;
+            tc_fence_after();
+            // a tile shared with other CTAs: how many of them have handed in their sums already (the answer is
+            // needed only after this CTA's own sums are complete, so the load costs nothing)
+            const bool whole = (seg_begin == tile * C) && (seg_end == (tile + 1) * C);
+            int nseg = 1, slot = 0;
+            uint32_t seen = 0;
             if (!whole) {
                 const int64_t c_first = cta_of_unit(tile * C, G, p.total);
                 const int64_t c_last = cta_of_unit((tile + 1) * C - 1, G, p.total);
-                const int nseg = (int)(c_last - c_first + 1), slot_i = (int)(blockIdx.x - c_first);
-                if (live && good) __stcg(reinterpret_cast<float4*>(p.partials + (((size_t)tile * p.maxseg + slot_i) * 128 + row) * 16 + 4 * tq), v);
-                __threadfence();
-                math_bar();
-                // the counter wraps to zero with the last arrival, so the workspace is ready for the next call
-                if (threadIdx.x == 0) s_misc[3] = (good && atomicInc(p.counters + tile, (uint32_t)(nseg - 1)) == (uint32_t)(nseg - 1)) ? 1u : 0u;
-                math_bar();
-                write_out = false;
-                if (s_misc[3]) {
+                nseg = (int)(c_last - c_first + 1);
+                slot = (int)(blockIdx.x - c_first);
+                if (lane == 0) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.counters + tile * 8 + q) : "memory");
+            }
+            uint32_t rr[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(accb * TOK), rr);
+            tc_fence_before();
+            mbar_arrive(acce0 + 8 * accb);
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
+            // corrections (2) and (3) of the segment: this row of every tile, in tile order; the rows of (2)
+            // are cleared for the next segment on the way
+            if (!(ok = mbar_wait(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 12))) break;
+#ifdef FGMP_DEBUG_PRINT
+            if (blockIdx.x == 0 && lane == 1) printf("epi warp %d row %d tile4 %f %f v0 %f\n", warp, row, tiles[4 * TILE_FLOATS + tile_idx(row, 0)], tiles[4 * TILE_FLOATS + tile_idx(row, 1)], v[0]);
+#endif
+            float c2[16];                              // (2): sums of the FP8 weight codes, still without 2^ratio
+#pragma unroll
+            for (int j = 0; j < 16; ++j) c2[j] = 0.f;
+#pragma unroll
+            for (int w = 0; w < NTILES; ++w) {
+                float4* src = reinterpret_cast<float4*>(tiles + w * TILE_FLOATS + row * TOK);
+                float4 x[4];
+#pragma unroll
+                for (int j = 0; j < 2 * NH; ++j) x[j] = src[(j ^ (row >> 1)) & 3];       // tokens 4j .. 4j+3
+#pragma unroll
+                for (int j = 0; j < 2 * NH; ++j) {
+                    if (w < 4) { c2[4 * j] += x[j].x; c2[4 * j + 1] += x[j].y; c2[4 * j + 2] += x[j].z; c2[4 * j + 3] += x[j].w; }
+                    else       { v[4 * j] += x[j].x; v[4 * j + 1] += x[j].y; v[4 * j + 2] += x[j].z; v[4 * j + 3] += x[j].w; }
+                    if (w < 4) src[(j ^ (row >> 1)) & 3] = make_float4(0.f, 0.f, 0.f, 0.f);   // the tile of (3) is overwritten
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] += c2[j] * r8;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tfree);
+
+            const int64_t n = tile * 128 + row;
+            bool write_out = whole;
+            if (!whole) {
+                // partial tile: publish, and let the warp that arrives last add everything up.  When all the
+                // others were seen to have arrived, this warp is the last without asking and skips the counter.
+                float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + row) * 16;
+#pragma unroll
+                for (int j = 0; j < 8 * NH; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+                // The counter wraps to zero with the last arrival (or is put back by the warp that skipped
+                // it), so the workspace is ready for the next call without being cleared.
+                uint32_t old = __shfl_sync(0xffffffffu, seen, 0);
+                if (old != (uint32_t)(nseg - 1)) {
                     __threadfence();
-                    v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (live)
-                        for (int sgi = 0; sgi < nseg; ++sgi) {
-                            const float4 x = __ldcg(reinterpret_cast<const float4*>(p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16 + 4 * tq));
-                            v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+                    __syncwarp();
+                    if (lane == 0) old = atomicInc(p.counters + tile * 8 + q, (uint32_t)(nseg - 1));
+                    old = __shfl_sync(0xffffffffu, old, 0);
+                } else if (lane == 0) {
+                    p.counters[tile * 8 + q] = 0u;
+                }
+                if (old == (uint32_t)(nseg - 1)) {
+                    __threadfence();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                    for (int sgi = 0; sgi < nseg; ++sgi) {       // one sum in slot order
+                        const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16;
+#pragma unroll
+                        for (int j = 0; j < 8 * NH; j += 4) {
+                            const float4 y4 = __ldcg(reinterpret_cast<const float4*>(src + j));
+                            v[j] += y4.x; v[j + 1] += y4.y; v[j + 2] += y4.z; v[j + 3] += y4.w;
                         }
+                    }
                     write_out = true;
                 }
             }
-            const int64_t n = tile * 128 + row;
-            if (write_out && good && live && n < p.N) {
-                const float y[4] = {v.x * alpha, v.y * alpha, v.z * alpha, v.w * alpha};
+            if (write_out && n < p.N) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int64_t m = 4 * tq + i;
-                    if (m < p.M) {
-                        if (p.y_is_bf16) reinterpret_cast<__nv_bfloat16*>(p.Ybf)[m * p.ldy + n] = __float2bfloat16_rn(y[i]);
-                        else p.Y[m * p.ldy + n] = y[i];
+                for (int j = 0; j < 8 * NH; ++j) {
+                    if (j < p.M) {
+                        if (p.y_is_bf16) reinterpret_cast<__nv_bfloat16*>(p.Ybf)[(int64_t)j * p.ldy + n] = __float2bfloat16_rn(v[j] * alpha);
+                        else p.Y[(int64_t)j * p.ldy + n] = v[j] * alpha;
                     }
                 }
             }
-            math_bar();                                // the next segment's sums overwrite the tile
-            sbeg = send;
         }
     }
 
     __syncthreads();
-    FGMP_STAMP(9);
     if (*abort_flag) {
         const unsigned long long t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
@@ -525,9 +753,13 @@ decode_kernel(DecParams p)
         if (atomicInc(p.cw + CW_DONE, (uint32_t)G - 1u) == (uint32_t)G - 1u)
             asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_EPOCH), "r"(tag) : "memory");
     }
+    if (warp == W_MMA) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, DEC_TMEM_COLS);
+    }
 }
 
-struct DecPlan { int64_t tiles, chunks, total; int grid; int maxseg; int64_t span; };
+struct DecPlan { int64_t tiles, chunks, total; int grid; int maxseg; };
 
 DecPlan decode_plan(int64_t N, int64_t K)
 {
@@ -538,7 +770,6 @@ DecPlan decode_plan(int64_t N, int64_t K)
     // a tile of `chunks` units meets at most this many CTA spans of >= floor(total/grid) units
     const int64_t span = d.total / d.grid;
     d.maxseg = (int)((d.chunks + span - 1) / span + 1);
-    d.span = (d.total + d.grid - 1) / d.grid;           // the longest span of a CTA
     return d;
 }
 
@@ -551,24 +782,20 @@ fgmp_status set_attrs_once()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
     std::lock_guard<std::mutex> lk(g_dec_mu);
     if (!g_attr_set[dev]) {
-        const int most = 232448;
-#define FGMP_SET(NG_) \
-        if (cudaFuncSetAttribute(decode_kernel<1, false, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess || \
-            cudaFuncSetAttribute(decode_kernel<2, false, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess || \
-            cudaFuncSetAttribute(decode_kernel<1, true, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess || \
-            cudaFuncSetAttribute(decode_kernel<2, true, NG_>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess) \
+        if (cudaFuncSetAttribute(decode_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DEC_SMEM) != cudaSuccess)
             return FGMP_ERR_CUDA;
-        FGMP_SET(1) FGMP_SET(2) FGMP_SET(4)
-#undef FGMP_SET
         g_attr_set[dev] = true;
     }
     return FGMP_OK;
 }
 
 // Workspace of the decode path, all inside the control area that must be zero before the first call and
-// that every call leaves zero (the call number excepted): status at 0, control words at 256, one
-// stream-K counter per tile from 1024; partial sums behind the control area, then (fused calls) the
-// activation records.
+// that every call leaves zero (the call number excepted): status at 0, control words at 256, stream-K
+// counters from 1024 (32 bytes per tile); partial sums behind the control area, then (fused calls
+// without a packed output) the activation records.
 DecParams base_params(const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                       void* workspace, const DecPlan& d)
 {
@@ -583,10 +810,6 @@ DecParams base_params(const void* packed_weights, void* Y, int y_is_bf16, int64_
     p.counters = reinterpret_cast<uint32_t*>(ws + 1024);
     p.partials = reinterpret_cast<float*>(ws + FGMP_WS_CONTROL_BYTES);
     p.maxseg = d.maxseg;
-    // Ring depth: long spans are bound by the weight stream and want every stage; short ones are bound by
-    // set-up, which a smaller footprint shortens.
-    p.stages = DEC_STAGES;
-    while (p.stages > 2 && dec_smem(p.stages, d.span) > 232448) --p.stages;      // very long spans: their table takes the room of a stage
     return p;
 }
 
@@ -594,17 +817,13 @@ template <bool FUSED>
 fgmp_status launch_decode(const DecParams& p, const DecPlan& d, bool programmatic, cudaStream_t s)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = dec_smem(p.stages, d.span); cfg.stream = s;
+    cfg.gridDim = dim3((unsigned)d.grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = DEC_SMEM; cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = programmatic ? 1 : 0;
-    const int ng = 4;       // measured on Llama-2 shapes: four groups of four warps are the fastest split
-#define FGMP_GO(NG_) \
-    if (p.M <= 8) { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<1, FUSED, NG_>, p)); } \
-    else          { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<2, FUSED, NG_>, p)); }
-    if (ng == 1) { FGMP_GO(1) } else if (ng == 4) { FGMP_GO(4) } else { FGMP_GO(2) }
-#undef FGMP_GO
+    if (p.M <= 8) { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<1, FUSED>, p)); }
+    else          { FGMP_LAUNCH(FGMP_K_DECODE, s, cudaLaunchKernelEx(&cfg, decode_kernel<2, FUSED>, p)); }
     return fgmp_launch_status();
 }
 
@@ -612,11 +831,8 @@ fgmp_status launch_decode(const DecParams& p, const DecPlan& d, bool programmati
 
 bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K)
 {
-    if (!(M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0 &&
-          1024 + ((N + 127) / 128) * 4 <= (int64_t)FGMP_WS_CONTROL_BYTES)) return false;
-    const int64_t total = ((N + 127) / 128) * (K / 256);
-    const int sms = fgmp_sm_count();
-    return (total + sms - 1) / sms <= MAX_SPAN;
+    return M >= 1 && M <= 16 && N >= 1 && K >= 256 && (K % 256) == 0 &&
+           1024 + ((N + 127) / 128) * 32 <= (int64_t)FGMP_WS_CONTROL_BYTES;
 }
 
 size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K)
@@ -643,7 +859,7 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
     p.ablob = (const uint8_t*)packed_acts;
     fgmp_status st = set_attrs_once();
     if (st != FGMP_OK) return st;
-    if (clear_first && cudaMemsetAsync(workspace, 0, 1024 + (size_t)d.tiles * 4, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    if (clear_first && cudaMemsetAsync(workspace, 0, 1024 + (size_t)d.tiles * 32, s) != cudaSuccess) return FGMP_ERR_CUDA;
     return launch_decode<false>(p, d, !clear_first, s);
 }
 

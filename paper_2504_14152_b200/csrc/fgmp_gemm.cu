@@ -57,7 +57,7 @@ __device__ __forceinline__ void nvfp4x16_scaled(const uint2& c, uint32_t scale_c
 // status word of the workspace says so and the kernel leaves.
 __device__ __forceinline__ bool header_matches(const fgmp_packed_header* h, int64_t rows, int64_t K, uint32_t kind, int* status, int where)
 {
-    const bool ok = h->magic == FGMP_MAGIC && h->version == 6u && h->rows == rows && h->K == K && h->kind == kind && h->error == 0;
+    const bool ok = h->magic == FGMP_MAGIC && h->version == 7u && h->rows == rows && h->K == K && h->kind == kind && h->error == 0;
     if (!ok && threadIdx.x == 0) { atomicCAS(status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(status + 1, where); }
     return ok;
 }
@@ -83,35 +83,47 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
     }
 }
 
-// packed weights -> bf16 plane; one CTA of 512 threads per unit, in record order (a thread has the
-// four blocks of one lane of the decode GEMM: all loads first, then the conversions)
-__global__ void __launch_bounds__(512) expand_w_kernel(const uint8_t* __restrict__ blob, int64_t rows, int64_t K, uint4* __restrict__ plane, int* status)
+// packed weights -> bf16 plane; one CTA of 128 threads per unit record, consecutive threads on
+// consecutive blocks of one row, four blocks per thread in flight at a time
+__global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* __restrict__ blob, int64_t rows, int64_t K, uint4* __restrict__ plane, int* status)
 {
-    if (!header_matches(reinterpret_cast<const fgmp_packed_header*>(blob), rows, K, 1u, status, 12)) return;
+    __shared__ UnitScratch sc;
+    const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
+    if (!header_matches(h, rows, K, 1u, status, 12)) return;
     const PackedLayout L = fgmp_layout(rows, K, 1, 0);
+    const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
     const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
-    const UnitLaneView u = fgmp_unit_lane(blob, L, unit);
-    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    const int64_t kb = c * 16 + fgmp_rec_col(w, lane);
+    const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
+    const uint8_t* rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
+    const uint8_t* halves = blob + L.off_ovf + (size_t)reinterpret_cast<const uint32_t*>(blob + L.off_uptr)[unit] * 16 + fgmp_list_halves_offset(cnt);
+    const int j = threadIdx.x & 15;
+    const int64_t kb = c * 16 + j;
     if (kb >= L.KB) return;
-    uint2 slot[4], hi[4];
-    uint32_t idx = u.idx;
+#pragma unroll 1
+    for (int i0 = 0; i0 < 16; i0 += 4) {
+        uint2 slot[4], hi[4];
+        uint32_t sfb[4], pos[4];
 #pragma unroll
-    for (uint32_t k = 0; k < 4; ++k) {
-        slot[k] = __ldg(reinterpret_cast<const uint2*>(u.rec + REC_W4 + w * 1024u + (k >> 1) * 512u + lane * 16u + (k & 1u) * 8u));
-        hi[k] = make_uint2(0u, 0u);
-        if ((u.sc4 >> (8 * k)) & 0x80u) hi[k] = __ldg(reinterpret_cast<const uint2*>(u.ovf + (size_t)(idx++) * 8));
-    }
+        for (int i = 0; i < 4; ++i) {
+            const int row = (threadIdx.x >> 4) + 8 * (i0 + i);
+            pos[i] = sc.pos[row * 16 + j];
+            slot[i] = __ldg(reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j)));
+            sfb[i] = __ldg(rec + REC_SF + fgmp_rec_sf_offset(row, j));
+            hi[i] = make_uint2(0u, 0u);
+            if (pos[i] != 0xffffu) hi[i] = __ldg(reinterpret_cast<const uint2*>(halves + (size_t)pos[i] * 8));
+        }
 #pragma unroll
-    for (uint32_t k = 0; k < 4; ++k) {
-        const int64_t r = tile * 128 + fgmp_rec_row(w, lane, k);
-        if (r >= L.rows) continue;
-        const uint32_t sb = (u.sc4 >> (8 * k)) & 0xffu;
-        float v[16];
-        // an FP8 block's scale byte holds the factor between the tensor scales, 2^ratio
-        if (sb & 0x80u) e4m3x16_scaled(make_uint4(slot[k].x, slot[k].y, hi[k].x, hi[k].y), e4m3_to_f32(sb & 0x7fu), v);
-        else nvfp4x16_scaled(slot[k], sb, v);
-        store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
+        for (int i = 0; i < 4; ++i) {
+            const int row = (threadIdx.x >> 4) + 8 * (i0 + i);
+            const int64_t r = tile * 128 + row;
+            if (r >= L.rows) continue;
+            float v[16];
+            if (pos[i] != 0xffffu) e4m3x16_scaled(make_uint4(slot[i].x, slot[i].y, hi[i].x, hi[i].y), r8, v);
+            else nvfp4x16_scaled(slot[i], sfb[i], v);
+            store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
+        }
     }
 }
 
@@ -280,7 +292,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
     if (p.q.codes4 && blockIdx.x == 0 && threadIdx.x == 0) {
         fgmp_packed_header* h = p.q.header;
-        h->magic = FGMP_MAGIC; h->version = 6; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
+        h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
         h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
         h->error = 0;
     }
@@ -456,7 +468,7 @@ static fgmp_status launch_prefill(const void* packed_acts, const void* packed_we
         const int g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
         FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, reinterpret_cast<uint4*>(planeA), status));
         const PackedLayout LW = fgmp_layout(N, K, 1, 0);
-        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_w_kernel<<<(unsigned)LW.units, 512, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW), status));
+        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_w_kernel<<<(unsigned)LW.units, 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW), status));
     }
     GemmParams p;
     p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K;

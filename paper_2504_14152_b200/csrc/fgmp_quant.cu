@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
     if (!SCORE_ONLY) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
-            h->magic = FGMP_MAGIC; h->version = 6; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
+            h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }
@@ -48,8 +48,10 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
             if (active) {
                 uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
                 const uint32_t j = (uint32_t)kb & 15u, m = (uint32_t)m0;
-                *reinterpret_cast<uint4*>(rec + fgmp_arec_offset(m, j, 0)) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(rec + fgmp_arec_offset(m, j, 1)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset(m, j)) = make_uint2(0u, 0u);
+                rec[AREC_SF + m * 16 + j] = 0;
+                uint4* at = reinterpret_cast<uint4*>(rec + fgmp_arec_at_offset(m, j));
+                at[0] = make_uint4(0, 0, 0, 0); at[1] = make_uint4(0, 0, 0, 0);
             }
             return;
         }
@@ -120,8 +122,14 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
                     }
                     uint8_t* rec = p.arec + (size_t)(kb >> 4) * AREC_BYTES;
                     const uint32_t j = (uint32_t)kb & 15u;
-                    *reinterpret_cast<uint4*>(rec + fgmp_arec_offset((uint32_t)m, j, 0)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    *reinterpret_cast<uint4*>(rec + fgmp_arec_offset((uint32_t)m, j, 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+                    uint4* at = reinterpret_cast<uint4*>(rec + fgmp_arec_at_offset((uint32_t)m, j));
+                    at[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    at[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                    // what the tensor core reads: codes and microscale (both zero for an FP8 block), and the
+                    // chunk's set of block columns that hold an FP8 block of some token
+                    *reinterpret_cast<uint2*>(rec + AREC_A4 + fgmp_rec_w4_offset((uint32_t)m, j)) = make_uint2(c4[0], c4[1]);
+                    rec[AREC_SF + (uint32_t)m * 16 + j] = (uint8_t)sc;
+                    if (is8) atomicOr(reinterpret_cast<unsigned int*>(rec + AREC_HOT), 1u << j);
                 }
                 *reinterpret_cast<uint2*>(p.codes4 + (m * p.K) / 2 + kb * 8) = make_uint2(c4[0], c4[1]);
                 p.sf[fgmp_sf_offset(m, kb, p.K)] = (uint8_t)sc;
@@ -162,33 +170,26 @@ __global__ void unpack_kernel(const uint8_t* blob, int64_t rows, int64_t K,
     }
 }
 
-// packed weights -> canonical arrays; one CTA of 512 threads per unit, in record order
-__global__ void __launch_bounds__(512) unpack_w_kernel(const uint8_t* blob, int64_t rows, int64_t K,
+// packed weights -> canonical arrays; one CTA of 128 threads per unit record
+__global__ void __launch_bounds__(128) unpack_w_kernel(const uint8_t* blob, int64_t rows, int64_t K,
                                                        uint8_t* codes4, uint8_t* codes8, uint8_t* scales, uint32_t* mask)
 {
+    __shared__ UnitScratch sc;
     const PackedLayout L = fgmp_layout(rows, K, 1, 0);
     if (mask) {
         const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-        for (int64_t i = (int64_t)blockIdx.x * 512 + threadIdx.x; i < rows * L.MW; i += (int64_t)gridDim.x * 512) mask[i] = pmask[i];
+        for (int64_t i = (int64_t)blockIdx.x * 128 + threadIdx.x; i < rows * L.MW; i += (int64_t)gridDim.x * 128) mask[i] = pmask[i];
     }
-    const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
-    const UnitLaneView u = fgmp_unit_lane(blob, L, unit);
-    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    const int64_t kb = c * 16 + fgmp_rec_col(w, lane);
-    uint32_t idx = u.idx;
-#pragma unroll 1
-    for (uint32_t k = 0; k < 4; ++k) {
-        const int64_t r = tile * 128 + fgmp_rec_row(w, lane, k);
-        const uint32_t sb = (u.sc4 >> (8 * k)) & 0xffu;
-        const uint2 slot = *reinterpret_cast<const uint2*>(u.rec + REC_W4 + w * 1024u + (k >> 1) * 512u + lane * 16u + (k & 1u) * 8u);
-        uint2 hi = make_uint2(0u, 0u);
-        const bool is8 = (sb & 0x80u) != 0;
-        if (is8) hi = *reinterpret_cast<const uint2*>(u.ovf + (size_t)(idx++) * 8);
-        if (r >= L.rows || kb >= L.KB) continue;
-        if (scales) scales[r * L.KB + kb] = is8 ? (uint8_t)0 : (uint8_t)sb;
-        if (codes4) *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) = is8 ? make_uint2(0u, 0u) : slot;
-        if (codes8) *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) = is8 ? make_uint4(slot.x, slot.y, hi.x, hi.y) : make_uint4(0, 0, 0, 0);
-    }
+    fgmp_for_each_block(blob, L, blockIdx.x, sc, [&](int64_t r, int64_t kb, int row, int j, const uint8_t* rec, const uint8_t* hi) {
+        const uint2 slot = *reinterpret_cast<const uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j));
+        if (scales) scales[r * L.KB + kb] = rec[REC_SF + fgmp_rec_sf_offset(row, j)];
+        if (codes4) *reinterpret_cast<uint2*>(codes4 + (r * K) / 2 + kb * 8) = hi ? make_uint2(0u, 0u) : slot;
+        if (codes8) {
+            uint4 c = make_uint4(0, 0, 0, 0);
+            if (hi) { const uint2 h = *reinterpret_cast<const uint2*>(hi); c = make_uint4(slot.x, slot.y, h.x, h.y); }
+            *reinterpret_cast<uint4*>(codes8 + r * K + kb * 16) = c;
+        }
+    });
 }
 
 // mean of squares per column of a bf16 matrix; thread per column, rows in order (one fp32 multiply
@@ -256,10 +257,12 @@ extern "C" fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx
     p.mask = reinterpret_cast<uint32_t*>(blob + L.off_mask); p.codes8 = blob + L.off_codes8;
     p.header = reinterpret_cast<fgmp_packed_header*>(blob);
     int64_t grid_rows = M;
-    if (M <= 16) {                     // decode-sized batch: also emit the fp16 copy, 16 token rows
+    if (M <= 16) {                     // decode-sized batch: also emit the records of the decode GEMM, 16 token rows
         p.arec = blob + L.off_arec;
         p.rows_per_cta = 1;
         grid_rows = 16;
+        // the sets of hot block columns are OR-ed together by the kernel's threads
+        if (cudaMemset2DAsync(blob + L.off_arec + AREC_HOT, AREC_BYTES, 0, 16, (size_t)L.chunks, s) != cudaSuccess) return FGMP_ERR_CUDA;
     }
     dim3 grid((unsigned)((p.KB + QA_THREADS - 1) / QA_THREADS), (unsigned)((grid_rows + p.rows_per_cta - 1) / p.rows_per_cta));
     if (sm == FGMP_SCORE_LP_ERROR) FGMP_LAUNCH(FGMP_K_ACT_QUANT, s, quant_act_kernel<0, false><<<grid, QA_THREADS, 0, s>>>(p));
@@ -299,7 +302,7 @@ extern "C" fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, 
     if (h.magic != FGMP_MAGIC || h.rows != rows || h.K != K || h.error != 0) return FGMP_ERR_INVALID_ARG;
     if (h.kind == 1) {
         const PackedLayout L = fgmp_layout(rows, K, 1, 0);
-        FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_w_kernel<<<(unsigned)L.units, 512, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
+        FGMP_LAUNCH(FGMP_K_UNPACK, s, unpack_w_kernel<<<(unsigned)L.units, 128, 0, s>>>((const uint8_t*)packed, rows, K, codes4, codes8, scales, mask));
     } else {
         int64_t nblk = rows * (K / 16);
         int grid = (int)((nblk + 255) / 256 < 148 * 16 ? (nblk + 255) / 256 : 148 * 16);

@@ -279,9 +279,9 @@ __global__ void __launch_bounds__(1024) scan_kernel(const uint32_t* in, uint32_t
     if (threadIdx.x == 0 && append_total) out[n] = (uint32_t)carry_s;
 }
 
-// per unit (128-row tile x 16-block K chunk): size of its overflow in 16-byte steps, and the
+// per unit (128-row tile x 16-block K chunk): size of its list of FP8 blocks in 16-byte steps, and the
 // running total of FP8 blocks.  One CTA of 128 threads per unit, a thread per row.
-__global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask, PackedLayout L, uint32_t* ovf_steps,
+__global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask, PackedLayout L, uint32_t* list_steps,
                                                            SelectState* st)
 {
     __shared__ uint32_t s_cnt[4];
@@ -293,17 +293,18 @@ __global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask,
     __syncthreads();
     if (threadIdx.x == 0) {
         const uint32_t cnt = s_cnt[0] + s_cnt[1] + s_cnt[2] + s_cnt[3];
-        ovf_steps[unit] = fgmp_ovf_steps(cnt);
+        list_steps[unit] = fgmp_list_steps(cnt);
         atomicAdd(&st->n_fp8, (unsigned long long)cnt);
     }
 }
 
-// Writes the record of one unit and its overflow entries.  One CTA of 512 threads per unit: thread
-// (w, lane) writes the four blocks that lane `lane` of the decode GEMM's warp w will take.
-__global__ void __launch_bounds__(512) w_emit_kernel(const uint4* W, int64_t ldw8, int ratio, const SelectState* st,
+// Writes the record of one unit (codes and microscales of its NVFP4 blocks, the first halves of its FP8
+// blocks, the per-column running counts) and the list of its FP8 blocks (rows, second halves).  One CTA
+// of 128 threads per unit.
+__global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw8, int ratio, const SelectState* st,
                                                      const uint8_t* sc_in, uint8_t* blob, PackedLayout L, int64_t room_steps)
 {
-    __shared__ uint32_t s_wtot[16];
+    __shared__ UnitScratch sc;
     const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
     const uint32_t* uptr = reinterpret_cast<const uint32_t*>(blob + L.off_uptr);
     const bool fits = (int64_t)uptr[unit + 1] <= room_steps;   // else the blob is too small: header.error says so
@@ -311,45 +312,40 @@ __global__ void __launch_bounds__(512) w_emit_kernel(const uint4* W, int64_t ldw
     const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
     const float inv8 = __fdiv_rn(1.0f, s8);
     const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    const uint32_t j = fgmp_rec_col(w, lane);
-    const int64_t kb = c * 16 + j;
-    uint32_t flags = 0;
-#pragma unroll
-    for (uint32_t k = 0; k < 4; ++k) {
-        const int64_t n = tile * 128 + fgmp_rec_row(w, lane, k);
-        if (kb < L.KB && ((fgmp_chunk_mask(mask, L, n, c) >> j) & 1u)) flags |= 1u << k;
-    }
-    uint32_t wtot;
-    uint32_t idx = fgmp_warp_excl_count(flags, wtot);
-    if (lane == 0) s_wtot[w] = wtot;
-    __syncthreads();
-    uint32_t before = 0, all = 0;
-#pragma unroll
-    for (uint32_t i = 0; i < 16; ++i) { if (i < w) before += s_wtot[i]; all += s_wtot[i]; }
-    idx += before;
+    const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
+    const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
     uint8_t* rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
-    uint8_t* ovf = blob + L.off_ovf + (size_t)uptr[unit] * 16;
-    if (lane == 0) reinterpret_cast<uint16_t*>(rec + REC_WSTART)[w] = (uint16_t)before;
-    if (threadIdx.x < 48) reinterpret_cast<uint16_t*>(rec + REC_WSTART)[16 + threadIdx.x] = threadIdx.x == 0 ? (uint16_t)all : (uint16_t)0;
-    if (fits && threadIdx.x == 0 && (all & 1u)) *reinterpret_cast<uint2*>(ovf + (size_t)all * 8) = make_uint2(0u, 0u);   // padding
-    uint32_t sc4 = 0;
+    uint8_t* rowid = blob + L.off_ovf + (size_t)uptr[unit] * 16;
+    uint8_t* halves = rowid + fgmp_list_halves_offset(cnt);
+    if (threadIdx.x < 64) {                                    // running sums of the per-column counts, then padding
+        uint32_t before = 0;
+        for (int i = 0; i < 16 && i < (int)threadIdx.x; ++i) before += sc.cnt[i];
+        reinterpret_cast<uint16_t*>(rec + REC_KBSTART)[threadIdx.x] = threadIdx.x <= 16 ? (uint16_t)before : (uint16_t)0;
+    }
+    if (fits) {                                                // padding behind the rows and behind the last half
+        for (uint32_t i = cnt + threadIdx.x; i < fgmp_list_halves_offset(cnt); i += 128) rowid[i] = 0;
+        if (threadIdx.x == 0 && (cnt & 1u)) *reinterpret_cast<uint2*>(halves + (size_t)cnt * 8) = make_uint2(0u, 0u);
+    }
+    const int j = threadIdx.x & 15;
 #pragma unroll 1
-    for (uint32_t k = 0; k < 4; ++k) {
-        const int64_t n = tile * 128 + fgmp_rec_row(w, lane, k);
+    for (int i = 0; i < 16; ++i) {
+        const int row = (threadIdx.x >> 4) + 8 * i;
+        const int64_t n = tile * 128 + row, kb = c * 16 + j;
         uint2 slot = make_uint2(0u, 0u);
         uint32_t scale = 0;
         if (n < L.rows && kb < L.KB) {
             float v[16], f[16];
             load_block(W, ldw8, nullptr, 0, n, kb, v, f);
-            if ((flags >> k) & 1u) {
+            const uint32_t pos = sc.pos[row * 16 + j];
+            if (pos != 0xffffu) {
                 uint32_t c8[4];
                 float dq8[16];
                 block_fp8(v, inv8, s8, c8, dq8);
                 slot = make_uint2(c8[0], c8[1]);
-                if (fits) *reinterpret_cast<uint2*>(ovf + (size_t)idx * 8) = make_uint2(c8[2], c8[3]);
-                ++idx;
-                scale = 0x80u | fgmp_pow2_e4m3(ratio);
+                if (fits) {
+                    *reinterpret_cast<uint2*>(halves + (size_t)pos * 8) = make_uint2(c8[2], c8[3]);
+                    rowid[pos] = (uint8_t)row;
+                }
             } else {
                 float dq4[16];
                 uint32_t c4[2];
@@ -358,10 +354,9 @@ __global__ void __launch_bounds__(512) w_emit_kernel(const uint4* W, int64_t ldw
                 slot = make_uint2(c4[0], c4[1]);
             }
         }
-        *reinterpret_cast<uint2*>(rec + REC_W4 + w * 1024u + (k >> 1) * 512u + lane * 16u + (k & 1u) * 8u) = slot;
-        sc4 |= scale << (8 * k);
+        *reinterpret_cast<uint2*>(rec + REC_W4 + fgmp_rec_w4_offset(row, j)) = slot;
+        rec[REC_SF + fgmp_rec_sf_offset(row, j)] = (uint8_t)scale;
     }
-    *reinterpret_cast<uint32_t*>(rec + REC_SF + (w >> 2) * 512u + lane * 16u + (w & 3u) * 4u) = sc4;
 }
 
 // With too little room the starts of the overflow entries are pulled back inside the blob, so that a
@@ -378,7 +373,7 @@ __global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, co
                                 float* tau_eff_out)
 {
     if (threadIdx.x == 0) {
-        h->magic = FGMP_MAGIC; h->version = 6; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
+        h->magic = FGMP_MAGIC; h->version = 7; h->rows = N; h->K = K; h->scale_fp4 = st->s4;
         h->fp8_log2_ratio = ratio; h->n_fp8 = (int64_t)st->n_fp8; h->kind = 1; h->capacity = room_steps;
         float teff = fraction_mode ? st->tau : tau_given;
         h->tau_eff = teff;
@@ -453,7 +448,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
         k = (int64_t)floor(fp8_fraction * (double)B + 0.5);
         if (k > B) k = B;
     }
-    // room for the overflow entries, in 16-byte steps
+    // room for the lists of FP8 blocks, in 16-byte steps
     const PackedLayout L = fgmp_layout(N, K, 1, 0);
     if (packed_bytes < L.total) return FGMP_ERR_WORKSPACE;
     const int64_t room_steps = (int64_t)((packed_bytes - L.off_ovf) / 16);
@@ -503,7 +498,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a));
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_unit_count_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, L, tmp_a, st));
     FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, uptr, NCT, nullptr, 1));
-    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<(unsigned)NCT, 512, 0, s>>>(W, ldw / 8, ratio, st, sc_tmp, blob, L, room_steps));
+    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<(unsigned)NCT, 128, 0, s>>>(W, ldw / 8, ratio, st, sc_tmp, blob, L, room_steps));
     FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, uptr, NCT, N, K, ratio,
                                      room_steps, fraction_mode ? 1 : 0, tau, tau_eff_out));
     FGMP_LAUNCH(FGMP_K_W_AUX, s, w_clamp_uptr_kernel<<<grid_for(NCT + 1, 256, 1), 256, 0, s>>>(reinterpret_cast<const fgmp_packed_header*>(blob), uptr, NCT + 1, room_steps));

@@ -7,14 +7,10 @@
 int main()
 {
     for (uint32_t m = 0; m < 16; ++m)
-        for (uint32_t j = 0; j < 16; ++j)
-            for (uint32_t half = 0; half < 2; ++half) printf("arec %u %u %u %u\n", m, j, half, fgmp_arec_offset(m, j, half));
+        for (uint32_t j = 0; j < 16; ++j) printf("arec %u %u %u %u\n", m, j, fgmp_arec_at_offset(m, j), fgmp_rec_w4_offset(m, j));
     for (uint32_t r = 0; r < 128; ++r)
-        for (uint32_t j = 0; j < 16; ++j)
-            printf("rec %u %u %u %u %u %u %u %u %u %u\n", r, j, fgmp_rec_w4_offset(r, j), fgmp_rec_sf_offset(r, j), fgmp_rec_order(r, j),
-                   fgmp_rec_warp(r, j), fgmp_rec_lane(r, j), fgmp_rec_slot(r, j),
-                   fgmp_rec_row(fgmp_rec_warp(r, j), fgmp_rec_lane(r, j), fgmp_rec_slot(r, j)), fgmp_rec_col(fgmp_rec_warp(r, j), fgmp_rec_lane(r, j)));
-    for (int ratio = -7; ratio <= 7; ++ratio) printf("pow2 %d %u\n", ratio, fgmp_pow2_e4m3(ratio));
-    printf("const %u %u %u %u %u\n", AREC_BYTES, REC_W4, REC_SF, REC_WSTART, REC_BYTES);
+        for (uint32_t j = 0; j < 16; ++j) printf("rec %u %u %u %u\n", r, j, fgmp_rec_w4_offset(r, j), fgmp_rec_sf_offset(r, j));
+    for (uint32_t cnt = 0; cnt < 40; ++cnt) printf("list %u %u %u\n", cnt, fgmp_list_halves_offset(cnt), fgmp_list_steps(cnt));
+    printf("const %u %u %u %u %u %u %u %u %u\n", AREC_BYTES, AREC_A4, AREC_SF, AREC_HOT, AREC_AT, REC_W4, REC_SF, REC_KBSTART, REC_BYTES);
     return 0;
 }
