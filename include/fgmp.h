@@ -34,28 +34,28 @@
  *                   0x00 for FP8 blocks
  *   mask          : rows * ceil(K/16/32) uint32; bit j of word w of a row = block 32w+j,
  *                   1 = FP8
- *   arec          : (rows <= 16 only) C records of 8192 bytes, one per chunk, holding what the
- *                   decode-sized GEMM streams: the quantized values of 16 token rows divided by
- *                   the tensor scale, in fp16 (exact), in the order that kernel's mma.sync
- *                   fragments take them: token octet m/8 in its own 4096 bytes; there piece
- *                   2*(j%4) + h of 512 bytes holds elements 8h .. 8h+7 of block column j of the
- *                   chunk for token m, 16 bytes at lane position 4*(m%8) + j/4; token rows >=
- *                   rows are zero
+ *   arec          : (rows <= 16 only) C records of 10752 bytes, one per chunk, holding what the
+ *                   decode-sized GEMM streams, for 16 token rows (rows >= M are zero):
+ *                   2048 B: the E2M1 codes as a 16-row x 128-byte tile, the 16-byte pieces of row m
+ *                   XOR-swizzled with m%8 (zero in FP8 blocks) | 256 B: E4M3 microscales [token][block
+ *                   column], 0x00 for FP8 blocks | 16 B: uint32 whose bit j says that block column j of
+ *                   some token is FP8, padding | 256 B padding | 8192 B: every element over the tensor
+ *                   scale in fp16 (exact for either format): token octet m/8 in its own 4096 bytes, there
+ *                   256 bytes per block column, there 32 bytes per token
  *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written (the
  *                   blob is sized for the worst case of every block being FP8)
  *
- * Weights: header | mask | uptr | records | overflow
- *   record        : 18560 bytes per unit, unit (t, c) at index t*C + c, in the order in which the
- *                   decode-sized GEMM's 16 warps read it: warp w = 4*(r/32) + j%4, lane 4*(r%8) + j/4
- *                   and slot k = (r/8)%4 hold block (row r of the tile, block column j of the chunk).
- *                   16384 B of 8-byte slots at w*1024 + (k/2)*512 + lane*16 + (k%2)*8: the 16 E2M1
- *                   codes of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block (zero beyond N)
- *                   | 2048 B of scale bytes at (w/4)*512 + lane*16 + (w%4)*4 + k: the E4M3 microscale of an NVFP4
- *                   block (bit 7 clear), or 0x80 | E4M3(2^fp8_log2_ratio) for an FP8 block
- *                   | 128 B: uint16 x 17, FP8 blocks of the unit before warp w's; entry 16 = all
- *   overflow      : E4M3 codes 8..15 of the FP8 blocks, 8 bytes each, unit by unit, inside a unit in
- *                   (w, lane, k) order, each unit padded to 16 bytes
- *   uptr          : uint32 [units + 1]: start of a unit's overflow entries in 16-byte steps
+ * Weights: header | mask | uptr | records | lists
+ *   record        : 18560 bytes per unit, unit (t, c) at index t*C + c:
+ *                   16384 B of 8-byte slots as a 128-row x 128-byte tile, the 16-byte pieces of row r
+ *                   XOR-swizzled with r%8 (the K-major layout the tensor core reads): the 16 E2M1 codes
+ *                   of an NVFP4 block, or E4M3 codes 0..7 of an FP8 block (zero beyond N)
+ *                   | 2048 B of E4M3 microscales, 0x00 for FP8 blocks, in the order they go to tensor
+ *                   memory: byte of (row r, block column j) = (j/4)*512 + (r%32)*16 + (r/32)*4 + j%4
+ *                   | 128 B: uint16 x 17, FP8 blocks of the unit before block column j; entry 16 = all
+ *   list          : per unit, its FP8 blocks ordered by (block column, row): the row of each (one byte,
+ *                   padded to 16), then E4M3 codes 8..15 of each (8 bytes, padded to 16)
+ *   uptr          : uint32 [units + 1]: start of a unit's list in 16-byte steps
  *                   fgmp_weights_bytes(N, K, max_fp8_blocks) leaves room for that many FP8 blocks.
  */
 #ifndef FGMP_H
@@ -98,14 +98,14 @@ typedef struct {
 /* First 256 bytes of a packed blob (device memory). */
 typedef struct {
     uint32_t magic;          /* 'FGMP' = 0x504d4746                                         */
-    uint32_t version;        /* layout version, 6                                           */
+    uint32_t version;        /* layout version, 7                                           */
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;
     int64_t n_fp8;           /* number of FP8 blocks                                        */
     float tau_eff;           /* weights, fraction mode: smallest selected score             */
     uint32_t kind;           /* 0 = activations, 1 = weights                                */
-    int64_t capacity;        /* weights: room for overflow entries, in 16-byte steps        */
+    int64_t capacity;        /* weights: room for the FP8 lists, in 16-byte steps            */
     int32_t error;           /* 0, or FGMP_ERR_CAPACITY                                     */
     int32_t reserved[49];
 } fgmp_packed_header;

@@ -31,8 +31,10 @@
 // order: results are reproducible bit for bit.
 //
 // Warp roles (576 threads): warp 0 = producer, warp 1 = MMA issuer and owner of the tensor memory,
-// warps 2-5 = block scales into tensor memory (one lane quadrant each), warps 6-9 = (2), four block
-// columns each, warps 10-13 = (3), 32 rows each, warps 14-17 = epilogue (one lane quadrant each).
+// warps 2-9 = (2): two sets of four warps that take alternate units, four block columns per warp (a warp
+// copies what it needs of a unit into registers and gives the stage back at once), warps 10-13 = block
+// scales into tensor memory (one lane quadrant each), then (3), 32 rows each, warps 14-17 = epilogue
+// (one lane quadrant each).
 #include "fgmp_common.cuh"
 #include "fgmp_actq.cuh"
 #include "fgmp_host.h"
@@ -45,15 +47,16 @@
 namespace {
 
 constexpr int DEC_WARPS = 18, DEC_THREADS = 32 * DEC_WARPS;
-constexpr int W_PROD = 0, W_MMA = 1, W_SCALE = 2, W_FP8 = 6, W_HOT = 10, W_EPI = 14;
+constexpr int W_PROD = 0, W_MMA = 1, W_FP8 = 2, W_HOT = 10, W_EPI = 14;
+constexpr int FP8_WARPS = W_HOT - W_FP8;        // two sets of four: a set takes every second unit
 constexpr int Q_THREADS = 32 * 16;              // warps 2..17 share out the prologue quantizer
 constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
 constexpr uint32_t LIST_CAP = 2944;             // bytes of a unit's FP8 list that fit a stage (about 320 blocks); more is read from global
 constexpr uint32_t STG_LIST = REC_BYTES;                                                         // 18560
 constexpr uint32_t STG_A = STG_LIST + LIST_CAP;                                                  // 21504, 1 KiB aligned
 constexpr uint32_t DEC_STAGE_BYTES = 32768;
-constexpr int DEC_STAGES = 5;
-constexpr int NTILES = 5;                       // [row][token] fp32 tiles: one per (2) warp, one shared by the (3) warps
+constexpr int DEC_STAGES = 4;
+constexpr int NTILES = FP8_WARPS + 1;           // [row][token] fp32 tiles: one per (2) warp, one shared by the (3) warps
 constexpr uint32_t TILE_FLOATS = 128 * TOK;
 constexpr uint32_t SF_COL0 = 32;                // tensor memory: 2 x 16 accumulator columns, then 32 scale columns per stage
 constexpr uint32_t DEC_TMEM_COLS = 256;
@@ -246,7 +249,7 @@ decode_kernel(DecParams p)
                 mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1 + 8); mbar_init(sfr0 + 8 * s, 4);
             }
             for (int b = 0; b < 2; ++b) {
-                mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); mbar_init(cdone0 + 8 * b, 8);
+                mbar_init(accf0 + 8 * b, 1); mbar_init(acce0 + 8 * b, 128); mbar_init(cdone0 + 8 * b, FP8_WARPS + 4);
             }
             mbar_init(tfree, 4);
             *abort_flag = 0;
@@ -274,7 +277,7 @@ decode_kernel(DecParams p)
     if (warp == W_MMA) tmem_alloc(smem_u32(tmem_slot), DEC_TMEM_COLS);
     if (warp >= W_FP8 && warp < W_EPI) {               // the tiles start at zero
         float4* z = reinterpret_cast<float4*>(tiles);
-        for (int i = (warp - W_FP8) * 32 + lane; i < (int)(NTILES * TILE_FLOATS / 4); i += 8 * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = (warp - W_FP8) * 32 + lane; i < (int)(NTILES * TILE_FLOATS / 4); i += (W_EPI - W_FP8) * 32) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     tc_fence_before();
     __syncthreads();
@@ -296,7 +299,7 @@ decode_kernel(DecParams p)
     const uint32_t tag = FUSED ? s_misc[0] : 0u;
     const bool dead = *abort_flag != 0;                // the weight blob does not belong to this call: nothing else is read
 
-    if (FUSED && !dead && warp >= W_SCALE) {
+    if (FUSED && !dead && warp >= W_FP8) {
         // The quantizer's work items (chunks) are handed out through a counter, so that every item is taken by
         // a CTA that is running: no CTA ever waits for one that has not started.  The counter and the count of
         // finished items wrap to zero with the call's last access.
@@ -394,58 +397,62 @@ decode_kernel(DecParams p)
             if (ok && lane == 0) umma_commit(accf0 + 8 * acc);
             __syncwarp();
         }
-    } else if (warp < W_FP8) {
-        // ------------------------------------------------------------ block scales into tensor memory, lane quadrant warp % 4
-        // Lane i holds, for MMA step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3 --
-        // 16 bytes of scale tile j of the record; the token scales follow in columns 16..31 (16 tokens: lanes
-        // 0..15, first column of every step), zeroed in the chunk's hot block columns.
-        int stage = 0; uint32_t phase = 0; bool ok = true;
-        for (int64_t u = u_begin; u < u_end && ok; ++u) {
-            if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 4))) break;
-            const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
-            const uint8_t* sa = sb + STG_A;
-            uint32_t r[16];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
-                r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
-            }
-            const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
-            tmem_st16(sf_t, r);
-            const uint32_t cold = ~*reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
-            const uint4 ts = *reinterpret_cast<const uint4*>(sa + AREC_SF + (lane & 15) * 16);
-            const uint32_t tsw[4] = {ts.x, ts.y, ts.z, ts.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                // bits 4j .. 4j+3 of `cold` spread to the four bytes of the step's scale word
-                const uint32_t keep = ((((cold >> (4 * j)) & 0xfu) * 0x00204081u) & 0x01010101u) * 0xffu;
-                r[4 * j] = lane < 16 ? (tsw[j] & keep) : 0u;
-                r[4 * j + 1] = 0u; r[4 * j + 2] = 0u; r[4 * j + 3] = 0u;
-            }
-            tmem_st16(sf_t + 16, r);
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
-            if (++stage == S) { stage = 0; phase ^= 1; }
-        }
     } else if (warp < W_HOT) {
         // ------------------------------------------------------------ (2): FP8 weight blocks of block columns bq, bq+4, bq+8, bq+12
-        // The E4M3 codes go into the MMA as they are; the factor 2^ratio between the FP8 and NVFP4
-        // tensor scales is applied once to the tile sums in the epilogue.
-        const int bq = warp - W_FP8;
+        // of every second unit.  The E4M3 codes go into the MMA as they are; the factor 2^ratio between the
+        // FP8 and NVFP4 tensor scales is applied once to the tile sums in the epilogue.
+        const int bq = (warp - W_FP8) & 3, par = (warp - W_FP8) >> 2;
         const uint32_t g = lane >> 2, t = lane & 3;
-        float* mytile = tiles + bq * TILE_FLOATS;
+        float* mytile = tiles + (warp - W_FP8) * TILE_FLOATS;
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
+        // tile[row][tokens] += sums of one group.  Within one column every block has its own row, so the
+        // read-modify-writes of a group touch distinct addresses: all loads first, then all stores.
+        auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t rowA, uint32_t rowB) {
+            float2 *pA = nullptr, *pB = nullptr;    // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on (piece ^ 2)
+            float2 vA0 = make_float2(0.f, 0.f), vA1 = vA0, vB0 = vA0, vB1 = vA0;
+            if (rowA != 0xffffffffu) {
+                pA = reinterpret_cast<float2*>(mytile + rowA * 16u + (((tpiece ^ (rowA >> 1)) & 3u) << 2) + tcol);
+                vA0 = pA[0];
+                if (NH == 2) vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
+            }
+            if (rowB != 0xffffffffu) {
+                pB = reinterpret_cast<float2*>(mytile + rowB * 16u + (((tpiece ^ (rowB >> 1)) & 3u) << 2) + tcol);
+                vB0 = pB[0];
+                if (NH == 2) vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
+            }
+            if (rowA != 0xffffffffu) {
+                pA[0] = make_float2(vA0.x + c[0], vA0.y + c[1]);
+                if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(vA1.x + d[0], vA1.y + d[1]);
+            }
+            if (rowB != 0xffffffffu) {
+                pB[0] = make_float2(vB0.x + c[2], vB0.y + c[3]);
+                if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(vB1.x + d[2], vB1.y + d[3]);
+            }
+            __syncwarp();                  // a later group may add to the same rows
+        };
+        // blocks iA = e + g and iB = e + g + 8 of a group as the M side of the mma.sync (tokens 0-7 and 8-15 as N);
+        // c/d[0..1]: block iA, tokens 2t, 2t+1 / 8+2t, 9+2t; [2..3]: block iB
+        auto group_mma = [&](uint32_t rawA, uint32_t rawB, const uint2& bt0, const uint2& bt1, float (&c)[4], float (&d)[4]) {
+            uint32_t a0, a1, a2, a3;
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a0) : "h"((uint16_t)rawA));
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a2) : "h"((uint16_t)(rawA >> 16)));
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a1) : "h"((uint16_t)rawB));
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a3) : "h"((uint16_t)(rawB >> 16)));
+            c[0] = c[1] = c[2] = c[3] = 0.f; d[0] = d[1] = d[2] = d[3] = 0.f;
+            mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);
+            if (NH == 2) mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);
+        };
 
-        int stage = 0; uint32_t phase = 0; bool ok = true;
+        bool ok = true;
         int seg = 0;
-        for (int64_t u = u_begin; u < u_end && ok; ++seg) {
-            const int64_t tile = u / C;
-            const int64_t seg_end = min(u_end, (tile + 1) * C);
+        const int n_units = (int)(u_end - u_begin);
+        for (int sbeg = 0; sbeg < n_units && ok; ++seg) {
+            const int64_t tile = (u_begin + sbeg) / C;
+            const int send = (int)min((int64_t)n_units, (tile + 1) * C - u_begin);
             // the epilogue has taken (and cleared) the previous segment's sums
             if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
-            for (; u < seg_end; ++u) {
+            for (int i = sbeg + ((par ^ sbeg) & 1); i < send; i += 2) {
+                const int stage = i % S; const uint32_t phase = (uint32_t)(i / S) & 1u;
                 if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
@@ -454,109 +461,86 @@ decode_kernel(DecParams p)
                 const uint16_t* kbs = reinterpret_cast<const uint16_t*>(sb + REC_KBSTART);
                 const uint32_t ntot = kbs[16];
                 const uint32_t hoff = fgmp_list_halves_offset(ntot);
-                // ALL = the whole list of the unit is in the stage (the usual case); otherwise its tail is read
-                // from global memory
-                auto body = [&](auto all_c) {
-                    constexpr bool ALL = decltype(all_c)::value;
-                    // One group of up to 16 blocks of column j: blocks e + g and e + g + 8 are the M side of the
-                    // mma.sync (tokens 0-7 and 8-15 as N).  Lane t has elements 4t .. 4t+3 of a block: from its slot
-                    // in the record (t < 2) or from the list (t >= 2).
-                    // c/d[0..1]: block iA, tokens 2t, 2t+1 / 8+2t, 9+2t; [2..3]: block iB.
-                    auto group_mma = [&](uint32_t j, uint32_t e, uint32_t end_, const uint2& bt0, const uint2& bt1, float (&c)[4], float (&d)[4],
-                                         uint32_t& rowA, uint32_t& rowB) {
-                        const uint32_t iA = e + g, iB = iA + 8;
-                        uint32_t rawA = 0, rawB = 0;
-                        rowA = 0xffffffffu; rowB = 0xffffffffu;
-                        auto fetch = [&](uint32_t i, uint32_t& row, uint32_t& raw) {
-                            row = (ALL || i < staged) ? sb[STG_LIST + i] : __ldg(list_g + i);
-                            if (t < 2) {
-                                raw = *reinterpret_cast<const uint32_t*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j) + 4 * t);
-                            } else {
-                                const uint32_t o = hoff + i * 8 + 4 * (t - 2);
-                                raw = (ALL || o + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + o)
-                                                               : __ldg(reinterpret_cast<const uint32_t*>(list_g + o));
-                            }
-                        };
-                        if (iA < end_) fetch(iA, rowA, rawA);
-                        if (iB < end_) fetch(iB, rowB, rawB);
-                        uint32_t a0, a1, a2, a3;
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a0) : "h"((uint16_t)rawA));
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a2) : "h"((uint16_t)(rawA >> 16)));
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a1) : "h"((uint16_t)rawB));
-                        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a3) : "h"((uint16_t)(rawB >> 16)));
-                        c[0] = c[1] = c[2] = c[3] = 0.f; d[0] = d[1] = d[2] = d[3] = 0.f;
-                        mma_f16_16816(c, a0, a1, a2, a3, bt0.x, bt0.y);
-                        if (NH == 2) mma_f16_16816(d, a0, a1, a2, a3, bt1.x, bt1.y);
-                    };
-                    // Within one column every block has its own row, so the read-modify-writes of a group touch
-                    // distinct addresses in every lane and across lanes: all loads first, then all stores.
-                    auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t rowA, uint32_t rowB) {
-                        float2 *pA = nullptr, *pB = nullptr;    // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on (piece ^ 2)
-                        float2 vA0 = make_float2(0.f, 0.f), vA1 = vA0, vB0 = vA0, vB1 = vA0;
-                        if (rowA != 0xffffffffu) {
-                            pA = reinterpret_cast<float2*>(mytile + rowA * 16u + (((tpiece ^ (rowA >> 1)) & 3u) << 2) + tcol);
-                            vA0 = pA[0];
-                            if (NH == 2) vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
+                const bool all = hoff + ntot * 8 <= staged;        // the whole list is in the stage (the usual case)
+                uint32_t st[4], en[4], rowA[8], rowB[8], rawA[8], rawB[8];     // [4 gr + cc]: group gr (blocks 16 gr ..) of column cc
+                uint2 bt0[4], bt1[4];
+                bool plain = all;                                  // ... and no column has more than two groups of 16
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const uint32_t j = (uint32_t)bq + 4u * cc;
+                    st[cc] = kbs[j]; en[cc] = kbs[j + 1];
+                    plain = plain && (en[cc] - st[cc] <= 32u);
+                    bt0[cc] = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g, j) + 8 * t);
+                    bt1[cc] = make_uint2(0u, 0u);
+                    if (NH == 2) bt1[cc] = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j) + 8 * t);
+                }
+                if (plain) {
+                    // Everything the four columns need, into registers.  Lane t has elements 4t .. 4t+3 of a block:
+                    // from its slot in the record (t < 2) or from the list (t >= 2).
+#pragma unroll
+                    for (int gr = 0; gr < 2; ++gr)
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) {
+                            const uint32_t j = (uint32_t)bq + 4u * cc;
+                            const uint32_t iA = st[cc] + 16u * gr + g, iB = iA + 8;
+                            const bool hasA = iA < en[cc], hasB = iB < en[cc];
+                            const uint32_t rA = hasA ? sb[STG_LIST + iA] : 0u, rB = hasB ? sb[STG_LIST + iB] : 0u;
+                            const uint32_t oA = t < 2 ? REC_W4 + fgmp_rec_w4_offset(rA, j) + 4 * t : STG_LIST + hoff + iA * 8 + 4 * (t - 2);
+                            const uint32_t oB = t < 2 ? REC_W4 + fgmp_rec_w4_offset(rB, j) + 4 * t : STG_LIST + hoff + iB * 8 + 4 * (t - 2);
+                            rawA[4 * gr + cc] = hasA ? *reinterpret_cast<const uint32_t*>(sb + oA) : 0u;
+                            rawB[4 * gr + cc] = hasB ? *reinterpret_cast<const uint32_t*>(sb + oB) : 0u;
+                            rowA[4 * gr + cc] = hasA ? rA : 0xffffffffu;
+                            rowB[4 * gr + cc] = hasB ? rB : 0xffffffffu;
                         }
-                        if (rowB != 0xffffffffu) {
-                            pB = reinterpret_cast<float2*>(mytile + rowB * 16u + (((tpiece ^ (rowB >> 1)) & 3u) << 2) + tcol);
-                            vB0 = pB[0];
-                            if (NH == 2) vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
+                } else {
+                    // a list that does not fit the stage, or a column with more than 32 FP8 blocks (rare): group by
+                    // group straight from the stage or from global memory, before the stage is given back
+                    auto fetch = [&](uint32_t j, uint32_t i_, uint32_t& row, uint32_t& raw) {
+                        row = (all || i_ < staged) ? sb[STG_LIST + i_] : __ldg(list_g + i_);
+                        if (t < 2) {
+                            raw = *reinterpret_cast<const uint32_t*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j) + 4 * t);
+                        } else {
+                            const uint32_t o = hoff + i_ * 8 + 4 * (t - 2);
+                            raw = (all || o + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + o)
+                                                           : __ldg(reinterpret_cast<const uint32_t*>(list_g + o));
                         }
-                        if (rowA != 0xffffffffu) {
-                            pA[0] = make_float2(vA0.x + c[0], vA0.y + c[1]);
-                            if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(vA1.x + d[0], vA1.y + d[1]);
-                        }
-                        if (rowB != 0xffffffffu) {
-                            pB[0] = make_float2(vB0.x + c[2], vB0.y + c[3]);
-                            if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(vB1.x + d[2], vB1.y + d[3]);
-                        }
-                        __syncwarp();                  // a later group may add to the same rows
                     };
 #pragma unroll 1
-                    for (int cp = 0; cp < 2; ++cp) {
-                        // two block columns side by side (their MMAs are independent), then their sums in order
-                        const uint32_t j0 = (uint32_t)bq + 8u * cp, j1 = j0 + 4u;
-                        const uint32_t st0 = kbs[j0], en0 = kbs[j0 + 1], st1 = kbs[j1], en1 = kbs[j1 + 1];
-                        // B fragments: true activation values of tokens g and g + 8, elements 4t..4t+3 of each column
-                        const uint2 b00 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g, j0) + 8 * t);
-                        const uint2 b10 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g, j1) + 8 * t);
-                        uint2 b01 = make_uint2(0u, 0u), b11 = b01;
-                        if (NH == 2) {
-                            b01 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j0) + 8 * t);
-                            b11 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j1) + 8 * t);
-                        }
-                        {
-                            float c0[4], d0[4], c1[4], d1[4];
-                            uint32_t rA0, rB0, rA1, rB1;
-                            group_mma(j0, st0, en0, b00, b01, c0, d0, rA0, rB0);
-                            group_mma(j1, st1, en1, b10, b11, c1, d1, rA1, rB1);
-                            group_add(c0, d0, rA0, rB0);
-                            group_add(c1, d1, rA1, rB1);
-                        }
-                        // columns with more than 16 FP8 blocks
-                        for (uint32_t e = st0 + 16; e < en0; e += 16) {
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const uint32_t j = (uint32_t)bq + 4u * cc;
+                        const uint32_t st_ = kbs[j], en_ = kbs[j + 1];
+                        const uint2 b0 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g, j) + 8 * t);
+                        uint2 b1 = make_uint2(0u, 0u);
+                        if (NH == 2) b1 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j) + 8 * t);
+                        for (uint32_t e = st_; e < en_; e += 16) {
+                            uint32_t rA = 0xffffffffu, rB = 0xffffffffu, wA = 0u, wB = 0u;
+                            if (e + g < en_) fetch(j, e + g, rA, wA);
+                            if (e + g + 8 < en_) fetch(j, e + g + 8, rB, wB);
                             float c[4], d[4];
-                            uint32_t rA, rB;
-                            group_mma(j0, e, en0, b00, b01, c, d, rA, rB);
-                            group_add(c, d, rA, rB);
-                        }
-                        for (uint32_t e = st1 + 16; e < en1; e += 16) {
-                            float c[4], d[4];
-                            uint32_t rA, rB;
-                            group_mma(j1, e, en1, b10, b11, c, d, rA, rB);
+                            group_mma(wA, wB, b0, b1, c, d);
                             group_add(c, d, rA, rB);
                         }
                     }
-                };
-                if (ntot && hoff + ntot * 8 <= staged) body(std::true_type{}); else if (ntot) body(std::false_type{});
+                }
+                // the stage is no longer needed
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-                if (++stage == S) { stage = 0; phase ^= 1; }
+                if (plain) {
+#pragma unroll
+                    for (int gr = 0; gr < 2; ++gr)
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) {
+                            if (gr == 1 && en[cc] - st[cc] <= 16u) continue;      // (the same for every lane)
+                            float c[4], d[4];
+                            group_mma(rawA[4 * gr + cc], rawB[4 * gr + cc], bt0[cc], bt1[cc], c, d);
+                            group_add(c, d, rowA[4 * gr + cc], rowB[4 * gr + cc]);
+                        }
+                }
             }
             if (!ok) break;
             __syncwarp();
             if (lane == 0) mbar_arrive(cdone0 + 8 * (seg & 1));
+            sbeg = send;
         }
     } else if (warp < W_EPI) {
         // ------------------------------------------------------------ (3): hot block columns, rows 32jr .. 32jr+31
@@ -564,7 +548,7 @@ decode_kernel(DecParams p)
         // bytes and the block's microscale (zero for an FP8 weight block, which (2) covers).
         const uint32_t jr = (uint32_t)(warp - W_HOT);
         const uint32_t g = lane >> 2, t = lane & 3;
-        float* tile3 = tiles + 4 * TILE_FLOATS;
+        float* tile3 = tiles + FP8_WARPS * TILE_FLOATS;
         int stage = 0; uint32_t phase = 0; bool ok = true;
         int seg = 0;
         for (int64_t u = u_begin; u < u_end && ok; ++seg) {
@@ -579,7 +563,36 @@ decode_kernel(DecParams p)
                 if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 6))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
-                uint32_t todo = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT) & 0xffffu;
+                const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
+                {
+                    // Block scales of the unit into tensor memory, lane quadrant warp % 4: lane i holds, for MMA step j,
+                    // the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3 -- 16 bytes of scale tile j of
+                    // the record; the token scales follow in columns 16..31 (16 tokens: lanes 0..15, first column of
+                    // every step), zeroed in the chunk's hot block columns.
+                    uint32_t r[16];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
+                        r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                    }
+                    const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
+                    tmem_st16(sf_t, r);
+                    const uint4 ts = *reinterpret_cast<const uint4*>(sa + AREC_SF + (lane & 15) * 16);
+                    const uint32_t tsw[4] = {ts.x, ts.y, ts.z, ts.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // bits 4j .. 4j+3 of the cold columns spread to the four bytes of the step's scale word
+                        const uint32_t keep = ((((~hot >> (4 * j)) & 0xfu) * 0x00204081u) & 0x01010101u) * 0xffu;
+                        r[4 * j] = lane < 16 ? (tsw[j] & keep) : 0u;
+                        r[4 * j + 1] = 0u; r[4 * j + 2] = 0u; r[4 * j + 3] = 0u;
+                    }
+                    tmem_st16(sf_t + 16, r);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
+                }
+                uint32_t todo = hot & 0xffffu;
 #ifdef FGMP_DEBUG_PRINT
                 if (blockIdx.x == 0 && lane == 5) printf("hot warp %d u %lld todo %x stage %d\n", warp, (long long)u, todo, stage);
 #endif
@@ -674,7 +687,7 @@ decode_kernel(DecParams p)
             // are cleared for the next segment on the way
             if (!(ok = mbar_wait(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 12))) break;
 #ifdef FGMP_DEBUG_PRINT
-            if (blockIdx.x == 0 && lane == 1) printf("epi warp %d row %d tile4 %f %f v0 %f\n", warp, row, tiles[4 * TILE_FLOATS + tile_idx(row, 0)], tiles[4 * TILE_FLOATS + tile_idx(row, 1)], v[0]);
+            if (blockIdx.x == 0 && lane == 1) printf("epi warp %d row %d tile4 %f %f v0 %f\n", warp, row, tiles[FP8_WARPS * TILE_FLOATS + tile_idx(row, 0)], tiles[FP8_WARPS * TILE_FLOATS + tile_idx(row, 1)], v[0]);
 #endif
             float c2[16];                              // (2): sums of the FP8 weight codes, still without 2^ratio
 #pragma unroll
@@ -687,9 +700,9 @@ decode_kernel(DecParams p)
                 for (int j = 0; j < 2 * NH; ++j) x[j] = src[(j ^ (row >> 1)) & 3];       // tokens 4j .. 4j+3
 #pragma unroll
                 for (int j = 0; j < 2 * NH; ++j) {
-                    if (w < 4) { c2[4 * j] += x[j].x; c2[4 * j + 1] += x[j].y; c2[4 * j + 2] += x[j].z; c2[4 * j + 3] += x[j].w; }
-                    else       { v[4 * j] += x[j].x; v[4 * j + 1] += x[j].y; v[4 * j + 2] += x[j].z; v[4 * j + 3] += x[j].w; }
-                    if (w < 4) src[(j ^ (row >> 1)) & 3] = make_float4(0.f, 0.f, 0.f, 0.f);   // the tile of (3) is overwritten
+                    if (w < FP8_WARPS) { c2[4 * j] += x[j].x; c2[4 * j + 1] += x[j].y; c2[4 * j + 2] += x[j].z; c2[4 * j + 3] += x[j].w; }
+                    else               { v[4 * j] += x[j].x; v[4 * j + 1] += x[j].y; v[4 * j + 2] += x[j].z; v[4 * j + 3] += x[j].w; }
+                    if (w < FP8_WARPS) src[(j ^ (row >> 1)) & 3] = make_float4(0.f, 0.f, 0.f, 0.f);   // the tile of (3) is overwritten
                 }
             }
 #pragma unroll
