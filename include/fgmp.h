@@ -53,8 +53,9 @@
  *                   | 2048 B of E4M3 microscales, 0x00 for FP8 blocks, in the order they go to tensor
  *                   memory: byte of (row r, block column j) = (j/4)*512 + (r%32)*16 + (r/32)*4 + j%4
  *                   | 128 B: uint16 x 17, FP8 blocks of the unit before block column j; entry 16 = all
- *   list          : per unit, its FP8 blocks ordered by (block column, row): the row of each (one byte,
- *                   padded to 16), then E4M3 codes 8..15 of each (8 bytes, padded to 16)
+ *   list          : per unit, its FP8 blocks ordered by (block column, row): one uint32 for each (padded
+ *                   to 16 bytes; low half = byte offset of the block's slot in the tile, high half =
+ *                   16 * row + 4 * ((row / 2) % 4)), then E4M3 codes 8..15 of each (8 bytes, padded to 16)
  *   uptr          : uint32 [units + 1]: start of a unit's list in 16-byte steps
  *                   fgmp_weights_bytes(N, K, max_fp8_blocks) leaves room for that many FP8 blocks.
  */

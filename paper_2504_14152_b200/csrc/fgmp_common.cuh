@@ -24,8 +24,9 @@
 //                       per r % 32, there 4 bytes per r / 32, there one byte per block of the step
 //   REC_KBSTART 128 B : uint16 x 17 (padded): FP8 blocks of the unit before block column j; entry 16 = all
 // List of a unit with cnt FP8 blocks, ordered by (block column, row) so that blocks meeting the same 16
-// activation elements are neighbours: the row of every block (cnt bytes, padded to 16), then E4M3 codes
-// 8..15 of every block (8 bytes each, padded to 16).  uptr[u] (uint32, units + 1 entries) = start of
+// activation elements are neighbours: one uint32 per block (padded to 16 bytes) -- low half: where the
+// block's slot sits in REC_W4, high half: 16 * row + 4 * ((row / 2) % 4), the place of its row in a swizzled
+// [row][16 tokens] fp32 tile -- then E4M3 codes 8..15 of every block (8 bytes each, padded to 16).  uptr[u] (uint32, units + 1 entries) = start of
 // unit u's list in 16-byte steps from off_ovf.
 //
 // Activations (kind 0): header | codes4 | sf | mask | arec | codes8.  codes4 is row-major, sf
@@ -58,7 +59,8 @@ struct PackedLayout {
 __host__ __device__ inline size_t fgmp_align1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 
 // list of a unit with cnt FP8 blocks: where the second halves start, and its size in 16-byte steps
-__host__ __device__ inline uint32_t fgmp_list_halves_offset(uint32_t cnt) { return (cnt + 15u) & ~15u; }
+__host__ __device__ inline uint32_t fgmp_list_halves_offset(uint32_t cnt) { return (cnt * 4u + 15u) & ~15u; }
+__host__ __device__ inline uint32_t fgmp_list_entry(uint32_t row, uint32_t j);
 __host__ __device__ inline uint32_t fgmp_list_steps(uint32_t cnt) { return (fgmp_list_halves_offset(cnt) + ((cnt * 8u + 15u) & ~15u)) >> 4; }
 
 // kind 0 = activations, 1 = weights (max_fp8 = room for that many FP8 blocks in the lists section)
@@ -79,8 +81,8 @@ __host__ __device__ inline PackedLayout fgmp_layout(int64_t rows, int64_t K, int
         L.off_mask = o;    o = fgmp_align1k(o + (size_t)rows * (size_t)L.MW * 4);
         L.off_uptr = o;    o = fgmp_align1k(o + ((size_t)L.units + 1) * 4);
         L.off_rec = o;     o = fgmp_align1k(o + (size_t)L.units * REC_BYTES);
-        // 9 bytes per FP8 block, and up to 30 bytes of padding per unit
-        L.off_ovf = o;     o = fgmp_align1k(o + (size_t)max_fp8 * 9 + (size_t)L.units * 32);
+        // 12 bytes per FP8 block, and up to 24 bytes of padding per unit
+        L.off_ovf = o;     o = fgmp_align1k(o + (size_t)max_fp8 * 12 + (size_t)L.units * 32);
     }
     L.total = o;
     return L;
@@ -102,6 +104,12 @@ __host__ __device__ inline uint32_t fgmp_rec_w4_offset(uint32_t r, uint32_t j)
 __host__ __device__ inline uint32_t fgmp_rec_sf_offset(uint32_t r, uint32_t j)
 {
     return (j >> 2) * 512u + (r & 31u) * 16u + (r >> 5) * 4u + (j & 3u);
+}
+
+// what a unit's list says about its FP8 block (row r of the tile, block column j)
+__host__ __device__ inline uint32_t fgmp_list_entry(uint32_t r, uint32_t j)
+{
+    return fgmp_rec_w4_offset(r, j) | ((r * 16u + (((r >> 1) & 3u) << 2)) << 16);
 }
 
 #ifdef __CUDACC__

@@ -51,10 +51,10 @@ constexpr int W_PROD = 0, W_MMA = 1, W_FP8 = 2, W_HOT = 10, W_EPI = 14;
 constexpr int FP8_WARPS = W_HOT - W_FP8;        // two sets of four: a set takes every second unit
 constexpr int Q_THREADS = 32 * 16;              // warps 2..17 share out the prologue quantizer
 constexpr int TOK = 16;                         // MMA N (token rows, zero padded)
-constexpr uint32_t LIST_CAP = 2944;             // bytes of a unit's FP8 list that fit a stage (about 320 blocks); more is read from global
+constexpr uint32_t LIST_CAP = 3968;             // bytes of a unit's FP8 list that fit a stage (about 330 blocks); more is read from global
 constexpr uint32_t STG_LIST = REC_BYTES;                                                         // 18560
-constexpr uint32_t STG_A = STG_LIST + LIST_CAP;                                                  // 21504, 1 KiB aligned
-constexpr uint32_t DEC_STAGE_BYTES = 32768;
+constexpr uint32_t STG_A = STG_LIST + LIST_CAP;                                                  // 22528, 1 KiB aligned
+constexpr uint32_t DEC_STAGE_BYTES = 33792;
 constexpr int DEC_STAGES = 4;
 constexpr int NTILES = FP8_WARPS + 1;           // [row][token] fp32 tiles: one per (2) warp, one shared by the (3) warps
 constexpr uint32_t TILE_FLOATS = 128 * TOK;
@@ -353,7 +353,7 @@ decode_kernel(DecParams p)
             const uint32_t step0 = __shfl_sync(0xffffffffu, pf, (int)(u - pf_base));
             const uint32_t step1 = __shfl_sync(0xffffffffu, pf, (int)(u + 1 - pf_base));
             if (lane == 0) {
-                ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1) ? 1 : 0;
+                ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1) ? 1 : 0;  /*lane*/
                 if (ok) { issue_w(u, stage, step0, step1); issue_a(u, stage); }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -370,13 +370,13 @@ decode_kernel(DecParams p)
             const int64_t tile = u / C;
             const int64_t seg_end = min(u_end, (tile + 1) * C);
             const int acc = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
-            if (!(ok = mbar_wait(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
+            if (!(ok = mbar_wait_warp(acce0 + 8 * acc, acc_phase ^ 1, abort_flag, p.status, 2))) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TOK);
             uint32_t accum = 0;
             for (; u < seg_end && ok; ++u) {
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
-                if (!(ok = mbar_wait(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;   // the scales are in tensor memory
+                if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
+                if (!(ok = mbar_wait_warp(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;   // the scales are in tensor memory
                 tc_fence_after();
                 const uint32_t sb = smem0 + (uint32_t)stage * DEC_STAGE_BYTES;
                 const uint32_t sf_t = tmem_base + SF_COL0 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
@@ -407,26 +407,26 @@ decode_kernel(DecParams p)
         const uint32_t tcol = (2 * t) & 3u, tpiece = t >> 1;
         // tile[row][tokens] += sums of one group.  Within one column every block has its own row, so the
         // read-modify-writes of a group touch distinct addresses: all loads first, then all stores.
-        auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t rowA, uint32_t rowB) {
-            float2 *pA = nullptr, *pB = nullptr;    // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on (piece ^ 2)
+        // (tlA, tlB: the rows' places in the tile as the list gives them, 0xffff = no block)
+        const uint32_t tx = tpiece << 2;
+        auto group_add = [&](const float (&c)[4], const float (&d)[4], uint32_t tlA, uint32_t tlB) {
+            const uint32_t iA = (tlA ^ tx) + tcol, iB = (tlB ^ tx) + tcol;      // tokens 2t, 2t+1; tokens 8+2t, 9+2t are 8 floats on
             float2 vA0 = make_float2(0.f, 0.f), vA1 = vA0, vB0 = vA0, vB1 = vA0;
-            if (rowA != 0xffffffffu) {
-                pA = reinterpret_cast<float2*>(mytile + rowA * 16u + (((tpiece ^ (rowA >> 1)) & 3u) << 2) + tcol);
-                vA0 = pA[0];
-                if (NH == 2) vA1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32);
+            if (tlA != 0xffffu) {
+                vA0 = *reinterpret_cast<const float2*>(mytile + iA);
+                if (NH == 2) vA1 = *reinterpret_cast<const float2*>(mytile + (iA ^ 8u));
             }
-            if (rowB != 0xffffffffu) {
-                pB = reinterpret_cast<float2*>(mytile + rowB * 16u + (((tpiece ^ (rowB >> 1)) & 3u) << 2) + tcol);
-                vB0 = pB[0];
-                if (NH == 2) vB1 = *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32);
+            if (tlB != 0xffffu) {
+                vB0 = *reinterpret_cast<const float2*>(mytile + iB);
+                if (NH == 2) vB1 = *reinterpret_cast<const float2*>(mytile + (iB ^ 8u));
             }
-            if (rowA != 0xffffffffu) {
-                pA[0] = make_float2(vA0.x + c[0], vA0.y + c[1]);
-                if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pA) ^ 32) = make_float2(vA1.x + d[0], vA1.y + d[1]);
+            if (tlA != 0xffffu) {
+                *reinterpret_cast<float2*>(mytile + iA) = make_float2(vA0.x + c[0], vA0.y + c[1]);
+                if (NH == 2) *reinterpret_cast<float2*>(mytile + (iA ^ 8u)) = make_float2(vA1.x + d[0], vA1.y + d[1]);
             }
-            if (rowB != 0xffffffffu) {
-                pB[0] = make_float2(vB0.x + c[2], vB0.y + c[3]);
-                if (NH == 2) *reinterpret_cast<float2*>(reinterpret_cast<uintptr_t>(pB) ^ 32) = make_float2(vB1.x + d[2], vB1.y + d[3]);
+            if (tlB != 0xffffu) {
+                *reinterpret_cast<float2*>(mytile + iB) = make_float2(vB0.x + c[2], vB0.y + c[3]);
+                if (NH == 2) *reinterpret_cast<float2*>(mytile + (iB ^ 8u)) = make_float2(vB1.x + d[2], vB1.y + d[3]);
             }
             __syncwarp();                  // a later group may add to the same rows
         };
@@ -450,10 +450,10 @@ decode_kernel(DecParams p)
             const int64_t tile = (u_begin + sbeg) / C;
             const int send = (int)min((int64_t)n_units, (tile + 1) * C - u_begin);
             // the epilogue has taken (and cleared) the previous segment's sums
-            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
+            if (seg > 0 && !(ok = mbar_wait_warp(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
             for (int i = sbeg + ((par ^ sbeg) & 1); i < send; i += 2) {
                 const int stage = i % S; const uint32_t phase = (uint32_t)(i / S) & 1u;
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
+                if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 5))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
                 const uint32_t staged = smeta[stage].staged;
@@ -481,24 +481,26 @@ decode_kernel(DecParams p)
                     for (int gr = 0; gr < 2; ++gr)
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) {
-                            const uint32_t j = (uint32_t)bq + 4u * cc;
                             const uint32_t iA = st[cc] + 16u * gr + g, iB = iA + 8;
                             const bool hasA = iA < en[cc], hasB = iB < en[cc];
-                            const uint32_t rA = hasA ? sb[STG_LIST + iA] : 0u, rB = hasB ? sb[STG_LIST + iB] : 0u;
-                            const uint32_t oA = t < 2 ? REC_W4 + fgmp_rec_w4_offset(rA, j) + 4 * t : STG_LIST + hoff + iA * 8 + 4 * (t - 2);
-                            const uint32_t oB = t < 2 ? REC_W4 + fgmp_rec_w4_offset(rB, j) + 4 * t : STG_LIST + hoff + iB * 8 + 4 * (t - 2);
+                            const uint32_t mA = hasA ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + 4 * iA) : 0xffffffffu;
+                            const uint32_t mB = hasB ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + 4 * iB) : 0xffffffffu;
+                            const uint32_t oA = t < 2 ? REC_W4 + (mA & 0xffffu) + 4 * t : STG_LIST + hoff + iA * 8 + 4 * (t - 2);
+                            const uint32_t oB = t < 2 ? REC_W4 + (mB & 0xffffu) + 4 * t : STG_LIST + hoff + iB * 8 + 4 * (t - 2);
                             rawA[4 * gr + cc] = hasA ? *reinterpret_cast<const uint32_t*>(sb + oA) : 0u;
                             rawB[4 * gr + cc] = hasB ? *reinterpret_cast<const uint32_t*>(sb + oB) : 0u;
-                            rowA[4 * gr + cc] = hasA ? rA : 0xffffffffu;
-                            rowB[4 * gr + cc] = hasB ? rB : 0xffffffffu;
+                            rowA[4 * gr + cc] = mA >> 16;
+                            rowB[4 * gr + cc] = mB >> 16;
                         }
                 } else {
                     // a list that does not fit the stage, or a column with more than 32 FP8 blocks (rare): group by
                     // group straight from the stage or from global memory, before the stage is given back
-                    auto fetch = [&](uint32_t j, uint32_t i_, uint32_t& row, uint32_t& raw) {
-                        row = (all || i_ < staged) ? sb[STG_LIST + i_] : __ldg(list_g + i_);
+                    auto fetch = [&](uint32_t i_, uint32_t& row, uint32_t& raw) {
+                        const uint32_t m_ = (all || 4 * i_ + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + 4 * i_)
+                                                                          : __ldg(reinterpret_cast<const uint32_t*>(list_g + 4 * i_));
+                        row = m_ >> 16;
                         if (t < 2) {
-                            raw = *reinterpret_cast<const uint32_t*>(sb + REC_W4 + fgmp_rec_w4_offset(row, j) + 4 * t);
+                            raw = *reinterpret_cast<const uint32_t*>(sb + REC_W4 + (m_ & 0xffffu) + 4 * t);
                         } else {
                             const uint32_t o = hoff + i_ * 8 + 4 * (t - 2);
                             raw = (all || o + 4 <= staged) ? *reinterpret_cast<const uint32_t*>(sb + STG_LIST + o)
@@ -513,9 +515,9 @@ decode_kernel(DecParams p)
                         uint2 b1 = make_uint2(0u, 0u);
                         if (NH == 2) b1 = *reinterpret_cast<const uint2*>(sa + fgmp_arec_at_offset(g + 8, j) + 8 * t);
                         for (uint32_t e = st_; e < en_; e += 16) {
-                            uint32_t rA = 0xffffffffu, rB = 0xffffffffu, wA = 0u, wB = 0u;
-                            if (e + g < en_) fetch(j, e + g, rA, wA);
-                            if (e + g + 8 < en_) fetch(j, e + g + 8, rB, wB);
+                            uint32_t rA = 0xffffu, rB = 0xffffu, wA = 0u, wB = 0u;
+                            if (e + g < en_) fetch(e + g, rA, wA);
+                            if (e + g + 8 < en_) fetch(e + g + 8, rB, wB);
                             float c[4], d[4];
                             group_mma(wA, wB, b0, b1, c, d);
                             group_add(c, d, rA, rB);
@@ -560,7 +562,7 @@ decode_kernel(DecParams p)
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) acc[mt][nh][0] = acc[mt][nh][1] = acc[mt][nh][2] = acc[mt][nh][3] = 0.f;
             for (; u < seg_end; ++u) {
-                if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 6))) break;
+                if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 6))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
                 const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
@@ -633,7 +635,7 @@ decode_kernel(DecParams p)
             if (!ok) break;
             // the epilogue has taken the previous segment's sums; now this segment's go in:
             // acc[mt][nh] = rows 32jr + 16mt + {g, g + 8} x tokens 8nh + {2t, 2t+1}
-            if (seg > 0 && !(ok = mbar_wait(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
+            if (seg > 0 && !(ok = mbar_wait_warp(tfree, (uint32_t)(seg - 1) & 1u, abort_flag, p.status, 7))) break;
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -662,7 +664,7 @@ decode_kernel(DecParams p)
             const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
             u = seg_end;
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
-            if (!(ok = mbar_wait(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 11))) break;
+            if (!(ok = mbar_wait_warp(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 11))) break;
             tc_fence_after();
             // a tile shared with other CTAs: how many of them have handed in their sums already (the answer is
             // needed only after this CTA's own sums are complete, so the load costs nothing)
@@ -685,7 +687,7 @@ decode_kernel(DecParams p)
             for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(rr[j]);
             // corrections (2) and (3) of the segment: this row of every tile, in tile order; the rows of (2)
             // are cleared for the next segment on the way
-            if (!(ok = mbar_wait(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 12))) break;
+            if (!(ok = mbar_wait_warp(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 12))) break;
 #ifdef FGMP_DEBUG_PRINT
             if (blockIdx.x == 0 && lane == 1) printf("epi warp %d row %d tile4 %f %f v0 %f\n", warp, row, tiles[FP8_WARPS * TILE_FLOATS + tile_idx(row, 0)], tiles[FP8_WARPS * TILE_FLOATS + tile_idx(row, 1)], v[0]);
 #endif

@@ -29,6 +29,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// the same, but the thread may stay suspended in hardware for up to `ns` before the answer comes
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns()
 {
     unsigned long long t;
@@ -37,15 +45,16 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
 }
 
 // Bounded wait: gives up after limit_ns (or when another thread of the CTA already gave up),
-// records the failure and returns false.  `abort_flag` lives in shared memory.
+// records the failure and returns false.  `abort_flag` lives in shared memory.  The waiting thread is
+// suspended by the hardware between looks at the barrier, so that waiting costs no issue slots and no
+// shared-memory traffic.
 constexpr unsigned long long MBAR_WAIT_LIMIT_NS = 2000000000ull;
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where,
                                             unsigned long long limit_ns)
 {
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_for(bar, parity, 100000u)) return true;
         if (*abort_flag) return false;
         if (globaltimer_ns() - t0 > limit_ns) {
             *abort_flag = 1;
@@ -53,7 +62,6 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
             atomicExch(status + 1, where);
             return false;
         }
-        __nanosleep(64);
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where,
@@ -61,6 +69,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, status, where, limit_ns);
+}
+// The same for a converged warp: one lane waits, the others are parked at the warp barrier; afterwards
+// every lane looks at the barrier once itself (it has completed: the look orders the lane's later reads).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait_slow(bar, parity, abort_flag, status, where, MBAR_WAIT_LIMIT_NS) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (ok) mbar_try_wait(bar, parity);
+    return ok != 0;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar)

@@ -315,15 +315,16 @@ __global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw
     const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
     const uint32_t cnt = fgmp_unit_positions(m16, sc.warp, sc.pos, sc.cnt);
     uint8_t* rec = blob + L.off_rec + (size_t)unit * REC_BYTES;
-    uint8_t* rowid = blob + L.off_ovf + (size_t)uptr[unit] * 16;
-    uint8_t* halves = rowid + fgmp_list_halves_offset(cnt);
+    uint8_t* list = blob + L.off_ovf + (size_t)uptr[unit] * 16;
+    uint32_t* entries = reinterpret_cast<uint32_t*>(list);
+    uint8_t* halves = list + fgmp_list_halves_offset(cnt);
     if (threadIdx.x < 64) {                                    // running sums of the per-column counts, then padding
         uint32_t before = 0;
         for (int i = 0; i < 16 && i < (int)threadIdx.x; ++i) before += sc.cnt[i];
         reinterpret_cast<uint16_t*>(rec + REC_KBSTART)[threadIdx.x] = threadIdx.x <= 16 ? (uint16_t)before : (uint16_t)0;
     }
-    if (fits) {                                                // padding behind the rows and behind the last half
-        for (uint32_t i = cnt + threadIdx.x; i < fgmp_list_halves_offset(cnt); i += 128) rowid[i] = 0;
+    if (fits) {                                                // padding behind the entries and behind the last half
+        for (uint32_t i = cnt + threadIdx.x; i < fgmp_list_halves_offset(cnt) / 4; i += 128) entries[i] = 0;
         if (threadIdx.x == 0 && (cnt & 1u)) *reinterpret_cast<uint2*>(halves + (size_t)cnt * 8) = make_uint2(0u, 0u);
     }
     const int j = threadIdx.x & 15;
@@ -344,7 +345,7 @@ __global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw
                 slot = make_uint2(c8[0], c8[1]);
                 if (fits) {
                     *reinterpret_cast<uint2*>(halves + (size_t)pos * 8) = make_uint2(c8[2], c8[3]);
-                    rowid[pos] = (uint8_t)row;
+                    entries[pos] = fgmp_list_entry((uint32_t)row, (uint32_t)j);
                 }
             } else {
                 float dq4[16];

@@ -40,7 +40,7 @@ def test_size_functions(lib):
     # sections: header + codes4 + sf + mask + FP8 plane, each rounded to 1 KiB
     assert fg.acts_bytes(64, 256) == 1024 + 8192 + 2048 + 1024 + 16384
     w0 = fg.weights_bytes(256, 256, 0)
-    assert fg.weights_bytes(256, 256, 410) - w0 == 3072          # 8 bytes per FP8 block beyond its slot, rounded to 1 KiB
+    assert fg.weights_bytes(256, 256, 410) - w0 == 4096          # 12 bytes per FP8 block beyond its slot (the first KiB is there already)
     assert fg.weights_bytes(256, 256, 4097) == 0                 # more blocks than exist
     # algorithmic payload versus the layout: an FP8 block's first half takes the place of the NVFP4 codes, so the
     # blob holds little beyond the payload (per-unit tables, the second copy of the mask bits, padding)
@@ -49,7 +49,7 @@ def test_size_functions(lib):
     n8 = B // 10
     algorithmic = (B - n8) * 9 + n8 * 16 + B / 8
     stored = fg.weights_bytes(N, K, n8)
-    assert 1.0 < stored / algorithmic < 1.03
+    assert 1.0 < stored / algorithmic < 1.07
     assert fg.workspace_bytes(1, 64, 0, 256) == 0
     assert fg.workspace_bytes(2, 64, 256, 256) >= 2 * (64 + 256) * 256
     assert fg.workspace_bytes(0, 0, 256, 250) == 0

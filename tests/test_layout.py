@@ -67,5 +67,5 @@ def test_weight_record_maps_are_bijections(maps):
 def test_fp8_list_sizes(maps):
     _, _, lists, _ = maps
     for cnt, (halves, steps) in lists.items():
-        assert halves % 16 == 0 and halves >= cnt and halves - cnt < 16       # row ids, padded to 16 bytes
+        assert halves % 16 == 0 and halves >= 4 * cnt and halves - 4 * cnt < 16     # one word per block, padded to 16 bytes
         assert steps * 16 >= halves + 8 * cnt and steps * 16 - (halves + 8 * cnt) < 16
