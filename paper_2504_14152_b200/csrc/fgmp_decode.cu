@@ -32,9 +32,9 @@
 //
 // Warp roles (576 threads): warp 0 = producer, warp 1 = MMA issuer and owner of the tensor memory,
 // warps 2-9 = (2): two sets of four warps that take alternate units, four block columns per warp (a warp
-// copies what it needs of a unit into registers and gives the stage back at once), warps 10-13 = block
-// scales into tensor memory (one lane quadrant each), then (3), 32 rows each, warps 14-17 = epilogue
-// (one lane quadrant each).
+// copies what it needs of a unit into registers and gives the stage back at once), warps 10-13 = (3), 32
+// rows each, warps 14-17 = block scales into tensor memory unit by unit and, at the end of a tile, the
+// epilogue (one lane quadrant each).
 #include "fgmp_common.cuh"
 #include "fgmp_actq.cuh"
 #include "fgmp_host.h"
@@ -153,6 +153,16 @@ __device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, ui
     if (tq == 0) *s_hot = 0u;
     quant_bar();
     const int octets = p.M > 8 ? 2 : 1;
+    // both token rows of this warp are on their way before either is worked on
+    uint2 xin[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+#pragma unroll
+    for (int o = 0; o < 2; ++o) {
+        const uint32_t m = 8u * (uint32_t)o + (wq >> 1);
+        if (o < octets && (int64_t)m < p.M)
+            xin[o] = __ldg(reinterpret_cast<const uint2*>(p.X + ((size_t)m * p.ldx + (size_t)kb * 16 + 4 * li) * 2));
+    }
+    const float4 f = __ldg(reinterpret_cast<const float4*>(p.fisher + kb * 16 + 4 * li));
+#pragma unroll
     for (int o = 0; o < 2; ++o) {
         const uint32_t m = 8u * (uint32_t)o + (wq >> 1);
         uint8_t* a4 = rec + AREC_A4 + fgmp_rec_w4_offset(m, j) + 2u * li;
@@ -163,9 +173,7 @@ __device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, ui
             if (li == 0) rec[AREC_SF + m * 16u + j] = 0;
             continue;
         }
-        const uint2 x = __ldg(reinterpret_cast<const uint2*>(p.X + ((size_t)m * p.ldx + (size_t)kb * 16 + 4 * li) * 2));
-        const float4 f = __ldg(reinterpret_cast<const float4*>(p.fisher + kb * 16 + 4 * li));
-        const BlockQuarter r = quantize_block_quarter<MODE>(x, f, p.q);
+        const BlockQuarter r = quantize_block_quarter<MODE>(xin[o], f, p.q);
         *reinterpret_cast<uint16_t*>(a4) = (uint16_t)r.c4;
         *reinterpret_cast<uint2*>(at) = r.h;
         if (li == 0) rec[AREC_SF + m * 16u + j] = (uint8_t)r.sc;
@@ -209,6 +217,7 @@ decode_kernel(DecParams p)
     volatile uint32_t* s_misc = reinterpret_cast<volatile uint32_t*>(abort_flag + 1);   // [0] tag, [1..2] claimed item, [3] hot columns of a chunk
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) FGMP_STAMP_ANY(0);
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, sfr0 = empty0 + 8 * S;
     const uint32_t accf0 = sfr0 + 8 * S, acce0 = accf0 + 16, cdone0 = acce0 + 16, tfree = cdone0 + 16;
     constexpr uint32_t A_BYTES = NH == 2 ? AREC_BYTES : AREC_AT + 4096u;
@@ -283,17 +292,20 @@ decode_kernel(DecParams p)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    FGMP_STAMP_ANY(warp == 0 && lane == 0 ? 1 : 15);
+    if (threadIdx.x == 0) FGMP_STAMP_ANY(1);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // Launched as a programmatic dependent of the preceding kernel in the stream, this kernel may have
     // started before that one finished: everything above touches neither its output nor the workspace.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 0) FGMP_STAMP_ANY(2);
     if (FUSED) {
         if (threadIdx.x == 0) {
             uint32_t e;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(e) : "l"(p.cw + CW_EPOCH) : "memory");
             s_misc[0] = e + 1u;
         }
+        // the first of the quantizer's work items is asked for at the same time
+        if (threadIdx.x == 64 && !*abort_flag) s_misc[1] = atomicInc(p.cw + CW_CLAIM, (uint32_t)C + (uint32_t)G - 1u);
         __syncthreads();
     }
     const uint32_t tag = FUSED ? s_misc[0] : 0u;
@@ -305,10 +317,10 @@ decode_kernel(DecParams p)
         // finished items wrap to zero with the call's last access.
         const uint32_t n_items = (uint32_t)C;
         for (uint32_t it = 0;; ++it) {
-            if (threadIdx.x == 64) s_misc[1 + (it & 1u)] = atomicInc(p.cw + CW_CLAIM, n_items + (uint32_t)G - 1u);
-            quant_bar();
             const uint32_t item = s_misc[1 + (it & 1u)];
             if (item >= n_items) break;
+            // the next item is asked for while this one is worked on
+            if (threadIdx.x == 64) s_misc[1 + ((it + 1u) & 1u)] = atomicInc(p.cw + CW_CLAIM, n_items + (uint32_t)G - 1u);
             if (item == 0 && threadIdx.x == 64 && p.q_header) {
                 fgmp_packed_header* h = p.q_header;
                 h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.q.s4;
@@ -324,6 +336,7 @@ decode_kernel(DecParams p)
         }
     }
 
+    if (threadIdx.x == 64) FGMP_STAMP_ANY(3);          // this CTA's share of the quantizer is done
     if (dead) {
     } else if (warp == W_PROD) {
         // ------------------------------------------------------------ producer (whole warp; lane 0 issues)
@@ -342,6 +355,7 @@ decode_kernel(DecParams p)
                 }
             }
             if (ok) for (int s = 0; s < pre; ++s) issue_a(u_begin + s, s);
+            FGMP_STAMP_ANY(4);                         // all activation records are in place
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         int stage = pre % S; uint32_t phase = (uint32_t)(pre / S) & 1u;
@@ -377,6 +391,8 @@ decode_kernel(DecParams p)
             for (; u < seg_end && ok; ++u) {
                 if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
                 if (!(ok = mbar_wait_warp(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;   // the scales are in tensor memory
+                if (u == u_begin && lane == 0) FGMP_STAMP_ANY(5);
+                if (u == u_end - 1 && lane == 0) FGMP_STAMP_ANY(6);
                 tc_fence_after();
                 const uint32_t sb = smem0 + (uint32_t)stage * DEC_STAGE_BYTES;
                 const uint32_t sf_t = tmem_base + SF_COL0 + (uint32_t)stage * 32;   // [0,16) weights, [16,32) tokens
@@ -566,34 +582,6 @@ decode_kernel(DecParams p)
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
                 const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
-                {
-                    // Block scales of the unit into tensor memory, lane quadrant warp % 4: lane i holds, for MMA step j,
-                    // the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3 -- 16 bytes of scale tile j of
-                    // the record; the token scales follow in columns 16..31 (16 tokens: lanes 0..15, first column of
-                    // every step), zeroed in the chunk's hot block columns.
-                    uint32_t r[16];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
-                        r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
-                    }
-                    const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
-                    tmem_st16(sf_t, r);
-                    const uint4 ts = *reinterpret_cast<const uint4*>(sa + AREC_SF + (lane & 15) * 16);
-                    const uint32_t tsw[4] = {ts.x, ts.y, ts.z, ts.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        // bits 4j .. 4j+3 of the cold columns spread to the four bytes of the step's scale word
-                        const uint32_t keep = ((((~hot >> (4 * j)) & 0xfu) * 0x00204081u) & 0x01010101u) * 0xffu;
-                        r[4 * j] = lane < 16 ? (tsw[j] & keep) : 0u;
-                        r[4 * j + 1] = 0u; r[4 * j + 2] = 0u; r[4 * j + 3] = 0u;
-                    }
-                    tmem_st16(sf_t + 16, r);
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
-                }
                 uint32_t todo = hot & 0xffffu;
 #ifdef FGMP_DEBUG_PRINT
                 if (blockIdx.x == 0 && lane == 5) printf("hot warp %d u %lld todo %x stage %d\n", warp, (long long)u, todo, stage);
@@ -659,10 +647,44 @@ decode_kernel(DecParams p)
         const int row = 32 * q + lane;
         bool ok = true;
         int seg = 0;
+        int stage = 0; uint32_t phase = 0;
         for (int64_t u = u_begin; u < u_end && ok; ++seg) {
             const int64_t tile = u / C;
             const int64_t seg_begin = u, seg_end = min(u_end, (tile + 1) * C);
-            u = seg_end;
+            // Block scales of the segment's units into tensor memory, lane quadrant warp % 4: lane i holds, for MMA
+            // step j, the four scale bytes of rows i, 32+i, 64+i, 96+i in columns 4j..4j+3 -- 16 bytes of scale tile j
+            // of the record; the token scales follow in columns 16..31 (16 tokens: lanes 0..15, first column of
+            // every step), zeroed in the chunk's hot block columns.
+            for (; u < seg_end; ++u) {
+                if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 4))) break;
+                const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
+                const uint8_t* sa = sb + STG_A;
+                const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
+                uint32_t r[16];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 x = *reinterpret_cast<const uint4*>(sb + REC_SF + 512 * j + lane * 16);
+                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                }
+                const uint32_t sf_t = tmem_base + ((uint32_t)(q * 32) << 16) + SF_COL0 + (uint32_t)stage * 32;
+                tmem_st16(sf_t, r);
+                const uint4 ts = *reinterpret_cast<const uint4*>(sa + AREC_SF + (lane & 15) * 16);
+                const uint32_t tsw[4] = {ts.x, ts.y, ts.z, ts.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    // bits 4j .. 4j+3 of the cold columns spread to the four bytes of the step's scale word
+                    const uint32_t keep = ((((~hot >> (4 * j)) & 0xfu) * 0x00204081u) & 0x01010101u) * 0xffu;
+                    r[4 * j] = lane < 16 ? (tsw[j] & keep) : 0u;
+                    r[4 * j + 1] = 0u; r[4 * j + 2] = 0u; r[4 * j + 3] = 0u;
+                }
+                tmem_st16(sf_t + 16, r);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
+                if (++stage == S) { stage = 0; phase ^= 1; }
+            }
+            if (!ok) break;
             const int accb = seg & 1; const uint32_t acc_phase = (uint32_t)((seg >> 1) & 1);
             if (!(ok = mbar_wait_warp(accf0 + 8 * accb, acc_phase, abort_flag, p.status, 11))) break;
             tc_fence_after();
@@ -746,6 +768,7 @@ decode_kernel(DecParams p)
                     write_out = true;
                 }
             }
+            if (u == u_end && threadIdx.x == W_EPI * 32) FGMP_STAMP_ANY(whole ? 7 : 8);    // last segment: sums complete / handed in
             if (write_out && n < p.N) {
 #pragma unroll
                 for (int j = 0; j < 8 * NH; ++j) {
@@ -759,6 +782,7 @@ decode_kernel(DecParams p)
     }
 
     __syncthreads();
+    if (threadIdx.x == 0) FGMP_STAMP_ANY(9);
     if (*abort_flag) {
         const unsigned long long t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
