@@ -78,7 +78,7 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi)
 }
 
 // control words of the workspace (int32, from byte 256): see fgmp_linear_fused
-enum { CW_EPOCH = 0, CW_DONE = 1, CW_CLAIM = 2, CW_QCOUNT = 3, CW_QREADY = 4 };
+enum { CW_DONE = 1, CW_CLAIM = 2, CW_QCOUNT = 3, CW_QREADY = 4 };
 
 struct DecParams {
     const uint8_t* wblob; const uint8_t* ablob;
@@ -214,7 +214,7 @@ decode_kernel(DecParams p)
     StageMeta* smeta = reinterpret_cast<StageMeta*>(bars + 3 * S + 8);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smeta + S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile uint32_t* s_misc = reinterpret_cast<volatile uint32_t*>(abort_flag + 1);   // [0] tag, [1..2] claimed item, [3] hot columns of a chunk
+    volatile uint32_t* s_misc = reinterpret_cast<volatile uint32_t*>(abort_flag + 1);   // [1..2] claimed item, [3] hot columns of a chunk
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) FGMP_STAMP_ANY(0);
@@ -299,16 +299,10 @@ decode_kernel(DecParams p)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (threadIdx.x == 0) FGMP_STAMP_ANY(2);
     if (FUSED) {
-        if (threadIdx.x == 0) {
-            uint32_t e;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(e) : "l"(p.cw + CW_EPOCH) : "memory");
-            s_misc[0] = e + 1u;
-        }
-        // the first of the quantizer's work items is asked for at the same time
+        // the first of the quantizer's work items is asked for right away
         if (threadIdx.x == 64 && !*abort_flag) s_misc[1] = atomicInc(p.cw + CW_CLAIM, (uint32_t)C + (uint32_t)G - 1u);
         __syncthreads();
     }
-    const uint32_t tag = FUSED ? s_misc[0] : 0u;
     const bool dead = *abort_flag != 0;                // the weight blob does not belong to this call: nothing else is read
 
     if (FUSED && !dead && warp >= W_FP8) {
@@ -332,7 +326,7 @@ decode_kernel(DecParams p)
             __threadfence();
             quant_bar();
             if (threadIdx.x == 64 && atomicInc(p.cw + CW_QCOUNT, n_items - 1u) == n_items - 1u)
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(tag) : "memory");
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(1u) : "memory");
         }
     }
 
@@ -344,7 +338,7 @@ decode_kernel(DecParams p)
         if (lane == 0) {
             if (FUSED) {
                 // every chunk's record is in place once the last work item of the quantizer has been handed in
-                ok = wait_global_equals(p.cw + CW_QREADY, tag, abort_flag, p.status, 8) ? 1 : 0;
+                ok = wait_global_equals(p.cw + CW_QREADY, 1u, abort_flag, p.status, 8) ? 1 : 0;
                 asm volatile("fence.proxy.async;" ::: "memory");   // records were written with ordinary stores, the bulk copy reads them
             } else {
                 const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
@@ -788,9 +782,9 @@ decode_kernel(DecParams p)
         while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
         __syncthreads();
     } else if (FUSED && threadIdx.x == 0) {
-        // the CTA that finishes last moves the call number on: the next call publishes under a new tag
+        // the CTA that finishes last takes the "records ready" word back, so that the control area is as the next call needs it
         if (atomicInc(p.cw + CW_DONE, (uint32_t)G - 1u) == (uint32_t)G - 1u)
-            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_EPOCH), "r"(tag) : "memory");
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(0u) : "memory");
     }
     if (warp == W_MMA) {
         tc_fence_after();
