@@ -301,12 +301,20 @@ fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, uint8_t* co
 
 /* ---- measurement support: tensor-core rate per operand kind ----
  * Runs, on every SM, mma_per_cta tcgen05 instructions of M = 128, N = 256 on operands resident in
- * shared memory (nothing is loaded or stored): kind 0 = bf16 (K = 16 per instruction), 1 = FP8 E4M3
+ * shared memory (nothing is loaded or stored; mma_per_cta <= 2^21): kind 0 = bf16 (K = 16 per instruction), 1 = FP8 E4M3
  * (K = 32), 2 = NVFP4 with E4M3 block scales (K = 64).  The caller times the call on the stream;
  * flops = 2 * 128 * 256 * K * mma_per_cta * (number of SMs).  These are the rates the block-pair
  * products of Section 4.1 can run at at best, i.e. the denominators of the prefill roofline.
  * workspace: >= 256 bytes, zeroed, 256-byte aligned (status word, read by fgmp_check). */
 fgmp_status fgmp_tensor_peak(int kind, int64_t mma_per_cta, void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- self-test of the failure path (the paper has no counterpart) ----
+ * Every wait inside the kernels is bounded: when it runs out the kernel records FGMP_ERR_TIMEOUT in
+ * the status word of its workspace and returns, instead of hanging the GPU.  This call exercises that
+ * path without any GEMM: a single thread block waits up to limit_ns (1e3 .. 1e8) for a barrier that
+ * nothing completes.  Afterwards fgmp_check(workspace) returns FGMP_ERR_TIMEOUT, fgmp_workspace_init
+ * clears it, and the workspace serves fgmp_linear again.  workspace: >= 256 bytes, 256-byte aligned. */
+fgmp_status fgmp_selftest_wait_timeout(void* workspace, size_t ws_bytes, int64_t limit_ns, void* cuda_stream);
 
 /* Block scores only (parity support and calibration): scores [M*K/16] fp32, activations. */
 fgmp_status fgmp_activation_scores(const void* X_bf16, int64_t ldx, const float* fisher_chan,

@@ -7,5 +7,5 @@ from .binding import (  # noqa: F401
     FgmpError, PackedTensor, SCORE_LP_ERROR, SCORE_HP_TO_LP, CLIP_NONE, CLIP_SW_BRUTE,
     acts_bytes, weights_bytes, workspace_bytes, workspace_init, alloc_workspace, quantize_weights, quantize_activations,
     calibrate_tau, activation_scores, weight_scores, global_tau, channel_mean_sq, linear_quantize, linear, linear_fused, check, unpack, version, status_string, library_path,
-    profile_begin, profile_end, kernel_names, linear_static, STATIC_SCRATCH_BYTES, tensor_peak,
+    profile_begin, profile_end, kernel_names, linear_static, STATIC_SCRATCH_BYTES, tensor_peak, selftest_wait_timeout,
 )

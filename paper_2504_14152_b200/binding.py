@@ -72,6 +72,8 @@ def _load():
     L.fgmp_global_tau.argtypes = [vp, vp, ci, ctypes.c_double, vp, vp, sz, vp]
     L.fgmp_tensor_peak.restype = ci
     L.fgmp_tensor_peak.argtypes = [ci, i64, vp, sz, vp]
+    L.fgmp_selftest_wait_timeout.restype = ci
+    L.fgmp_selftest_wait_timeout.argtypes = [vp, sz, i64, vp]
     L.fgmp_workspace_init.restype = ci
     L.fgmp_workspace_init.argtypes = [vp, sz, vp]
     L.fgmp_unpack.restype = ci
@@ -354,6 +356,12 @@ def linear_static(acts: PackedTensor, weights: PackedTensor, *, out: torch.Tenso
 def tensor_peak(kind: int, mma_per_cta: int, workspace: torch.Tensor) -> None:
     """Launch the MMA-only loop of fgmp_tensor_peak (kind 0 bf16, 1 E4M3, 2 NVFP4); the caller times it."""
     _ok(_load().fgmp_tensor_peak(kind, mma_per_cta, workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_tensor_peak")
+
+
+def selftest_wait_timeout(workspace: torch.Tensor, limit_ns: int = 1_000_000) -> None:
+    """Launch the one-block kernel whose bounded wait runs out (fgmp_selftest_wait_timeout)."""
+    _ok(_load().fgmp_selftest_wait_timeout(workspace.data_ptr(), workspace.numel(), int(limit_ns), _stream()),
+        "fgmp_selftest_wait_timeout")
 
 
 def check(workspace: torch.Tensor) -> None:

@@ -99,14 +99,37 @@ tensor_peak_kernel(int kind, int64_t n_mma, int* status)
         tc_fence_after();
     }
     __syncthreads();
+    if (*abort_flag) {                                  // MMAs may still be in flight: let them drain before the tensor memory goes back
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
     if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
+// One CTA waits, with the library's bounded wait, for a barrier that nothing completes: the wait runs out
+// after limit_ns, FGMP_ERR_TIMEOUT goes into the status word like in the GEMM kernels, and the kernel returns.
+__global__ void __launch_bounds__(32, 1) wait_selftest_kernel(unsigned long long limit_ns, int* status)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_s;
+    volatile int* abort_flag = &abort_s;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, abort_flag, status, 30, limit_ns);
+    __syncwarp();
 }
 
 }  // namespace
 
 extern "C" fgmp_status fgmp_tensor_peak(int kind, int64_t mma_per_cta, void* workspace, size_t ws_bytes, void* cuda_stream)
 {
-    if (kind < 0 || kind > 2 || mma_per_cta < 1 || mma_per_cta > (int64_t)1 << 24 || !workspace || ws_bytes < 256 ||
+    // (at about 0.1 us per instruction 2^21 of them stay far inside the bounded wait at the end of the loop)
+    if (kind < 0 || kind > 2 || mma_per_cta < 1 || mma_per_cta > (int64_t)1 << 21 || !workspace || ws_bytes < 256 ||
         ((uintptr_t)workspace & 255)) return FGMP_ERR_INVALID_ARG;
     fgmp_status st;
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
@@ -120,5 +143,15 @@ extern "C" fgmp_status fgmp_tensor_peak(int kind, int64_t mma_per_cta, void* wor
     }
     cudaStream_t s = (cudaStream_t)cuda_stream;
     tensor_peak_kernel<<<fgmp_sm_count(), PK_THREADS, PK_SMEM, s>>>(kind, mma_per_cta, reinterpret_cast<int*>(workspace));
+    return fgmp_launch_status();
+}
+
+extern "C" fgmp_status fgmp_selftest_wait_timeout(void* workspace, size_t ws_bytes, int64_t limit_ns, void* cuda_stream)
+{
+    if (!workspace || ws_bytes < 256 || ((uintptr_t)workspace & 255)) return FGMP_ERR_INVALID_ARG;
+    if (limit_ns < 1000 || limit_ns > 100000000) return FGMP_ERR_INVALID_ARG;      // 1 us .. 0.1 s
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>((unsigned long long)limit_ns, reinterpret_cast<int*>(workspace));
     return fgmp_launch_status();
 }

@@ -1,0 +1,91 @@
+"""GPU parity at the full sizes of the five benchmark configurations: sampled GEMM outputs against the
+oracle (after the packed operands have been compared with the oracle's bit for bit), the clip-search packer
+at full width, and the hand-derived tie cases of the clip search."""
+import numpy as np
+import pytest
+import torch
+
+import fgmp_inputs as gi
+import oracle
+from test_gpu_parity import GEMM_TOL, compare_packed, fg, quantize_both, _sampled_linear_check  # noqa: F401
+from test_oracle_quant import clip_tie_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("M", [2, 4, 8])
+def test_config2_llama2_7b_fc1_decode_token_counts(fg, M):
+    """Config 2 says M = 1..16 tokens: the counts between the two that the other tests use."""
+    _sampled_linear_check(fg, gi.llama("cfg2", M, 11008, 4096, seed=8), 0.1, 4000, 10 + M)
+
+
+@pytest.mark.parametrize("N,K", [(11008, 4096), (4096, 11008)])
+def test_config3_llama2_7b_prefill_fc1_and_fc2(fg, N, K):
+    """Config 3 at M = 4096: FC1 / gate (4096 -> 11008) and FC2 (11008 -> 4096); the 4096 x 4096 projections are
+    test_linear_prefill_shape_sampled."""
+    _sampled_linear_check(fg, gi.llama("cfg3", 4096, N, K, seed=9), 0.1, 2500, 20)
+
+
+@pytest.mark.parametrize("N,K", [(13824, 5120), (5120, 13824)])
+def test_config4_llama2_13b_at_ten_percent(fg, N, K):
+    """Config 4 at M = 2048: both layers at the 10 % point of the sweep (0 / 20 / 30 % of FC1 are swept elsewhere)."""
+    _sampled_linear_check(fg, gi.llama("cfg4", 2048, N, K, seed=10), 0.1, 2500, 21)
+
+
+def test_config5_llama2_70b_prefill(fg):
+    """Config 5 at M = 8192: the 8192 x 8192 activations through the quantizer and the 28672 x 8192 FC1 GEMM."""
+    _sampled_linear_check(fg, gi.llama("cfg5", 8192, 28672, 8192, seed=11), 0.1, 2500, 22)
+
+
+def test_config3_fc2_activation_quantizer_full_size(fg):
+    """The activation quantizer on the 4096 x 11008 input of FC2, every block against the oracle."""
+    wl = gi.llama("cfg3a", 4096, 1, 11008, seed=12)
+    x, fx = wl.x(), wl.fx()
+    s4 = gi.tensor_scale(x)
+    xb = gi.bf16_bits(x)
+    scores = oracle.quantize_activations(xb, fx.numpy(), s4, tau=np.inf).scores
+    k = int(np.floor(0.1 * scores.size + 0.5))
+    srt = np.sort(scores)[::-1]
+    tau = float(np.float32(0.5) * (srt[k - 1] + srt[k]))
+    q = oracle.quantize_activations(xb, fx.numpy(), s4, tau=tau)
+    p = fg.quantize_activations(x.cuda(), fx.cuda(), scale_fp4=s4, tau=tau)
+    compare_packed(fg, p, q, tau, "4096 x 11008")
+
+
+def test_config5_clip_search_packer_at_full_width(fg):
+    """The packer with the Eq. 11 clip search on a full-width tensor (11008 x 4096, threshold mode, tensor scale
+    given, so that every block's outcome depends on that block alone): the blocks of the first 512 rows against
+    the oracle run on those rows."""
+    wl = gi.llama("cfg5w", 1, 11008, 4096, seed=13)
+    w, fw = wl.w(), wl.fw()
+    rows = 512
+    s4 = float(np.float32(w.float().abs().max().item() / 2688.0))
+    q0 = oracle.quantize_weights(gi.bf16_bits(w)[:rows].copy(), fw.numpy()[:rows].copy(), scale_fp4=s4, clip=True, fp8_fraction=0.0)
+    tau = float(np.sort(q0.scores)[::-1][int(0.1 * q0.scores.size)])
+    q = oracle.quantize_weights(gi.bf16_bits(w)[:rows].copy(), fw.numpy()[:rows].copy(), scale_fp4=s4, clip=True,
+                                fp8_fraction=-1.0, tau=tau)
+    p = fg.quantize_weights(w.cuda(), fw.cuda(), scale_fp4=s4, clip_mode=1, fp8_fraction=-1.0, tau=tau)
+    assert p.header()["error"] == 0
+    c4, c8, sc, mk = [t.cpu().numpy() for t in fg.unpack(p)]
+    K, KB = 4096, 256
+    MW = KB // 32
+    g = oracle.Quantized(rows, K, c4[: rows * K // 2], c8[: rows * K], sc[: rows * KB], mk.view(np.uint32)[: rows * MW],
+                         q.scores, s4, 3)
+    excused = np.abs(q.scores.reshape(rows, KB) - np.float32(tau)) <= 1e-6 * tau
+    keep = ~excused
+    assert ((g.mask_bits() == q.mask_bits()) | excused).all()
+    assert np.array_equal(g.scales.reshape(rows, KB)[keep], q.scales.reshape(rows, KB)[keep])
+    assert not ((g.codes4.reshape(rows, KB, 8) != q.codes4.reshape(rows, KB, 8)).any(-1) & keep).any()
+    assert not ((g.codes8.reshape(rows, KB, 16) != q.codes8.reshape(rows, KB, 16)).any(-1) & keep).any()
+    assert 0.05 < q.mask_bits().mean() < 0.2
+
+
+def test_clip_search_tie_cases_on_the_gpu(fg):
+    """The two tie cases whose outcome is derived by hand in tests/test_oracle_quant.py (an all-zero block; a block
+    that four scale codes represent exactly): the GPU packer gives the derived codes and scales."""
+    w, bits, codes4, scales = clip_tie_case()
+    wt = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    p = fg.quantize_weights(wt.cuda(), torch.ones(2, 64).cuda(), scale_fp4=1.0, clip_mode=1, fp8_fraction=0.0)
+    c4, c8, sc, mk = [t.cpu().numpy() for t in fg.unpack(p)]
+    assert np.array_equal(sc, scales) and np.array_equal(c4, codes4)
+    assert not c8.any() and not mk.any()

@@ -220,8 +220,11 @@ def quantize_both(fg, wl, frac_a, frac_w, mode=0, clip=True):
         w, fw = wl.w(), wl.fw()
         qw = oracle.quantize_weights(gi.bf16_bits(w), fw.numpy(), clip=clip, mode=mode, fp8_fraction=frac_w)
         pw = fg.quantize_weights(w.cuda(), fw.cuda(), clip_mode=int(clip), score_mode=mode, fp8_fraction=frac_w)
+        # the GEMM tests below must not be able to hide a wrong block inside their tolerance
+        compare_packed(fg, pw, qw, None, f"weights of {wl.name}")
         _last_weights[key] = (qw, pw)
     qw, pw = _last_weights[key]
+    compare_packed(fg, pa, qa, tau, f"activations of {wl.name}")
     return qa, qw, pa, pw
 
 
@@ -585,3 +588,23 @@ def test_linear_with_next_layer_quantizer_in_the_epilogue(fg, M, N, K, mode):
     Y, S = oracle.linear_sampled(qa, qw, ms, nn)
     got = y16.float().cpu().numpy().astype(np.float64)[ms, nn]
     assert (np.abs(got - Y) <= GEMM_TOL * S + np.abs(Y) * 2.0 ** -8 + 1e-30).all()
+
+
+def test_bounded_wait_runs_out_and_the_workspace_recovers(fg):
+    """The failure path of the kernels' waits, made to happen safely: one thread block waits 1 ms for a barrier
+    that nothing completes; the status word then says FGMP_ERR_TIMEOUT, clearing the workspace removes it, and
+    the same workspace serves a correct fgmp_linear afterwards."""
+    M, N, K = 16, 640, 1024
+    wl = gi.llama("d", M, N, K, seed=11)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+    ws = fg.alloc_workspace(fg.binding.OP_LINEAR, M, N, K, torch.device("cuda"))
+    y0 = fg.linear(pa, pw, workspace=ws)
+    fg.check(ws)
+    fg.selftest_wait_timeout(ws, 1_000_000)
+    with pytest.raises(fg.FgmpError) as e:
+        fg.check(ws)
+    assert e.value.code == -6 and "timed out" in str(e.value)
+    fg.workspace_init(ws)
+    fg.check(ws)
+    assert torch.equal(fg.linear(pa, pw, workspace=ws), y0)
+    fg.check(ws)

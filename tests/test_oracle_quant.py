@@ -374,3 +374,44 @@ def test_channel_mean_sq_against_float64():
     assert got.shape == (64,)
     assert np.all(np.abs(got - ref) <= 200 * 2.0 ** -24 * ref)
     assert not np.allclose((x.double().abs()).mean(0).numpy(), ref)
+
+
+# ------------------------------------------------------------------ tie rule of the clip search
+
+def clip_tie_case():
+    """Weights whose clip objective (Eq. 11) ties, with the outcome derived by hand.  Tensor scale 1.
+    * An all-zero block: every scale code gives J = 0; the incumbent is the dynamic-max code E4M3(0) = 0x00 and
+      a candidate replaces it only on strict improvement, so the scale stays 0x00 and all codes are +0.
+    * A block of +-2 and 0: amax / 6 = 0.3333 rounds to the E4M3 value 0.34375 (code 0x2b), under which 2 becomes
+      6 * 0.34375 = 2.0625 (J > 0).  J = 0 exactly for the scales 0.5, 1, 2 and 4 (2 / d in the E2M1 set); the
+      ascending scan meets 0.5 = code 0x30 first and later ties do not replace it: scale 0x30, 2 -> 2 / 0.5 = 4 =
+      E2M1 index 6 (code 0x6, negative 0xe), 0 -> code 0x0."""
+    pattern = np.array([2, -2, 2, 2, 0, -2, 0, 2, -2, -2, 2, 0, 2, 2, -2, 2], np.float32)
+    w = np.zeros((2, 64), np.float32)
+    w[0, 16:32] = pattern
+    w[1, 48:64] = pattern[::-1]
+    bits = (w.view(np.uint32) >> 16).astype(np.uint16)
+    codes = np.where(w == 2, 0x6, np.where(w == -2, 0xE, 0x0)).astype(np.uint8)
+    packed = (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)          # even element in the low nibble
+    scales = np.zeros((2, 4), np.uint8)
+    scales[0, 1] = 0x30
+    scales[1, 3] = 0x30
+    return w, bits, packed.ravel(), scales.ravel()
+
+
+def test_clip_search_ties_keep_the_incumbent_then_the_lowest_code():
+    w, bits, codes4, scales = clip_tie_case()
+    f = np.ones_like(w)
+    q = oracle.quantize_weights(bits, f, scale_fp4=1.0, clip=True, fp8_fraction=0.0)
+    assert np.array_equal(q.scales, scales), (q.scales, scales)
+    assert np.array_equal(q.codes4, codes4)
+    assert not q.mask_bits().any() and (q.scores == 0).all()
+    # the single-block entry point agrees, and the objective really ties where the derivation says
+    assert oracle.clip_search(w[0, 16:32], f[0, 16:32], 1.0) == 0x30
+    assert oracle.clip_search(np.zeros(16, np.float32), np.ones(16, np.float32), 1.0) == 0x00
+    for c in (0x30, 0x38, 0x40, 0x48):
+        assert oracle.clip_objective(w[0, 16:32], f[0, 16:32], c, 1.0) == 0.0
+    assert oracle.clip_objective(w[0, 16:32], f[0, 16:32], 0x2B, 1.0) > 0.0
+    # without the search the dynamic-max code stays
+    q0 = oracle.quantize_weights(bits, f, scale_fp4=1.0, clip=False, fp8_fraction=0.0)
+    assert q0.scales[1] == 0x2B and q0.scales[0] == 0x00
