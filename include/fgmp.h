@@ -103,7 +103,7 @@ typedef struct {
     int64_t rows, K;
     float scale_fp4;         /* tensor scale actually used                                  */
     int32_t fp8_log2_ratio;
-    int64_t n_fp8;           /* number of FP8 blocks                                        */
+    int64_t n_fp8;           /* number of FP8 blocks (activations: 0 if tau = +inf, else -1) */
     float tau_eff;           /* weights, fraction mode: smallest selected score             */
     uint32_t kind;           /* 0 = activations, 1 = weights                                */
     int64_t capacity;        /* weights: room for the FP8 lists, in 16-byte steps            */

@@ -318,7 +318,7 @@ decode_kernel(DecParams p)
             if (item == 0 && threadIdx.x == 64 && p.q_header) {
                 fgmp_packed_header* h = p.q_header;
                 h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.q.s4;
-                h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+                h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = (p.q.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
                 h->error = 0;
             }
             if (p.q_mode == 0) quantize_chunk<0>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));

@@ -65,6 +65,7 @@ __device__ __forceinline__ bool header_matches(const fgmp_packed_header* h, int6
 // packed activations -> bf16 plane; one thread per block
 __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane, int* status)
 {
+    if (status[2]) return;                              // the all-NVFP4 GEMM has produced the result already
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
     if (!header_matches(h, rows, K, 0u, status, 11)) return;
     const PackedLayout L = fgmp_layout(rows, K, 0, 0);
@@ -88,6 +89,7 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
 __global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* __restrict__ blob, int64_t rows, int64_t K, uint4* __restrict__ plane, int* status)
 {
     __shared__ UnitScratch sc;
+    if (status[2]) return;                              // the all-NVFP4 GEMM has produced the result already
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
     if (!header_matches(h, rows, K, 1u, status, 12)) return;
     const PackedLayout L = fgmp_layout(rows, K, 1, 0);
@@ -265,6 +267,7 @@ __device__ __forceinline__ void store_chunk32(const GemmParams& p, int64_t row, 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p)
 {
+    if (p.status[2]) return;                            // the all-NVFP4 GEMM has produced the result already (every thread of every CTA sees the same word)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // offset from the array: stays known as shared memory
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)P_STAGES * P_STAGE_BYTES);
@@ -293,7 +296,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     if (p.q.codes4 && blockIdx.x == 0 && threadIdx.x == 0) {
         fgmp_packed_header* h = p.q.header;
         h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
-        h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+        h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = (p.q.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
         h->error = 0;
     }
     const int64_t tiles_m = (p.M + P_BM - 1) / P_BM, tiles_n = (p.N + P_BN - 1) / P_BN;
@@ -462,6 +465,14 @@ static fgmp_status launch_prefill(const void* packed_acts, const void* packed_we
     if (!make_tmap_bf16(&tmA, planeA, M, K, 128) || !make_tmap_bf16(&tmB, planeW, N, K, 128)) return FGMP_ERR_CUDA;
 
     if (cudaMemsetAsync(status, 0, 256, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    // Operands without any FP8 block go through the NVFP4 tensor-core kind straight from the packed form; whether
+    // that is the case is written in the two headers, so the kernel looks itself and leaves word 2 of the status
+    // area at 1 if it has done the work.  (The variant with the next layer's quantizer in the epilogue has the
+    // general path only.)
+    if (!qn.codes4) {
+        const fgmp_status st4 = fgmp_launch_gemm_nvfp4(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, status, s);
+        if (st4 != FGMP_OK) return st4;
+    }
     const int sms = fgmp_sm_count();
     {
         const int64_t nb = M * (K / 16);

@@ -1,0 +1,320 @@
+// fgmp_linear for prefill-sized batches whose operands hold no FP8 block at all (threshold +inf for the
+// activations, FP8 fraction 0 for the weights: the all-NVFP4 end of the method's range): every block pair is
+// an FP4 x FP4 product (Section 4.1), and the GEMM runs on tcgen05.mma kind::mxf4nvf4 straight from the
+// packed operands -- no expansion pass, a quarter of the operand bytes of the bf16 container, four times its
+// MMA rate.
+//
+// The packed layouts were made for this: a weight record's code tile is the 128-byte-swizzled K-major tile
+// of 128 rows x 256 elements that the tensor core reads, its scale bytes are in tensor-memory order; the
+// activations' code plane is row-major (a TMA tile load swizzles it on the way in) and their scale section
+// consists of 512-byte tiles in the same tensor-memory order.
+//
+// One CTA per SM, persistent over 128 (tokens) x 256 (weight rows) output tiles; a stage holds one K chunk of
+// 256 elements: 16 KiB of activation codes, 2 x 16 KiB of weight codes, 3 x 2 KiB of scales.  Warp 0 = producer
+// (TMA / bulk copies), warp 1 = MMA issuer and owner of the tensor memory, warps 2-5 = block scales into
+// tensor memory (one lane quadrant each), warps 6-9 = epilogue (one lane quadrant each).  Every wait is bounded.
+#include <cuda.h>
+#include <mutex>
+#include "fgmp_common.cuh"
+#include "fgmp_host.h"
+#include "fgmp_ptx.cuh"
+
+namespace {
+
+constexpr int G4_THREADS = 320;
+constexpr int G4_STAGES = 4;
+constexpr uint32_t G4_A4 = 0, G4_B0 = 16384, G4_B1 = 32768, G4_SFB0 = 49152, G4_SFB1 = 51200, G4_SFA = 53248;
+constexpr uint32_t G4_STAGE_BYTES = 55296;
+constexpr size_t G4_SMEM = (size_t)G4_STAGES * G4_STAGE_BYTES + 1024 /*alignment*/ + 512 /*barriers*/;
+constexpr uint32_t G4_SF_COL0 = 256;            // tensor memory: 256 accumulator columns, then 48 scale columns per stage
+constexpr uint32_t G4_TMEM_COLS = 512;
+static_assert(G4_SMEM <= 232448, "shared memory of one CTA");
+static_assert(G4_SF_COL0 + 48 * G4_STAGES <= G4_TMEM_COLS, "tensor memory columns");
+
+// kind::mxf4nvf4, E2M1 x E2M1, UE4M3 scales, K-major operands, M = 128, dense K = 64; N = 256 or 128
+constexpr uint32_t G4_IDESC_BASE = (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 4) << 24);
+constexpr uint32_t G4_IDESC_N256 = G4_IDESC_BASE | ((uint32_t)(256 >> 3) << 17);
+constexpr uint32_t G4_IDESC_N128 = G4_IDESC_BASE | ((uint32_t)(128 >> 3) << 17);
+constexpr uint32_t G4_SW128_LO = 1u << 16, G4_SW128_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+
+__device__ __forceinline__ uint64_t g4_desc(uint32_t lo)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(G4_SW128_HI));
+    return d;
+}
+
+struct Gemm4Params {
+    const uint8_t* ablob; const uint8_t* wblob;
+    PackedLayout LA, LW;
+    void* Y; int64_t ldy; int y_is_bf16;
+    int64_t M, N, K;
+    int* status;                          // [0..1] device-side status, [2] 1 = this kernel has produced Y
+};
+
+__device__ __forceinline__ bool g4_applicable(const Gemm4Params& p)
+{
+    const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
+    const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+    return ha->magic == FGMP_MAGIC && ha->version == 7u && ha->rows == p.M && ha->K == p.K && ha->kind == 0u && ha->n_fp8 == 0 &&
+           hw->magic == FGMP_MAGIC && hw->version == 7u && hw->rows == p.N && hw->K == p.K && hw->kind == 1u && hw->error == 0 &&
+           hw->n_fp8 == 0;
+}
+
+__global__ void __launch_bounds__(G4_THREADS, 1)
+gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, Gemm4Params p)
+{
+    // operands with FP8 blocks (or headers that do not match the call) are left to the general path
+    if (!g4_applicable(p)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) p.status[2] = 0;
+        return;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) p.status[2] = 1;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    constexpr int S = G4_STAGES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * G4_STAGE_BYTES);
+    // bars: [0,S) full, [S,2S) empty, [2S,3S) scales in tensor memory, then acc_full, acc_empty
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, sfr0 = empty0 + 8 * S, accf = sfr0 + 8 * S, acce = accf + 8;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); mbar_init(sfr0 + 8 * s, 4); }
+        mbar_init(accf, 1); mbar_init(acce, 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), G4_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int64_t tiles_m = (p.M + 127) / 128, wtiles = p.LW.tiles, tiles_n = (wtiles + 1) / 2;
+    const int64_t num_tiles = tiles_m * tiles_n;
+    const int64_t chunks = p.LW.chunks;
+    const int64_t ksteps_total = p.K / 64;
+    const uint8_t* recs = p.wblob + p.LW.off_rec;
+    const uint8_t* asf = p.ablob + p.LA.off_sf;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                const int64_t tm = t % tiles_m, tn = t / tiles_m;             // token tiles fastest: CTAs that run together share weights
+                const bool two = 2 * tn + 1 < wtiles;
+                for (int64_t c = 0; c < chunks; ++c) {
+                    if (!(ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1))) break;
+                    const uint32_t ks = (uint32_t)min((int64_t)4, ksteps_total - 4 * c);
+                    const uint32_t fb = full0 + 8 * stage;
+                    const uint32_t dst = smem_u32(smem + (size_t)stage * G4_STAGE_BYTES);
+                    mbar_expect_tx(fb, 16384u + (two ? 2u : 1u) * (16384u + 2048u) + ks * 512u);
+                    tma_load_2d(dst + G4_A4, &tmA, (int32_t)(c * 128), (int32_t)(tm * 128), fb);
+                    const uint8_t* r0 = recs + (size_t)((2 * tn) * chunks + c) * REC_BYTES;
+                    bulk_load(dst + G4_B0, r0 + REC_W4, 16384, fb);
+                    bulk_load(dst + G4_SFB0, r0 + REC_SF, 2048, fb);
+                    if (two) {
+                        const uint8_t* r1 = recs + (size_t)((2 * tn + 1) * chunks + c) * REC_BYTES;
+                        bulk_load(dst + G4_B1, r1 + REC_W4, 16384, fb);
+                        bulk_load(dst + G4_SFB1, r1 + REC_SF, 2048, fb);
+                    }
+                    bulk_load(dst + G4_SFA, asf + ((size_t)tm * (size_t)ksteps_total + (size_t)(4 * c)) * 512, ks * 512u, fb);
+                    if (++stage == S) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t smem0 = smem_u32(smem);
+            int stage = 0; uint32_t phase = 0; bool ok = true;
+            int64_t it = 0;
+            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+                const int64_t tn = t / tiles_m;
+                const uint32_t idesc = (2 * tn + 1 < wtiles) ? G4_IDESC_N256 : G4_IDESC_N128;
+                if (!(ok = mbar_wait(acce, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status, 2))) break;    // the epilogue has drained the accumulator
+                tc_fence_after();
+                uint32_t accum = 0;
+                for (int64_t c = 0; c < chunks; ++c) {
+                    if (!(ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3))) break;
+                    if (!(ok = mbar_wait(sfr0 + 8 * stage, phase, abort_flag, p.status, 8))) break;
+                    tc_fence_after();
+                    const uint32_t ks = (uint32_t)min((int64_t)4, ksteps_total - 4 * c);
+                    const uint32_t sb = smem0 + (uint32_t)stage * G4_STAGE_BYTES;
+                    const uint32_t sf_t = tmem_base + G4_SF_COL0 + (uint32_t)stage * 48;     // [0,16) tokens, [16,48) weight rows
+                    const uint32_t a_lo = ((sb + G4_A4) >> 4) | G4_SW128_LO, b_lo = ((sb + G4_B0) >> 4) | G4_SW128_LO;
+                    for (uint32_t j = 0; j < ks; ++j) {
+                        umma_nvf4(tmem_base, g4_desc(a_lo + 2 * j), g4_desc(b_lo + 2 * j), idesc, sf_t + 4 * j, sf_t + 16 + 8 * j, accum);
+                        accum = 1;
+                    }
+                    umma_commit(empty0 + 8 * stage);
+                    if (++stage == S) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(accf);
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ block scales into tensor memory, lane quadrant warp % 4
+        // Lane i holds, for MMA step j, the scale bytes of operand rows i, 32+i, ... : one column per 32 rows, i.e.
+        // 16 bytes of a 512-byte scale tile per 128 rows.
+        int stage = 0; uint32_t phase = 0; bool ok = true;
+        for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            const int64_t tn = t / tiles_m;
+            const bool two = 2 * tn + 1 < wtiles;
+            for (int64_t c = 0; c < chunks; ++c) {
+                if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 4))) break;
+                const uint32_t ks = (uint32_t)min((int64_t)4, ksteps_total - 4 * c);
+                const uint8_t* sb = smem + (size_t)stage * G4_STAGE_BYTES;
+                const uint32_t sf_t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + G4_SF_COL0 + (uint32_t)stage * 48;
+                uint32_t r[16];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 x = make_uint4(0u, 0u, 0u, 0u);
+                    if ((uint32_t)j < ks) x = *reinterpret_cast<const uint4*>(sb + G4_SFA + 512 * j + lane * 16);
+                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                }
+                tmem_st16(sf_t, r);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {              // MMA steps 2 half, 2 half + 1: eight columns each
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int j = 2 * half + jj;
+                        const uint4 x = *reinterpret_cast<const uint4*>(sb + G4_SFB0 + 512 * j + lane * 16);
+                        uint4 y = make_uint4(0u, 0u, 0u, 0u);
+                        if (two) y = *reinterpret_cast<const uint4*>(sb + G4_SFB1 + 512 * j + lane * 16);
+                        r[8 * jj] = x.x; r[8 * jj + 1] = x.y; r[8 * jj + 2] = x.z; r[8 * jj + 3] = x.w;
+                        r[8 * jj + 4] = y.x; r[8 * jj + 5] = y.y; r[8 * jj + 6] = y.z; r[8 * jj + 7] = y.w;
+                    }
+                    tmem_st16(sf_t + 16 + 16 * half, r);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sfr0 + 8 * stage);
+                if (++stage == S) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: lane quadrant warp % 4, a token row per thread
+        const int q = warp & 3;
+        const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
+        const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
+        const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
+        bool ok = true;
+        int64_t it = 0;
+        for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
+            const int64_t tm = t % tiles_m, tn = t / tiles_m;
+            if (!(ok = mbar_wait_warp(accf, (uint32_t)(it & 1), abort_flag, p.status, 5))) break;
+            tc_fence_after();
+            const int64_t row = tm * 128 + q * 32 + lane, n0 = tn * 256;
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                if (n0 + c * 32 >= p.N) break;
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+                if (row < p.M) {
+                    const int64_t col0 = n0 + c * 32;
+                    if (p.y_is_bf16) {
+                        __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
+                        if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t o[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * u]) * alpha, __uint_as_float(r[j + 2 * u + 1]) * alpha);
+                                    o[u] = *reinterpret_cast<uint32_t*>(&h);
+                                }
+                                *reinterpret_cast<uint4*>(y + j) = make_uint4(o[0], o[1], o[2], o[3]);
+                            }
+                        } else {
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) y[j] = __float2bfloat16_rn(__uint_as_float(r[j]) * alpha);
+                        }
+                    } else {
+                        float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
+                        if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
+                                                                                __uint_as_float(r[j + 2]) * alpha, __uint_as_float(r[j + 3]) * alpha);
+                        } else {
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) y[j] = __uint_as_float(r[j]) * alpha;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce);
+        }
+    }
+
+    __syncthreads();
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, G4_TMEM_COLS);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g4_mu;
+EncodeTiledFn g4_encode = nullptr;
+bool g4_attr_set[64] = {};
+
+}  // namespace
+
+// Launches the all-NVFP4 GEMM; it decides on the device (from the two headers) whether it applies and says so in
+// status[2], which the general path's kernels read.
+fgmp_status fgmp_launch_gemm_nvfp4(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
+                                   int64_t M, int64_t N, int64_t K, int* status, cudaStream_t s)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lk(g4_mu);
+        if (!g4_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+                q != cudaDriverEntryPointSuccess) return FGMP_ERR_CUDA;
+            g4_encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        if (!g4_attr_set[dev]) {
+            if (cudaFuncSetAttribute(gemm_nvfp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G4_SMEM) != cudaSuccess)
+                return FGMP_ERR_CUDA;
+            g4_attr_set[dev] = true;
+        }
+    }
+    Gemm4Params p;
+    p.ablob = (const uint8_t*)packed_acts; p.wblob = (const uint8_t*)packed_weights;
+    p.LA = fgmp_layout(M, K, 0, 0); p.LW = fgmp_layout(N, K, 1, 0);
+    p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K; p.status = status;
+    // the activations' code plane: bytes [M, K/2] row-major, boxes of 128 rows x 128 bytes, swizzled on the way in
+    CUtensorMap tmA;
+    cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)M};
+    cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    cuuint32_t box[2] = {128, 128};
+    cuuint32_t estr[2] = {1, 1};
+    if (g4_encode(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(p.ablob + p.LA.off_codes4), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return FGMP_ERR_CUDA;
+    const int64_t tiles = ((M + 127) / 128) * ((p.LW.tiles + 1) / 2);
+    const int sms = fgmp_sm_count();
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    FGMP_LAUNCH(FGMP_K_GEMM_NVFP4, s, gemm_nvfp4_kernel<<<grid, G4_THREADS, G4_SMEM, s>>>(tmA, p));
+    return fgmp_launch_status();
+}

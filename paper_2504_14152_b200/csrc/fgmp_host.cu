@@ -80,7 +80,7 @@ std::vector<ProfRec> g_prof_recs;
 std::vector<cudaEvent_t> g_event_pool;
 const char* const g_kernel_names[FGMP_K_COUNT] = {
     "quant_act", "act_aux", "unpack", "expand_acts", "expand_weights", "gemm_bf16_tcgen05",
-    "w_amax", "w_score_clip", "select", "w_mask", "scan", "w_emit", "w_aux", "act_scores", "decode_gemm"};
+    "w_amax", "w_score_clip", "select", "w_mask", "scan", "w_emit", "w_aux", "act_scores", "decode_gemm", "gemm_nvfp4_tcgen05"};
 cudaEvent_t get_event()
 {
     if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }

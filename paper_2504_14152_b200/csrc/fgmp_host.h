@@ -22,11 +22,15 @@ size_t fgmp_ws_decode(int64_t M, int64_t N, int64_t K);
 fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
                                int64_t M, int64_t N, int64_t K, void* workspace, bool clear_first, cudaStream_t s);
 
+// all-NVFP4 prefill GEMM (fgmp_gemm4.cu): decides on the device whether it applies, answer in status[2]
+fgmp_status fgmp_launch_gemm_nvfp4(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
+                                   int64_t M, int64_t N, int64_t K, int* status, cudaStream_t s);
+
 // ---- launch accounting (see fgmp_profile_begin in fgmp.h) ----
 enum FgmpKernelId {
     FGMP_K_ACT_QUANT = 0, FGMP_K_ACT_AUX, FGMP_K_UNPACK, FGMP_K_EXPAND_A, FGMP_K_EXPAND_W, FGMP_K_GEMM_BF16,
     FGMP_K_W_AMAX, FGMP_K_W_SCORE, FGMP_K_SELECT, FGMP_K_W_MASK, FGMP_K_SCAN, FGMP_K_W_EMIT, FGMP_K_W_AUX,
-    FGMP_K_ACT_SCORES, FGMP_K_DECODE, FGMP_K_COUNT
+    FGMP_K_ACT_SCORES, FGMP_K_DECODE, FGMP_K_GEMM_NVFP4, FGMP_K_COUNT
 };
 // Brackets one kernel launch: counts it and, when event timing of this kernel id is on,
 // records a CUDA event before and after it on the launch stream.

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
             fgmp_packed_header* h = p.header;
             h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
-            h->fp8_log2_ratio = p.ratio; h->n_fp8 = -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
+            h->fp8_log2_ratio = p.ratio; h->n_fp8 = (p.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
             h->error = 0;
         }
         // token rows M..15 of the decode records are zero (the grid covers 16 rows in that mode)

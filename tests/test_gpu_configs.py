@@ -89,3 +89,30 @@ def test_clip_search_tie_cases_on_the_gpu(fg):
     c4, c8, sc, mk = [t.cpu().numpy() for t in fg.unpack(p)]
     assert np.array_equal(sc, scales) and np.array_equal(c4, codes4)
     assert not c8.any() and not mk.any()
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 256, 256), (77, 300, 1024), (129, 136, 64), (384, 1000, 2048), (1000, 640, 320)])
+def test_all_nvfp4_operands_take_the_fp4_tensor_core_kernel(fg, M, N, K):
+    """With no FP8 block on either side (threshold +inf, fraction 0) the prefill GEMM runs on the NVFP4 tensor-core
+    kind straight from the packed operands (word 2 of the workspace status says which kernel produced Y): every
+    output against the oracle, fp32 and bf16; one FP8 block anywhere sends the call down the general path."""
+    wl = gi.llama("n4", M, N, K, seed=50 + M)
+    qa, qw, pa, pw = quantize_both(fg, wl, 0.0, 0.0, clip=True)
+    Y, S = oracle.linear(qa, qw)
+    y = fg.linear(pa, pw)
+    ws = fg.linear.last_workspace
+    fg.check(ws)
+    assert int(ws[8:12].view(torch.int32).item()) == 1, "the NVFP4 kernel did not take the call"
+    err = np.abs(y.cpu().numpy().astype(np.float64) - Y)
+    assert (err <= 1e-5 * S + 1e-30).all(), f"max err/S = {(err / np.maximum(S, 1e-300)).max():.3e}"
+    assert torch.equal(fg.linear(pa, pw), y)
+    yb = fg.linear(pa, pw, out_dtype=torch.bfloat16).float().cpu().numpy().astype(np.float64)
+    assert (np.abs(yb - Y) <= GEMM_TOL * S + np.abs(Y) * 2.0 ** -8 + 1e-30).all()
+    # FP8 blocks in the weights: the general path, same bar
+    qa2, qw2, pa2, pw2 = quantize_both(fg, wl, 0.0, 0.1, clip=True)
+    y2 = fg.linear(pa2, pw2)
+    ws2 = fg.linear.last_workspace
+    fg.check(ws2)
+    assert int(ws2[8:12].view(torch.int32).item()) == 0
+    Y2, S2 = oracle.linear(qa2, qw2)
+    assert (np.abs(y2.cpu().numpy().astype(np.float64) - Y2) <= 1e-5 * S2 + 1e-30).all()
