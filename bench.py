@@ -6,9 +6,11 @@
 Default workload: Llama-2-7B FC1 at decode (M=16 tokens, K=4096, N=11008, 10% FP8 blocks in
 weights and activations); metric = packed-weight GB/s.  One step = the online path: quantize
 the step's activations (bf16 -> mixed NVFP4/FP8) and run the mixed-precision GEMM against
-offline-packed weights.  Weight packing is offline in the method and is timed separately
-(reported under "offline").  The step rotates over several weight copies so that the working
-set exceeds L2.  Prints ONE JSON line (rank 0).
+offline-packed weights -- one fused launch at decode, two calls at prefill.  Weight packing is
+offline in the method and is timed separately (reported under "offline").  The step rotates
+over several weight copies so that the working set exceeds L2.  `value` is the median of
+--replays timed runs of exactly --steps steps.  The default run adds the 70B decode layer and
+a prefill layer as side objects ("decode_70b", "prefill").  Prints ONE JSON line (rank 0).
 
 With N > 1 (torchrun) every rank runs an independent replica of the same workload on its own
 GPU ("weak" scaling, no data-path collective); the time is the max over ranks.
@@ -313,7 +315,7 @@ def roofline_of(fg, wk, prof, step_ms, dev, peaks):
         if "decode_gemm" in prof and prof["decode_gemm"][1]:
             ev_us = prof["decode_gemm"][1] / prof["decode_gemm"][0] * 1e3
         return {"kernel": "decode_gemm", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                "frac": ach / peaks["hbm_gbs"], "traffic": traffic_bytes("decode_gemm", wk.name),
                 "traffic_from_profile": load_traffic("decode_gemm", wk.name),
                 "peak_source": peaks["source"], "avg_kernel_us": avg_s * 1e6,
                 "avg_kernel_us_note": "timed region / launches: the step is one launch of this kernel (activation quantizer inside)",
@@ -333,7 +335,7 @@ def roofline_of(fg, wk, prof, step_ms, dev, peaks):
     blended_s = wk.flops * (f4 / p4 + (1 - f4) / p8) / 1e12
     blended_peak = wk.flops / blended_s / 1e12
     return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": blended_peak, "unit": "TFLOP/s",
-            "frac": ach / blended_peak, "traffic": None, "traffic_from_profile": load_traffic(name, wk.name),
+            "frac": ach / blended_peak, "traffic": traffic_bytes(name, wk.name), "traffic_from_profile": load_traffic(name, wk.name),
             "peak_source": "blend of the NVFP4 and E4M3 tcgen05 rates measured in this run for this FP8 fraction",
             "avg_kernel_us": avg_s * 1e6,
             "frac_of_fp8_roofline": (wk.flops / p8 / 1e12) / avg_s,
@@ -455,12 +457,19 @@ def run_ours(args, world, rank, local):
 # DRAM bytes (read + write) per launch from the committed ncu captures (profiles/*.md).  An entry is
 # removed when its kernel changes after the capture.
 NCU_TRAFFIC = {
+    ("llama2-7b-fc1-decode", "decode_gemm"): {"bytes": 29194240, "file": "profiles/decode_kernel_llama2-7b-fc1-decode.md"},
+    ("llama2-13b-fc1-prefill", "gemm_nvfp4_tcgen05"): {"bytes": 106512640, "file": "profiles/gemm_nvfp4_kernel_llama2-13b-fc1-prefill.md"},
     ("llama2-7b-fc2-prefill", "gemm_bf16_tcgen05"): {"bytes": 535152896, "file": "profiles/gemm_bf16_pair_kernel_llama2-7b-fc2-prefill.md"},
 }
 
 
 def load_traffic(kernel: str, workload: str):
     return NCU_TRAFFIC.get((workload, kernel))
+
+
+def traffic_bytes(kernel: str, workload: str):
+    e = load_traffic(kernel, workload)
+    return e["bytes"] if e else None
 
 
 def cpu_baseline(args, wl, p, kind, per_step_units, unit, budget_s=20.0, max_steps=None):

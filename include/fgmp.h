@@ -231,8 +231,9 @@ fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
  *     caller that wants them (fgmp_unpack, or a later fgmp_linear with other weights); if NULL only the
  *     fp16 records the GEMM streams are kept, in the workspace.
  *   workspace: fgmp_workspace_bytes(FGMP_OP_LINEAR_FUSED, M, N, K), cleared once with
- *     fgmp_workspace_init.  Beside fgmp_linear's words the control area holds a call number, which
- *     tags what the blocks publish to each other, so nothing has to be cleared between calls; after an
+ *     fgmp_workspace_init.  Beside fgmp_linear's words the control area holds the work-item counters of
+ *     the quantizer and a "records ready" word; the counters wrap to zero by themselves and the block that
+ *     finishes last clears the word, so nothing has to be cleared between calls; after an
  *     error reported by fgmp_check clear the workspace again.  Calls that share a workspace must not
  *     overlap on the GPU.
  *   The kernel is launched as a programmatic dependent like fgmp_linear's (same condition on

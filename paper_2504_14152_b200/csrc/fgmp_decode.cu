@@ -40,7 +40,6 @@
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
 #include <cuda_fp16.h>
-#include <cstdio>
 #include <mutex>
 #include <type_traits>
 
@@ -577,9 +576,6 @@ decode_kernel(DecParams p)
                 const uint8_t* sa = sb + STG_A;
                 const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
                 uint32_t todo = hot & 0xffffu;
-#ifdef FGMP_DEBUG_PRINT
-                if (blockIdx.x == 0 && lane == 5) printf("hot warp %d u %lld todo %x stage %d\n", warp, (long long)u, todo, stage);
-#endif
                 while (todo) {
                     const uint32_t j = (uint32_t)__ffs(todo) - 1u;
                     todo &= todo - 1;
@@ -605,9 +601,6 @@ decode_kernel(DecParams p)
                         }
 #pragma unroll
                         for (int nh = 0; nh < NH; ++nh) mma_f16_16816(acc[mt][nh], x[0][0], x[1][0], x[0][1], x[1][1], b[nh].x, b[nh].y);
-#ifdef FGMP_DEBUG_PRINT
-                        if (blockIdx.x == 0 && lane == 5 && mt == 0 && j < 2) printf("  w %d j %u x %08x %08x b %08x %08x acc %f\n", warp, j, x[0][0], x[1][0], b[0].x, b[0].y, acc[0][0][0]);
-#endif
                     }
                 }
                 __syncwarp();
@@ -704,9 +697,6 @@ decode_kernel(DecParams p)
             // corrections (2) and (3) of the segment: this row of every tile, in tile order; the rows of (2)
             // are cleared for the next segment on the way
             if (!(ok = mbar_wait_warp(cdone0 + 8 * accb, acc_phase, abort_flag, p.status, 12))) break;
-#ifdef FGMP_DEBUG_PRINT
-            if (blockIdx.x == 0 && lane == 1) printf("epi warp %d row %d tile4 %f %f v0 %f\n", warp, row, tiles[FP8_WARPS * TILE_FLOATS + tile_idx(row, 0)], tiles[FP8_WARPS * TILE_FLOATS + tile_idx(row, 1)], v[0]);
-#endif
             float c2[16];                              // (2): sums of the FP8 weight codes, still without 2^ratio
 #pragma unroll
             for (int j = 0; j < 16; ++j) c2[j] = 0.f;
@@ -826,7 +816,7 @@ fgmp_status set_attrs_once()
 }
 
 // Workspace of the decode path, all inside the control area that must be zero before the first call and
-// that every call leaves zero (the call number excepted): status at 0, control words at 256, stream-K
+// that every call leaves zero: status at 0, control words at 256, stream-K
 // counters from 1024 (32 bytes per tile); partial sums behind the control area, then (fused calls
 // without a packed output) the activation records.
 DecParams base_params(const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
