@@ -182,6 +182,14 @@ WORKLOADS = {
     "llama2-70b-fc1-prefill": (8192, 28672, 8192, 0.10, "prefill"),
     "llama2-70b-fc2-decode": (16, 8192, 28672, 0.10, "decode"),
     "llama2-13b-fc1-decode": (16, 13824, 5120, 0.10, "decode"),
+    # the other families Section 5.1 names (hidden / feed-forward widths of the models' public descriptions)
+    "gpt3-1.3b-fc1-decode": (16, 8192, 2048, 0.10, "decode"),
+    "gpt3-8.3b-fc1-decode": (16, 12288, 3072, 0.10, "decode"),
+    "gpt3-8.3b-fc1-prefill": (2048, 12288, 3072, 0.10, "prefill"),
+    "gpt3-22b-fc1-decode": (16, 24576, 6144, 0.10, "decode"),
+    "nemotron4-15b-fc1-decode": (16, 24576, 6144, 0.10, "decode"),
+    "nemotron4-15b-fc2-decode": (16, 6144, 24576, 0.10, "decode"),
+    "nemotron4-15b-fc1-prefill": (4096, 24576, 6144, 0.10, "prefill"),
     "tiny": (64, 256, 256, 0.10, "decode"),
 }
 

@@ -116,3 +116,93 @@ def test_all_nvfp4_operands_take_the_fp4_tensor_core_kernel(fg, M, N, K):
     assert int(ws2[8:12].view(torch.int32).item()) == 0
     Y2, S2 = oracle.linear(qa2, qw2)
     assert (np.abs(y2.cpu().numpy().astype(np.float64) - Y2) <= 1e-5 * S2 + 1e-30).all()
+
+
+# ------------------------------------------------------------ the other model families of Section 5.1
+
+# FC1 / FC2 shapes (N, K) of the GPT3 and Nemotron-4 models that Section 5.1 evaluates beside Llama-2; hidden and
+# feed-forward widths as in the models' public descriptions (the paper gives the names only)
+OTHER_FAMILIES = {
+    "gpt3-1.3b": (2048, 8192),
+    "gpt3-8.3b": (3072, 12288),
+    "gpt3-22b": (6144, 24576),
+    "nemotron4-15b": (6144, 24576),
+}
+
+
+@pytest.mark.parametrize("model,M", [("gpt3-1.3b", 16), ("gpt3-8.3b", 3), ("gpt3-22b", 16), ("nemotron4-15b", 1)])
+def test_section_5_1_other_families_decode(fg, model, M):
+    """GPT3 and Nemotron-4 feed-forward layers at decode size: FC1 and FC2, sampled outputs against the oracle
+    (packed operands compared bit for bit first)."""
+    h, f = OTHER_FAMILIES[model]
+    _sampled_linear_check(fg, gi.llama(model + "-fc1", M, f, h, seed=60), 0.1, 3000, 30)
+    _sampled_linear_check(fg, gi.llama(model + "-fc2", M, h, f, seed=61), 0.1, 3000, 31)
+
+
+@pytest.mark.parametrize("model,M", [("gpt3-8.3b", 2048), ("nemotron4-15b", 1024)])
+def test_section_5_1_other_families_prefill(fg, model, M):
+    h, f = OTHER_FAMILIES[model]
+    _sampled_linear_check(fg, gi.llama(model + "-fc1p", M, f, h, seed=62), 0.1, 2500, 32)
+
+
+# ------------------------------------------------------------ guard bands
+
+CANARY = 0xA5
+
+
+class Guarded:
+    """A device buffer with 4 KiB of canary bytes before and after the part that is handed to the library."""
+
+    def __init__(self, nbytes, device="cuda", fill=None):
+        self.n = int(nbytes)
+        self.raw = torch.full((self.n + 2 * 4096 + 1024,), CANARY, dtype=torch.uint8, device=device)
+        off = 4096 + ((-(self.raw.data_ptr() + 4096)) % 1024)
+        self.off = off
+        self.view = self.raw[off:off + self.n]
+        if fill is not None:
+            self.view.fill_(fill)
+
+    def intact(self):
+        before, after = self.raw[: self.off], self.raw[self.off + self.n:]
+        return bool((before == CANARY).all().item()) and bool((after == CANARY).all().item())
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 1000, 1024), (200, 392, 512)])
+def test_no_call_writes_outside_its_buffers(fg, M, N, K):
+    """Every buffer a call writes (packed activations, packed weights, workspaces, Y) sits between canary bytes
+    that must be unchanged afterwards: the packer, the activation quantizer, fgmp_linear at decode and prefill
+    size and the fused decode step, with results equal to those of the same calls on ordinary buffers."""
+    wl = gi.llama("guard", M, N, K, seed=70)
+    x, fx, w, fw = wl.x().cuda(), wl.fx().cuda(), wl.w().cuda(), wl.fw().cuda()
+    s4 = gi.tensor_scale(wl.x())
+    tau = float(fg.calibrate_tau(x, fx, scale_fp4=s4, fp8_fraction=0.1))
+    B = N * K // 16
+    n8 = int(0.1 * B + 0.5) + 1
+    gw = Guarded(fg.weights_bytes(N, K, n8))
+    gws = Guarded(fg.workspace_bytes(fg.OP_QUANTIZE_WEIGHTS, 0, N, K))
+    pw = fg.quantize_weights(w, fw, fp8_fraction=0.1, out=gw.view, workspace=gws.view)
+    ga = Guarded(fg.acts_bytes(M, K))
+    pa = fg.quantize_activations(x, fx, scale_fp4=s4, tau=tau, out=ga.view)
+    gy = Guarded(M * N * 4)
+    gl = Guarded(fg.workspace_bytes(fg.OP_LINEAR, M, N, K), fill=0)
+    fg.workspace_init(gl.view)
+    y = fg.linear(pa, pw, out=gy.view.view(torch.float32).view(M, N), workspace=gl.view)
+    fg.check(gl.view)
+    torch.cuda.synchronize()
+    for name, g in (("packed weights", gw), ("packer workspace", gws), ("packed activations", ga), ("Y", gy), ("workspace", gl)):
+        assert g.intact(), f"bytes around {name} were written"
+    pw0 = fg.quantize_weights(w, fw, fp8_fraction=0.1)
+    pa0 = fg.quantize_activations(x, fx, scale_fp4=s4, tau=tau)
+    assert torch.equal(fg.linear(pa0, pw0), y)
+    if M <= 16:
+        gy2 = Guarded(M * N * 2)
+        gf = Guarded(fg.workspace_bytes(fg.OP_LINEAR_FUSED, M, N, K), fill=0)
+        gp = Guarded(fg.acts_bytes(M, K))
+        fg.workspace_init(gf.view)
+        y2, _ = fg.linear_fused(x, fx, pw, scale_fp4=s4, tau=tau, out=gy2.view.view(torch.bfloat16).view(M, N),
+                                packed_out=gp.view, workspace=gf.view)
+        fg.check(gf.view)
+        torch.cuda.synchronize()
+        for name, g in (("Y (bf16)", gy2), ("fused workspace", gf), ("packed activations of the fused call", gp), ("packed weights", gw)):
+            assert g.intact(), f"bytes around {name} were written"
+        assert torch.equal(y2.float(), fg.linear(pa0, pw0, out_dtype=torch.bfloat16).float())
