@@ -93,7 +93,13 @@ typedef enum { FGMP_CLIP_NONE = 0, FGMP_CLIP_SW_BRUTE = 1 } fgmp_clip_mode;
 typedef struct {
     float scale_fp4;    /* FP32 tensor scale of the NVFP4 part; 0 = derive amax/(6*448)
                            on the device (weights only)                                     */
-    int fp8_log2_ratio; /* FP8 tensor scale = scale_fp4 * 2^ratio, -7 <= ratio <= 7        */
+    int fp8_log2_ratio; /* FP8 tensor scale = scale_fp4 * 2^ratio, -7 <= ratio <= 7 (used
+                           when scale_fp8 is 0)                                             */
+    float scale_fp8;    /* 0, or an FP32 tensor scale of the FP8 part of its own (Section
+                           5.1: FP8 blocks carry no microscale, only a per-tensor scale),
+                           in any ratio to scale_fp4.  Operands packed with such a scale
+                           are multiplied by fgmp_linear_classes; fgmp_linear, whose single
+                           accumulator needs the power-of-two ratio, refuses them.          */
 } fgmp_scales;
 
 /* First 256 bytes of a packed blob (device memory). */
@@ -108,13 +114,15 @@ typedef struct {
     uint32_t kind;           /* 0 = activations, 1 = weights                                */
     int64_t capacity;        /* weights: room for the FP8 lists, in 16-byte steps            */
     int32_t error;           /* 0, or FGMP_ERR_CAPACITY                                     */
-    int32_t reserved[49];
+    float scale_fp8;         /* FP8 tensor scale actually used                              */
+    int32_t fp8_scale_free;  /* 1 if scale_fp8 was given on its own (fgmp_scales.scale_fp8) */
+    int32_t reserved[47];
 } fgmp_packed_header;
 
 enum { FGMP_OP_QUANTIZE_WEIGHTS = 0, FGMP_OP_QUANTIZE_ACTIVATIONS = 1, FGMP_OP_LINEAR = 2,
        FGMP_OP_CALIBRATE_TAU = 3,
        FGMP_OP_GLOBAL_TAU = 4,      /* M = total number of scores; N, K ignored */
-       FGMP_OP_LINEAR_QUANTIZE = 5, FGMP_OP_LINEAR_FUSED = 6 };
+       FGMP_OP_LINEAR_QUANTIZE = 5, FGMP_OP_LINEAR_FUSED = 6, FGMP_OP_LINEAR_CLASSES = 7 };
 
 /* ---- sizes (pure host functions; return 0 for invalid shapes) ---- */
 size_t fgmp_weights_bytes(int64_t N, int64_t K, int64_t max_fp8_blocks);
@@ -218,6 +226,19 @@ fgmp_status fgmp_workspace_init(void* workspace, size_t ws_bytes, void* cuda_str
 fgmp_status fgmp_linear(const void* packed_acts, const void* packed_weights,
                         void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
                         void* workspace, size_t ws_bytes, void* cuda_stream);
+
+/* ---- the same GEMM with one accumulation per class of block pair (Section 4.1: the four dot-product
+ * units; Section 5.1: FP8 blocks under a per-tensor scale of their own) ----
+ * For operands whose FP8 tensor scale is not tied to the NVFP4 one by a power of two (fgmp_scales.scale_fp8 > 0
+ * at packing time; operands with tied scales are accepted too).  The four classes FP4xFP4, FP4xFP8, FP8xFP4 and
+ * FP8xFP8 are accumulated separately in FP32 -- four passes of the tensor-core GEMM over operands in which the
+ * blocks of the other format are zero -- and each sum is multiplied by the product of its own two tensor scales
+ * before it is added to Y.  About four times the cost of fgmp_linear: the price of the free scale.
+ * Y is fp32 [M, ldy] (y_is_bf16 must be 0).  workspace: fgmp_workspace_bytes(FGMP_OP_LINEAR_CLASSES, M, N, K),
+ * cleared once with fgmp_workspace_init; any M >= 1. */
+fgmp_status fgmp_linear_classes(const void* packed_acts, const void* packed_weights,
+                                void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                void* workspace, size_t ws_bytes, void* cuda_stream);
 
 /* ---- one decode step in one launch: activation quantizer + GEMM (Section 4.2 into Section 4.1) ----
  * For decode-sized batches (the shapes of fgmp_linear's weight-streaming kernel: 1 <= M <= 16,

@@ -51,25 +51,25 @@ def lib():
         L.oracle_quantize_activations.restype = None
         L.oracle_quantize_activations.argtypes = [
             ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
-            ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+            ctypes.c_float, ctypes.c_int, ctypes.c_float, ctypes.c_int, ctypes.c_float,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.oracle_quantize_weights.restype = ctypes.c_float
         L.oracle_quantize_weights.argtypes = [
             ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64,
-            ctypes.c_int64, ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctypes.c_float, ctypes.c_int, ctypes.c_int,
             ctypes.c_double, ctypes.c_float,
             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
             ctypes.c_void_p]
         L.oracle_decode.restype = None
         L.oracle_decode.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64, ctypes.c_int64,
-                                                            ctypes.c_float, ctypes.c_int, ctypes.c_void_p]
+                                                            ctypes.c_float, ctypes.c_int, ctypes.c_float, ctypes.c_void_p]
         L.oracle_linear.restype = None
         L.oracle_linear.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
         L.oracle_linear_sampled.restype = None
         L.oracle_linear_sampled.argtypes = (
-            [ctypes.c_void_p] * 4 + [ctypes.c_float, ctypes.c_int] +
-            [ctypes.c_void_p] * 4 + [ctypes.c_float, ctypes.c_int, ctypes.c_int64,
+            [ctypes.c_void_p] * 4 + [ctypes.c_float, ctypes.c_int, ctypes.c_float] +
+            [ctypes.c_void_p] * 4 + [ctypes.c_float, ctypes.c_int, ctypes.c_float, ctypes.c_int64,
                                      ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
                                      ctypes.c_void_p, ctypes.c_void_p])
         L.oracle_num_threads.restype = ctypes.c_int
@@ -95,6 +95,7 @@ class Quantized:
     scale_fp4: float
     ratio: int
     tau_eff: float = float("nan")
+    scale_fp8: float = 0.0   # 0: tied to scale_fp4 by 2^ratio; else the FP8 tensor scale given on its own
 
     def mask_bits(self) -> np.ndarray:
         """bool [rows, K/16]: True = FP8 block."""
@@ -130,21 +131,21 @@ def _alloc(rows: int, K: int):
 
 
 def quantize_activations(x_bf16_bits: np.ndarray, fisher: np.ndarray, scale_fp4: float,
-                         ratio: int = 3, mode: int = 0, tau: float = float("inf")) -> Quantized:
+                         ratio: int = 3, mode: int = 0, tau: float = float("inf"), scale_fp8: float = 0.0) -> Quantized:
     """x_bf16_bits: uint16 [M, K] (bf16 bit patterns); fisher: float32 [K]."""
     M, K = x_bf16_bits.shape
     assert K % BS == 0 and x_bf16_bits.dtype == np.uint16
     x = np.ascontiguousarray(x_bf16_bits)
     f = np.ascontiguousarray(fisher, dtype=np.float32)
     c4, c8, sc, mk, scr = _alloc(M, K)
-    lib().oracle_quantize_activations(_p(x), K, _p(f), M, K, float(np.float32(scale_fp4)), ratio, mode,
+    lib().oracle_quantize_activations(_p(x), K, _p(f), M, K, float(np.float32(scale_fp4)), ratio, float(np.float32(scale_fp8)), mode,
                                       float(np.float32(tau)), _p(c4), _p(c8), _p(sc), _p(mk), _p(scr))
-    return Quantized(M, K, c4, c8, sc, mk, scr, float(np.float32(scale_fp4)), ratio, float(tau))
+    return Quantized(M, K, c4, c8, sc, mk, scr, float(np.float32(scale_fp4)), ratio, float(tau), float(np.float32(scale_fp8)))
 
 
 def quantize_weights(w_bf16_bits: np.ndarray, fisher: np.ndarray, scale_fp4: float = 0.0,
                      ratio: int = 3, mode: int = 0, clip: bool = True,
-                     fp8_fraction: float = 0.1, tau: float = 0.0) -> Quantized:
+                     fp8_fraction: float = 0.1, tau: float = 0.0, scale_fp8: float = 0.0) -> Quantized:
     """w_bf16_bits: uint16 [N, K]; fisher: float32 [N, K] (per element)."""
     N, K = w_bf16_bits.shape
     assert K % BS == 0 and w_bf16_bits.dtype == np.uint16 and fisher.shape == (N, K)
@@ -152,17 +153,17 @@ def quantize_weights(w_bf16_bits: np.ndarray, fisher: np.ndarray, scale_fp4: flo
     f = np.ascontiguousarray(fisher, dtype=np.float32)
     c4, c8, sc, mk, scr = _alloc(N, K)
     teff = ctypes.c_float(0.0)
-    s4 = lib().oracle_quantize_weights(_p(w), K, _p(f), K, N, K, float(np.float32(scale_fp4)), ratio, mode,
+    s4 = lib().oracle_quantize_weights(_p(w), K, _p(f), K, N, K, float(np.float32(scale_fp4)), ratio, float(np.float32(scale_fp8)), mode,
                                        int(bool(clip)), float(fp8_fraction), float(np.float32(tau)),
                                        _p(c4), _p(c8), _p(sc), _p(mk), _p(scr), ctypes.byref(teff))
-    return Quantized(N, K, c4, c8, sc, mk, scr, float(s4), ratio, float(teff.value))
+    return Quantized(N, K, c4, c8, sc, mk, scr, float(s4), ratio, float(teff.value), float(np.float32(scale_fp8)))
 
 
 def decode(q: Quantized) -> np.ndarray:
     """float64 [rows, K]: exact values of the quantized tensor."""
     out = np.zeros((q.rows, q.K), np.float64)
     lib().oracle_decode(_p(q.codes4), _p(q.codes8), _p(q.scales), _p(q.mask), q.rows, q.K,
-                        float(np.float32(q.scale_fp4)), q.ratio, _p(out))
+                        float(np.float32(q.scale_fp4)), q.ratio, float(np.float32(q.scale_fp8)), _p(out))
     return out
 
 
@@ -183,9 +184,9 @@ def linear_sampled(a: Quantized, w: Quantized, ms: np.ndarray, ns: np.ndarray):
     Y = np.zeros(len(ms), np.float64)
     S = np.zeros(len(ms), np.float64)
     lib().oracle_linear_sampled(_p(a.codes4), _p(a.codes8), _p(a.scales), _p(a.mask),
-                                float(np.float32(a.scale_fp4)), a.ratio,
+                                float(np.float32(a.scale_fp4)), a.ratio, float(np.float32(a.scale_fp8)),
                                 _p(w.codes4), _p(w.codes8), _p(w.scales), _p(w.mask),
-                                float(np.float32(w.scale_fp4)), w.ratio, a.K, len(ms), _p(ms), _p(ns),
+                                float(np.float32(w.scale_fp4)), w.ratio, float(np.float32(w.scale_fp8)), a.K, len(ms), _p(ms), _p(ns),
                                 _p(Y), _p(S))
     return Y, S
 

@@ -26,7 +26,9 @@
  *
  * Single-precision steps are single IEEE operations (compile with
  * -ffp-contract=off, no fast-math).  The sequence is, per block of 16 values v_i
- * with tensor scale s4 (FP32) and s8 = s4 * 2^ratio:
+ * with tensor scale s4 (FP32) and the FP8 tensor scale s8 (FP32): given on its own
+ * (Section 5.1: FP8 blocks have no microscale, only a per-tensor scale), or, when
+ * the argument is 0, tied to s4 as s8 = s4 * 2^ratio:
  *     amax = max |v_i|;  k6 = 1 / (6 * s4);  c0 = E4M3(amax * k6)     (dynamic max)
  *     d = e4m3val(c) * s4;  inv = 1 / d;  code_i = E2M1(v_i * inv);  dq4_i = e2m1val(code_i) * d
  *     inv8 = 1 / s8;  code8_i = E4M3(v_i * inv8);  dq8_i = e4m3val(code8_i) * s8
@@ -224,12 +226,12 @@ static void write_block(int fp8, const int *c4, const int *c8, int sc,
  *   scores [M*K/16] fp32 block scores
  * A block is FP8 iff score > tau (strict). */
 void oracle_quantize_activations(const uint16_t *X, int64_t ldx, const float *fisher,
-                                 int64_t M, int64_t K, float s4, int ratio, int mode, float tau,
+                                 int64_t M, int64_t K, float s4, int ratio, float s8_given, int mode, float tau,
                                  uint8_t *codes4, uint8_t *codes8, uint8_t *scales,
                                  uint32_t *mask, float *scores)
 {
     int64_t KB = K / BS, MW = (KB + 31) / 32;
-    float s8 = ldexpf(s4, ratio);
+    float s8 = s8_given > 0.0f ? s8_given : ldexpf(s4, ratio);
     init_tables();
     memset(mask, 0, (size_t)(M * MW) * 4);
     #pragma omp parallel for schedule(static)
@@ -267,7 +269,7 @@ static int cmp_scored(const void *a, const void *b)
  * smallest selected score; fp8_fraction < 0 -> FP8 iff score > tau.
  * Returns the tensor scale used. */
 float oracle_quantize_weights(const uint16_t *W, int64_t ldw, const float *fisher, int64_t ldf,
-                              int64_t N, int64_t K, float s4_in, int ratio, int mode, int clip,
+                              int64_t N, int64_t K, float s4_in, int ratio, float s8_given, int mode, int clip,
                               double fp8_fraction, float tau,
                               uint8_t *codes4, uint8_t *codes8, uint8_t *scales,
                               uint32_t *mask, float *scores, float *tau_eff)
@@ -284,7 +286,7 @@ float oracle_quantize_weights(const uint16_t *W, int64_t ldw, const float *fishe
             }
         s4 = amax / 2688.0f;
     }
-    float s8 = ldexpf(s4, ratio);
+    float s8 = s8_given > 0.0f ? s8_given : ldexpf(s4, ratio);
     uint8_t *sc_all = (uint8_t *)malloc((size_t)B);
     memset(mask, 0, (size_t)(N * MW) * 4);
 
@@ -348,9 +350,9 @@ static double decode_elem(const uint8_t *codes4, const uint8_t *codes8, const ui
 }
 
 void oracle_decode(const uint8_t *codes4, const uint8_t *codes8, const uint8_t *scales,
-                   const uint32_t *mask, int64_t rows, int64_t K, float s4, int ratio, double *out)
+                   const uint32_t *mask, int64_t rows, int64_t K, float s4, int ratio, float s8_given, double *out)
 {
-    double s8 = ldexp((double)s4, ratio);
+    double s8 = s8_given > 0.0f ? (double)s8_given : ldexp((double)s4, ratio);
     #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t k = 0; k < K; ++k)
@@ -379,12 +381,13 @@ void oracle_linear(const double *A, const double *Wd, int64_t M, int64_t N, int6
 /* the same sum for a list of output coordinates, decoding on the fly (full-size
  * configurations, sampled outputs) */
 void oracle_linear_sampled(const uint8_t *a4, const uint8_t *a8, const uint8_t *asc, const uint32_t *am,
-                           float a_s4, int a_ratio,
+                           float a_s4, int a_ratio, float a_s8_given,
                            const uint8_t *w4, const uint8_t *w8, const uint8_t *wsc, const uint32_t *wm,
-                           float w_s4, int w_ratio, int64_t K,
+                           float w_s4, int w_ratio, float w_s8_given, int64_t K,
                            int64_t nsamp, const int64_t *ms, const int64_t *ns, double *Y, double *S)
 {
-    double as8 = ldexp((double)a_s4, a_ratio), ws8 = ldexp((double)w_s4, w_ratio);
+    double as8 = a_s8_given > 0.0f ? (double)a_s8_given : ldexp((double)a_s4, a_ratio);
+    double ws8 = w_s8_given > 0.0f ? (double)w_s8_given : ldexp((double)w_s4, w_ratio);
     #pragma omp parallel for schedule(static)
     for (int64_t j = 0; j < nsamp; ++j) {
         double y = 0.0, s = 0.0;

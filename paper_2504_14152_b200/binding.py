@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libfgmp.so")
 
 SCORE_LP_ERROR, SCORE_HP_TO_LP = 0, 1
 CLIP_NONE, CLIP_SW_BRUTE = 0, 1
-OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU, OP_LINEAR_QUANTIZE, OP_LINEAR_FUSED = 0, 1, 2, 3, 4, 5, 6
+OP_QUANTIZE_WEIGHTS, OP_QUANTIZE_ACTIVATIONS, OP_LINEAR, OP_CALIBRATE_TAU, OP_GLOBAL_TAU, OP_LINEAR_QUANTIZE, OP_LINEAR_FUSED, OP_LINEAR_CLASSES = 0, 1, 2, 3, 4, 5, 6, 7
 
 
 class FgmpError(RuntimeError):
@@ -22,7 +22,7 @@ class FgmpError(RuntimeError):
 
 
 class _Scales(ctypes.Structure):
-    _fields_ = [("scale_fp4", ctypes.c_float), ("fp8_log2_ratio", ctypes.c_int)]
+    _fields_ = [("scale_fp4", ctypes.c_float), ("fp8_log2_ratio", ctypes.c_int), ("scale_fp8", ctypes.c_float)]
 
 
 _lib = None
@@ -56,6 +56,8 @@ def _load():
     L.fgmp_calibrate_tau.argtypes = [vp, i64, vp, i64, i64, _Scales, ci, f64, vp, vp, sz, vp]
     L.fgmp_linear.restype = ci
     L.fgmp_linear.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp]
+    L.fgmp_linear_classes.restype = ci
+    L.fgmp_linear_classes.argtypes = [vp, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp]
     L.fgmp_linear_fused.restype = ci
     L.fgmp_linear_fused.argtypes = [vp, i64, vp, _Scales, ci, f32, vp, vp, ci, i64, i64, i64, i64, vp, sz, vp, sz, vp]
     L.fgmp_linear_static.restype = ci
@@ -151,16 +153,17 @@ class PackedTensor:
     rows: int
     K: int
     kind: int               # 0 activations, 1 weights
+    fp8_free: bool = False  # packed with an FP8 tensor scale of its own (scale_fp8 > 0): multiplied by linear_classes
 
     def header(self) -> dict:
-        h = self.blob[:64].cpu().numpy().tobytes()
+        h = self.blob[:128].cpu().numpy().tobytes()
         import struct
-        magic, ver, rows, K, s4, ratio, n8, tau, kind, cap, err = struct.unpack("<IIqqfiqfIqi", h[:60])
+        magic, ver, rows, K, s4, ratio, n8, tau, kind, cap, err, s8, free = struct.unpack("<IIqqfiqfIqifi", h[:68])
         return dict(magic=magic, version=ver, rows=rows, K=K, scale_fp4=s4, fp8_log2_ratio=ratio, n_fp8=n8,
-                    tau_eff=tau, kind=kind, capacity=cap, error=err)
+                    tau_eff=tau, kind=kind, capacity=cap, error=err, scale_fp8=s8, fp8_scale_free=free)
 
 
-def quantize_weights(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float = 0.0, ratio: int = 3,
+def quantize_weights(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float = 0.0, ratio: int = 3, scale_fp8: float = 0.0,
                      score_mode: int = SCORE_LP_ERROR, clip_mode: int = CLIP_SW_BRUTE,
                      fp8_fraction: float = 0.1, tau: float = 0.0, max_fp8_blocks: int | None = None,
                      workspace: torch.Tensor | None = None, out: torch.Tensor | None = None) -> PackedTensor:
@@ -180,13 +183,13 @@ def quantize_weights(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float 
     if workspace is None:
         workspace = _alloc_aligned(ws_bytes, W.device)
     _ok(L.fgmp_quantize_weights(W.data_ptr(), W.stride(0), fisher.data_ptr(), fisher.stride(0), N, K,
-                                _Scales(scale_fp4, ratio), score_mode, clip_mode, float(fp8_fraction), tau,
+                                _Scales(scale_fp4, ratio, scale_fp8), score_mode, clip_mode, float(fp8_fraction), tau,
                                 out.data_ptr(), out.numel(), None, workspace.data_ptr(), workspace.numel(),
                                 _stream()), "fgmp_quantize_weights")
-    return PackedTensor(out, N, K, 1)
+    return PackedTensor(out, N, K, 1, scale_fp8 > 0)
 
 
-def quantize_activations(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ratio: int = 3,
+def quantize_activations(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ratio: int = 3, scale_fp8: float = 0.0,
                          score_mode: int = SCORE_LP_ERROR, tau: float,
                          out: torch.Tensor | None = None) -> PackedTensor:
     """X bf16 [M, K], fisher fp32 [K] -> packed activations."""
@@ -198,13 +201,13 @@ def quantize_activations(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: fl
         raise FgmpError(-2, "fgmp_acts_bytes")
     if out is None:
         out = _alloc_aligned(nbytes, X.device)
-    _ok(L.fgmp_quantize_activations(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio),
+    _ok(L.fgmp_quantize_activations(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio, scale_fp8),
                                     score_mode, tau, out.data_ptr(), out.numel(), None, 0, _stream()),
         "fgmp_quantize_activations")
-    return PackedTensor(out, M, K, 0)
+    return PackedTensor(out, M, K, 0, scale_fp8 > 0)
 
 
-def calibrate_tau(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ratio: int = 3,
+def calibrate_tau(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ratio: int = 3, scale_fp8: float = 0.0,
                   score_mode: int = SCORE_LP_ERROR, fp8_fraction: float,
                   workspace: torch.Tensor | None = None) -> torch.Tensor:
     """Returns a 1-element fp32 device tensor holding the threshold for this batch."""
@@ -214,7 +217,7 @@ def calibrate_tau(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ra
     ws_bytes = L.fgmp_workspace_bytes(OP_CALIBRATE_TAU, M, 0, K)
     if workspace is None:
         workspace = _alloc_aligned(ws_bytes, X.device)
-    _ok(L.fgmp_calibrate_tau(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio),
+    _ok(L.fgmp_calibrate_tau(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio, scale_fp8),
                              score_mode, float(fp8_fraction), tau.data_ptr(), workspace.data_ptr(),
                              workspace.numel(), _stream()), "fgmp_calibrate_tau")
     return tau
@@ -230,7 +233,7 @@ def channel_mean_sq(X: torch.Tensor) -> torch.Tensor:
     return out
 
 
-def weight_scores(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float = 0.0, ratio: int = 3,
+def weight_scores(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float = 0.0, ratio: int = 3, scale_fp8: float = 0.0,
                   score_mode: int = SCORE_LP_ERROR, clip_mode: int = CLIP_SW_BRUTE) -> torch.Tensor:
     """Block scores [N, K/16] of a weight tensor, as fgmp_quantize_weights ranks them."""
     L = _load()
@@ -238,7 +241,7 @@ def weight_scores(W: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float = 0
     scores = torch.empty(N, K // 16, dtype=torch.float32, device=W.device)
     workspace = _alloc_aligned(L.fgmp_workspace_bytes(OP_QUANTIZE_WEIGHTS, 0, N, K), W.device)
     _ok(L.fgmp_weight_scores(W.data_ptr(), W.stride(0), fisher.data_ptr(), fisher.stride(0), N, K,
-                             _Scales(scale_fp4, ratio), score_mode, clip_mode, scores.data_ptr(),
+                             _Scales(scale_fp4, ratio, scale_fp8), score_mode, clip_mode, scores.data_ptr(),
                              workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_weight_scores")
     return scores
 
@@ -260,21 +263,24 @@ def global_tau(score_tensors, fp8_fraction: float) -> torch.Tensor:
     return tau
 
 
-def activation_scores(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ratio: int = 3,
+def activation_scores(X: torch.Tensor, fisher: torch.Tensor, *, scale_fp4: float, ratio: int = 3, scale_fp8: float = 0.0,
                       score_mode: int = SCORE_LP_ERROR) -> torch.Tensor:
     L = _load()
     M, K = X.shape
     scores = torch.empty(M, K // 16, dtype=torch.float32, device=X.device)
-    _ok(L.fgmp_activation_scores(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio),
+    _ok(L.fgmp_activation_scores(X.data_ptr(), X.stride(0), fisher.data_ptr(), M, K, _Scales(scale_fp4, ratio, scale_fp8),
                                  score_mode, scores.data_ptr(), _stream()), "fgmp_activation_scores")
     return scores
 
 
 def linear(acts: PackedTensor, weights: PackedTensor, *, out_dtype=torch.float32,
            out: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
-    """Y [M, N] = acts x weights^T (FP32 accumulation)."""
+    """Y [M, N] = acts x weights^T (FP32 accumulation).  Operands packed with an FP8 tensor scale of their
+    own go through linear_classes (one accumulation per class of block pair, fp32 output)."""
     L = _load()
     assert acts.K == weights.K and acts.kind == 0 and weights.kind == 1
+    if acts.fp8_free or weights.fp8_free:
+        return linear_classes(acts, weights, out=out, workspace=workspace)
     M, N, K = acts.rows, weights.rows, acts.K
     if out is None:
         out = torch.empty(M, N, dtype=out_dtype, device=acts.blob.device)
@@ -284,6 +290,24 @@ def linear(acts: PackedTensor, weights: PackedTensor, *, out_dtype=torch.float32
     _ok(L.fgmp_linear(acts.blob.data_ptr(), weights.blob.data_ptr(), out.data_ptr(),
                       1 if out.dtype == torch.bfloat16 else 0, out.stride(0), M, N, K,
                       workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear")
+    linear.last_workspace = workspace
+    return out
+
+
+def linear_classes(acts: PackedTensor, weights: PackedTensor, *, out: torch.Tensor | None = None,
+                   workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """Y fp32 [M, N] with the four classes of block pair accumulated separately, each under its own pair of
+    tensor scales: the GEMM for operands whose FP8 scale is not a power of two times the NVFP4 scale."""
+    L = _load()
+    assert acts.K == weights.K and acts.kind == 0 and weights.kind == 1
+    M, N, K = acts.rows, weights.rows, acts.K
+    if out is None:
+        out = torch.empty(M, N, dtype=torch.float32, device=acts.blob.device)
+    assert out.dtype == torch.float32
+    if workspace is None:
+        workspace = alloc_workspace(OP_LINEAR_CLASSES, M, N, K, acts.blob.device)
+    _ok(L.fgmp_linear_classes(acts.blob.data_ptr(), weights.blob.data_ptr(), out.data_ptr(), 0, out.stride(0), M, N, K,
+                              workspace.data_ptr(), workspace.numel(), _stream()), "fgmp_linear_classes")
     linear.last_workspace = workspace
     return out
 

@@ -269,7 +269,7 @@ decode_kernel(DecParams p)
         if (lane == 0) {
             const uint2 mv = __ldg(reinterpret_cast<const uint2*>(hw));
             okh = mv.x == FGMP_MAGIC && mv.y == 7u && __ldg(&hw->rows) == p.N && __ldg(&hw->K) == p.K &&
-                  __ldg(&hw->kind) == 1u && __ldg(&hw->error) == 0;
+                  __ldg(&hw->kind) == 1u && __ldg(&hw->error) == 0 && __ldg(&hw->fp8_scale_free) == 0;
             if (!okh) { *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 9); }
         }
         okh = __shfl_sync(0xffffffffu, okh, 0);
@@ -318,7 +318,7 @@ decode_kernel(DecParams p)
                 fgmp_packed_header* h = p.q_header;
                 h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.q.s4;
                 h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = (p.q.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
-                h->error = 0;
+                h->error = 0; h->scale_fp8 = p.q.s8; h->fp8_scale_free = 0;
             }
             if (p.q_mode == 0) quantize_chunk<0>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
             else               quantize_chunk<1>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
@@ -342,7 +342,7 @@ decode_kernel(DecParams p)
             } else {
                 const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
                 const uint2 mv = __ldg(reinterpret_cast<const uint2*>(ha));
-                if (!(mv.x == FGMP_MAGIC && mv.y == 7u && __ldg(&ha->rows) == p.M && __ldg(&ha->K) == p.K && __ldg(&ha->kind) == 0u)) {
+                if (!(mv.x == FGMP_MAGIC && mv.y == 7u && __ldg(&ha->rows) == p.M && __ldg(&ha->K) == p.K && __ldg(&ha->kind) == 0u && __ldg(&ha->fp8_scale_free) == 0)) {
                     *abort_flag = 1; atomicCAS(p.status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(p.status + 1, 10);
                     ok = 0;
                 }
@@ -895,7 +895,7 @@ extern "C" fgmp_status fgmp_linear_fused(const void* X_bf16, int64_t ldx, const 
     if (!X_bf16 || !fisher_chan || !packed_weights || !Y || !workspace) return FGMP_ERR_INVALID_ARG;
     if ((int)sm < 0 || (int)sm > 1 || tau != tau) return FGMP_ERR_INVALID_ARG;
     if (!(sc.scale_fp4 > 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    if (!fgmp_scales_valid(sc) || fgmp_fp8_free(sc)) return FGMP_ERR_INVALID_ARG;   // a free FP8 scale: the two calls and fgmp_linear_classes
     if (M < 1 || N < 1 || K < 64 || (K % 64) != 0 || ldy < N || ldx < K || (ldx % 8) != 0) return FGMP_ERR_SHAPE;
     if (((uintptr_t)X_bf16 & 15) || ((uintptr_t)fisher_chan & 15) || ((uintptr_t)packed_weights & 1023) ||
         ((uintptr_t)workspace & 1023) || ((uintptr_t)Y & 15) || ((uintptr_t)packed_acts_out & 1023)) return FGMP_ERR_SHAPE;

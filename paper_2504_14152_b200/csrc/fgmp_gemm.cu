@@ -16,6 +16,7 @@
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
+#include <mutex>
 
 namespace {
 
@@ -55,22 +56,25 @@ __device__ __forceinline__ void nvfp4x16_scaled(const uint2& c, uint32_t scale_c
 
 // A packed tensor is read only if its header describes the tensor the call was given; otherwise the
 // status word of the workspace says so and the kernel leaves.
-__device__ __forceinline__ bool header_matches(const fgmp_packed_header* h, int64_t rows, int64_t K, uint32_t kind, int* status, int where)
+// cls: 0 = every block on the NVFP4 tensor scale (needs the power-of-two tie of the two scales), 1 / 2 = only the
+// NVFP4 / only the FP8 blocks, each over its own tensor scale (the per-class passes of fgmp_linear_classes)
+__device__ __forceinline__ bool header_matches(const fgmp_packed_header* h, int64_t rows, int64_t K, uint32_t kind, int* status, int where, int cls = 0)
 {
-    const bool ok = h->magic == FGMP_MAGIC && h->version == 7u && h->rows == rows && h->K == K && h->kind == kind && h->error == 0;
+    const bool ok = h->magic == FGMP_MAGIC && h->version == 7u && h->rows == rows && h->K == K && h->kind == kind && h->error == 0 &&
+                    (cls != 0 || h->fp8_scale_free == 0);
     if (!ok && threadIdx.x == 0) { atomicCAS(status, 0, (int)FGMP_ERR_INVALID_ARG); atomicExch(status + 1, where); }
     return ok;
 }
 
 // packed activations -> bf16 plane; one thread per block
-__global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane, int* status)
+__global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_t rows, int64_t K, uint4* plane, int* status, int cls)
 {
     if (status[2]) return;                              // the all-NVFP4 GEMM has produced the result already
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
-    if (!header_matches(h, rows, K, 0u, status, 11)) return;
+    if (!header_matches(h, rows, K, 0u, status, 11, cls)) return;
     const PackedLayout L = fgmp_layout(rows, K, 0, 0);
     const uint32_t* pmask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
-    const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
+    const float r8 = cls ? 1.0f : __int_as_float((127 + h->fp8_log2_ratio) << 23);
     const int64_t nblk = rows * L.KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
         int64_t r = b / L.KB, kb = b % L.KB;
@@ -80,20 +84,24 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint8_t* blob, int64_
         if (is8) e4m3x16_scaled(*reinterpret_cast<const uint4*>(blob + L.off_codes8 + (size_t)(r * K + kb * 16)), r8, v);
         else nvfp4x16_scaled(*reinterpret_cast<const uint2*>(blob + L.off_codes4 + (r * K) / 2 + kb * 8),
                              blob[L.off_sf + fgmp_sf_offset(r, kb, K)], v);
+        if (cls && (is8 != (cls == 2))) {               // a block of the other class
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
         store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
     }
 }
 
 // packed weights -> bf16 plane; one CTA of 128 threads per unit record, consecutive threads on
 // consecutive blocks of one row, four blocks per thread in flight at a time
-__global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* __restrict__ blob, int64_t rows, int64_t K, uint4* __restrict__ plane, int* status)
+__global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* __restrict__ blob, int64_t rows, int64_t K, uint4* __restrict__ plane, int* status, int cls)
 {
     __shared__ UnitScratch sc;
     if (status[2]) return;                              // the all-NVFP4 GEMM has produced the result already
     const fgmp_packed_header* h = reinterpret_cast<const fgmp_packed_header*>(blob);
-    if (!header_matches(h, rows, K, 1u, status, 12)) return;
+    if (!header_matches(h, rows, K, 1u, status, 12, cls)) return;
     const PackedLayout L = fgmp_layout(rows, K, 1, 0);
-    const float r8 = __int_as_float((127 + h->fp8_log2_ratio) << 23);
+    const float r8 = cls ? 1.0f : __int_as_float((127 + h->fp8_log2_ratio) << 23);
     const int64_t unit = blockIdx.x, tile = unit / L.chunks, c = unit % L.chunks;
     const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
     const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
@@ -124,6 +132,10 @@ __global__ void __launch_bounds__(128) expand_w_kernel(const uint8_t* __restrict
             float v[16];
             if (pos[i] != 0xffffu) e4m3x16_scaled(make_uint4(slot[i].x, slot[i].y, hi[i].x, hi[i].y), r8, v);
             else nvfp4x16_scaled(slot[i], sfb[i], v);
+            if (cls && ((pos[i] != 0xffffu) != (cls == 2))) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0.f;
+            }
             store_bf16x16(plane + (r * K) / 8 + kb * 2, v);
         }
     }
@@ -167,7 +179,7 @@ __device__ __forceinline__ void pair_tile_coords(int64_t t, int64_t tiles_m, int
 struct QuantNext {
     const float* fisher;                 // [N] per-channel sensitivity of the next layer's input
     float s4, k6, s8, inv8, tau;
-    int mode, ratio;
+    int mode, ratio, free8;
     uint8_t* codes4; uint8_t* sf; uint32_t* mask; uint8_t* codes8;
     fgmp_packed_header* header;
     int64_t MW;                          // mask words per output row
@@ -179,6 +191,8 @@ struct GemmParams {
     const fgmp_packed_header* ha; const fgmp_packed_header* hw;
     int* status;
     QuantNext q;
+    int cls_a, cls_w;       // 0, or the class of each operand's plane (1 = NVFP4 blocks, 2 = FP8 blocks): picks the tensor scales
+    int accumulate;         // add to Y (fp32) instead of storing
 };
 
 // One row of 32 accumulator columns = two blocks of the next layer's activations: round to bf16 (what an
@@ -252,7 +266,10 @@ __device__ __forceinline__ void store_chunk32(const GemmParams& p, int64_t row, 
         }
     } else {
         float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
-        if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
+        if (p.accumulate) {
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) y[j] = __fadd_rn(y[j], __fmul_rn(__uint_as_float(r[j]), alpha));
+        } else if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
                 *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
@@ -297,7 +314,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         fgmp_packed_header* h = p.q.header;
         h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.N; h->scale_fp4 = p.q.s4;
         h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = (p.q.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
-        h->error = 0;
+        h->error = 0; h->scale_fp8 = p.q.s8; h->fp8_scale_free = p.q.free8;
     }
     const int64_t tiles_m = (p.M + P_BM - 1) / P_BM, tiles_n = (p.N + P_BN - 1) / P_BN;
     const int64_t num_tiles = tiles_m * tiles_n;
@@ -349,7 +366,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
     } else {
         const int q = warp & 3;                        // TMEM lane quadrant this warp may read
-        const float alpha = __fmul_rn(p.ha->scale_fp4, p.hw->scale_fp4);
+        const float alpha = __fmul_rn(p.cls_a == 2 ? p.ha->scale_fp8 : p.ha->scale_fp4, p.cls_w == 2 ? p.hw->scale_fp8 : p.hw->scale_fp4);
         bool ok = true;
         int64_t it = 0;
         for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++it) {
@@ -438,20 +455,15 @@ size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K)
     return (size_t)FGMP_WS_CONTROL_BYTES + fgmp_align1k((size_t)M * K * 2) + fgmp_align1k((size_t)N * K * 2);
 }
 
-// expand both operands and run the pair GEMM (M > 16 or a shape the weight-streaming kernel does not take)
-static fgmp_status launch_prefill(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
-                                  int64_t M, int64_t N, int64_t K, void* workspace, const QuantNext& qn, cudaStream_t s)
+// CTA pairs that can be resident at once on this device (a pair needs two SMs of one cluster domain)
+static fgmp_status resident_pairs(int* pairs)
 {
-    uint8_t* ws = (uint8_t*)workspace;
-    int* status = reinterpret_cast<int*>(ws);
-    uint8_t* planeA = ws + FGMP_WS_CONTROL_BYTES;       // the control area stays as the decode-sized calls need it
-    uint8_t* planeW = planeA + fgmp_align1k((size_t)M * K * 2);
-
-    // CTA pairs that can be resident at once on this device (a pair needs two SMs of one cluster domain)
+    static std::mutex mu;
     static int pairs_of_device[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(mu);
     if (!pairs_of_device[dev]) {
         if (cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PAIR_SMEM) != cudaSuccess)
             return FGMP_ERR_CUDA;
@@ -461,6 +473,22 @@ static fgmp_status launch_prefill(const void* packed_acts, const void* packed_we
         if (cudaOccupancyMaxActiveClusters(&n, gemm_bf16_pair_kernel, &qc) != cudaSuccess || n < 1) return FGMP_ERR_CUDA;
         pairs_of_device[dev] = n;
     }
+    *pairs = pairs_of_device[dev];
+    return FGMP_OK;
+}
+
+// expand both operands and run the pair GEMM (M > 16 or a shape the weight-streaming kernel does not take)
+static fgmp_status launch_prefill(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
+                                  int64_t M, int64_t N, int64_t K, void* workspace, const QuantNext& qn, cudaStream_t s)
+{
+    uint8_t* ws = (uint8_t*)workspace;
+    int* status = reinterpret_cast<int*>(ws);
+    uint8_t* planeA = ws + FGMP_WS_CONTROL_BYTES;       // the control area stays as the decode-sized calls need it
+    uint8_t* planeW = planeA + fgmp_align1k((size_t)M * K * 2);
+
+    int pairs_avail = 0;
+    fgmp_status stp = resident_pairs(&pairs_avail);
+    if (stp != FGMP_OK) return stp;
     CUtensorMap tmA, tmB;
     if (!make_tmap_bf16(&tmA, planeA, M, K, 128) || !make_tmap_bf16(&tmB, planeW, N, K, 128)) return FGMP_ERR_CUDA;
 
@@ -477,9 +505,9 @@ static fgmp_status launch_prefill(const void* packed_acts, const void* packed_we
     {
         const int64_t nb = M * (K / 16);
         const int g = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
-        FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, reinterpret_cast<uint4*>(planeA), status));
+        FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<g, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, reinterpret_cast<uint4*>(planeA), status, 0));
         const PackedLayout LW = fgmp_layout(N, K, 1, 0);
-        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_w_kernel<<<(unsigned)LW.units, 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW), status));
+        FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_w_kernel<<<(unsigned)LW.units, 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW), status, 0));
     }
     GemmParams p;
     p.Y = Y; p.ldy = ldy; p.y_is_bf16 = y_is_bf16; p.M = M; p.N = N; p.K = K;
@@ -487,8 +515,9 @@ static fgmp_status launch_prefill(const void* packed_acts, const void* packed_we
     p.hw = reinterpret_cast<const fgmp_packed_header*>(packed_weights);
     p.status = status;
     p.q = qn;
+    p.cls_a = 0; p.cls_w = 0; p.accumulate = 0;
     const int64_t tiles = ((M + P_BM - 1) / P_BM) * ((N + P_BN - 1) / P_BN);
-    const int pairs = (int)(tiles < pairs_of_device[dev] ? tiles : pairs_of_device[dev]);
+    const int pairs = (int)(tiles < pairs_avail ? tiles : pairs_avail);
     FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_pair_kernel<<<2 * pairs, GEMM_THREADS, PAIR_SMEM, s>>>(tmA, tmB, p));
     return fgmp_launch_status();
 }
@@ -511,6 +540,66 @@ extern "C" fgmp_status fgmp_linear(const void* packed_acts, const void* packed_w
     return launch_prefill(packed_acts, packed_weights, Y, y_is_bf16, ldy, M, N, K, workspace, off, s);
 }
 
+size_t fgmp_ws_linear_classes(int64_t M, int64_t N, int64_t K)
+{
+    return (size_t)FGMP_WS_CONTROL_BYTES + fgmp_align1k((size_t)M * K * 2) + fgmp_align1k((size_t)N * K * 2);
+}
+
+// One accumulation per class of block pair: FP4 x FP4, FP4 x FP8, FP8 x FP8, FP8 x FP4, each a pass of the pair
+// GEMM over planes that hold the blocks of one format (over their own tensor scale) and zeros elsewhere; the
+// epilogue multiplies by the two scales of the pass and adds to Y.
+extern "C" fgmp_status fgmp_linear_classes(const void* packed_acts, const void* packed_weights,
+                                           void* Y, int y_is_bf16, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                           void* workspace, size_t ws_bytes, void* cuda_stream)
+{
+    if (!packed_acts || !packed_weights || !Y || !workspace || y_is_bf16) return FGMP_ERR_INVALID_ARG;
+    if (M < 1 || N < 1 || K < 64 || (K % 64) != 0 || ldy < N) return FGMP_ERR_SHAPE;
+    if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
+        ((uintptr_t)Y & 15)) return FGMP_ERR_SHAPE;
+    if (ws_bytes < fgmp_ws_linear_classes(M, N, K)) return FGMP_ERR_WORKSPACE;
+    fgmp_status st;
+    if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    int* status = reinterpret_cast<int*>(ws);
+    uint8_t* planeA = ws + FGMP_WS_CONTROL_BYTES;
+    uint8_t* planeW = planeA + fgmp_align1k((size_t)M * K * 2);
+    int pairs_avail = 0;
+    if ((st = resident_pairs(&pairs_avail)) != FGMP_OK) return st;
+    CUtensorMap tmA, tmB;
+    if (!make_tmap_bf16(&tmA, planeA, M, K, 128) || !make_tmap_bf16(&tmB, planeW, N, K, 128)) return FGMP_ERR_CUDA;
+    if (cudaMemsetAsync(status, 0, 256, s) != cudaSuccess) return FGMP_ERR_CUDA;
+    const int sms = fgmp_sm_count();
+    const int64_t nb = M * (K / 16);
+    const int ga = (int)((nb + 255) / 256 < (int64_t)sms * 8 ? (nb + 255) / 256 : (int64_t)sms * 8);
+    const PackedLayout LW = fgmp_layout(N, K, 1, 0);
+    GemmParams p;
+    p.Y = Y; p.ldy = ldy; p.y_is_bf16 = 0; p.M = M; p.N = N; p.K = K;
+    p.ha = reinterpret_cast<const fgmp_packed_header*>(packed_acts);
+    p.hw = reinterpret_cast<const fgmp_packed_header*>(packed_weights);
+    p.status = status;
+    p.q = QuantNext{};
+    const int64_t tiles = ((M + P_BM - 1) / P_BM) * ((N + P_BN - 1) / P_BN);
+    const int pairs = (int)(tiles < pairs_avail ? tiles : pairs_avail);
+    // (activation class, weight class) in an order that re-expands one operand per pass
+    const int order[4][2] = {{1, 1}, {1, 2}, {2, 2}, {2, 1}};
+    int have_a = 0, have_w = 0;
+    for (int i = 0; i < 4; ++i) {
+        const int ca = order[i][0], cw = order[i][1];
+        if (ca != have_a) {
+            FGMP_LAUNCH(FGMP_K_EXPAND_A, s, expand_kernel<<<ga, 256, 0, s>>>((const uint8_t*)packed_acts, M, K, reinterpret_cast<uint4*>(planeA), status, ca));
+            have_a = ca;
+        }
+        if (cw != have_w) {
+            FGMP_LAUNCH(FGMP_K_EXPAND_W, s, expand_w_kernel<<<(unsigned)LW.units, 128, 0, s>>>((const uint8_t*)packed_weights, N, K, reinterpret_cast<uint4*>(planeW), status, cw));
+            have_w = cw;
+        }
+        p.cls_a = ca; p.cls_w = cw; p.accumulate = i > 0;
+        FGMP_LAUNCH(FGMP_K_GEMM_BF16, s, gemm_bf16_pair_kernel<<<2 * pairs, GEMM_THREADS, PAIR_SMEM, s>>>(tmA, tmB, p));
+    }
+    return fgmp_launch_status();
+}
+
 extern "C" fgmp_status fgmp_linear_quantize(const void* packed_acts, const void* packed_weights,
                                             int64_t M, int64_t N, int64_t K,
                                             const float* fisher_chan_next, fgmp_scales sc_next, fgmp_score_mode sm,
@@ -520,7 +609,7 @@ extern "C" fgmp_status fgmp_linear_quantize(const void* packed_acts, const void*
     if (!packed_acts || !packed_weights || !fisher_chan_next || !packed_out || !workspace) return FGMP_ERR_INVALID_ARG;
     if ((int)sm < 0 || (int)sm > 1 || tau_next != tau_next) return FGMP_ERR_INVALID_ARG;
     if (!(sc_next.scale_fp4 > 0.f) || !isfinite(sc_next.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc_next.fp8_log2_ratio < -7 || sc_next.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    if (!fgmp_scales_valid(sc_next)) return FGMP_ERR_INVALID_ARG;
     // the output is a packed activation tensor [M, N]: N is the next layer's K
     if (M < 1 || N < 64 || (N % 64) != 0 || K < 64 || (K % 64) != 0) return FGMP_ERR_SHAPE;
     if (((uintptr_t)packed_acts & 1023) || ((uintptr_t)packed_weights & 1023) || ((uintptr_t)workspace & 1023) ||
@@ -545,7 +634,7 @@ extern "C" fgmp_status fgmp_linear_quantize(const void* packed_acts, const void*
     // the same scalars, computed the same way, as fgmp_quantize_activations uses
     q.s4 = sc_next.scale_fp4;
     q.k6 = 1.0f / (6.0f * sc_next.scale_fp4);
-    q.s8 = ldexpf(sc_next.scale_fp4, sc_next.fp8_log2_ratio);
+    q.s8 = fgmp_fp8_scale(sc_next); q.free8 = fgmp_fp8_free(sc_next) ? 1 : 0;
     q.inv8 = 1.0f / q.s8;
     q.tau = tau_next; q.mode = (int)sm; q.ratio = sc_next.fp8_log2_ratio;
     q.codes4 = blob + L.off_codes4; q.sf = blob + L.off_sf;
@@ -584,6 +673,7 @@ extern "C" size_t fgmp_workspace_bytes(int op, int64_t M, int64_t N, int64_t K)
         case FGMP_OP_CALIBRATE_TAU: return M >= 1 ? fgmp_ws_calibrate(M, K) : 0;
         case FGMP_OP_LINEAR_QUANTIZE: return (M >= 1 && N >= 1) ? fgmp_ws_linear_quantize(M, N, K) : 0;
         case FGMP_OP_LINEAR_FUSED: return (M >= 1 && N >= 1) ? fgmp_ws_linear_fused(M, N, K) : 0;
+        case FGMP_OP_LINEAR_CLASSES: return (M >= 1 && N >= 1) ? fgmp_ws_linear_classes(M, N, K) : 0;
     }
     return 0;
 }

@@ -15,6 +15,7 @@ size_t fgmp_ws_calibrate(int64_t M, int64_t K);
 size_t fgmp_ws_linear(int64_t M, int64_t N, int64_t K);
 size_t fgmp_ws_linear_quantize(int64_t M, int64_t N, int64_t K);
 size_t fgmp_ws_linear_fused(int64_t M, int64_t N, int64_t K);
+size_t fgmp_ws_linear_classes(int64_t M, int64_t N, int64_t K);
 size_t fgmp_ws_global_tau(int64_t total_scores);
 // weight-streaming kernel for M <= 16 tokens and K % 256 == 0
 bool fgmp_decode_supported(int64_t M, int64_t N, int64_t K);
@@ -25,6 +26,15 @@ fgmp_status fgmp_linear_decode(const void* packed_acts, const void* packed_weigh
 // all-NVFP4 prefill GEMM (fgmp_gemm4.cu): decides on the device whether it applies, answer in status[2]
 fgmp_status fgmp_launch_gemm_nvfp4(const void* packed_acts, const void* packed_weights, void* Y, int y_is_bf16, int64_t ldy,
                                    int64_t M, int64_t N, int64_t K, int* status, cudaStream_t s);
+
+// ---- the FP8 tensor scale of a call (fgmp_scales): given on its own, or scale_fp4 * 2^ratio ----
+#include <math.h>
+inline bool fgmp_scales_valid(const fgmp_scales& sc)
+{
+    return sc.fp8_log2_ratio >= -7 && sc.fp8_log2_ratio <= 7 && sc.scale_fp8 >= 0.f && isfinite(sc.scale_fp8);
+}
+inline bool fgmp_fp8_free(const fgmp_scales& sc) { return sc.scale_fp8 > 0.f; }
+inline float fgmp_fp8_scale(const fgmp_scales& sc) { return sc.scale_fp8 > 0.f ? sc.scale_fp8 : ldexpf(sc.scale_fp4, sc.fp8_log2_ratio); }
 
 // ---- launch accounting (see fgmp_profile_begin in fgmp.h) ----
 enum FgmpKernelId {

@@ -23,6 +23,7 @@ struct ActParams {
     fgmp_packed_header* header;
     float r8;                            // 2^ratio
     int ratio;
+    int free8;                           // the FP8 tensor scale was given on its own
     int rows_per_cta;
 };
 
@@ -41,7 +42,7 @@ __global__ void __launch_bounds__(QA_THREADS) quant_act_kernel(ActParams p)
             fgmp_packed_header* h = p.header;
             h->magic = FGMP_MAGIC; h->version = 7; h->rows = p.M; h->K = p.K; h->scale_fp4 = p.s4;
             h->fp8_log2_ratio = p.ratio; h->n_fp8 = (p.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
-            h->error = 0;
+            h->error = 0; h->scale_fp8 = p.s8; h->fp8_scale_free = p.free8;
         }
         // token rows M..15 of the decode records are zero (the grid covers 16 rows in that mode)
         if (p.arec && m0 >= p.M) {
@@ -211,7 +212,7 @@ fgmp_status check_act_args(const void* X, int64_t ldx, const float* fisher, int6
     if (!X || !fisher) return FGMP_ERR_INVALID_ARG;
     if (sm != 0 && sm != 1) return FGMP_ERR_INVALID_ARG;
     if (!(sc.scale_fp4 > 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    if (!fgmp_scales_valid(sc)) return FGMP_ERR_INVALID_ARG;
     if (M < 1 || K < 64 || (K % 64) != 0 || ldx < K || (ldx % 8) != 0) return FGMP_ERR_SHAPE;
     if (((uintptr_t)X & 15) || ((uintptr_t)fisher & 15)) return FGMP_ERR_SHAPE;
     return FGMP_OK;
@@ -224,8 +225,9 @@ ActParams make_act_params(const void* X, int64_t ldx, const float* fisher, int64
     p.M = M; p.K = K; p.KB = K / 16; p.MW = (p.KB + 31) / 32;
     p.s4 = sc.scale_fp4;
     p.k6 = 1.0f / (6.0f * sc.scale_fp4);
-    p.s8 = ldexpf(sc.scale_fp4, sc.fp8_log2_ratio);
+    p.s8 = fgmp_fp8_scale(sc);
     p.inv8 = 1.0f / p.s8;
+    p.free8 = fgmp_fp8_free(sc) ? 1 : 0;
     p.tau = tau;
     p.ratio = sc.fp8_log2_ratio;
     p.r8 = ldexpf(1.0f, sc.fp8_log2_ratio);
@@ -257,7 +259,7 @@ extern "C" fgmp_status fgmp_quantize_activations(const void* X_bf16, int64_t ldx
     p.mask = reinterpret_cast<uint32_t*>(blob + L.off_mask); p.codes8 = blob + L.off_codes8;
     p.header = reinterpret_cast<fgmp_packed_header*>(blob);
     int64_t grid_rows = M;
-    if (M <= 16) {                     // decode-sized batch: also emit the records of the decode GEMM, 16 token rows
+    if (M <= 16 && !p.free8) {         // decode-sized batch: also emit the records of the decode GEMM, 16 token rows (tied scales only)
         p.arec = blob + L.off_arec;
         p.rows_per_cta = 1;
         grid_rows = 16;

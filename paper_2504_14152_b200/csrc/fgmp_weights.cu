@@ -76,7 +76,7 @@ __device__ __forceinline__ void load_block(const uint4* W, int64_t ldw8, const f
 // per block: microscale (dynamic max or Eq. 11 brute force) and the score under it
 template <int MODE, bool CLIP>
 __global__ void __launch_bounds__(256) w_score_kernel(const uint4* W, int64_t ldw8, const float* F, int64_t ldf,
-                                                      int64_t N, int64_t KB, int ratio, const SelectState* st,
+                                                      int64_t N, int64_t KB, int ratio, float s8_given, const SelectState* st,
                                                       uint8_t* sc_out, float* scores)
 {
     __shared__ float s_d[128], s_inv[128];
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(256) w_score_kernel(const uint4* W, int64_t ld
         __syncthreads();
     }
     const float k6 = __fdiv_rn(1.0f, __fmul_rn(6.0f, s4));
-    const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
+    const float s8 = s8_given > 0.f ? s8_given : __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
     const float inv8 = __fdiv_rn(1.0f, s8);
     const int64_t B = N * KB;
     for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
@@ -301,7 +301,7 @@ __global__ void __launch_bounds__(128) w_unit_count_kernel(const uint32_t* mask,
 // Writes the record of one unit (codes and microscales of its NVFP4 blocks, the first halves of its FP8
 // blocks, the per-column running counts) and the list of its FP8 blocks (rows, second halves).  One CTA
 // of 128 threads per unit.
-__global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw8, int ratio, const SelectState* st,
+__global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw8, int ratio, float s8_given, const SelectState* st,
                                                      const uint8_t* sc_in, uint8_t* blob, PackedLayout L, int64_t room_steps)
 {
     __shared__ UnitScratch sc;
@@ -309,7 +309,7 @@ __global__ void __launch_bounds__(128) w_emit_kernel(const uint4* W, int64_t ldw
     const uint32_t* uptr = reinterpret_cast<const uint32_t*>(blob + L.off_uptr);
     const bool fits = (int64_t)uptr[unit + 1] <= room_steps;   // else the blob is too small: header.error says so
     const float s4 = st->s4;
-    const float s8 = __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
+    const float s8 = s8_given > 0.f ? s8_given : __fmul_rn(s4, __int_as_float((127 + ratio) << 23));
     const float inv8 = __fdiv_rn(1.0f, s8);
     const uint32_t* mask = reinterpret_cast<const uint32_t*>(blob + L.off_mask);
     const uint32_t m16 = fgmp_chunk_mask(mask, L, tile * 128 + threadIdx.x, c);
@@ -370,7 +370,7 @@ __global__ void w_clamp_uptr_kernel(const fgmp_packed_header* h, uint32_t* uptr,
 }
 
 __global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, const uint32_t* uptr, int64_t units,
-                                int64_t N, int64_t K, int ratio, int64_t room_steps, int fraction_mode, float tau_given,
+                                int64_t N, int64_t K, int ratio, float s8_given, int64_t room_steps, int fraction_mode, float tau_given,
                                 float* tau_eff_out)
 {
     if (threadIdx.x == 0) {
@@ -379,6 +379,8 @@ __global__ void w_header_kernel(fgmp_packed_header* h, const SelectState* st, co
         float teff = fraction_mode ? st->tau : tau_given;
         h->tau_eff = teff;
         h->error = ((int64_t)uptr[units] > room_steps) ? (int32_t)FGMP_ERR_CAPACITY : 0;
+        h->scale_fp8 = s8_given > 0.f ? s8_given : __fmul_rn(st->s4, __int_as_float((127 + ratio) << 23));
+        h->fp8_scale_free = s8_given > 0.f ? 1 : 0;
         if (tau_eff_out) *tau_eff_out = teff;
     }
 }
@@ -435,7 +437,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     if (!W_bf16 || !fisher_elem || !packed_out || !workspace) return FGMP_ERR_INVALID_ARG;
     if ((int)sm < 0 || (int)sm > 1 || (int)cm < 0 || (int)cm > 1) return FGMP_ERR_INVALID_ARG;
     if (!(sc.scale_fp4 >= 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    if (!fgmp_scales_valid(sc)) return FGMP_ERR_INVALID_ARG;
     if (fp8_fraction != fp8_fraction || fp8_fraction > 1.0) return FGMP_ERR_INVALID_ARG;
     if (fp8_fraction < 0 && tau != tau) return FGMP_ERR_INVALID_ARG;
     if (N < 1 || K < 64 || (K % 64) != 0 || ldw < K || (ldw % 8) != 0 || ldf < K || (ldf % 4) != 0) return FGMP_ERR_SHAPE;
@@ -468,6 +470,7 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     uint8_t* blob = (uint8_t*)packed_out;
     const uint4* W = reinterpret_cast<const uint4*>(W_bf16);
     const int ratio = sc.fp8_log2_ratio;
+    const float s8_given = sc.scale_fp8;
 
     FGMP_LAUNCH(FGMP_K_W_AUX, s, state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, (unsigned long long)k));
     if (sc.scale_fp4 == 0.f) {
@@ -477,11 +480,11 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     {
         int g = grid_for(B, 256, 4);
         if (sm == FGMP_SCORE_LP_ERROR) {
-            if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
-            else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+            if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
+            else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
         } else {
-            if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
-            else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+            if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
+            else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
         }
     }
     uint32_t* mask = reinterpret_cast<uint32_t*>(blob + L.off_mask);
@@ -499,8 +502,8 @@ extern "C" fgmp_status fgmp_quantize_weights(const void* W_bf16, int64_t ldw, co
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_mask_kernel<<<gw, 256, 0, s>>>(scores, N, KB, MW, st, tmp_b, mask, tmp_a));
     FGMP_LAUNCH(FGMP_K_W_MASK, s, w_unit_count_kernel<<<(unsigned)NCT, 128, 0, s>>>(mask, L, tmp_a, st));
     FGMP_LAUNCH(FGMP_K_SCAN, s, scan_kernel<<<1, 1024, 0, s>>>(tmp_a, uptr, NCT, nullptr, 1));
-    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<(unsigned)NCT, 128, 0, s>>>(W, ldw / 8, ratio, st, sc_tmp, blob, L, room_steps));
-    FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, uptr, NCT, N, K, ratio,
+    FGMP_LAUNCH(FGMP_K_W_EMIT, s, w_emit_kernel<<<(unsigned)NCT, 128, 0, s>>>(W, ldw / 8, ratio, s8_given, st, sc_tmp, blob, L, room_steps));
+    FGMP_LAUNCH(FGMP_K_W_AUX, s, w_header_kernel<<<1, 32, 0, s>>>(reinterpret_cast<fgmp_packed_header*>(blob), st, uptr, NCT, N, K, ratio, s8_given,
                                      room_steps, fraction_mode ? 1 : 0, tau, tau_eff_out));
     FGMP_LAUNCH(FGMP_K_W_AUX, s, w_clamp_uptr_kernel<<<grid_for(NCT + 1, 256, 1), 256, 0, s>>>(reinterpret_cast<const fgmp_packed_header*>(blob), uptr, NCT + 1, room_steps));
     return fgmp_launch_status();
@@ -543,7 +546,7 @@ extern "C" fgmp_status fgmp_weight_scores(const void* W_bf16, int64_t ldw, const
     if (!W_bf16 || !fisher_elem || !scores || !workspace) return FGMP_ERR_INVALID_ARG;
     if ((int)sm < 0 || (int)sm > 1 || (int)cm < 0 || (int)cm > 1) return FGMP_ERR_INVALID_ARG;
     if (!(sc.scale_fp4 >= 0.f) || !isfinite(sc.scale_fp4)) return FGMP_ERR_INVALID_ARG;
-    if (sc.fp8_log2_ratio < -7 || sc.fp8_log2_ratio > 7) return FGMP_ERR_INVALID_ARG;
+    if (!fgmp_scales_valid(sc)) return FGMP_ERR_INVALID_ARG;
     if (N < 1 || K < 64 || (K % 64) != 0 || ldw < K || (ldw % 8) != 0 || ldf < K || (ldf % 4) != 0) return FGMP_ERR_SHAPE;
     if (((uintptr_t)W_bf16 & 15) || ((uintptr_t)fisher_elem & 15) || ((uintptr_t)scores & 15) || ((uintptr_t)workspace & 255))
         return FGMP_ERR_SHAPE;
@@ -558,6 +561,7 @@ extern "C" fgmp_status fgmp_weight_scores(const void* W_bf16, int64_t ldw, const
     uint8_t* sc_tmp = ws + STATE_BYTES + fgmp_align1k((size_t)B * 4);
     const uint4* W = reinterpret_cast<const uint4*>(W_bf16);
     const int ratio = sc.fp8_log2_ratio;
+    const float s8_given = sc.scale_fp8;
     FGMP_LAUNCH(FGMP_K_W_AUX, s, state_init_kernel<<<1, 256, 0, s>>>(st, sc.scale_fp4, 0ull));
     if (sc.scale_fp4 == 0.f) {
         FGMP_LAUNCH(FGMP_K_W_AMAX, s, w_amax_kernel<<<grid_for(N * (K / 8), 256, 8), 256, 0, s>>>(W, ldw / 8, N, K / 8, st));
@@ -565,11 +569,11 @@ extern "C" fgmp_status fgmp_weight_scores(const void* W_bf16, int64_t ldw, const
     }
     const int g = grid_for(B, 256, 4);
     if (sm == FGMP_SCORE_LP_ERROR) {
-        if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
-        else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+        if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
+        else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<0, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
     } else {
-        if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
-        else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, st, sc_tmp, scores));
+        if (cm == FGMP_CLIP_SW_BRUTE) FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, true><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
+        else                          FGMP_LAUNCH(FGMP_K_W_SCORE, s, w_score_kernel<1, false><<<g, 256, 0, s>>>(W, ldw / 8, fisher_elem, ldf, N, KB, ratio, s8_given, st, sc_tmp, scores));
     }
     return fgmp_launch_status();
 }

@@ -415,3 +415,80 @@ def test_clip_search_ties_keep_the_incumbent_then_the_lowest_code():
     # without the search the dynamic-max code stays
     q0 = oracle.quantize_weights(bits, f, scale_fp4=1.0, clip=False, fp8_fraction=0.0)
     assert q0.scales[1] == 0x2B and q0.scales[0] == 0x00
+
+
+# ------------------------------------------------------------------ FP8 tensor scale given on its own (Section 5.1)
+
+def _free_scales(x, w):
+    """amax / 448 for the FP8 part, amax / (6 * 448) for the NVFP4 part: a ratio of 6, not a power of two."""
+    ax, aw = float(x.float().abs().max()), float(w.float().abs().max())
+    return (np.float32(ax / 2688.0), np.float32(ax / 448.0)), (np.float32(aw / 2688.0), np.float32(aw / 448.0))
+
+
+def test_free_fp8_scale_rounds_to_nearest_under_that_scale():
+    """FP8 codes are the E4M3 values nearest to x / s8 (brute force over the 253 finite values, fp64) for an s8 that
+    is not s4 times a power of two; the NVFP4 side does not depend on s8; mode-1 scores are Eq. 8 in fp64 with
+    this s8."""
+    wl, x, _, fx, _ = _tiny()
+    (s4, s8), _ = _free_scales(x, x)
+    q = oracle.quantize_activations(gi.bf16_bits(x), fx, s4, tau=-1.0, mode=1, scale_fp8=s8)
+    xv = _bf16_to_f32(gi.bf16_bits(x)).astype(np.float64)
+    e4 = _e4m3_vals()
+    y8 = xv / np.float64(s8)
+    c8 = q.codes8.reshape(wl.M, wl.K)
+    finite = e4[np.r_[0:0x7F, 0x80:0xFF]]
+    best8 = np.abs(y8[..., None] - finite[None, None, :]).min(-1)
+    assert np.all(np.abs(y8 - e4[c8]) <= best8 + 1e-5 * np.abs(y8) + 1e-12)
+    assert np.abs(e4[c8]).max() > 224          # the scale uses the E4M3 range (amax lands near 448)
+    q4 = oracle.quantize_activations(gi.bf16_bits(x), fx, s4, tau=np.inf, mode=0, scale_fp8=s8)
+    q4t = oracle.quantize_activations(gi.bf16_bits(x), fx, s4, tau=np.inf, mode=0)
+    assert np.array_equal(q4.codes4, q4t.codes4) and np.array_equal(q4.scales, q4t.scales) and np.array_equal(q4.scores, q4t.scores)
+    # Eq. 8 with this s8: sum f (Q4(x) - Q8(x))^2
+    d4 = oracle.decode(q4)
+    d8 = e4[c8] * np.float64(s8)
+    ref = (fx.astype(np.float64)[None, :] * (d4 - d8) ** 2).reshape(wl.M, -1, 16).sum(-1)
+    assert np.allclose(q.scores.reshape(wl.M, -1), ref, rtol=2e-5, atol=1e-30)
+
+
+def test_free_fp8_scale_equal_to_the_tied_one_changes_nothing():
+    """Passing s8 = s4 * 2^3 explicitly gives the arrays of the tied default, and decode / linear use the given value."""
+    wl, x, w, fx, fw = _tiny()
+    s4 = gi.tensor_scale(x)
+    a = oracle.quantize_activations(gi.bf16_bits(x), fx, s4, tau=1e-4, mode=1)
+    b = oracle.quantize_activations(gi.bf16_bits(x), fx, s4, tau=1e-4, mode=1, scale_fp8=float(np.float32(s4) * np.float32(8)))
+    for n in ("codes4", "codes8", "scales", "mask", "scores"):
+        assert np.array_equal(getattr(a, n), getattr(b, n)), n
+    assert np.array_equal(oracle.decode(a), oracle.decode(b))
+
+
+def test_free_fp8_scale_decode_and_linear():
+    """Decoded FP8 blocks are e4m3 * s8 with the given s8 (NVFP4 blocks unchanged); the layer is the fp64 library
+    matmul of the decoded operands; with every block in FP8 it is the plain per-tensor-scaled E4M3 GEMM through
+    torch's own cast."""
+    wl, x, w, fx, fw = _tiny()
+    (as4, as8), (ws4, ws8) = _free_scales(x, w)
+    e4 = _e4m3_vals()
+    for frac in (0.1, 1.0):
+        sa = oracle.quantize_activations(gi.bf16_bits(x), fx, as4, tau=np.inf, scale_fp8=as8).scores
+        tau = -1.0 if frac == 1.0 else _tau_for_fraction(sa, frac)[0]
+        qa = oracle.quantize_activations(gi.bf16_bits(x), fx, as4, tau=tau, scale_fp8=as8)
+        qw = oracle.quantize_weights(gi.bf16_bits(w), fw, scale_fp4=ws4, fp8_fraction=frac, scale_fp8=ws8)
+        for q, s8 in ((qa, as8), (qw, ws8)):
+            mb = np.repeat(q.mask_bits(), 16, axis=1)
+            sc = np.repeat(q.scales.reshape(q.rows, -1), 16, axis=1)
+            v4 = E2M1[_unpack4(q)] * e4[sc] * np.float64(np.float32(q.scale_fp4))
+            v8 = e4[q.codes8.reshape(q.rows, q.K)] * np.float64(s8)
+            assert np.array_equal(oracle.decode(q), np.where(mb, v8, v4))
+        Y, S = oracle.linear(qa, qw)
+        A, Wd = torch.from_numpy(oracle.decode(qa)), torch.from_numpy(oracle.decode(qw))
+        assert np.allclose(Y, (A @ Wd.T).numpy(), rtol=0, atol=1e-12 * S.max())
+        ms = np.array([0, 5, 63, 17]); ns = np.array([0, 255, 128, 3])
+        Ys, _ = oracle.linear_sampled(qa, qw, ms, ns)
+        assert np.allclose(Ys, Y[ms, ns], rtol=0, atol=1e-12 * S.max())
+        if frac == 1.0:
+            xa = (x.float() * (np.float32(1.0) / as8)).to(torch.float8_e4m3fn).double() * np.float64(as8)
+            ww = (w.float() * (np.float32(1.0) / ws8)).to(torch.float8_e4m3fn).double() * np.float64(ws8)
+            assert np.allclose(Y, (xa @ ww.T).numpy(), rtol=0, atol=1e-12 * np.abs(Y).max())
+            # a free scale uses the whole E4M3 range: the FP8 layer is closer to the bf16 layer than with s8 = 8 s4 > amax / 448
+            ref = (x.double() @ w.double().T).numpy()
+            assert np.abs(Y - ref).sum() / np.abs(ref).sum() < 0.05
