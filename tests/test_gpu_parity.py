@@ -385,15 +385,23 @@ def test_fused_decode_step_equals_the_two_calls_and_the_oracle(fg, M, N, K, mode
     fg.check(ws)
 
 
-def test_fused_step_for_a_prefill_sized_batch_runs_the_two_calls(fg):
-    wl = gi.llama("f", 40, 300, 512, seed=70)
-    qa, qw, pa, pw = quantize_both(fg, wl, 0.1, 0.1, clip=False)
+@pytest.mark.parametrize("M,N,K,mode,frac", [(40, 300, 512, 0, 0.1), (333, 520, 1024, 1, 0.1), (130, 136, 320, 0, 1.0),
+                                             (12, 300, 320, 0, 0.1), (200, 392, 512, 0, 0.0)])
+def test_fused_step_for_a_prefill_sized_batch(fg, M, N, K, mode, frac):
+    """Beyond the decode kernel's shapes the fused call runs the two calls: packed activations bit for bit as the
+    oracle's, Y bit for bit as the two calls give (all-FP8, mixed, and the all-NVFP4 operands that take the FP4
+    tensor-core kernel)."""
+    wl = gi.llama("f", M, N, K, seed=70)
+    qa, qw, pa, pw = quantize_both(fg, wl, frac, frac, mode=mode, clip=False)
     x, fx = wl.x(), wl.fx()
     s4 = gi.tensor_scale(x)
-    tau = tau_for_fraction(qa.scores, 0.1)
-    y, pf = fg.linear_fused(x.cuda(), fx.cuda(), pw, scale_fp4=s4, tau=tau, want_packed=True)
+    tau = tau_for_fraction(qa.scores, frac)
+    y, pf = fg.linear_fused(x.cuda(), fx.cuda(), pw, scale_fp4=s4, score_mode=mode, tau=tau, want_packed=True)
+    fg.check(fg.linear.last_workspace)
     compare_packed(fg, pf, qa, tau, "fused prefill-sized")
     assert torch.equal(y, fg.linear(pa, pw))
+    Y, S = oracle.linear(qa, qw)
+    assert (np.abs(y.cpu().numpy().astype(np.float64) - Y) <= 1e-5 * S + 1e-30).all()
 
 
 def test_weight_blob_that_does_not_match_the_call_is_refused_on_the_device(fg):
