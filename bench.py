@@ -351,9 +351,9 @@ def roofline_of(fg, wk, prof, step_ms, dev, peaks):
             "tensor_peaks_tflops": tp}
 
 
-def side_measurement(fg, dev, name, steps, replays, world, peaks, use_graph):
+def side_measurement(fg, dev, name, steps, replays, world, peaks, use_graph, fp8=None):
     """A shorter measurement of another workload for the same JSON line."""
-    wk = Workload(fg, dev, name)
+    wk = Workload(fg, dev, name, fp8=fp8)
     for i in range(3):
         wk.step(i)
     fg.check(wk.ws)
@@ -363,7 +363,7 @@ def side_measurement(fg, dev, name, steps, replays, world, peaks, use_graph):
     ms = statistics.median(runs)
     prof = kernel_pass(fg, wk, steps, world)
     metric, unit = wk.metric_unit
-    out = {"workload": name, "M": wk.M, "N": wk.N, "K": wk.K, "metric": metric, "unit": unit,
+    out = {"workload": name, "M": wk.M, "N": wk.N, "K": wk.K, "fp8_fraction": wk.p, "metric": metric, "unit": unit,
            "value": world * wk.units_per_step * steps / (ms / 1e3), "step_us": ms / steps * 1e3,
            "steps": steps, "replays": replays, "launch": note,
            "kernels": {k: {"launches": v[0], "avg_us": (v[1] / v[0] * 1e3 if v[1] else None)} for k, v in prof.items()},
@@ -496,6 +496,11 @@ def run_ours(args, world, rank, local):
     if not args.no_extras and args.workload == "llama2-7b-fc1-decode" and not args.m:
         out["decode_70b"] = side_measurement(fg, dev, "llama2-70b-fc1-decode", 20, 11, world, peaks, use_graph)
         out["prefill"] = side_measurement(fg, dev, "llama2-7b-fc1-prefill", 5, 7, world, peaks, use_graph)
+    if args.sweep:
+        # the FP8 fraction of both operands swept over the given points (config 4: 0 / 10 / 20 / 30 %), each point
+        # measured like the side objects above: step time, kernel times and the roofline of the mix at that point
+        out["sweep"] = [side_measurement(fg, dev, args.workload, 5, 7, world, peaks, use_graph, fp8=float(f))
+                        for f in args.sweep.split(",")]
     if rank == 0 and not args.no_cpu_baseline and world >= 1:
         out["cpu_baseline"] = cpu_baseline(args, wl, p, kind, per_step_units, unit)
         out["cpu_baseline"]["single_thread"] = cpu_baseline_single_thread(args)
@@ -647,6 +652,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2-7b-fc1-decode", choices=sorted(WORKLOADS))
     ap.add_argument("--m", type=int, default=0, help="override the token count M")
+    ap.add_argument("--sweep", default="", help="comma-separated FP8 fractions: adds a measurement of the workload at each (e.g. 0,0.1,0.2,0.3)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the timed steps eagerly")
     ap.add_argument("--replays", type=int, default=25, help="how often the K steps are timed (the median run is reported)")

@@ -324,8 +324,9 @@ fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, uint8_t* co
 /* ---- measurement support: tensor-core rate per operand kind ----
  * Runs, on every SM, mma_per_cta tcgen05 instructions of M = 128, N = 256 on operands resident in
  * shared memory (nothing is loaded or stored; mma_per_cta <= 2^21): kind 0 = bf16 (K = 16 per instruction), 1 = FP8 E4M3
- * (K = 32), 2 = NVFP4 with E4M3 block scales (K = 64).  The caller times the call on the stream;
- * flops = 2 * 128 * 256 * K * mma_per_cta * (number of SMs).  These are the rates the block-pair
+ * (K = 32), 2 = NVFP4 with E4M3 block scales (K = 64); kind + 4 = the same on CTA pairs (cta_group::2, M = 256 per
+ * pair, the leader issues mma_per_cta instructions; an odd SM stays idle).  The caller times the call on the stream;
+ * flops = 2 * 128 * 256 * K * mma_per_cta * (number of CTAs launched: the SMs, or the SMs in pairs).  These are the rates the block-pair
  * products of Section 4.1 can run at at best, i.e. the denominators of the prefill roofline.
  * workspace: >= 256 bytes, zeroed, 256-byte aligned (status word, read by fgmp_check). */
 fgmp_status fgmp_tensor_peak(int kind, int64_t mma_per_cta, void* workspace, size_t ws_bytes, void* cuda_stream);

@@ -6,6 +6,7 @@
 #include "fgmp_common.cuh"
 #include "fgmp_host.h"
 #include "fgmp_ptx.cuh"
+#include <mutex>
 
 namespace {
 
@@ -107,6 +108,100 @@ tensor_peak_kernel(int kind, int64_t n_mma, int* status)
     if (warp == 0) tmem_dealloc(tmem_base, 512);
 }
 
+
+// The same loop on CTA pairs: tcgen05.mma cta_group::2, M = 256 (128 rows of A per CTA), N = 256 (128 rows of B per
+// CTA), issued by the pair's leader; each CTA's tensor memory holds its 128 rows of the accumulator (and, for the
+// block-scaled kind, the scales of its rows of A and of all rows of B).
+__device__ __forceinline__ void umma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+constexpr uint32_t PKP_B_BYTES = 128 * 128;
+constexpr size_t PKP_SMEM = PK_A_BYTES + PKP_B_BYTES + 1024 + 64;
+constexpr uint32_t PKP_IDESC_NM = ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PK_THREADS, 1)
+tensor_peak_pair_kernel(int kind, int64_t n_mma, int* status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem + PK_A_BYTES + PKP_B_BYTES);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t done = smem_u32(bar);
+    {
+        uint32_t* w = reinterpret_cast<uint32_t*>(smem);
+        for (uint32_t i = threadIdx.x; i < (PK_A_BYTES + PKP_B_BYTES) / 4; i += PK_THREADS) {
+            uint32_t h = (i + 7919u * rank) * 2654435761u; h ^= h >> 15;
+            uint32_t v;
+            if (kind == 0)      v = 0x3c003c00u | (h & 0x807f807fu);
+            else if (kind == 1) v = 0x38383838u | (h & 0x87078707u) | ((h >> 3) & 0x00080008u);
+            else                v = (h & 0x77777777u) | 0x11111111u | ((h >> 7) & 0x88888888u);
+            w[i] = v;
+        }
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(done, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc_pair(smem_u32(tmem_slot), 512);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (kind == 2) {
+        uint32_t r[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = 0x38383838u;
+        const uint32_t t = tmem_base + ((uint32_t)(warp * 32) << 16) + PK_SF_COL0;
+        tmem_st16(t, r); tmem_st16(t + 16, r); tmem_st16(t + 32, r);
+        tmem_wait_st();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();                                     // both CTAs' operands and scales are in place
+    tc_fence_after();
+
+    if (warp == 0) {
+        if (rank == 0) {
+            const uint32_t a_lo = (smem_u32(smem) >> 4) | (1u << 16), b_lo = (smem_u32(smem + PK_A_BYTES) >> 4) | (1u << 16);
+            if (lane == 0) {
+                for (int64_t i = 0; i < n_mma; ++i) {
+                    const uint32_t k = (uint32_t)(i & 3) * 2u;
+                    uint64_t ad, bd;
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(ad) : "r"(a_lo + k), "r"(PK_SW128_HI));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(bd) : "r"(b_lo + k), "r"(PK_SW128_HI));
+                    const uint32_t acc = i ? 1u : 0u;
+                    if (kind == 0)      umma_f16_pair(tmem_base, ad, bd, (1u << 4) | (1u << 7) | (1u << 10) | PKP_IDESC_NM, acc);
+                    else if (kind == 1) umma_f8_pair(tmem_base, ad, bd, (1u << 4) | PKP_IDESC_NM, acc);
+                    else                umma_nvf4_pair(tmem_base, ad, bd, (1u << 7) | (1u << 10) | PKP_IDESC_NM,
+                                                       tmem_base + PK_SF_COL0 + 4 * (k >> 1), tmem_base + PK_SF_COL0 + 16 + 8 * (k >> 1), acc);
+                }
+                umma_commit_pair(done, 3);
+            }
+            __syncwarp();
+        }
+        mbar_wait(done, 0, abort_flag, status, 21);     // both CTAs wait for the leader's last MMA
+        tc_fence_after();
+    }
+    __syncthreads();
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    cluster_sync();
+    if (warp == 0) tmem_dealloc_pair(tmem_base, 512);
+}
+
 // One CTA waits, with the library's bounded wait, for a barrier that nothing completes: the wait runs out
 // after limit_ns, FGMP_ERR_TIMEOUT goes into the status word like in the GEMM kernels, and the kernel returns.
 __global__ void __launch_bounds__(32, 1) wait_selftest_kernel(unsigned long long limit_ns, int* status)
@@ -129,19 +224,31 @@ __global__ void __launch_bounds__(32, 1) wait_selftest_kernel(unsigned long long
 extern "C" fgmp_status fgmp_tensor_peak(int kind, int64_t mma_per_cta, void* workspace, size_t ws_bytes, void* cuda_stream)
 {
     // (at about 0.1 us per instruction 2^21 of them stay far inside the bounded wait at the end of the loop)
+    const bool pair = kind >= 4;
+    if (pair) kind -= 4;
     if (kind < 0 || kind > 2 || mma_per_cta < 1 || mma_per_cta > (int64_t)1 << 21 || !workspace || ws_bytes < 256 ||
         ((uintptr_t)workspace & 255)) return FGMP_ERR_INVALID_ARG;
     fgmp_status st;
     if ((st = fgmp_require_sm100()) != FGMP_OK) return st;
+    static std::mutex mu;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(tensor_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PK_SMEM) != cudaSuccess)
-            return FGMP_ERR_CUDA;
-        attr_set[dev] = true;
+    if (dev < 0 || dev >= 64) return FGMP_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (!attr_set[dev]) {
+            if (cudaFuncSetAttribute(tensor_peak_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PK_SMEM) != cudaSuccess ||
+                cudaFuncSetAttribute(tensor_peak_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PKP_SMEM) != cudaSuccess)
+                return FGMP_ERR_CUDA;
+            attr_set[dev] = true;
+        }
     }
     cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (pair) {
+        tensor_peak_pair_kernel<<<(fgmp_sm_count() / 2) * 2, PK_THREADS, PKP_SMEM, s>>>(kind, mma_per_cta, reinterpret_cast<int*>(workspace));
+        return fgmp_launch_status();
+    }
     tensor_peak_kernel<<<fgmp_sm_count(), PK_THREADS, PK_SMEM, s>>>(kind, mma_per_cta, reinterpret_cast<int*>(workspace));
     return fgmp_launch_status();
 }
