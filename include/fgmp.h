@@ -43,7 +43,11 @@
  *                   scale in fp16 (exact for either format): token octet m/8 in its own 4096 bytes, there
  *                   256 bytes per block column, there 32 bytes per token
  *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written (the
- *                   blob is sized for the worst case of every block being FP8)
+ *                   blob is sized for the worst case of every block being FP8).  Footprint of packed
+ *                   activations: 1.57 bytes per element reserved (codes4 0.5 + sf 1/16 + mask 1/128 + codes8 1),
+ *                   of which a quantizer pass with FP8 fraction p writes and a GEMM reads
+ *                   (1-p)*9/16 + p + 1/128 bytes per element (0.61 at p = 0.1): the plane costs address space,
+ *                   not traffic, and keeps the single-pass quantizer free of a compaction step
  *
  * Weights: header | mask | uptr | records | lists
  *   record        : 18560 bytes per unit, unit (t, c) at index t*C + c:
@@ -317,7 +321,8 @@ fgmp_status fgmp_check(const void* workspace, void* cuda_stream);
 /* ---- parity support: packed -> canonical arrays (device) ----
  * codes4 [rows*K/2] (0 for FP8 blocks), codes8 [rows*K] (0 for FP4 blocks), scales
  * [rows*K/16] E4M3 (0 for FP8 blocks), mask [rows*ceil(K/16/32)], scores is not stored.
- * Any output pointer may be NULL. */
+ * Any output pointer may be NULL.  The tensor scales are not among the outputs: they are in the blob's
+ * header (scale_fp4, fp8_log2_ratio, scale_fp8), 256 bytes that the caller can copy. */
 fgmp_status fgmp_unpack(const void* packed, int64_t rows, int64_t K, uint8_t* codes4, uint8_t* codes8,
                         uint8_t* scales, uint32_t* mask, void* cuda_stream);
 
