@@ -39,8 +39,9 @@ __device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&v)[16])
 #pragma unroll
     for (int i = 0; i < 8; ++i)
         o[i] = (__float_as_uint(v[2 * i]) >> 16) | (__float_as_uint(v[2 * i + 1]) & 0xffff0000u);
-    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    // one 32-byte store (the planes are 32-byte aligned and a block is 32 bytes): whole sectors per lane
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
 }
 
 __device__ __forceinline__ void nvfp4x16_scaled(const uint2& c, uint32_t scale_code, float (&v)[16])
