@@ -32,6 +32,12 @@ __device__ __forceinline__ void e4m3x16_scaled(const uint4& c, float r8, float (
     }
 }
 
+__device__ __forceinline__ void store_256(void* dst, const uint32_t (&o)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+}
+
 // 16 values that are exact in bf16 (the low 16 bits of every float are zero) -> 32 bytes
 __device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&v)[16])
 {
@@ -39,9 +45,7 @@ __device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&v)[16])
 #pragma unroll
     for (int i = 0; i < 8; ++i)
         o[i] = (__float_as_uint(v[2 * i]) >> 16) | (__float_as_uint(v[2 * i + 1]) & 0xffff0000u);
-    // one 32-byte store (the planes are 32-byte aligned and a block is 32 bytes): whole sectors per lane
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"l"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+    store_256(dst, o);        // one 32-byte store (the planes are 32-byte aligned and a block is 32 bytes): whole sectors per lane
 }
 
 __device__ __forceinline__ void nvfp4x16_scaled(const uint2& c, uint32_t scale_code, float (&v)[16])
@@ -247,6 +251,33 @@ __device__ __forceinline__ uint32_t quantize_chunk32(const GemmParams& p, int64_
 __device__ __forceinline__ void store_chunk32(const GemmParams& p, int64_t row, int64_t col0, const uint32_t (&r)[32], float alpha)
 {
     if (row >= p.M) return;
+    // Y and its row pitch 32-byte aligned: a lane writes whole 32-byte sectors
+    const bool wide = !p.accumulate && ((uintptr_t)p.Y & 31) == 0 && ((p.ldy * (p.y_is_bf16 ? 2 : 4)) % 32) == 0 && col0 + 32 <= p.N;
+    if (wide) {
+        if (p.y_is_bf16) {
+            __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
+#pragma unroll
+            for (int j = 0; j < 32; j += 16) {
+                uint32_t o[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * u]) * alpha, __uint_as_float(r[j + 2 * u + 1]) * alpha);
+                    o[u] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                store_256(y + j, o);
+            }
+        } else {
+            float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+                uint32_t o[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) o[u] = __float_as_uint(__uint_as_float(r[j + u]) * alpha);
+                store_256(y + j, o);
+            }
+        }
+        return;
+    }
     if (p.y_is_bf16) {
         __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
         if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {

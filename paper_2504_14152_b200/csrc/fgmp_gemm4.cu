@@ -44,6 +44,12 @@ __device__ __forceinline__ uint64_t g4_desc(uint32_t lo)
     return d;
 }
 
+__device__ __forceinline__ void st_global_256(void* dst, const uint32_t (&o)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+}
+
 struct Gemm4Params {
     const uint8_t* ablob; const uint8_t* wblob;
     PackedLayout LA, LW;
@@ -204,6 +210,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, Gemm4Params p)
         const fgmp_packed_header* ha = reinterpret_cast<const fgmp_packed_header*>(p.ablob);
         const fgmp_packed_header* hw = reinterpret_cast<const fgmp_packed_header*>(p.wblob);
         const float alpha = __fmul_rn(ha->scale_fp4, hw->scale_fp4);
+        // Y and its row pitch 32-byte aligned: a lane writes whole sectors
+        const bool wide = ((uintptr_t)p.Y & 31) == 0 && ((p.ldy * (p.y_is_bf16 ? 2 : 4)) % 32) == 0;
         bool ok = true;
         int64_t it = 0;
         for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++it) {
@@ -220,7 +228,19 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, Gemm4Params p)
                     const int64_t col0 = n0 + c * 32;
                     if (p.y_is_bf16) {
                         __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(p.Y) + row * p.ldy + col0;
-                        if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {
+                        if (col0 + 32 <= p.N && wide) {
+                            // whole 32-byte sectors per lane
+#pragma unroll
+                            for (int j = 0; j < 32; j += 16) {
+                                uint32_t o[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[j + 2 * u]) * alpha, __uint_as_float(r[j + 2 * u + 1]) * alpha);
+                                    o[u] = *reinterpret_cast<uint32_t*>(&h);
+                                }
+                                st_global_256(y + j, o);
+                            }
+                        } else if (col0 + 32 <= p.N && (p.ldy % 8) == 0) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 8) {
                                 uint32_t o[4];
@@ -237,7 +257,15 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, Gemm4Params p)
                         }
                     } else {
                         float* y = reinterpret_cast<float*>(p.Y) + row * p.ldy + col0;
-                        if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
+                        if (col0 + 32 <= p.N && wide) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t o[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) o[u] = __float_as_uint(__uint_as_float(r[j + u]) * alpha);
+                                st_global_256(y + j, o);
+                            }
+                        } else if (col0 + 32 <= p.N && (p.ldy % 4) == 0) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
                                 *reinterpret_cast<float4*>(y + j) = make_float4(__uint_as_float(r[j]) * alpha, __uint_as_float(r[j + 1]) * alpha,
