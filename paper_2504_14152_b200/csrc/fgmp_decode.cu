@@ -724,8 +724,13 @@ decode_kernel(DecParams p)
                 // partial tile: publish, and let the warp that arrives last add everything up.  When all the
                 // others were seen to have arrived, this warp is the last without asking and skips the counter.
                 float* dst = p.partials + (((size_t)tile * p.maxseg + slot) * 128 + row) * 16;
+                // (32 bytes per store: whole sectors)
 #pragma unroll
-                for (int j = 0; j < 8 * NH; j += 4) __stcg(reinterpret_cast<float4*>(dst + j), make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+                for (int j = 0; j < 8 * NH; j += 8)
+                    asm volatile("st.global.cg.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                 ::"l"(dst + j), "r"(__float_as_uint(v[j])), "r"(__float_as_uint(v[j + 1])), "r"(__float_as_uint(v[j + 2])),
+                                   "r"(__float_as_uint(v[j + 3])), "r"(__float_as_uint(v[j + 4])), "r"(__float_as_uint(v[j + 5])),
+                                   "r"(__float_as_uint(v[j + 6])), "r"(__float_as_uint(v[j + 7])) : "memory");
                 // The counter wraps to zero with the last arrival (or is put back by the warp that skipped
                 // it), so the workspace is ready for the next call without being cleared.
                 uint32_t old = __shfl_sync(0xffffffffu, seen, 0);
@@ -744,9 +749,13 @@ decode_kernel(DecParams p)
                     for (int sgi = 0; sgi < nseg; ++sgi) {       // one sum in slot order
                         const float* src = p.partials + (((size_t)tile * p.maxseg + sgi) * 128 + row) * 16;
 #pragma unroll
-                        for (int j = 0; j < 8 * NH; j += 4) {
-                            const float4 y4 = __ldcg(reinterpret_cast<const float4*>(src + j));
-                            v[j] += y4.x; v[j + 1] += y4.y; v[j + 2] += y4.z; v[j + 3] += y4.w;
+                        for (int j = 0; j < 8 * NH; j += 8) {
+                            uint32_t y8[8];
+                            asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                         : "=r"(y8[0]), "=r"(y8[1]), "=r"(y8[2]), "=r"(y8[3]), "=r"(y8[4]), "=r"(y8[5]), "=r"(y8[6]), "=r"(y8[7])
+                                         : "l"(src + j) : "memory");
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) v[j + e] += __uint_as_float(y8[e]);
                         }
                     }
                     write_out = true;
