@@ -322,10 +322,15 @@ decode_kernel(DecParams p)
             }
             if (p.q_mode == 0) quantize_chunk<0>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
             else               quantize_chunk<1>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
-            __threadfence();
+            // The item's stores become visible with the counter: the barrier orders them before the one thread's
+            // release, and the last arrival's acquire sees every earlier release of the counter.
             quant_bar();
-            if (threadIdx.x == 64 && atomicInc(p.cw + CW_QCOUNT, n_items - 1u) == n_items - 1u)
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(1u) : "memory");
+            if (threadIdx.x == 64) {
+                uint32_t old;
+                asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.cw + CW_QCOUNT), "r"(n_items - 1u) : "memory");
+                if (old == n_items - 1u)
+                    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.cw + CW_QREADY), "r"(1u) : "memory");
+            }
         }
     }
 
