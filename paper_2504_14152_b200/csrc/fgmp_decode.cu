@@ -740,15 +740,15 @@ decode_kernel(DecParams p)
                 // it), so the workspace is ready for the next call without being cleared.
                 uint32_t old = __shfl_sync(0xffffffffu, seen, 0);
                 if (old != (uint32_t)(nseg - 1)) {
-                    __threadfence();
+                    // the warp's stores are ordered before lane 0's release of the counter; its acquire sees the others'
                     __syncwarp();
-                    if (lane == 0) old = atomicInc(p.counters + tile * 8 + q, (uint32_t)(nseg - 1));
+                    if (lane == 0)
+                        asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.counters + tile * 8 + q), "r"((uint32_t)(nseg - 1)) : "memory");
                     old = __shfl_sync(0xffffffffu, old, 0);
                 } else if (lane == 0) {
                     p.counters[tile * 8 + q] = 0u;
                 }
                 if (old == (uint32_t)(nseg - 1)) {
-                    __threadfence();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) v[j] = 0.f;
                     for (int sgi = 0; sgi < nseg; ++sgi) {       // one sum in slot order
