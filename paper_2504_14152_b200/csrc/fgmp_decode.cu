@@ -138,11 +138,11 @@ __device__ __noinline__ bool wait_global_equals(const uint32_t* addr, uint32_t v
     }
 }
 
-// One work item of the prologue quantizer: chunk c (256 elements) of every token row.  Run by the 16
-// warps 2..17: warp wq takes, per token octet o, token 8o + wq/2 and the eight blocks 8(wq%2) .. +7 of
-// the chunk, four lanes per block.  s_hot: one word of shared memory.
+// One work item of the prologue quantizer: chunk c (256 elements) of the eight token rows of octet o.  Run by
+// the 16 warps 2..17: warp wq takes token 8o + wq/2 and the eight blocks 8(wq%2) .. +7 of the chunk, four lanes
+// per block.  s_hot: one word of shared memory.  Each octet has its own word for the chunk's hot block columns.
 template <int MODE>
-__device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, uint32_t* s_hot)
+__device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, int o, uint32_t* s_hot)
 {
     const uint32_t tq = threadIdx.x - 64u;                 // index among the quantizer's threads
     const uint32_t wq = tq >> 5, lane = tq & 31u, li = lane & 3u;
@@ -151,28 +151,23 @@ __device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, ui
     uint8_t* rec = p.arec + (size_t)c * AREC_BYTES;
     if (tq == 0) *s_hot = 0u;
     quant_bar();
-    const int octets = p.M > 8 ? 2 : 1;
-    // both token rows of this warp are on their way before either is worked on
-    uint2 xin[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
-#pragma unroll
-    for (int o = 0; o < 2; ++o) {
-        const uint32_t m = 8u * (uint32_t)o + (wq >> 1);
-        if (o < octets && (int64_t)m < p.M)
-            xin[o] = __ldg(reinterpret_cast<const uint2*>(p.X + ((size_t)m * p.ldx + (size_t)kb * 16 + 4 * li) * 2));
+    const uint32_t m = 8u * (uint32_t)o + (wq >> 1);
+    const bool live = (int64_t)m < p.M;
+    uint2 xin = make_uint2(0u, 0u);
+    float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (live) {
+        xin = __ldg(reinterpret_cast<const uint2*>(p.X + ((size_t)m * p.ldx + (size_t)kb * 16 + 4 * li) * 2));
+        f = __ldg(reinterpret_cast<const float4*>(p.fisher + kb * 16 + 4 * li));
     }
-    const float4 f = __ldg(reinterpret_cast<const float4*>(p.fisher + kb * 16 + 4 * li));
-#pragma unroll
-    for (int o = 0; o < 2; ++o) {
-        const uint32_t m = 8u * (uint32_t)o + (wq >> 1);
+    {
         uint8_t* a4 = rec + AREC_A4 + fgmp_rec_w4_offset(m, j) + 2u * li;
         uint8_t* at = rec + fgmp_arec_at_offset(m, j) + 8u * li;
-        if (o >= octets || (int64_t)m >= p.M) {             // token rows beyond the batch are zero
+        if (!live) {                                        // token rows beyond the batch are zero
             *reinterpret_cast<uint16_t*>(a4) = 0;
             *reinterpret_cast<uint2*>(at) = make_uint2(0u, 0u);
             if (li == 0) rec[AREC_SF + m * 16u + j] = 0;
-            continue;
-        }
-        const BlockQuarter r = quantize_block_quarter<MODE>(xin[o], f, p.q);
+        } else {
+        const BlockQuarter r = quantize_block_quarter<MODE>(xin, f, p.q);
         *reinterpret_cast<uint16_t*>(a4) = (uint16_t)r.c4;
         *reinterpret_cast<uint2*>(at) = r.h;
         if (li == 0) rec[AREC_SF + m * 16u + j] = (uint8_t)r.sc;
@@ -192,9 +187,10 @@ __device__ __forceinline__ void quantize_chunk(const DecParams& p, int64_t c, ui
                 if (kb + 8 == p.LA.KB && (p.LA.KB & 31) != 0) { mb[1] = 0; mb[2] = 0; }   // rest of the row's last mask word
             }
         }
+        }
     }
     quant_bar();
-    if (tq == 0) *reinterpret_cast<uint32_t*>(rec + AREC_HOT) = *s_hot;
+    if (tq == 0) reinterpret_cast<uint32_t*>(rec + AREC_HOT)[o] = *s_hot;
 }
 
 // NH = token octets in use: 1 for M <= 8, else 2.  FUSED: the activation quantizer runs in the prologue.
@@ -299,7 +295,7 @@ decode_kernel(DecParams p)
     if (threadIdx.x == 0) FGMP_STAMP_ANY(2);
     if (FUSED) {
         // the first of the quantizer's work items is asked for right away
-        if (threadIdx.x == 64 && !*abort_flag) s_misc[1] = atomicInc(p.cw + CW_CLAIM, (uint32_t)C + (uint32_t)G - 1u);
+        if (threadIdx.x == 64 && !*abort_flag) s_misc[1] = atomicInc(p.cw + CW_CLAIM, 2u * (uint32_t)C + (uint32_t)G - 1u);
         __syncthreads();
     }
     const bool dead = *abort_flag != 0;                // the weight blob does not belong to this call: nothing else is read
@@ -308,7 +304,7 @@ decode_kernel(DecParams p)
         // The quantizer's work items (chunks) are handed out through a counter, so that every item is taken by
         // a CTA that is running: no CTA ever waits for one that has not started.  The counter and the count of
         // finished items wrap to zero with the call's last access.
-        const uint32_t n_items = (uint32_t)C;
+        const uint32_t n_items = 2u * (uint32_t)C;          // (chunk, token octet)
         for (uint32_t it = 0;; ++it) {
             const uint32_t item = s_misc[1 + (it & 1u)];
             if (item >= n_items) break;
@@ -320,8 +316,8 @@ decode_kernel(DecParams p)
                 h->fp8_log2_ratio = p.q.ratio; h->n_fp8 = (p.q.tau == INFINITY) ? 0 : -1; h->tau_eff = 0.f; h->kind = 0; h->capacity = 0;
                 h->error = 0; h->scale_fp8 = p.q.s8; h->fp8_scale_free = 0;
             }
-            if (p.q_mode == 0) quantize_chunk<0>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
-            else               quantize_chunk<1>(p, (int64_t)item, const_cast<uint32_t*>(s_misc + 3));
+            if (p.q_mode == 0) quantize_chunk<0>(p, (int64_t)(item >> 1), (int)(item & 1u), const_cast<uint32_t*>(s_misc + 3));
+            else               quantize_chunk<1>(p, (int64_t)(item >> 1), (int)(item & 1u), const_cast<uint32_t*>(s_misc + 3));
             // The item's stores become visible with the counter: the barrier orders them before the one thread's
             // release, and the last arrival's acquire sees every earlier release of the counter.
             quant_bar();
@@ -579,7 +575,8 @@ decode_kernel(DecParams p)
                 if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 6))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
-                const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
+                const uint2 hw2 = *reinterpret_cast<const uint2*>(sa + AREC_HOT);      // one word per token octet
+                const uint32_t hot = hw2.x | hw2.y;
                 uint32_t todo = hot & 0xffffu;
                 while (todo) {
                     const uint32_t j = (uint32_t)__ffs(todo) - 1u;
@@ -651,7 +648,8 @@ decode_kernel(DecParams p)
                 if (!(ok = mbar_wait_warp(full0 + 8 * stage, phase, abort_flag, p.status, 4))) break;
                 const uint8_t* sb = smem + (size_t)stage * DEC_STAGE_BYTES;
                 const uint8_t* sa = sb + STG_A;
-                const uint32_t hot = *reinterpret_cast<const uint32_t*>(sa + AREC_HOT);
+                const uint2 hw2 = *reinterpret_cast<const uint2*>(sa + AREC_HOT);      // one word per token octet
+                const uint32_t hot = hw2.x | hw2.y;
                 uint32_t r[16];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
