@@ -512,7 +512,7 @@ def run_ours(args, world, rank, local):
 NCU_TRAFFIC = {
     ("llama2-7b-fc1-decode", "decode_gemm"): {"bytes": 29184000, "file": "profiles/decode_kernel_llama2-7b-fc1-decode.md"},
     ("llama2-13b-fc1-prefill", "gemm_nvfp4_tcgen05"): {"bytes": 109814016, "file": "profiles/gemm_nvfp4_kernel_llama2-13b-fc1-prefill.md"},
-    ("llama2-7b-fc2-prefill", "gemm_bf16_tcgen05"): {"bytes": 535152896, "file": "profiles/gemm_bf16_pair_kernel_llama2-7b-fc2-prefill.md"},
+    ("llama2-7b-fc2-prefill", "gemm_bf16_tcgen05"): {"bytes": 536672512, "file": "profiles/gemm_bf16_pair_kernel_llama2-7b-fc2-prefill.md"},
 }
 
 
