@@ -433,8 +433,9 @@ def test_weight_blob_that_does_not_match_the_call_is_refused_on_the_device(fg):
     fg.check(fg.linear.last_workspace)
 
 
-@pytest.mark.parametrize("kind", [0, 1, 2])
+@pytest.mark.parametrize("kind", [0, 1, 2, 4, 5, 6])
 def test_tensor_peak_loop_runs(fg, kind):
+    """Kinds 0-2: one CTA per SM; kinds 4-6: the same operand kinds on CTA pairs (cta_group::2)."""
     ws = fg.binding._alloc_aligned(1024, torch.device("cuda"))
     ws.zero_()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -445,6 +446,8 @@ def test_tensor_peak_loop_runs(fg, kind):
     torch.cuda.synchronize()
     fg.check(ws)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
+    if kind >= 4:
+        sms, kind = (sms // 2) * 2, kind - 4
     tflops = 2.0 * 128 * 256 * (16, 32, 64)[kind] * 50000 * sms / (e0.elapsed_time(e1) * 1e-3) / 1e12
     # far below the rate means the loop did not run on the tensor cores, far above that it did not run at all
     assert 0.3 * (2250, 4500, 9000)[kind] < tflops < 1.05 * (2250, 4500, 9000)[kind], tflops
