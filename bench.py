@@ -351,9 +351,9 @@ def roofline_of(fg, wk, prof, step_ms, dev, peaks):
             "tensor_peaks_tflops": tp}
 
 
-def side_measurement(fg, dev, name, steps, replays, world, peaks, use_graph, fp8=None):
+def side_measurement(fg, dev, name, steps, replays, world, peaks, use_graph, fp8=None, m=0):
     """A shorter measurement of another workload for the same JSON line."""
-    wk = Workload(fg, dev, name, fp8=fp8)
+    wk = Workload(fg, dev, name, m, fp8=fp8)
     for i in range(3):
         wk.step(i)
     fg.check(wk.ws)
@@ -495,6 +495,7 @@ def run_ours(args, world, rank, local):
     # ---- the other halves of the metric, measured the same way in the same run (shorter)
     if not args.no_extras and args.workload == "llama2-7b-fc1-decode" and not args.m:
         out["decode_70b"] = side_measurement(fg, dev, "llama2-70b-fc1-decode", 20, 11, world, peaks, use_graph)
+        out["decode_70b_m1"] = side_measurement(fg, dev, "llama2-70b-fc1-decode", 20, 11, world, peaks, use_graph, m=1)
         out["prefill"] = side_measurement(fg, dev, "llama2-7b-fc1-prefill", 5, 7, world, peaks, use_graph)
     if args.sweep:
         # the FP8 fraction of both operands swept over the given points (config 4: 0 / 10 / 20 / 30 %), each point
