@@ -38,8 +38,8 @@
  *                   decode-sized GEMM streams, for 16 token rows (rows >= M are zero):
  *                   2048 B: the E2M1 codes as a 16-row x 128-byte tile, the 16-byte pieces of row m
  *                   XOR-swizzled with m%8 (zero in FP8 blocks) | 256 B: E4M3 microscales [token][block
- *                   column], 0x00 for FP8 blocks | 16 B: uint32 whose bit j says that block column j of
- *                   some token is FP8, padding | 256 B padding | 8192 B: every element over the tensor
+ *                   column], 0x00 for FP8 blocks | 16 B: two uint32 (one per token octet; their OR is used) whose
+ *                   bit j says that block column j of some token is FP8, padding | 256 B padding | 8192 B: every element over the tensor
  *                   scale in fp16 (exact for either format): token octet m/8 in its own 4096 bytes, there
  *                   256 bytes per block column, there 32 bytes per token
  *   codes8        : a dense rows*K byte plane of which only the FP8 blocks are written (the

@@ -35,7 +35,8 @@
 // token rows (rows >= M are zero):
 //   AREC_A4   2048 B : the E2M1 codes as a 16-row x 128-byte tile, swizzled like REC_W4 (zero in FP8 blocks)
 //   AREC_SF    256 B : E4M3 microscales, [token][block column], 0x00 for FP8 blocks
-//   AREC_HOT    16 B : uint32: bit j set if block column j of some token is FP8 ("hot" column), then padding
+//   AREC_HOT    16 B : two uint32, one per token octet (readers use their OR): bit j set if block column j of some token is
+//                      FP8 ("hot" column); then padding
 //   AREC_AT   8192 B : the value over the tensor scale of every element in fp16 (E2M1 x microscale, or E4M3 x
 //                      2^ratio; exact): token octet m / 8 in its own 4096 bytes, there 256 bytes per block
 //                      column, there 32 bytes per token -- what a warp reads for one column is contiguous
